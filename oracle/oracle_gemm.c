@@ -1,0 +1,229 @@
+/*
+ * CPU oracle for C = alpha*A*B + beta*C  --  TEST INFRASTRUCTURE ONLY.
+ *
+ * This file is the independent reference the CUDA path is checked against.  It
+ * is imported only by the tests, by the smoke check and by the benchmark's
+ * cpu_baseline / reference legs; the product never calls it, and it shares no
+ * code (no header, helper, table or constant) with the CUDA path.
+ *
+ * What it computes.  The paper names the operation only as a matrix-multiply
+ * accumulate, "D += matmul(A, B)" (Section 2.2, the asynchronous-MMA listings),
+ * and measures it against the BLAS routine Sgemm (Section 6, Evaluation), whose
+ * definition C = alpha*A*B + beta*C is therefore the definition used here,
+ * written out as the plain triple loop in fp64:
+ *
+ *     S_ij    = sum_{k=0..K-1} a_ik * b_kj               (k ascending, fp64)
+ *     D_ij    = sum_{k=0..K-1} |a_ik * b_kj|             (fp64)
+ *     Cref_ij = alpha * S_ij + (beta != 0 ? beta * c_ij : 0)
+ *     Den_ij  = D_ij + |beta * c_ij|
+ *
+ * with a, b, c the stored 16-bit / 32-bit values widened exactly to fp64.  A
+ * product of two bf16 or two fp16 numbers is exact in fp64, so the only error
+ * of S is fp64 summation error (<= K * 2^-53 * D_ij).  beta == 0 means C_in is
+ * never read (BLAS convention), so NaN there cannot reach the result.
+ *
+ * There is no blocking, no reordering and no library call.  The only
+ * preparation step is a layout copy: A is widened to a dense row-major double
+ * array and B to a dense transposed (N x K) double array, so that the k loop
+ * walks two contiguous streams whatever the input layouts were.  Rows of C are
+ * distributed over threads with OpenMP; each entry is still one thread's plain
+ * k loop.
+ *
+ * Parity status: pinned for finite inputs (identity, permutation, rank-1,
+ * all-ones, hand-expanded tiny cases, transpose / layout invariants, linearity,
+ * a float64 library matmul on small shapes).  Behaviour on Inf/NaN *operands*
+ * is "parity unpinned".
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+enum { ORC_BF16 = 0, ORC_FP16 = 1, ORC_FP32 = 2 };
+enum { ORC_ROW = 0, ORC_COL = 1 };
+
+/* bf16: the upper 16 bits of an IEEE binary32. */
+static double widen_bf16(uint16_t h) {
+    uint32_t w = (uint32_t)h << 16;
+    float f;
+    memcpy(&f, &w, sizeof f);
+    return (double)f;
+}
+
+/* IEEE binary16: 1 sign, 5 exponent (bias 15), 10 fraction bits. */
+static double widen_fp16(uint16_t h) {
+    int sign = (h >> 15) & 1;
+    int e = (h >> 10) & 0x1F;
+    int frac = h & 0x3FF;
+    double v;
+    if (e == 0) {
+        v = ldexp((double)frac, -24);               /* zero and subnormals */
+    } else if (e == 31) {
+        v = frac ? NAN : INFINITY;
+    } else {
+        v = ldexp((double)(frac | 0x400), e - 25);  /* (1 + frac/1024) * 2^(e-15) */
+    }
+    return sign ? -v : v;
+}
+
+static double widen_at(const void* base, int dtype, int64_t idx) {
+    switch (dtype) {
+        case ORC_BF16: return widen_bf16(((const uint16_t*)base)[idx]);
+        case ORC_FP16: return widen_fp16(((const uint16_t*)base)[idx]);
+        default:       return (double)((const float*)base)[idx];
+    }
+}
+
+/* element (r, c) of a matrix stored with the given layout and leading dimension */
+static int64_t offset_of(int64_t r, int64_t c, int layout, int64_t ld) {
+    return layout == ORC_ROW ? r * ld + c : c * ld + r;
+}
+
+int oracle_num_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+void oracle_set_num_threads(int n) {
+#ifdef _OPENMP
+    if (n > 0) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
+
+/* Widen one stored value; exported so tests can pin the decoders. */
+double oracle_widen(uint32_t bits, int dtype) {
+    if (dtype == ORC_FP32) {
+        float f;
+        memcpy(&f, &bits, sizeof f);
+        return (double)f;
+    }
+    return dtype == ORC_BF16 ? widen_bf16((uint16_t)bits) : widen_fp16((uint16_t)bits);
+}
+
+static int bad_args(int64_t M, int64_t N, int64_t K, int ab_dtype, int c_dtype, int a_layout,
+                    int b_layout, int c_layout, int64_t lda, int64_t ldb, int64_t ldc) {
+    if (M < 0 || N < 0 || K < 0) return 1;
+    if (ab_dtype != ORC_BF16 && ab_dtype != ORC_FP16) return 1;
+    if (c_dtype != ORC_BF16 && c_dtype != ORC_FP16 && c_dtype != ORC_FP32) return 1;
+    if ((a_layout | b_layout | c_layout) & ~1) return 1;
+    if (lda < (a_layout == ORC_ROW ? K : M)) return 1;
+    if (ldb < (b_layout == ORC_ROW ? N : K)) return 1;
+    if (ldc < (c_layout == ORC_ROW ? N : M)) return 1;
+    return 0;
+}
+
+/*
+ * Rows [row_begin, row_end) of the reference result.
+ *   cref, den : dense row-major (row_end-row_begin) x N doubles
+ * Returns 0 on success, 1 on bad arguments, 2 on allocation failure.
+ */
+int oracle_gemm_rows(int64_t M, int64_t N, int64_t K,
+                     const void* A, const void* B, const void* Cin,
+                     int ab_dtype, int c_dtype,
+                     int a_layout, int b_layout, int c_layout,
+                     int64_t lda, int64_t ldb, int64_t ldc,
+                     double alpha, double beta,
+                     int64_t row_begin, int64_t row_end,
+                     double* cref, double* den) {
+    if (bad_args(M, N, K, ab_dtype, c_dtype, a_layout, b_layout, c_layout, lda, ldb, ldc)) return 1;
+    if (row_begin < 0 || row_end > M || row_begin > row_end) return 1;
+    int64_t R = row_end - row_begin;
+    if (R == 0 || N == 0) return 0;
+
+    /* layout copy: Aw is R x K row-major, Bt is N x K row-major (B transposed) */
+    double* Aw = (double*)malloc(sizeof(double) * (size_t)(R * K + 1));
+    double* Bt = (double*)malloc(sizeof(double) * (size_t)(N * K + 1));
+    if (!Aw || !Bt) { free(Aw); free(Bt); return 2; }
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < R; ++i)
+        for (int64_t k = 0; k < K; ++k)
+            Aw[i * K + k] = widen_at(A, ab_dtype, offset_of(row_begin + i, k, a_layout, lda));
+#pragma omp parallel for schedule(static)
+    for (int64_t j = 0; j < N; ++j)
+        for (int64_t k = 0; k < K; ++k)
+            Bt[j * K + k] = widen_at(B, ab_dtype, offset_of(k, j, b_layout, ldb));
+
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t i = 0; i < R; ++i) {
+        for (int64_t j = 0; j < N; ++j) {
+            const double* a = Aw + i * K;
+            const double* b = Bt + j * K;
+            double s = 0.0, d = 0.0;
+            for (int64_t k = 0; k < K; ++k) {
+                double p = a[k] * b[k];
+                s += p;
+                d += fabs(p);
+            }
+            double r = alpha * s;
+            double dd = d;
+            if (beta != 0.0) {
+                double c = widen_at(Cin, c_dtype, offset_of(row_begin + i, j, c_layout, ldc));
+                r += beta * c;
+                dd += fabs(beta * c);
+            }
+            cref[i * N + j] = r;
+            den[i * N + j] = dd;
+        }
+    }
+    free(Aw);
+    free(Bt);
+    return 0;
+}
+
+/* Whole matrix. */
+int oracle_gemm(int64_t M, int64_t N, int64_t K,
+                const void* A, const void* B, const void* Cin,
+                int ab_dtype, int c_dtype,
+                int a_layout, int b_layout, int c_layout,
+                int64_t lda, int64_t ldb, int64_t ldc,
+                double alpha, double beta,
+                double* cref, double* den) {
+    return oracle_gemm_rows(M, N, K, A, B, Cin, ab_dtype, c_dtype, a_layout, b_layout, c_layout,
+                            lda, ldb, ldc, alpha, beta, 0, M, cref, den);
+}
+
+/*
+ * Selected entries (rows[e], cols[e]), each by the same definition, read straight
+ * through the layout accessor (no layout copy).  Used where the whole matrix is
+ * too large to evaluate: sampling only chooses which entries are evaluated.
+ */
+int oracle_gemm_entries(int64_t M, int64_t N, int64_t K,
+                        const void* A, const void* B, const void* Cin,
+                        int ab_dtype, int c_dtype,
+                        int a_layout, int b_layout, int c_layout,
+                        int64_t lda, int64_t ldb, int64_t ldc,
+                        double alpha, double beta,
+                        int64_t n_entries, const int64_t* rows, const int64_t* cols,
+                        double* cref, double* den) {
+    if (bad_args(M, N, K, ab_dtype, c_dtype, a_layout, b_layout, c_layout, lda, ldb, ldc)) return 1;
+    for (int64_t e = 0; e < n_entries; ++e)
+        if (rows[e] < 0 || rows[e] >= M || cols[e] < 0 || cols[e] >= N) return 1;
+#pragma omp parallel for schedule(dynamic, 64)
+    for (int64_t e = 0; e < n_entries; ++e) {
+        int64_t i = rows[e], j = cols[e];
+        double s = 0.0, d = 0.0;
+        for (int64_t k = 0; k < K; ++k) {
+            double p = widen_at(A, ab_dtype, offset_of(i, k, a_layout, lda)) *
+                       widen_at(B, ab_dtype, offset_of(k, j, b_layout, ldb));
+            s += p;
+            d += fabs(p);
+        }
+        double r = alpha * s;
+        if (beta != 0.0) {
+            double c = widen_at(Cin, c_dtype, offset_of(i, j, c_layout, ldc));
+            r += beta * c;
+            d += fabs(beta * c);
+        }
+        cref[e] = r;
+        den[e] = d;
+    }
+    return 0;
+}
