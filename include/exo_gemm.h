@@ -1,0 +1,191 @@
+/*
+ * exo_gemm.h -- C ABI of the B200 (sm_100a) tensor-core GEMM library.
+ *
+ * Operation.  C = alpha * A * B + beta * C with 16-bit floating-point operands
+ * (bf16 or fp16) and fp32 accumulation: the matrix-multiply-accumulate the
+ * paper's kernels implement ("D += matmul(A, B)", Section 2.2 listings; the
+ * GEMM kernels of Section 6, "Evaluation", measured against BLAS Sgemm, whose
+ * alpha/beta/layout/leading-dimension conventions this interface follows).
+ *
+ * Every compute step runs in hand-written CUDA kernels on the device; there is
+ * no CPU path and no fallback: on a device that is not compute capability 10.x
+ * exo_gemm_create fails with EXO_GEMM_ERR_ARCH.
+ *
+ * Plain C.  Callers need no CUDA headers: the stream is passed as void*.
+ */
+#ifndef EXO_GEMM_H_
+#define EXO_GEMM_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct exo_gemm_plan* exo_gemm_handle_t; /* opaque; owned by the library */
+
+typedef enum {
+  EXO_GEMM_OK = 0,
+  EXO_GEMM_ERR_NULL = 1,           /* a required pointer argument is NULL                         */
+  EXO_GEMM_ERR_INVALID_ARG = 2,    /* negative or oversized dimension, ld below extent, bad enum   */
+  EXO_GEMM_ERR_UNSUPPORTED = 3,    /* legal BLAS call outside the supported set (see below)       */
+  EXO_GEMM_ERR_ALIGNMENT = 4,      /* a matrix base pointer is not 16-byte aligned (run)          */
+  EXO_GEMM_ERR_ARCH = 5,           /* device is not compute capability 10.x                        */
+  EXO_GEMM_ERR_CUDA = 6,           /* a CUDA runtime/driver call failed                            */
+  EXO_GEMM_ERR_DEVICE_TIMEOUT = 7  /* a bounded device-side wait gave up in an earlier launch      */
+} exo_gemm_status_t;
+
+typedef enum { EXO_GEMM_BF16 = 0, EXO_GEMM_FP16 = 1, EXO_GEMM_FP32 = 2 } exo_gemm_dtype_t;
+typedef enum { EXO_GEMM_ROW_MAJOR = 0, EXO_GEMM_COL_MAJOR = 1 } exo_gemm_layout_t;
+
+/*
+ * Tuning overrides, OR-ed into exo_gemm_desc_t.flags.  0 = let the library choose.
+ *   bits 0..1   cta_group: 1 = one SM per tile, 2 = a pair of SMs (2-CTA cluster) per tile
+ *   bits 2..5   tile N / 64 (1, 2 or 4  =>  64, 128 or 256 columns per tile)
+ *   bits 6..9   raster band width in tiles (1..15)
+ *   bit  10     raster direction: 0 = library choice, set = bands along M instead of N
+ *   bits 12..19 grid limit: launch at most this many CTAs (multiple of cta_group), 0 = all SMs
+ */
+#define EXO_GEMM_FLAG_CTA_GROUP(g)  ((uint32_t)(g) & 3u)
+#define EXO_GEMM_FLAG_TILE_N(n)     ((((uint32_t)(n) / 64u) & 15u) << 2)
+#define EXO_GEMM_FLAG_BAND(b)       (((uint32_t)(b) & 15u) << 6)
+#define EXO_GEMM_FLAG_BANDS_ALONG_M (1u << 10)
+#define EXO_GEMM_FLAG_GRID_LIMIT(c) (((uint32_t)(c) & 255u) << 12)
+
+/*
+ * Problem descriptor.  Logical shapes: A is M x K, B is K x N, C is M x N.
+ * Leading dimensions are in elements: for a row-major matrix ld >= #columns, for
+ * a column-major matrix ld >= #rows.
+ *
+ * Supported set: ab_dtype in {BF16, FP16}; c_dtype FP32 or equal to ab_dtype; any
+ * of the 8 layout combinations; 0 <= M, N, K <= 2^31 - 1.  Because operands and
+ * results move by TMA, every leading dimension times its element size must be a
+ * multiple of 16 bytes (16-bit: ld % 8 == 0, fp32 C: ldc % 4 == 0) and every base
+ * pointer passed to exo_gemm_run must be 16-byte aligned.  Legal BLAS calls
+ * outside this set return EXO_GEMM_ERR_UNSUPPORTED.
+ */
+typedef struct {
+  int64_t M, N, K;
+  int32_t ab_dtype;                     /* exo_gemm_dtype_t: BF16 or FP16, both operands       */
+  int32_t c_dtype;                      /* exo_gemm_dtype_t: FP32 or the same as ab_dtype      */
+  int32_t a_layout, b_layout, c_layout; /* exo_gemm_layout_t                                   */
+  int32_t device;                       /* CUDA device ordinal; -1 = the current device        */
+  int64_t lda, ldb, ldc;                /* elements                                            */
+  uint32_t flags;                       /* 0, or EXO_GEMM_FLAG_* overrides                     */
+  uint32_t reserved;                    /* must be 0                                           */
+} exo_gemm_desc_t;
+
+/* What a plan decided; filled by exo_gemm_get_info. */
+typedef struct {
+  int32_t cta_group;      /* 1 or 2 SMs per tile                                               */
+  int32_t tile_m, tile_n; /* output tile of one CTA group (tile_m = 128 * cta_group)           */
+  int32_t tile_k;         /* k-block staged per pipeline stage (64 elements = 128 bytes)       */
+  int32_t stages;         /* depth of the shared-memory operand ring                           */
+  int32_t grid;           /* CTAs launched (persistent)                                        */
+  int32_t smem_bytes;     /* dynamic shared memory per CTA                                     */
+  int32_t tmem_columns;   /* tensor-memory columns allocated per CTA (2 accumulators)          */
+  int32_t tiles_m, tiles_n;
+  int32_t raster_along_m; /* 1: bands run along M, tiles inside a band walk N first            */
+  int32_t raster_band;    /* band width in tiles                                               */
+  int32_t swapped;        /* 1: column-major C computed as C^T = B^T A^T                       */
+  int32_t sm_count;
+  int32_t kernel_launches_per_run; /* 1, or 0 for an empty problem                             */
+  int32_t reserved[5];
+} exo_gemm_info_t;
+
+/*
+ * Pure argument check; needs no GPU and touches no CUDA state.  Returns OK,
+ * ERR_NULL, ERR_INVALID_ARG or ERR_UNSUPPORTED by the rules above.
+ */
+exo_gemm_status_t exo_gemm_validate(const exo_gemm_desc_t* desc);
+
+/*
+ * Builds a plan for one problem descriptor: validates, canonicalises
+ * (column-major C becomes the transposed product), picks the tile shape, the
+ * cta_group, the pipeline depth and the raster, and sizes the persistent grid
+ * (the paper's counterpart is the device-function configuration of Section 3.2,
+ * clusterDim and warp configuration, and the persistent task loop of
+ * Section 4.2).  Allocates host state and one 32-byte device status block;
+ * touches no user matrix.  *out is written only on success.
+ */
+exo_gemm_status_t exo_gemm_create(exo_gemm_handle_t* out, const exo_gemm_desc_t* desc);
+
+/*
+ * Enqueues C = alpha*A*B + beta*C on cuda_stream (a cudaStream_t; NULL = the
+ * legacy default stream) and returns without synchronising.
+ *
+ *   A, B, C   DEVICE pointers, 16-byte aligned, laid out as the descriptor says.
+ *             The caller owns them and keeps them alive until the stream has
+ *             passed the kernel.  C is updated in place; A and B must not
+ *             overlap C.  The library never allocates, frees or copies them.
+ *   alpha, beta   host floats.  beta == 0: C is never read (NaN/Inf or
+ *             uninitialised memory in C do not propagate).  alpha == 0 or K == 0:
+ *             A and B are not read and C = beta*C.
+ *   M == 0 or N == 0: returns OK without launching.
+ *
+ * The result is alpha*acc + beta*C_in evaluated in fp32, where acc is the fp32
+ * tensor-core accumulation over k, then rounded to nearest-even into c_dtype.
+ * For a fixed plan the result is bitwise reproducible from run to run.
+ *
+ * All checks happen before the launch; on any error nothing is enqueued.  A
+ * handle may be used from several host threads (tensor maps are built on the
+ * caller's stack).  Device-side waits are bounded: if one gives up, the kernel
+ * records where in the plan's status block and exits cleanly; a later
+ * exo_gemm_check reports EXO_GEMM_ERR_DEVICE_TIMEOUT.
+ */
+exo_gemm_status_t exo_gemm_run(exo_gemm_handle_t plan, const void* A, const void* B, void* C,
+                               float alpha, float beta, void* cuda_stream);
+
+/*
+ * Reads the plan's device status block (a blocking 32-byte copy; call it after
+ * synchronising the stream(s) the plan ran on).  Returns OK or
+ * ERR_DEVICE_TIMEOUT, and clears the block.  detail, if not NULL, receives 8
+ * words: {code, role, barrier, tile, k_block, cta, 0, 0}.
+ */
+exo_gemm_status_t exo_gemm_check(exo_gemm_handle_t plan, uint32_t* detail);
+
+/*
+ * What exo_gemm_create would choose for `desc` on a device with `sm_count` SMs
+ * (all of them pairable).  Pure; needs no GPU.  Same status codes as
+ * exo_gemm_validate, plus ERR_NULL for info == NULL.
+ */
+exo_gemm_status_t exo_gemm_plan_preview(const exo_gemm_desc_t* desc, int32_t sm_count, exo_gemm_info_t* info);
+
+/* Reports what the plan chose. */
+exo_gemm_status_t exo_gemm_get_info(exo_gemm_handle_t plan, exo_gemm_info_t* info);
+
+/* Frees the plan and its device status block.  NULL is a no-op returning OK. */
+exo_gemm_status_t exo_gemm_destroy(exo_gemm_handle_t plan);
+
+/* Static string for a status code. */
+const char* exo_gemm_status_string(exo_gemm_status_t status);
+
+/* The CUDA error code (cudaError_t / CUresult as int) behind the last ERR_CUDA of this thread. */
+int exo_gemm_last_cuda_error(void);
+
+/*
+ * Host-side enumeration of the persistent tile schedule (Section 4.2 of the
+ * paper distributes tasks round-robin in lexicographic order and names a
+ * swizzled order as future work; this library uses a band-swizzled raster).
+ * Writes the (tile_m, tile_n) indices that worker `worker` of `num_workers`
+ * visits, in order, into out_m/out_n (capacity `cap`), and returns how many it
+ * visits (which may exceed cap), or -1 on bad arguments.  Needs no GPU; it
+ * compiles the same function the kernel uses.
+ */
+int64_t exo_gemm_schedule_enumerate(int32_t tiles_m, int32_t tiles_n, int32_t band, int32_t along_m,
+                                    int32_t num_workers, int32_t worker, int32_t* out_m,
+                                    int32_t* out_n, int64_t cap);
+
+/*
+ * Test hook for the bounded waits: the next exo_gemm_run on this plan uses
+ * `timeout_ms` as the device-side wait limit and, if skip_k_block >= 0, its
+ * first CTA's producer skips issuing the loads of that k-block (counted from the
+ * start of the CTA's work), so that one wait runs out and the kernel returns an
+ * error status without trapping.  The settings apply to one run, then reset.
+ */
+exo_gemm_status_t exo_gemm_debug_set(exo_gemm_handle_t plan, int32_t timeout_ms, int64_t skip_k_block);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EXO_GEMM_H_ */

@@ -1,0 +1,365 @@
+// C-ABI entry points: plan creation, tensor-map encoding and the launch.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <string.h>
+
+#include <atomic>
+#include <mutex>
+#include <new>
+
+#include "../../include/exo_gemm.h"
+#include "gemm_kernel.cuh"
+#include "plan.h"
+
+namespace exo {
+
+using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const GemmParams);
+
+template <int G, int BN>
+static KernelFn pick_out(int out) {
+  switch (out) {
+    case EXO_GEMM_BF16: return exo_gemm_kernel<G, BN, kOutBf16>;
+    case EXO_GEMM_FP16: return exo_gemm_kernel<G, BN, kOutFp16>;
+    default:            return exo_gemm_kernel<G, BN, kOutFp32>;
+  }
+}
+
+static KernelFn pick_kernel(int cta_group, int bn, int out) {
+  if (cta_group == 2) return bn == 256 ? pick_out<2, 256>(out) : pick_out<2, 128>(out);
+  if (bn == 256) return pick_out<1, 256>(out);
+  if (bn == 128) return pick_out<1, 128>(out);
+  return pick_out<1, 64>(out);
+}
+
+static thread_local int g_last_cuda_error = 0;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode_fn() {
+  static std::once_flag once;
+  static EncodeTiledFn fn = nullptr;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q);
+    if (e == cudaSuccess && q == cudaDriverEntryPointSuccess) fn = (EncodeTiledFn)p;
+    else g_last_cuda_error = (int)e;
+  });
+  return fn;
+}
+
+// 2-D tensor map over a matrix whose contiguous dimension has `inner` elements and
+// whose other dimension has `outer` elements `ld` elements apart.
+static CUresult encode_2d(CUtensorMap* map, int dtype, const void* base, uint64_t inner, uint64_t outer,
+                          uint64_t ld, uint32_t box_inner, uint32_t box_outer, bool operand) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return CUDA_ERROR_NOT_FOUND;
+  const CUtensorMapDataType dt = dtype == EXO_GEMM_FP32   ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                                 : dtype == EXO_GEMM_FP16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
+                                                          : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+  cuuint64_t dims[2] = {inner, outer};
+  cuuint64_t strides[1] = {ld * (uint64_t)elem_bytes(dtype)};
+  cuuint32_t box[2] = {box_inner, box_outer};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B,
+            operand ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_NONE,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+}
+
+}  // namespace exo
+
+struct exo_gemm_plan {
+  exo_gemm_desc_t desc;
+  exo::Canonical canon;
+  exo::TileConfig cfg;
+  exo::KernelFn kernel;
+  int device;
+  int sm_count;
+  int smem_bytes;
+  uint32_t* d_status;
+  std::atomic<int32_t> dbg_timeout_ms;
+  std::atomic<int64_t> dbg_skip_k_block;
+};
+
+using namespace exo;
+
+namespace {
+
+struct DeviceGuard {
+  int prev = -1;
+  bool switched = false;
+  cudaError_t err = cudaSuccess;
+  explicit DeviceGuard(int dev) {
+    err = cudaGetDevice(&prev);
+    if (err == cudaSuccess && dev >= 0 && dev != prev) {
+      err = cudaSetDevice(dev);
+      switched = err == cudaSuccess;
+    }
+  }
+  ~DeviceGuard() {
+    if (switched) cudaSetDevice(prev);
+  }
+};
+
+exo_gemm_status_t cuda_fail(cudaError_t e) {
+  g_last_cuda_error = (int)e;
+  cudaGetLastError();  // clear the sticky-free error state of the runtime
+  return EXO_GEMM_ERR_CUDA;
+}
+
+void fill_info(const exo_gemm_plan* p, exo_gemm_info_t* info) {
+  memset(info, 0, sizeof(*info));
+  info->cta_group = p->cfg.cta_group;
+  info->tile_m = 128 * p->cfg.cta_group;
+  info->tile_n = p->cfg.tile_n;
+  info->tile_k = kBlockK;
+  info->stages = p->cfg.stages;
+  info->grid = p->cfg.workers * p->cfg.cta_group;
+  info->smem_bytes = p->smem_bytes;
+  info->tmem_columns = 2 * p->cfg.tile_n;
+  info->tiles_m = p->cfg.tiles_m;
+  info->tiles_n = p->cfg.tiles_n;
+  info->raster_along_m = p->cfg.along_m;
+  info->raster_band = p->cfg.band;
+  info->swapped = p->canon.swapped;
+  info->sm_count = p->sm_count;
+  info->kernel_launches_per_run = (p->canon.M == 0 || p->canon.N == 0) ? 0 : 1;
+}
+
+}  // namespace
+
+extern "C" {
+
+exo_gemm_status_t exo_gemm_validate(const exo_gemm_desc_t* desc) { return validate_desc(desc); }
+
+const char* exo_gemm_status_string(exo_gemm_status_t s) {
+  switch (s) {
+    case EXO_GEMM_OK: return "ok";
+    case EXO_GEMM_ERR_NULL: return "null pointer argument";
+    case EXO_GEMM_ERR_INVALID_ARG: return "invalid argument";
+    case EXO_GEMM_ERR_UNSUPPORTED: return "unsupported configuration";
+    case EXO_GEMM_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
+    case EXO_GEMM_ERR_ARCH: return "device is not compute capability 10.x";
+    case EXO_GEMM_ERR_CUDA: return "CUDA call failed";
+    case EXO_GEMM_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+int exo_gemm_last_cuda_error(void) { return g_last_cuda_error; }
+
+int64_t exo_gemm_schedule_enumerate(int32_t tiles_m, int32_t tiles_n, int32_t band, int32_t along_m,
+                                    int32_t num_workers, int32_t worker, int32_t* out_m, int32_t* out_n,
+                                    int64_t cap) {
+  if (tiles_m < 0 || tiles_n < 0 || band < 1 || num_workers < 1 || worker < 0 || worker >= num_workers ||
+      cap < 0 || (cap > 0 && (!out_m || !out_n)))
+    return -1;
+  Raster r{tiles_m, tiles_n, band, along_m ? 1 : 0};
+  int64_t n = 0;
+  for (int64_t t = worker; t < raster_total(r); t += num_workers, ++n) {
+    if (n < cap) {
+      const TileCoord c = raster_decode(r, t);
+      out_m[n] = c.m;
+      out_n[n] = c.n;
+    }
+  }
+  return n;
+}
+
+exo_gemm_status_t exo_gemm_plan_preview(const exo_gemm_desc_t* desc, int32_t sm_count, exo_gemm_info_t* info) {
+  if (!info) return EXO_GEMM_ERR_NULL;
+  exo_gemm_status_t st = validate_desc(desc);
+  if (st != EXO_GEMM_OK) return st;
+  if (sm_count < 1) return EXO_GEMM_ERR_INVALID_ARG;
+  exo_gemm_plan p{};
+  p.desc = *desc;
+  p.canon = canonicalize(*desc);
+  p.sm_count = sm_count;
+  p.cfg = choose_config(p.canon, decode_flags(desc->flags), sm_count, sm_count / 2);
+  p.smem_bytes = smem_bytes_for(p.cfg.cta_group, p.cfg.tile_n);
+  fill_info(&p, info);
+  return EXO_GEMM_OK;
+}
+
+exo_gemm_status_t exo_gemm_create(exo_gemm_handle_t* out, const exo_gemm_desc_t* desc) {
+  if (!out) return EXO_GEMM_ERR_NULL;
+  exo_gemm_status_t st = validate_desc(desc);
+  if (st != EXO_GEMM_OK) return st;
+
+  int device = desc->device;
+  cudaError_t e;
+  if (device < 0) {
+    e = cudaGetDevice(&device);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
+  DeviceGuard guard(device);
+  if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+  int major = 0, sms = 0;
+  e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (major != 10) return EXO_GEMM_ERR_ARCH;  // no fallback path by design
+  e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (!get_encode_fn()) return EXO_GEMM_ERR_CUDA;
+
+  exo_gemm_plan* p = new (std::nothrow) exo_gemm_plan{};
+  if (!p) return EXO_GEMM_ERR_CUDA;
+  p->desc = *desc;
+  p->canon = canonicalize(*desc);
+  p->device = device;
+  p->sm_count = sms;
+  p->dbg_timeout_ms = 0;
+  p->dbg_skip_k_block = -1;
+  const FlagOverrides ov = decode_flags(desc->flags);
+
+  // How many 2-CTA clusters can be resident at once (GPC shapes may leave SMs unpaired).
+  int max_pairs = 0;
+  if (ov.cta_group != 1) {
+    KernelFn probe = pick_kernel(2, 256, desc->c_dtype);
+    const int smem = smem_bytes_for(2, 256);
+    e = cudaFuncSetAttribute((const void*)probe, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) { delete p; return cuda_fail(e); }
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3((unsigned)sms & ~1u, 1, 1);
+    lc.blockDim = dim3(kNumThreads, 1, 1);
+    lc.dynamicSmemBytes = smem;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    lc.attrs = at;
+    lc.numAttrs = 1;
+    int n = 0;
+    e = cudaOccupancyMaxActiveClusters(&n, (const void*)probe, &lc);
+    if (e != cudaSuccess) { delete p; return cuda_fail(e); }
+    max_pairs = n < sms / 2 ? n : sms / 2;
+  }
+
+  p->cfg = choose_config(p->canon, ov, sms, max_pairs);
+  p->kernel = pick_kernel(p->cfg.cta_group, p->cfg.tile_n, desc->c_dtype);
+  p->smem_bytes = smem_bytes_for(p->cfg.cta_group, p->cfg.tile_n);
+  e = cudaFuncSetAttribute((const void*)p->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, p->smem_bytes);
+  if (e != cudaSuccess) { delete p; return cuda_fail(e); }
+  e = cudaMalloc((void**)&p->d_status, 32);
+  if (e != cudaSuccess) { delete p; return cuda_fail(e); }
+  e = cudaMemset(p->d_status, 0, 32);
+  if (e != cudaSuccess) { cudaFree(p->d_status); delete p; return cuda_fail(e); }
+  *out = p;
+  return EXO_GEMM_OK;
+}
+
+exo_gemm_status_t exo_gemm_get_info(exo_gemm_handle_t plan, exo_gemm_info_t* info) {
+  if (!plan || !info) return EXO_GEMM_ERR_NULL;
+  fill_info(plan, info);
+  return EXO_GEMM_OK;
+}
+
+exo_gemm_status_t exo_gemm_debug_set(exo_gemm_handle_t plan, int32_t timeout_ms, int64_t skip_k_block) {
+  if (!plan) return EXO_GEMM_ERR_NULL;
+  if (timeout_ms < 0 || timeout_ms > 10000) return EXO_GEMM_ERR_INVALID_ARG;
+  plan->dbg_timeout_ms = timeout_ms;
+  plan->dbg_skip_k_block = skip_k_block;
+  return EXO_GEMM_OK;
+}
+
+exo_gemm_status_t exo_gemm_run(exo_gemm_handle_t plan, const void* A, const void* B, void* C, float alpha,
+                               float beta, void* cuda_stream) {
+  if (!plan) return EXO_GEMM_ERR_NULL;
+  const Canonical& cn = plan->canon;
+  if (cn.M == 0 || cn.N == 0) return EXO_GEMM_OK;
+  const bool read_ab = alpha != 0.f && cn.K > 0;
+  if (!C || (read_ab && (!A || !B))) return EXO_GEMM_ERR_NULL;
+  if (((uintptr_t)C & 15u) || (read_ab && (((uintptr_t)A | (uintptr_t)B) & 15u))) return EXO_GEMM_ERR_ALIGNMENT;
+
+  const exo_gemm_desc_t& d = plan->desc;
+  const TileConfig& cfg = plan->cfg;
+  const void* opA = cn.swapped ? B : A;
+  const void* opB = cn.swapped ? A : B;
+
+  GemmParams prm{};
+  prm.M = (int32_t)cn.M;
+  prm.N = (int32_t)cn.N;
+  prm.K = (int32_t)cn.K;
+  prm.num_k_blocks = read_ab ? (int32_t)((cn.K + kBlockK - 1) / kBlockK) : 0;
+  prm.raster = Raster{cfg.tiles_m, cfg.tiles_n, cfg.band, cfg.along_m};
+  prm.alpha = read_ab ? alpha : 0.f;
+  prm.beta = beta;
+  prm.idesc = make_idesc(d.ab_dtype, cn.a_mn_major, cn.b_mn_major, 128 * cfg.cta_group, cfg.tile_n);
+  prm.a = make_staging(cn.a_mn_major);
+  prm.b = make_staging(cn.b_mn_major);
+  prm.status = plan->d_status;
+  const int32_t dbg_ms = plan->dbg_timeout_ms.exchange(0);
+  prm.timeout_ns = dbg_ms > 0 ? (uint64_t)dbg_ms * 1000000ull : 4000000000ull;
+  prm.debug_skip_k_block = plan->dbg_skip_k_block.exchange(-1);
+
+  CUtensorMap tm_a, tm_b, tm_c;
+  memset(&tm_a, 0, sizeof tm_a);
+  memset(&tm_b, 0, sizeof tm_b);
+  CUresult r;
+  const int b_rows = cfg.tile_n / cfg.cta_group;
+  if (read_ab) {
+    r = cn.a_mn_major ? encode_2d(&tm_a, d.ab_dtype, opA, cn.M, cn.K, cn.lda, 64, kBlockK, true)
+                      : encode_2d(&tm_a, d.ab_dtype, opA, cn.K, cn.M, cn.lda, kBlockK, kBlockM, true);
+    if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return EXO_GEMM_ERR_CUDA; }
+    r = cn.b_mn_major ? encode_2d(&tm_b, d.ab_dtype, opB, cn.N, cn.K, cn.ldb, 64, kBlockK, true)
+                      : encode_2d(&tm_b, d.ab_dtype, opB, cn.K, cn.N, cn.ldb, kBlockK, b_rows, true);
+    if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return EXO_GEMM_ERR_CUDA; }
+  }
+  r = encode_2d(&tm_c, d.c_dtype, C, cn.N, cn.M, cn.ldc, d.c_dtype == EXO_GEMM_FP32 ? 32 : 64, 32, false);
+  if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return EXO_GEMM_ERR_CUDA; }
+  if (!read_ab) { tm_a = tm_c; tm_b = tm_c; }  // never dereferenced for data; keeps the prefetch valid
+
+  DeviceGuard guard(plan->device);
+  if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+  cudaLaunchConfig_t lc{};
+  lc.gridDim = dim3((unsigned)(cfg.workers * cfg.cta_group), 1, 1);
+  lc.blockDim = dim3(kNumThreads, 1, 1);
+  lc.dynamicSmemBytes = plan->smem_bytes;
+  lc.stream = (cudaStream_t)cuda_stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = cfg.cta_group;
+  at[0].val.clusterDim.y = 1;
+  at[0].val.clusterDim.z = 1;
+  lc.attrs = at;
+  lc.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&lc, plan->kernel, tm_a, tm_b, tm_c, prm);
+  if (e != cudaSuccess) return cuda_fail(e);
+  return EXO_GEMM_OK;
+}
+
+exo_gemm_status_t exo_gemm_check(exo_gemm_handle_t plan, uint32_t* detail) {
+  if (!plan) return EXO_GEMM_ERR_NULL;
+  DeviceGuard guard(plan->device);
+  if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+  uint32_t h[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  cudaError_t e = cudaMemcpy(h, plan->d_status, 32, cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (detail) memcpy(detail, h, 32);
+  if (h[0] == kStatusOk) return EXO_GEMM_OK;
+  e = cudaMemset(plan->d_status, 0, 32);
+  if (e != cudaSuccess) return cuda_fail(e);
+  return EXO_GEMM_ERR_DEVICE_TIMEOUT;
+}
+
+exo_gemm_status_t exo_gemm_destroy(exo_gemm_handle_t plan) {
+  if (!plan) return EXO_GEMM_OK;
+  exo_gemm_status_t st = EXO_GEMM_OK;
+  {
+    DeviceGuard guard(plan->device);
+    if (plan->d_status) {
+      cudaError_t e = cudaFree(plan->d_status);
+      if (e != cudaSuccess) st = cuda_fail(e);
+    }
+  }
+  delete plan;
+  return st;
+}
+
+}  // extern "C"

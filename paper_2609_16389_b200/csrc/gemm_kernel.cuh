@@ -1,0 +1,403 @@
+// Persistent warp-specialised tcgen05 GEMM kernel for sm_100a.
+//
+// One CTA (CTA_GROUP == 1) or a pair of CTAs on two SMs (CTA_GROUP == 2, a
+// 2-CTA cluster) computes output tiles of (128 * CTA_GROUP) x BN, one after
+// another, taken round-robin from a band-swizzled raster.  Roles per CTA:
+//
+//   warp 0, one lane   producer: TMA loads of the A and B k-blocks into a ring
+//                      of shared-memory stages (full/empty mbarriers)
+//   warp 1, one lane   MMA issuer (leader CTA only): tcgen05.mma from shared
+//                      memory into one of two TMEM accumulators; tcgen05.commit
+//                      releases stages and publishes finished accumulators
+//   warp 1             owns the TMEM allocation
+//   warps 2..5         epilogue: tcgen05.ld the accumulator (warp w reads TMEM
+//                      lanes 32*(w%4)..), alpha*acc + beta*C_in in fp32, convert,
+//                      write a 128B-swizzled staging buffer, TMA store
+//
+// The structure follows the kernel class of the paper's Section 6 (persistent,
+// warp-specialised, TMA + swizzled shared memory + asynchronous tensor-core
+// MMA, 2-CTA clusters), re-designed for Blackwell: the accumulator lives in
+// tensor memory instead of registers, one thread issues the MMA, and completion
+// is tracked by tcgen05.commit on mbarriers instead of commit groups.  The
+// synchronisation rules it obeys are the ones the paper's Section 2.2 bug
+// catalogue spells out: a stage is refilled only after the *asynchronous* MMAs
+// that read it completed (commit -> empty barrier), an accumulator is read only
+// after the MMAs that write it completed (commit -> tmem_full barrier), and a
+// release that covers another CTA's shared memory is cluster-scoped.
+//
+// Every wait is bounded: when one gives up, the kernel records where, all roles
+// leave their loops, TMEM is freed and the kernel returns.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <stdint.h>
+
+#include "gemm_params.h"
+#include "ptx.cuh"
+
+namespace exo {
+
+enum OutKind : int { kOutBf16 = 0, kOutFp16 = 1, kOutFp32 = 2 };
+
+struct WaitSite {
+  uint32_t role, barrier, tile, k_block;
+};
+
+template <bool CLUSTER>
+__device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, const GemmParams& p, WaitSite site) {
+  const uint64_t t0 = ptx::globaltimer_ns();
+  uint32_t n = 0;
+  for (;;) {
+    const bool done = CLUSTER ? ptx::mbar_try_wait_cluster(bar, parity) : ptx::mbar_try_wait(bar, parity);
+    if (done) return true;
+    if ((++n & 15u) == 0u) {
+      if (*(volatile uint32_t*)p.status != kStatusOk) return false;  // another role gave up
+      if (ptx::globaltimer_ns() - t0 > p.timeout_ns) {
+        if (atomicCAS(p.status, (uint32_t)kStatusOk, (uint32_t)kStatusTimeout) == kStatusOk) {
+          p.status[1] = site.role;
+          p.status[2] = site.barrier;
+          p.status[3] = site.tile;
+          p.status[4] = site.k_block;
+          p.status[5] = blockIdx.x;
+          __threadfence();
+        }
+        return false;
+      }
+    }
+  }
+}
+
+// Bounded mbarrier wait.  Returns false if the wait was abandoned.
+template <bool CLUSTER>
+__device__ __forceinline__ bool wait_barrier(uint32_t bar, uint32_t parity, const GemmParams& p,
+                                             WaitSite site) {
+  const bool done = CLUSTER ? ptx::mbar_try_wait_cluster(bar, parity) : ptx::mbar_try_wait(bar, parity);
+  if (done) return true;
+  return wait_slow<CLUSTER>(bar, parity, p, site);
+}
+
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr, const OperandStaging& op) {
+  const uint32_t lo = ((smem_addr & 0x3FFFFu) >> 4) | (op.lbo_enc << 16);
+  return ((uint64_t)op.desc_hi << 32) | lo;
+}
+
+template <int OUT>
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+  if constexpr (OUT == kOutBf16) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+  } else {
+    __half2 v = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+  }
+}
+
+template <int OUT>
+__device__ __forceinline__ float2 unpack2(uint32_t w) {
+  if constexpr (OUT == kOutBf16) {
+    return __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&w));
+  } else {
+    return __half22float2(*reinterpret_cast<__half2*>(&w));
+  }
+}
+
+template <int CTA_GROUP, int BN, int OUT>
+__global__ void __launch_bounds__(kNumThreads, 1)
+exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+                const __grid_constant__ CUtensorMap tm_c, const GemmParams p) {
+  constexpr int STAGES = max_stages(CTA_GROUP, BN);
+  constexpr int B_ROWS = BN / CTA_GROUP;             // rows of the B tile this CTA stages
+  constexpr int STAGE_BYTES = stage_bytes(CTA_GROUP, BN);
+  constexpr uint32_t TMEM_COLS = 2 * BN;             // two accumulators; 128, 256 or 512 columns
+  constexpr int CW = (OUT == kOutFp32) ? 32 : 64;    // columns per epilogue chunk = 128 bytes of C
+  constexpr int NCHUNK = BN / CW;
+  constexpr bool PAIR = CTA_GROUP == 2;
+  static_assert(BN == 64 || BN == 128 || BN == 256, "tile N");
+  static_assert(STAGES >= 2, "ring too shallow");
+
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;  // swizzle atoms are 1 KB
+  const uint32_t stage0 = smem_base;
+  const uint32_t epi0 = smem_base + STAGES * STAGE_BYTES;
+  const uint32_t bar0 = epi0 + kEpiWarps * kEpiBufsPerWarp * kEpiBufBytes;
+  auto full_bar = [&](uint32_t s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](uint32_t s) { return bar0 + 8u * (STAGES + s); };
+  auto tfull_bar = [&](uint32_t a) { return bar0 + 8u * (2 * STAGES + a); };
+  auto tempty_bar = [&](uint32_t a) { return bar0 + 8u * (2 * STAGES + 2 + a); };
+  auto cin_bar = [&](uint32_t w, uint32_t b) { return bar0 + 8u * (2 * STAGES + 4 + 2 * w + b); };
+  const uint32_t tmem_slot = bar0 + 8u * (2 * STAGES + 12);
+
+  const uint32_t warp = threadIdx.x >> 5;
+  const uint32_t lane = threadIdx.x & 31u;
+  const uint32_t cta_rank = PAIR ? ptx::cluster_ctarank() : 0u;
+  const int64_t worker = blockIdx.x / CTA_GROUP;
+  const int64_t num_workers = gridDim.x / CTA_GROUP;
+  const int64_t total_tiles = raster_total(p.raster);
+  const int32_t nkb = p.num_k_blocks;
+
+  // ---------------------------------------------------------------- setup
+  if (threadIdx.x == 0) {
+    for (uint32_t s = 0; s < STAGES; ++s) {
+      ptx::mbar_init(full_bar(s), 1);
+      ptx::mbar_init(empty_bar(s), 1);
+    }
+    for (uint32_t a = 0; a < 2; ++a) {
+      ptx::mbar_init(tfull_bar(a), 1);
+      ptx::mbar_init(tempty_bar(a), kEpiWarps * CTA_GROUP);
+    }
+    for (uint32_t w = 0; w < kEpiWarps; ++w)
+      for (uint32_t b = 0; b < 2; ++b) ptx::mbar_init(cin_bar(w, b), 1);
+    ptx::fence_mbar_init();
+    ptx::prefetch_tensormap(&tm_a);
+    ptx::prefetch_tensormap(&tm_b);
+    ptx::prefetch_tensormap(&tm_c);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc<CTA_GROUP>(tmem_slot, TMEM_COLS);
+    ptx::tmem_relinquish<CTA_GROUP>();
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  if constexpr (PAIR) {  // peer barriers must be initialised before anything remote touches them
+    ptx::cluster_arrive();
+    ptx::cluster_wait();
+  }
+  ptx::tc_fence_after_sync();
+  uint32_t tmem_base;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot) : "memory");
+
+  bool ok = true;
+
+  if (warp == 0) {
+    // ============================================================ producer
+    if (lane == 0) {
+      uint32_t s = 0, ph = 0;
+      int64_t issued = 0;
+      // in a pair, both CTAs' loads are counted on the leader's full barrier
+      const uint32_t full0 = PAIR ? ptx::map_to_cta(full_bar(0), 0) : full_bar(0);
+      for (int64_t t = worker; t < total_tiles && ok; t += num_workers) {
+        const TileCoord tc = raster_decode(p.raster, t);
+        const int32_t a_mn0 = tc.m * (kBlockM * CTA_GROUP) + (int32_t)cta_rank * kBlockM;
+        const int32_t b_mn0 = tc.n * BN + (int32_t)cta_rank * B_ROWS;
+        for (int32_t kb = 0; kb < nkb; ++kb) {
+          ok = wait_barrier<PAIR>(empty_bar(s), ph ^ 1u, p,
+                                  WaitSite{kRoleProducer, s, (uint32_t)t, (uint32_t)kb});
+          if (!ok) break;
+          if (cta_rank == 0) ptx::mbar_arrive_expect_tx(full_bar(s), STAGE_BYTES * CTA_GROUP);
+          const bool skip = (p.debug_skip_k_block == issued) && blockIdx.x == 0;
+          ++issued;
+          if (!skip) {
+            const uint32_t a_dst = stage0 + s * STAGE_BYTES;
+            const uint32_t b_dst = a_dst + kATileBytes;
+            const uint32_t bar = full0 + 8u * s;
+            const int32_t k0 = kb * kBlockK;
+            auto load = [&](uint32_t dst, const CUtensorMap* map, int32_t x, int32_t y) {
+              if constexpr (PAIR) ptx::tma_load_2d_pair(dst, map, x, y, bar);
+              else ptx::tma_load_2d(dst, map, x, y, bar);
+            };
+            if (!p.a.mn_major) {
+              load(a_dst, &tm_a, k0, a_mn0);
+            } else {
+#pragma unroll
+              for (int b = 0; b < kBlockM / 64; ++b) load(a_dst + b * 8192, &tm_a, a_mn0 + 64 * b, k0);
+            }
+            if (!p.b.mn_major) {
+              load(b_dst, &tm_b, k0, b_mn0);
+            } else {
+#pragma unroll
+              for (int b = 0; b < B_ROWS / 64; ++b) load(b_dst + b * 8192, &tm_b, b_mn0 + 64 * b, k0);
+            }
+          }
+          if (++s == STAGES) { s = 0; ph ^= 1u; }
+        }
+      }
+      // Tail: do not leave while stage releases addressed to this CTA are still in flight.
+      for (uint32_t i = 0; i < STAGES && ok; ++i) {
+        ok = wait_barrier<PAIR>(empty_bar(s), ph ^ 1u, p, WaitSite{kRoleProducerTail, s, 0, 0});
+        if (++s == STAGES) { s = 0; ph ^= 1u; }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ============================================================ MMA issuer
+    if (lane == 0 && cta_rank == 0 && nkb > 0) {
+      uint32_t s = 0, ph = 0, acc = 0, acc_ph = 0;
+      constexpr uint16_t kMask = PAIR ? 3 : 1;
+      for (int64_t t = worker; t < total_tiles && ok; t += num_workers) {
+        // the epilogue (of both CTAs) must have drained this accumulator
+        ok = wait_barrier<PAIR>(tempty_bar(acc), acc_ph ^ 1u, p, WaitSite{kRoleMma, 100 + acc, (uint32_t)t, 0});
+        if (!ok) break;
+        ptx::tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int32_t kb = 0; kb < nkb; ++kb) {
+          ok = wait_barrier<PAIR>(full_bar(s), ph, p, WaitSite{kRoleMma, s, (uint32_t)t, (uint32_t)kb});
+          if (!ok) break;
+          ptx::tc_fence_after_sync();
+          const uint32_t a_addr = stage0 + s * STAGE_BYTES;
+          const uint64_t a_desc = make_smem_desc(a_addr, p.a);
+          const uint64_t b_desc = make_smem_desc(a_addr + kATileBytes, p.b);
+          const int32_t k_left = p.K - kb * kBlockK;
+          const int32_t n_mma = k_left >= kBlockK ? kBlockK / kUmmaK : (k_left + kUmmaK - 1) / kUmmaK;
+          for (int32_t k = 0; k < n_mma; ++k) {
+            ptx::umma_f16<CTA_GROUP>(d_tmem, a_desc + (uint64_t)(k * p.a.k_step_enc),
+                                     b_desc + (uint64_t)(k * p.b.k_step_enc), p.idesc,
+                                     (kb | k) != 0 ? 1u : 0u);
+          }
+          ptx::umma_commit<CTA_GROUP>(empty_bar(s), kMask);  // stage free once these MMAs completed
+          if (++s == STAGES) { s = 0; ph ^= 1u; }
+        }
+        if (!ok) break;
+        ptx::umma_commit<CTA_GROUP>(tfull_bar(acc), kMask);  // accumulator complete
+        if ((acc ^= 1u) == 0u) acc_ph ^= 1u;
+      }
+    }
+    __syncwarp();
+  } else {
+    // ============================================================ epilogue
+    const uint32_t quad = warp & 3u;  // TMEM lanes 32*quad .. 32*quad+31 belong to this warp
+    const uint32_t ew = warp - 2u;
+    const uint32_t buf0 = epi0 + ew * (kEpiBufsPerWarp * kEpiBufBytes);
+    const uint32_t tempty0 = PAIR ? ptx::map_to_cta(tempty_bar(0), 0) : tempty_bar(0);
+    const bool has_beta = p.beta != 0.f;
+    const bool has_acc = nkb > 0;
+    const float alpha = p.alpha, beta = p.beta;
+    const uint32_t row_off = lane * 128u;
+    const uint32_t sw = lane & 7u;
+    uint32_t g = 0;  // running chunk counter: staging buffer g & 1, its C_in barrier phase (g >> 1) & 1
+    uint32_t acc = 0, acc_ph = 0;
+
+    for (int64_t t = worker; t < total_tiles; t += num_workers) {
+      const TileCoord tc = raster_decode(p.raster, t);
+      const int32_t row0 = tc.m * (kBlockM * CTA_GROUP) + (int32_t)cta_rank * kBlockM + (int32_t)quad * 32;
+      const int32_t col0 = tc.n * BN;
+      int32_t nch = 0;
+      if (row0 < p.M) {
+        nch = (p.N - col0 + CW - 1) / CW;
+        if (nch > NCHUNK) nch = NCHUNK;
+      }
+      if (has_acc) {
+        ok = wait_barrier<PAIR>(tfull_bar(acc), acc_ph, p, WaitSite{kRoleEpilogue, 200 + acc, (uint32_t)t, 0});
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        ptx::tc_fence_after_sync();
+      }
+      auto release_acc = [&]() {
+        ptx::tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) {
+          if constexpr (PAIR) ptx::mbar_arrive_cluster(tempty0 + 8u * acc);
+          else ptx::mbar_arrive(tempty0 + 8u * acc);
+        }
+      };
+      auto issue_cin = [&](uint32_t gg, int32_t chunk) {  // lane 0 only
+        const uint32_t b = gg & 1u;
+        ptx::mbar_arrive_expect_tx(cin_bar(ew, b), kEpiBufBytes);
+        ptx::tma_load_2d(buf0 + b * kEpiBufBytes, &tm_c, col0 + chunk * CW, row0, cin_bar(ew, b));
+      };
+      if (nch == 0) {
+        if (has_acc) release_acc();
+      } else if (has_beta) {
+        if (lane == 0) {
+          ptx::bulk_wait_read<0>();
+          issue_cin(g, 0);
+        }
+      }
+      for (int32_t c = 0; c < nch; ++c) {
+        const uint32_t buf = buf0 + (g & 1u) * kEpiBufBytes;
+        if (has_beta) {
+          if (c + 1 < nch && lane == 0) {
+            ptx::bulk_wait_read<0>();  // the other buffer's last store has been read out
+            issue_cin(g + 1, c + 1);
+          }
+          ok = wait_barrier<false>(cin_bar(ew, g & 1u), (g >> 1) & 1u, p,
+                                   WaitSite{kRoleEpilogueCin, 300 + (g & 1u), (uint32_t)t, (uint32_t)c});
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+        } else {
+          if (lane == 0) ptx::bulk_wait_read<1>();  // this buffer's last store (two chunks ago) is read out
+          __syncwarp();
+        }
+
+        uint32_t v[CW];
+        if (has_acc) {
+          const uint32_t taddr = tmem_base + ((quad * 32u) << 16) + acc * BN + c * CW;
+          ptx::tmem_ld_32x32(taddr, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
+          if constexpr (CW == 64) ptx::tmem_ld_32x32(taddr + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
+          ptx::tmem_ld_wait();
+          if (c == nch - 1) release_acc();  // last read of this accumulator: hand it back early
+        } else {
+#pragma unroll
+          for (int i = 0; i < CW; ++i) v[i] = 0u;
+        }
+
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {  // eight 16-byte pieces of this thread's 128-byte row segment
+          const uint32_t addr = buf + row_off + ((j ^ sw) << 4);
+          if constexpr (OUT == kOutFp32) {
+            float x0 = alpha * __uint_as_float(v[4 * j + 0]);
+            float x1 = alpha * __uint_as_float(v[4 * j + 1]);
+            float x2 = alpha * __uint_as_float(v[4 * j + 2]);
+            float x3 = alpha * __uint_as_float(v[4 * j + 3]);
+            if (has_beta) {
+              uint32_t c0, c1, c2, c3;
+              ptx::ld_shared_v4(addr, c0, c1, c2, c3);
+              x0 = fmaf(beta, __uint_as_float(c0), x0);
+              x1 = fmaf(beta, __uint_as_float(c1), x1);
+              x2 = fmaf(beta, __uint_as_float(c2), x2);
+              x3 = fmaf(beta, __uint_as_float(c3), x3);
+            }
+            ptx::st_shared_v4(addr, __float_as_uint(x0), __float_as_uint(x1), __float_as_uint(x2),
+                              __float_as_uint(x3));
+          } else {
+            float x[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) x[i] = alpha * __uint_as_float(v[8 * j + i]);
+            if (has_beta) {
+              uint32_t cw[4];
+              ptx::ld_shared_v4(addr, cw[0], cw[1], cw[2], cw[3]);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const float2 cc = unpack2<OUT>(cw[i]);
+                x[2 * i] = fmaf(beta, cc.x, x[2 * i]);
+                x[2 * i + 1] = fmaf(beta, cc.y, x[2 * i + 1]);
+              }
+            }
+            ptx::st_shared_v4(addr, pack2<OUT>(x[0], x[1]), pack2<OUT>(x[2], x[3]), pack2<OUT>(x[4], x[5]),
+                              pack2<OUT>(x[6], x[7]));
+          }
+        }
+        ptx::fence_proxy_async_smem();  // generic-proxy writes -> visible to the TMA store
+        __syncwarp();
+        if (lane == 0) {
+          ptx::tma_store_2d(&tm_c, col0 + c * CW, row0, buf);
+          ptx::bulk_commit();
+        }
+        ++g;
+      }
+      if (!ok) break;
+      if ((acc ^= 1u) == 0u) acc_ph ^= 1u;
+    }
+    if (lane == 0) ptx::bulk_wait<0>();  // all stores of this warp have completed
+    __syncwarp();
+  }
+
+  // ---------------------------------------------------------------- teardown
+  if (*(volatile uint32_t*)p.status != kStatusOk) {
+    // Some wait was abandoned: give copies and MMAs still in flight time to land
+    // before shared and tensor memory are released.
+    for (int i = 0; i < 200; ++i) __nanosleep(1000);
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  if constexpr (PAIR) {  // the peer's shared and tensor memory stay valid until both CTAs are done
+    ptx::cluster_arrive();
+    ptx::cluster_wait();
+  }
+  if (warp == 1) {
+    ptx::tc_fence_after_sync();
+    ptx::tmem_dealloc<CTA_GROUP>(tmem_base, TMEM_COLS);
+  }
+}
+
+}  // namespace exo

@@ -1,0 +1,69 @@
+// Kernel parameter block and compile-time geometry shared by the host plan and
+// the device kernel.
+#pragma once
+#include <stdint.h>
+
+#include "tile_scheduler.h"
+
+namespace exo {
+
+constexpr int kBlockM = 128;        // rows of C per CTA (one TMEM lane per row)
+constexpr int kBlockK = 64;         // elements of K per stage: 128 bytes = one swizzle span
+constexpr int kUmmaK = 16;          // K of one tcgen05.mma for 16-bit inputs
+constexpr int kNumThreads = 192;    // warp 0 producer, warp 1 MMA issuer + TMEM owner, warps 2..5 epilogue
+constexpr int kEpiWarps = 4;
+constexpr int kEpiBufBytes = 4096;  // one staging buffer: 32 rows x 128 bytes
+constexpr int kEpiBufsPerWarp = 2;
+constexpr int kSmemLimit = 232448;  // 227 KB opt-in limit per CTA
+constexpr int kBarrierBytes = 512;
+constexpr int kATileBytes = kBlockM * kBlockK * 2;  // 16 KB
+
+// Bytes of one pipeline stage in one CTA: its A rows plus its share of B.
+#if defined(__CUDACC__)
+#define EXO_CX __host__ __device__ constexpr
+#else
+#define EXO_CX constexpr
+#endif
+EXO_CX int stage_bytes(int cta_group, int bn) { return kATileBytes + (bn / cta_group) * kBlockK * 2; }
+
+EXO_CX int max_stages(int cta_group, int bn) {
+  return (kSmemLimit - 1024 /*alignment slack*/ - kBarrierBytes -
+          kEpiWarps * kEpiBufsPerWarp * kEpiBufBytes) /
+         stage_bytes(cta_group, bn);
+}
+
+// How one operand is staged.  K-major: one TMA box {64 k, rows}.  MN-major: rows/64
+// boxes {64 mn, 64 k}, 8 KB apart.
+struct OperandStaging {
+  uint32_t mn_major;   // 0: K contiguous in memory, 1: M/N contiguous
+  uint32_t desc_hi;    // upper half of the UMMA shared-memory descriptor
+  uint32_t lbo_enc;    // leading byte offset >> 4
+  uint32_t k_step_enc; // descriptor start-address increment per UMMA_K (bytes >> 4)
+};
+
+enum StatusCode : uint32_t {
+  kStatusOk = 0,
+  kStatusTimeout = 1,
+};
+
+enum WaitRole : uint32_t {
+  kRoleProducer = 1,
+  kRoleMma = 2,
+  kRoleEpilogue = 3,
+  kRoleProducerTail = 4,
+  kRoleEpilogueCin = 5,
+};
+
+struct GemmParams {
+  int32_t M, N, K;          // canonical problem (C row-major; operands possibly swapped)
+  int32_t num_k_blocks;     // ceil(K / 64), or 0 when alpha == 0 / K == 0
+  Raster raster;
+  float alpha, beta;
+  uint32_t idesc;           // tcgen05 instruction descriptor
+  OperandStaging a, b;
+  uint32_t* status;         // device: 8 words {code, role, barrier, tile, k_block, cta, -, -}
+  uint64_t timeout_ns;      // bound of every device-side wait
+  int64_t debug_skip_k_block;  // -1, or the producer k-block of CTA 0 whose loads are skipped
+};
+
+}  // namespace exo

@@ -1,0 +1,202 @@
+// Host-side planning: argument validation, canonical form, tile-shape choice.
+// Pure functions (no CUDA calls), so they can be exercised without a GPU.
+#pragma once
+#include <math.h>
+#include <stdint.h>
+
+#include "../../include/exo_gemm.h"
+#include "gemm_params.h"
+
+namespace exo {
+
+inline int elem_bytes(int dtype) { return dtype == EXO_GEMM_FP32 ? 4 : 2; }
+
+struct FlagOverrides {
+  int cta_group;   // 0 = auto
+  int tile_n;      // 0 = auto
+  int band;        // 0 = auto
+  int along_m;     // 0 = auto/default, 1 = forced
+  int grid_limit;  // 0 = none
+};
+
+inline FlagOverrides decode_flags(uint32_t f) {
+  FlagOverrides o;
+  o.cta_group = (int)(f & 3u);
+  o.tile_n = (int)((f >> 2) & 15u) * 64;
+  o.band = (int)((f >> 6) & 15u);
+  o.along_m = (int)((f >> 10) & 1u);
+  o.grid_limit = (int)((f >> 12) & 255u);
+  return o;
+}
+
+inline exo_gemm_status_t validate_desc(const exo_gemm_desc_t* d) {
+  if (!d) return EXO_GEMM_ERR_NULL;
+  if (d->reserved != 0) return EXO_GEMM_ERR_INVALID_ARG;
+  const int64_t kMaxDim = 2147483647LL;
+  if (d->M < 0 || d->N < 0 || d->K < 0 || d->M > kMaxDim || d->N > kMaxDim || d->K > kMaxDim)
+    return EXO_GEMM_ERR_INVALID_ARG;
+  auto bad_dtype = [](int32_t t) { return t < EXO_GEMM_BF16 || t > EXO_GEMM_FP32; };
+  auto bad_layout = [](int32_t l) { return l != EXO_GEMM_ROW_MAJOR && l != EXO_GEMM_COL_MAJOR; };
+  if (bad_dtype(d->ab_dtype) || bad_dtype(d->c_dtype)) return EXO_GEMM_ERR_INVALID_ARG;
+  if (bad_layout(d->a_layout) || bad_layout(d->b_layout) || bad_layout(d->c_layout))
+    return EXO_GEMM_ERR_INVALID_ARG;
+  if (d->device < -1) return EXO_GEMM_ERR_INVALID_ARG;
+  auto extent = [](int32_t layout, int64_t rows, int64_t cols) {
+    const int64_t e = layout == EXO_GEMM_ROW_MAJOR ? cols : rows;
+    return e < 1 ? 1 : e;
+  };
+  const int64_t kMaxLd = (1LL << 36);
+  if (d->lda < extent(d->a_layout, d->M, d->K) || d->ldb < extent(d->b_layout, d->K, d->N) ||
+      d->ldc < extent(d->c_layout, d->M, d->N) || d->lda > kMaxLd || d->ldb > kMaxLd || d->ldc > kMaxLd)
+    return EXO_GEMM_ERR_INVALID_ARG;
+  if (d->flags >> 20) return EXO_GEMM_ERR_INVALID_ARG;
+  if (d->flags & (1u << 11)) return EXO_GEMM_ERR_INVALID_ARG;
+  const FlagOverrides o = decode_flags(d->flags);
+  if (o.cta_group == 3) return EXO_GEMM_ERR_INVALID_ARG;
+  if (o.tile_n != 0 && o.tile_n != 64 && o.tile_n != 128 && o.tile_n != 256) return EXO_GEMM_ERR_INVALID_ARG;
+  if (o.cta_group == 2 && o.tile_n == 64) return EXO_GEMM_ERR_INVALID_ARG;
+  if (o.grid_limit != 0 && o.cta_group == 2 && (o.grid_limit & 1)) return EXO_GEMM_ERR_INVALID_ARG;
+  // beyond here the call is a legal BLAS call; what follows is this library's supported set
+  if (d->ab_dtype == EXO_GEMM_FP32) return EXO_GEMM_ERR_UNSUPPORTED;
+  if (d->c_dtype != EXO_GEMM_FP32 && d->c_dtype != d->ab_dtype) return EXO_GEMM_ERR_UNSUPPORTED;
+  if ((d->lda * 2) % 16 || (d->ldb * 2) % 16 || (d->ldc * elem_bytes(d->c_dtype)) % 16)
+    return EXO_GEMM_ERR_UNSUPPORTED;
+  return EXO_GEMM_OK;
+}
+
+// The problem after canonicalisation: C is always written row-major.  A
+// column-major C is computed as C^T = B^T A^T, which only swaps the operands and
+// M with N; an operand's "major-ness" (is K or M/N contiguous) carries over.
+struct Canonical {
+  int64_t M, N, K;
+  int a_mn_major, b_mn_major;  // of the canonical operands
+  int64_t lda, ldb, ldc;
+  int swapped;
+};
+
+inline Canonical canonicalize(const exo_gemm_desc_t& d) {
+  Canonical c;
+  const int a_mn = d.a_layout == EXO_GEMM_COL_MAJOR;  // A (M x K) col-major: M contiguous
+  const int b_mn = d.b_layout == EXO_GEMM_ROW_MAJOR;  // B (K x N) row-major: N contiguous
+  c.swapped = d.c_layout == EXO_GEMM_COL_MAJOR;
+  c.K = d.K;
+  c.ldc = d.ldc;
+  if (!c.swapped) {
+    c.M = d.M; c.N = d.N;
+    c.a_mn_major = a_mn; c.b_mn_major = b_mn;
+    c.lda = d.lda; c.ldb = d.ldb;
+  } else {
+    c.M = d.N; c.N = d.M;
+    c.a_mn_major = b_mn; c.b_mn_major = a_mn;
+    c.lda = d.ldb; c.ldb = d.lda;
+  }
+  return c;
+}
+
+struct TileConfig {
+  int cta_group, tile_n, stages;
+  int tiles_m, tiles_n;
+  int band, along_m;
+  int workers;  // CTA groups launched
+};
+
+// Relative tensor-pipe efficiency of a tile shape in the main loop (1 = the MMA
+// rate): smaller N per CTA re-reads A from shared memory more often per flop.
+inline double shape_efficiency(int cta_group, int bn) {
+  if (cta_group == 2) return bn == 256 ? 1.0 : 0.9;
+  return bn == 256 ? 0.93 : (bn == 128 ? 0.8 : 0.55);
+}
+
+// Estimated time of the whole problem in SM clocks for one candidate shape.
+inline double estimate_clocks(int64_t M, int64_t N, int64_t K, int cta_group, int bn, int max_workers) {
+  const int64_t tm = (M + 128 * cta_group - 1) / (128 * cta_group);
+  const int64_t tn = (N + bn - 1) / bn;
+  const int64_t tiles = tm * tn;
+  const int64_t workers = tiles < max_workers ? tiles : max_workers;
+  const int64_t waves = (tiles + workers - 1) / workers;
+  const int64_t nkb = (K + kBlockK - 1) / kBlockK;
+  const double mainloop = (double)nkb * 2.0 * bn / shape_efficiency(cta_group, bn);  // clocks per tile
+  const double epilogue = 6.0 * bn + 1500.0;  // drain of one accumulator: exposed once, plus fill latency
+  const double per_tile = mainloop > 4.0 * bn ? mainloop : 4.0 * bn;  // epilogue-bound tiles
+  return (double)waves * per_tile + epilogue;
+}
+
+inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int sm_count,
+                                int max_pairs /* co-resident 2-CTA clusters */) {
+  static const int cand[5][2] = {{2, 256}, {2, 128}, {1, 256}, {1, 128}, {1, 64}};
+  int best_g = 0, best_n = 0;
+  double best = 0;
+  for (int i = 0; i < 5; ++i) {
+    const int g = cand[i][0], n = cand[i][1];
+    if (o.cta_group && o.cta_group != g) continue;
+    if (o.tile_n && o.tile_n != n) continue;
+    if (g == 2 && max_pairs < 1) continue;
+    const int workers = g == 2 ? max_pairs : sm_count;
+    const double t = estimate_clocks(c.M, c.N, c.K, g, n, workers);
+    if (best_g == 0 || t < best * 0.999) { best = t; best_g = g; best_n = n; }
+  }
+  if (best_g == 0) { best_g = o.cta_group ? o.cta_group : 1; best_n = o.tile_n ? o.tile_n : 128; }
+  TileConfig cfg;
+  cfg.cta_group = best_g;
+  cfg.tile_n = best_n;
+  cfg.stages = max_stages(best_g, best_n);
+  cfg.tiles_m = (int)((c.M + 128 * best_g - 1) / (128 * best_g));
+  cfg.tiles_n = (int)((c.N + best_n - 1) / best_n);
+  int64_t workers = best_g == 2 ? max_pairs : sm_count;
+  if (o.grid_limit && o.grid_limit / best_g < workers) workers = o.grid_limit / best_g;
+  if (workers < 1) workers = 1;
+  const int64_t tiles = (int64_t)cfg.tiles_m * cfg.tiles_n;
+  if (tiles < workers) workers = tiles < 1 ? 1 : tiles;
+  cfg.workers = (int)workers;
+  cfg.along_m = o.along_m;
+  // Tiles that run together should cover a square patch of C: band width G along
+  // the banded dimension minimises (W/G)*extent_other + G*extent_banded.
+  const double tile_m = 128.0 * best_g, tile_n = best_n;
+  const double ratio = cfg.along_m ? tile_n / tile_m : tile_m / tile_n;
+  int band = o.band ? o.band : (int)floor(sqrt((double)workers * ratio) + 0.5);
+  const int major = cfg.along_m ? cfg.tiles_m : cfg.tiles_n;
+  if (band > major) band = major;
+  if (band > 15) band = 15;
+  if (band < 1) band = 1;
+  cfg.band = band;
+  return cfg;
+}
+
+inline int smem_bytes_for(int cta_group, int bn) {
+  return 1024 + max_stages(cta_group, bn) * stage_bytes(cta_group, bn) +
+         kEpiWarps * kEpiBufsPerWarp * kEpiBufBytes + kBarrierBytes;
+}
+
+// tcgen05 instruction descriptor for kind::f16 with fp32 accumulation.
+inline uint32_t make_idesc(int ab_dtype, int a_mn_major, int b_mn_major, int umma_m, int umma_n) {
+  const uint32_t fmt = ab_dtype == EXO_GEMM_BF16 ? 1u : 0u;  // 0 = fp16, 1 = bf16
+  uint32_t d = 0;
+  d |= 1u << 4;                        // D format: fp32
+  d |= fmt << 7;                       // A format
+  d |= fmt << 10;                      // B format
+  d |= (uint32_t)(a_mn_major & 1) << 15;
+  d |= (uint32_t)(b_mn_major & 1) << 16;
+  d |= (uint32_t)(umma_n >> 3) << 17;
+  d |= (uint32_t)(umma_m >> 4) << 24;
+  return d;
+}
+
+// How an operand tile sits in shared memory (128-byte swizzle, 8-row atoms of 1 KB).
+inline OperandStaging make_staging(int mn_major) {
+  OperandStaging s;
+  s.mn_major = (uint32_t)mn_major;
+  const uint32_t sbo = 1024u >> 4;       // between 8-row groups of a swizzle atom column
+  const uint32_t version = 1u << 14;     // descriptor bits 46..47 = 1 on sm_100
+  const uint32_t swizzle128 = 2u << 29;  // descriptor bits 61..63
+  s.desc_hi = sbo | version | swizzle128;
+  if (!mn_major) {
+    s.lbo_enc = 1;                                   // unused for swizzled K-major tiles
+    s.k_step_enc = (kUmmaK * 2) >> 4;                // 32 bytes along the 128-byte row
+  } else {
+    s.lbo_enc = (kBlockK * 128u) >> 4;               // next 64 M/N elements: next 8 KB box
+    s.k_step_enc = (kUmmaK * 128u) >> 4;             // 16 k-rows of 128 bytes
+  }
+  return s;
+}
+
+}  // namespace exo
