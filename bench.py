@@ -1,0 +1,414 @@
+#!/usr/bin/env python
+"""Benchmark of the GEMM hot path: one step = one C = alpha*A*B + beta*C through the C ABI.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+Prints one JSON line (rank 0).  ``value`` is whole-job TFLOP/s (2*M*N*K per GEMM)
+with the matrices already resident in HBM; ``e2e`` is the same metric through
+the same C-ABI call with host buffers (pinned), host<->device copies inside the
+timed region.  With N > 1 (torchrun, one rank per GPU) every rank runs its own
+independent GEMMs of the same shape (weak scaling, no collective on the data
+path); the time is the maximum over ranks.
+
+``--impl reference`` times the CPU oracle (oracle/) on the host cores, on
+bounded row bands of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+METRIC = "GEMM TFLOP/s on 1 B200 and % of dense bf16 tensor-core roofline"
+UNIT = "TFLOP/s"
+L2_BYTES = 126 * 1024 * 1024
+
+WORKLOADS = {
+    # name: (config index, variant)
+    "cfg1_256": (0, None), "cfg2_4096": (1, None), "cfg3_8192": (2, None),
+    "cfg4a_skinny": (3, "a"), "cfg4b_skinny": (3, "b"),
+}
+DEFAULT_WORKLOAD = "cfg2_4096"   # the configuration the metric is quoted on; fits one GPU
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-cublas", action="store_true")
+    ap.add_argument("--flags", type=int, default=0, help="EXO_GEMM_FLAG_* overrides (experiments)")
+    return ap.parse_args()
+
+
+def make_problem(name: str, rank: int = 0):
+    from paper_2609_16389_b200 import synth
+    if name.startswith("sweep_"):
+        M, N, K = (int(x) for x in name[len("sweep_"):].split("x"))
+        p = synth.sweep_problem(M, N, K)
+    else:
+        idx, variant = WORKLOADS[name]
+        p = synth.config(idx, variant)
+    p.seed += 7919 * rank      # independent problems per rank
+    return p.generate()
+
+
+def peaks():
+    """Measured roofline denominators (generated file), else the stated fallback."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": d["hbm_gbs"], "tflops_burst": d["bf16_tflops"],
+                "tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "tflops_burst": 1590.0, "tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def profiled_traffic(workload: str):
+    """DRAM bytes per launch from the committed ncu summary for this workload, if any."""
+    path = os.path.join(ROOT, "profiles", f"exo_gemm_kernel_{workload}.md")
+    if not os.path.exists(path):
+        return None
+    for ln in open(path):
+        if ln.startswith("dram_bytes_per_launch:"):
+            try:
+                return float(ln.split(":", 1)[1].split()[0])
+            except ValueError:
+                return None
+    return None
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.samples = []
+        self._stop = threading.Event()
+        self._thr = None
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.QUERY}",
+                                      "--format=csv,noheader,nounits"], capture_output=True, text=True,
+                                     timeout=5).stdout.strip()
+                if out:
+                    self.samples.append([x.strip() for x in out.split(",")])
+            except Exception:
+                pass
+            self._stop.wait(0.05)
+
+    def start(self):
+        self._thr = threading.Thread(target=self._run, daemon=True)
+        self._thr.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thr:
+            self._thr.join(timeout=10)
+        sm = [float(s[0]) for s in self.samples if s and s[0].replace(".", "").isdigit()]
+        mx = [float(s[1]) for s in self.samples if len(s) > 1 and s[1].replace(".", "").isdigit()]
+        reasons = set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for s in self.samples:
+            for i, n in enumerate(names):
+                if len(s) > 3 + i and s[3 + i].lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def aggregate_over_ranks(local_ms: float, local_flop: float, world: int, device=None):
+    """Whole-job throughput: all ranks' work divided by the slowest rank's time.
+
+    Returns (tflops, max_ms).  Uses one all_reduce(MAX) and one all_reduce(SUM) on
+    the default process group when world > 1 (control path only, not data path).
+    """
+    if world <= 1:
+        return local_flop / (local_ms * 1e-3) / 1e12, local_ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([local_ms], dtype=torch.float64, device=device)
+    f = torch.tensor([local_flop], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(f, op=dist.ReduceOp.SUM)
+    return float(f.item()) / (float(t.item()) * 1e-3) / 1e12, float(t.item())
+
+
+# ---------------------------------------------------------------------------------------
+# reference arm: the CPU oracle, as it stands, on the host cores
+# ---------------------------------------------------------------------------------------
+def run_reference(args, rank, world):
+    if rank != 0:
+        return
+    import oracle
+    p = make_problem(args.workload)
+    cores = oracle.num_threads()
+    # calibrate on a thin band, then size the per-step band so the whole run stays bounded
+    cal_rows = min(p.M, 16)
+    t0 = time.perf_counter()
+    oracle.gemm_problem(p, rows=(0, cal_rows))
+    cal = time.perf_counter() - t0
+    budget_s = 90.0
+    per_row = max(cal / cal_rows, 1e-9)
+    rows = int(budget_s / ((args.steps + args.warmup) * per_row))
+    rows = max(1, min(p.M, rows))
+    for w in range(args.warmup):
+        r0 = (w * rows) % max(1, p.M - rows + 1)
+        oracle.gemm_problem(p, rows=(r0, r0 + rows))
+    t0 = time.perf_counter()
+    for s in range(args.steps):
+        r0 = ((s + args.warmup) * rows) % max(1, p.M - rows + 1)
+        oracle.gemm_problem(p, rows=(r0, r0 + rows))
+    dt = time.perf_counter() - t0
+    flop = 2.0 * rows * p.N * p.K * args.steps
+    tflops = flop / dt / 1e12
+    sample = f"each step = a band of {rows} rows of C ({rows}x{p.N}x{p.K}) of {args.workload}"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": tflops, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": args.workload, "M": p.M, "N": p.N, "K": p.K, "sample": sample},
+        "cpu_baseline": {"value": tflops, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": tflops, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------
+# our arm
+# ---------------------------------------------------------------------------------------
+def run_ours(args, rank, world, local_rank):
+    import torch
+    from paper_2609_16389_b200 import binding as B
+    from paper_2609_16389_b200 import harness, synth
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the GEMM path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    p = make_problem(args.workload, rank)
+    flop = p.flop
+    set_bytes = p.A.nbytes + p.B.nbytes + p.C.nbytes
+    n_sets = max(2, int(np.ceil(2.0 * L2_BYTES / set_bytes)))     # rotate through > 2x L2 of operands
+    n_sets = min(n_sets, 64)
+    sets = []
+    for _ in range(n_sets):
+        sets.append((harness._to_device(p.A, dev), harness._to_device(p.B, dev), harness._to_device(p.C, dev)))
+    plan = B.Plan(harness.desc_of(p, args.flags, local_rank))
+    info = plan.info()
+    stream = torch.cuda.current_stream(dev)
+
+    def step(i):
+        a, b, c = sets[i % n_sets]
+        plan.run(a.data_ptr(), b.data_ptr(), c.data_ptr(), p.alpha, p.beta, stream.cuda_stream)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    barrier()
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    # --- device-resident timing: K steps bracketed by events on the launching stream
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    barrier()
+    ev[0].record(stream)
+    for i in range(args.steps):
+        step(i)
+        ev[i + 1].record(stream)
+    barrier()
+    total_ms = ev[0].elapsed_time(ev[-1])
+    per_step = np.array([ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)])
+    plan.check()
+
+    # --- cuBLAS on the same box, same shapes (reference point only), interleaved order
+    cublas = None
+    if rank == 0 and not args.no_cublas:
+        cublas = time_cublas(p, dev, args.steps, n_sets)
+
+    # --- end to end: pinned host buffers, H2D + GEMM + D2H inside the timed region
+    e2e_steps = max(3, min(args.steps, 20))
+    hA = torch.from_numpy(p.A.view(np.uint8)).pin_memory()
+    hB = torch.from_numpy(p.B.view(np.uint8)).pin_memory()
+    hC = torch.from_numpy(p.C.view(np.uint8)).pin_memory()
+    hOut = torch.empty_like(hC).pin_memory()
+    dA, dB, dC = sets[0]
+    need_c_in = p.beta != 0.0
+    h2d = hA.numel() + hB.numel() + (hC.numel() if need_c_in else 0)
+    d2h = hOut.numel()
+
+    def e2e_step():
+        dA.copy_(hA, non_blocking=True)
+        dB.copy_(hB, non_blocking=True)
+        if need_c_in:
+            dC.copy_(hC, non_blocking=True)
+        plan.run(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), p.alpha, p.beta, stream.cuda_stream)
+        hOut.copy_(dC, non_blocking=True)
+
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    clocks = sampler.stop()
+    plan.check()
+
+    value, max_ms = aggregate_over_ranks(total_ms, flop * args.steps, world, dev)
+    e2e_value, _ = aggregate_over_ranks(e2e_ms, flop, world, dev)
+
+    if rank == 0:
+        pk = peaks()
+        ms_per_step = max_ms / args.steps
+        avg_kernel_ms = total_ms / args.steps          # one kernel per step, back to back
+        achieved = flop / (avg_kernel_ms * 1e-3) / 1e12
+        timed_region_s = total_ms * 1e-3
+        peak = pk["tflops_burst"] if timed_region_s < 1.0 else pk["tflops_sustained"]
+        ai = flop / p.algorithmic_bytes
+        hbm_bound_tflops = ai * pk["hbm_gbs"] / 1e3
+        tensor_bound = hbm_bound_tflops >= peak
+        q1, q3 = np.percentile(per_step, [25, 75])
+        iqr = per_step[(per_step >= q1) & (per_step <= q3)]
+        roofline = {
+            "bound": "tensor" if tensor_bound else "hbm",
+            "achieved": achieved if tensor_bound else p.algorithmic_bytes / (avg_kernel_ms * 1e-3) / 1e9,
+            "peak": peak if tensor_bound else pk["hbm_gbs"],
+            "unit": "TFLOP/s" if tensor_bound else "GB/s",
+            "traffic": profiled_traffic(args.workload),
+            "peak_source": f"{pk['source']} ({'burst' if timed_region_s < 1.0 else 'sustained'} cuBLAS bf16)"
+                           if tensor_bound else f"{pk['source']} (copy bandwidth)",
+            "kernel": f"exo_gemm_kernel<{info['cta_group']},{info['tile_n']}>",
+            "avg_kernel_ms": avg_kernel_ms,
+            "algorithmic_bytes": p.algorithmic_bytes, "flop": flop,
+            "frac_of_nominal_2250": achieved / 2250.0,
+        }
+        roofline["frac"] = roofline["achieved"] / roofline["peak"]
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None,
+            "dtype": ("bf16" if p.ab_dtype == synth.BF16 else "fp16") + " in, fp32 accumulate",
+            "data": "synthetic",
+            "config": {"workload": args.workload, "M": p.M, "N": p.N, "K": p.K,
+                       "ab_dtype": synth.dtype_name(p.ab_dtype), "c_dtype": synth.dtype_name(p.c_dtype),
+                       "layouts": "A%s B%s C%s" % tuple("rc"[x] for x in (p.a_layout, p.b_layout, p.c_layout)),
+                       "alpha": p.alpha, "beta": p.beta,
+                       "l2": f"rotating {n_sets} operand sets ({n_sets * set_bytes >> 20} MiB > 126 MiB L2)",
+                       "plan": info},
+            "iqr_mean_ms": float(iqr.mean()) if iqr.size else None, "min_ms": float(per_step.min()),
+            "roofline": roofline,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+                    "d2h_bytes_per_step": int(d2h), "ms_per_step": e2e_ms, "steps": e2e_steps},
+            "gpu_launches": args.steps,
+            "clocks": clocks,
+        }
+        if cublas is not None:
+            line["cublas"] = cublas
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(p, args.workload)
+        print(json.dumps(line), flush=True)
+
+    plan.close()
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def time_cublas(p, dev, steps, n_sets):
+    """torch.matmul / addmm (cuBLAS) on the same shapes: a same-box reference point."""
+    import torch
+    from paper_2609_16389_b200 import synth
+    try:
+        tdt = torch.bfloat16 if p.ab_dtype == synth.BF16 else torch.float16
+        sets = []
+        for _ in range(n_sets):
+            a = torch.randn(p.M, p.K, device=dev, dtype=torch.float32).to(tdt)
+            if p.a_layout == synth.COL_MAJOR:
+                a = a.t().contiguous().t()
+            if p.b_layout == synth.COL_MAJOR:      # K x N view of an N x K row-major buffer
+                b = torch.randn(p.N, p.K, device=dev, dtype=torch.float32).to(tdt).t()
+            else:
+                b = torch.randn(p.K, p.N, device=dev, dtype=torch.float32).to(tdt)
+            sets.append((a, b, torch.empty(p.M, p.N, device=dev, dtype=tdt)))
+        for i in range(3):
+            a, b, c = sets[i % n_sets]
+            torch.matmul(a, b, out=c)
+        torch.cuda.synchronize(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(steps):
+            a, b, c = sets[i % n_sets]
+            torch.matmul(a, b, out=c)
+        e1.record()
+        torch.cuda.synchronize(dev)
+        ms = e0.elapsed_time(e1) / steps
+        return {"tflops": p.flop / (ms * 1e-3) / 1e12, "ms_per_step": ms,
+                "note": "torch.matmul, 16-bit output, alpha=1 beta=0, same M,N,K and operand layouts"}
+    except Exception as e:  # a reference point only; never fails the bench
+        return {"error": repr(e)}
+
+
+def cpu_baseline(p, workload):
+    import oracle
+    cores = oracle.num_threads()
+    cal_rows = min(p.M, 16)
+    t0 = time.perf_counter()
+    oracle.gemm_problem(p, rows=(0, cal_rows))
+    cal = time.perf_counter() - t0
+    target_wall = 20.0 / max(cores, 1)       # about 20 s of CPU work in total
+    rows = int(max(1, min(p.M, target_wall / max(cal / cal_rows, 1e-9))))
+    t0 = time.perf_counter()
+    oracle.gemm_problem(p, rows=(0, rows))
+    dt = time.perf_counter() - t0
+    return {"value": 2.0 * rows * p.N * p.K / dt / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"rows 0..{rows} of C ({rows}x{p.N}x{p.K}) of {workload}, {dt:.1f} s wall"}
+
+
+def main():
+    args = parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.workload not in WORKLOADS and not args.workload.startswith("sweep_"):
+        raise SystemExit(f"unknown workload {args.workload}")
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+    run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

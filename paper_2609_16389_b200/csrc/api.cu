@@ -295,7 +295,8 @@ exo_gemm_status_t exo_gemm_run(exo_gemm_handle_t plan, const void* A, const void
   prm.b = make_staging(cn.b_mn_major);
   prm.status = plan->d_status;
   const int32_t dbg_ms = plan->dbg_timeout_ms.exchange(0);
-  prm.timeout_ns = dbg_ms > 0 ? (uint64_t)dbg_ms * 1000000ull : 4000000000ull;
+  // SM clocks, converted at 2 GHz (an upper bound of the SM clock, so the real limit is not shorter)
+  prm.timeout_cycles = (uint64_t)(dbg_ms > 0 ? dbg_ms : 4000) * 2000000ull;
   prm.debug_skip_k_block = plan->dbg_skip_k_block.exchange(-1);
 
   CUtensorMap tm_a, tm_b, tm_c;

@@ -46,14 +46,14 @@ struct WaitSite {
 
 template <bool CLUSTER>
 __device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, const GemmParams& p, WaitSite site) {
-  const uint64_t t0 = ptx::globaltimer_ns();
+  const long long t0 = clock64();
   uint32_t n = 0;
   for (;;) {
     const bool done = CLUSTER ? ptx::mbar_try_wait_cluster(bar, parity) : ptx::mbar_try_wait(bar, parity);
     if (done) return true;
-    if ((++n & 15u) == 0u) {
+    if ((++n & 63u) == 0u) {
       if (*(volatile uint32_t*)p.status != kStatusOk) return false;  // another role gave up
-      if (ptx::globaltimer_ns() - t0 > p.timeout_ns) {
+      if ((uint64_t)(clock64() - t0) > p.timeout_cycles) {
         if (atomicCAS(p.status, (uint32_t)kStatusOk, (uint32_t)kStatusTimeout) == kStatusOk) {
           p.status[1] = site.role;
           p.status[2] = site.barrier;
@@ -72,8 +72,11 @@ __device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, const Gemm
 template <bool CLUSTER>
 __device__ __forceinline__ bool wait_barrier(uint32_t bar, uint32_t parity, const GemmParams& p,
                                              WaitSite site) {
-  const bool done = CLUSTER ? ptx::mbar_try_wait_cluster(bar, parity) : ptx::mbar_try_wait(bar, parity);
-  if (done) return true;
+#pragma unroll 1
+  for (int i = 0; i < 8; ++i) {
+    const bool done = CLUSTER ? ptx::mbar_try_wait_cluster(bar, parity) : ptx::mbar_try_wait(bar, parity);
+    if (done) return true;
+  }
   return wait_slow<CLUSTER>(bar, parity, p, site);
 }
 

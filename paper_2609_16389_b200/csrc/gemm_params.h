@@ -62,7 +62,7 @@ struct GemmParams {
   uint32_t idesc;           // tcgen05 instruction descriptor
   OperandStaging a, b;
   uint32_t* status;         // device: 8 words {code, role, barrier, tile, k_block, cta, -, -}
-  uint64_t timeout_ns;      // bound of every device-side wait
+  uint64_t timeout_cycles;  // bound of every device-side wait, in SM clocks
   int64_t debug_skip_k_block;  // -1, or the producer k-block of CTA 0 whose loads are skipped
 };
 

@@ -59,8 +59,11 @@ inline exo_gemm_status_t validate_desc(const exo_gemm_desc_t* d) {
   // beyond here the call is a legal BLAS call; what follows is this library's supported set
   if (d->ab_dtype == EXO_GEMM_FP32) return EXO_GEMM_ERR_UNSUPPORTED;
   if (d->c_dtype != EXO_GEMM_FP32 && d->c_dtype != d->ab_dtype) return EXO_GEMM_ERR_UNSUPPORTED;
-  if ((d->lda * 2) % 16 || (d->ldb * 2) % 16 || (d->ldc * elem_bytes(d->c_dtype)) % 16)
-    return EXO_GEMM_ERR_UNSUPPORTED;
+  // a matrix that is never touched (empty problem, K == 0) has no stride rule
+  const bool c_used = d->M > 0 && d->N > 0;
+  const bool ab_used = c_used && d->K > 0;
+  if (ab_used && ((d->lda * 2) % 16 || (d->ldb * 2) % 16)) return EXO_GEMM_ERR_UNSUPPORTED;
+  if (c_used && (d->ldc * elem_bytes(d->c_dtype)) % 16) return EXO_GEMM_ERR_UNSUPPORTED;
   return EXO_GEMM_OK;
 }
 
@@ -112,6 +115,7 @@ inline double estimate_clocks(int64_t M, int64_t N, int64_t K, int cta_group, in
   const int64_t tm = (M + 128 * cta_group - 1) / (128 * cta_group);
   const int64_t tn = (N + bn - 1) / bn;
   const int64_t tiles = tm * tn;
+  if (tiles == 0) return 0.0;
   const int64_t workers = tiles < max_workers ? tiles : max_workers;
   const int64_t waves = (tiles + workers - 1) / workers;
   const int64_t nkb = (K + kBlockK - 1) / kBlockK;

@@ -1,0 +1,174 @@
+"""Host-side tests of the C-ABI library that need no GPU: the library loads and
+exports what the header declares, argument validation, plan preview, and the
+persistent tile schedule."""
+import os
+import re
+
+import pytest
+
+from paper_2609_16389_b200 import binding as B
+from paper_2609_16389_b200 import synth
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "exo_gemm.h")
+
+
+def _declared_functions():
+    text = open(HEADER).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(exo_gemm_[a-z_]+)\s*\(", text)))
+
+
+def test_library_loads_and_exports_every_declared_symbol():
+    lib = B.lib()
+    declared = _declared_functions()
+    assert "exo_gemm_create" in declared and "exo_gemm_run" in declared and "exo_gemm_destroy" in declared
+    for name in declared:
+        assert hasattr(lib, name), f"{name} declared in exo_gemm.h but not exported"
+    assert set(declared) == set(B.EXPORTED_SYMBOLS)
+
+
+def test_status_strings():
+    for code in range(8):
+        assert B.exo_gemm_status_string(code)
+    assert B.exo_gemm_status_string(B.OK) == "ok"
+    assert "unknown" in B.exo_gemm_status_string(99)
+
+
+def good(**kw):
+    d = dict(M=256, N=192, K=128, ab_dtype=B.BF16, c_dtype=B.FP32, a_layout=0, b_layout=1, c_layout=0)
+    d.update(kw)
+    return B.make_desc(**d)
+
+
+def test_validate_accepts_the_supported_set():
+    assert B.exo_gemm_validate(good()) == B.OK
+    for ab in (B.BF16, B.FP16):
+        for cd in (B.FP32, ab):
+            for la in (0, 1):
+                for lb in (0, 1):
+                    for lc in (0, 1):
+                        assert B.exo_gemm_validate(good(ab_dtype=ab, c_dtype=cd, a_layout=la, b_layout=lb,
+                                                        c_layout=lc)) == B.OK
+    assert B.exo_gemm_validate(good(M=0)) == B.OK
+    assert B.exo_gemm_validate(good(K=0)) == B.OK
+    assert B.exo_gemm_validate(good(M=1000, N=1000, K=1000)) == B.OK
+    assert B.exo_gemm_validate(good(lda=136, ldb=160, ldc=200)) == B.OK
+
+
+def test_validate_rejects_bad_arguments():
+    assert B.lib().exo_gemm_validate(None) == B.ERR_NULL
+    assert B.exo_gemm_validate(good(M=-1)) == B.ERR_INVALID_ARG
+    assert B.exo_gemm_validate(good(N=2 ** 31)) == B.ERR_INVALID_ARG
+    assert B.exo_gemm_validate(good(ab_dtype=7)) == B.ERR_INVALID_ARG
+    assert B.exo_gemm_validate(good(c_layout=2)) == B.ERR_INVALID_ARG
+    assert B.exo_gemm_validate(good(lda=64)) == B.ERR_INVALID_ARG          # row-major A needs lda >= K
+    assert B.exo_gemm_validate(good(ldb=120)) == B.ERR_INVALID_ARG         # col-major B needs ldb >= K
+    assert B.exo_gemm_validate(good(ldc=100)) == B.ERR_INVALID_ARG
+    assert B.exo_gemm_validate(good(device=-2)) == B.ERR_INVALID_ARG
+    d = good()
+    d.reserved = 1
+    assert B.exo_gemm_validate(d) == B.ERR_INVALID_ARG
+    assert B.exo_gemm_validate(good(flags=3)) == B.ERR_INVALID_ARG                       # cta_group 3
+    assert B.exo_gemm_validate(good(flags=B.flag_tile_n(192))) == B.ERR_INVALID_ARG
+    assert B.exo_gemm_validate(good(flags=B.flag_cta_group(2) | B.flag_tile_n(64))) == B.ERR_INVALID_ARG
+    assert B.exo_gemm_validate(good(flags=1 << 25)) == B.ERR_INVALID_ARG
+
+
+def test_validate_unsupported_but_legal_blas_calls():
+    assert B.exo_gemm_validate(good(ab_dtype=B.FP32)) == B.ERR_UNSUPPORTED
+    assert B.exo_gemm_validate(good(ab_dtype=B.BF16, c_dtype=B.FP16)) == B.ERR_UNSUPPORTED
+    assert B.exo_gemm_validate(good(K=100)) == B.ERR_UNSUPPORTED            # lda = 100: 200 bytes, not 16 | it
+    assert B.exo_gemm_validate(good(K=100, lda=104, ldb=104)) == B.OK
+    assert B.exo_gemm_validate(good(N=190)) == B.ERR_UNSUPPORTED            # fp32 C, ldc = 190
+    assert B.exo_gemm_validate(good(N=190, ldc=192)) == B.OK
+
+
+def test_benchmark_configs_are_in_the_supported_set():
+    for idx, var in ((0, None), (1, None), (2, None), (3, "a"), (3, "b")):
+        p = synth.config(idx, var)
+        d = B.make_desc(p.M, p.N, p.K, p.ab_dtype, p.c_dtype, p.a_layout, p.b_layout, p.c_layout,
+                        p.lda, p.ldb, p.ldc)
+        assert B.exo_gemm_validate(d) == B.OK
+    for M in synth.SWEEP_DIMS:
+        for N in synth.SWEEP_DIMS:
+            for K in synth.SWEEP_DIMS:
+                p = synth.sweep_problem(M, N, K)
+                d = B.make_desc(p.M, p.N, p.K, p.ab_dtype, p.c_dtype, p.a_layout, p.b_layout, p.c_layout)
+                assert B.exo_gemm_validate(d) == B.OK, (M, N, K)
+
+
+def test_plan_preview_geometry_and_overrides():
+    st, info = B.exo_gemm_plan_preview(good(M=4096, N=4096, K=4096, c_dtype=B.BF16), 148)
+    assert st == B.OK
+    i = info.as_dict()
+    assert i["tile_m"] == 128 * i["cta_group"] and i["tile_k"] == 64
+    assert i["tiles_m"] * i["tile_m"] >= 4096 and i["tiles_n"] * i["tile_n"] >= 4096
+    assert i["grid"] <= 148 and i["grid"] % i["cta_group"] == 0
+    assert i["smem_bytes"] <= 232448 and i["tmem_columns"] == 2 * i["tile_n"] <= 512
+    assert i["kernel_launches_per_run"] == 1 and i["swapped"] == 0
+    for g, bn in ((1, 64), (1, 128), (1, 256), (2, 128), (2, 256)):
+        st, info = B.exo_gemm_plan_preview(good(M=1000, N=520, K=264,
+                                                flags=B.flag_cta_group(g) | B.flag_tile_n(bn)), 148)
+        i = info.as_dict()
+        assert (i["cta_group"], i["tile_n"]) == (g, bn)
+        assert i["tiles_m"] == -(-1000 // (128 * g)) and i["tiles_n"] == -(-520 // bn)
+        assert i["grid"] == min(148 // g, i["tiles_m"] * i["tiles_n"]) * g
+        assert i["stages"] * (16384 + bn // g * 128) + 32768 + 1536 <= 232448
+    # column-major C is computed as the transposed product
+    st, info = B.exo_gemm_plan_preview(good(M=512, N=2048, K=64, c_layout=1, ldc=512), 148)
+    i = info.as_dict()
+    assert i["swapped"] == 1 and i["tiles_m"] * i["tile_m"] >= 2048 and i["tiles_n"] * i["tile_n"] >= 512
+    # grid limit and band override
+    st, info = B.exo_gemm_plan_preview(good(M=4096, N=4096, K=512, flags=B.flag_grid_limit(8) | B.flag_band(3)
+                                            | B.flag_cta_group(2) | B.flag_tile_n(256)), 148)
+    assert info.grid == 8 and info.raster_band == 3
+    st, info = B.exo_gemm_plan_preview(good(M=0), 148)
+    assert st == B.OK and info.kernel_launches_per_run == 0
+    assert B.exo_gemm_plan_preview(good(), 0)[0] == B.ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("tiles_m,tiles_n", [(1, 1), (4, 4), (16, 16), (3, 5), (4, 64), (64, 4), (48, 47), (7, 1)])
+@pytest.mark.parametrize("band", [1, 2, 3, 8, 15])
+@pytest.mark.parametrize("along_m", [0, 1])
+def test_schedule_visits_every_tile_exactly_once(tiles_m, tiles_n, band, along_m):
+    for workers in (1, 2, 7, 74, 148):
+        seen = {}
+        longest, shortest = 0, 10 ** 9
+        for w in range(workers):
+            seq = B.exo_gemm_schedule_enumerate(tiles_m, tiles_n, band, along_m, workers, w)
+            longest, shortest = max(longest, len(seq)), min(shortest, len(seq))
+            for t in seq:
+                assert 0 <= t[0] < tiles_m and 0 <= t[1] < tiles_n
+                assert t not in seen, f"tile {t} visited twice"
+                seen[t] = w
+        assert len(seen) == tiles_m * tiles_n
+        assert longest - shortest <= 1                     # round-robin: balanced to within one tile
+
+
+def test_schedule_order_is_band_swizzled():
+    # 3 x 5 tiles, bands of 2 tile columns: walk a band's columns first, then the next tile row
+    seq = B.exo_gemm_schedule_enumerate(3, 5, 2, 0, 1, 0)
+    assert seq[:6] == [(0, 0), (0, 1), (1, 0), (1, 1), (2, 0), (2, 1)]
+    assert seq[6:12] == [(0, 2), (0, 3), (1, 2), (1, 3), (2, 2), (2, 3)]
+    assert seq[12:] == [(0, 4), (1, 4), (2, 4)]                       # narrower last band
+    seq = B.exo_gemm_schedule_enumerate(3, 5, 2, 1, 1, 0)              # transposed raster
+    assert seq[:4] == [(0, 0), (1, 0), (0, 1), (1, 1)]
+    assert seq[-5:] == [(2, 0), (2, 1), (2, 2), (2, 3), (2, 4)]
+    # a wave of consecutive indices covers a compact patch: 8 workers on 16x16 tiles, band 4
+    first_wave = [B.exo_gemm_schedule_enumerate(16, 16, 4, 0, 8, w)[0] for w in range(8)]
+    assert {t[0] for t in first_wave} == {0, 1} and {t[1] for t in first_wave} == {0, 1, 2, 3}
+    with pytest.raises(ValueError):
+        B.exo_gemm_schedule_enumerate(3, 5, 0, 0, 1, 0)
+
+
+def test_create_fails_cleanly_without_a_gpu():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a GPU is present")
+    st, h = B.exo_gemm_create(good())
+    assert st in (B.ERR_CUDA, B.ERR_ARCH) and h is None      # no CPU fallback: an error, not a result
+    with pytest.raises(B.ExoGemmError):
+        B.Plan(good())
+    assert B.exo_gemm_destroy(None) == B.OK
+    assert B.exo_gemm_run(None, 0, 0, 0, 1.0, 0.0, 0) == B.ERR_NULL

@@ -1,0 +1,258 @@
+"""Parity tests proper: the CUDA path, called through the C ABI, against the CPU oracle
+on the same seeded inputs.  Tolerance (written here, from the benchmark spec):
+
+    max_ij |C - Cref| / (sum_k |a_ik b_kj| + |beta c_ij|) <= 1e-3
+
+For 16-bit outputs at small K the rounding of the result into bf16/fp16 is itself
+larger than 1e-3 of the denominator on some entries, so those cases use the
+widened gate |dC| <= 1e-3 * Den + u_out * |Cref| (u_out = 2^-8 bf16, 2^-11 fp16);
+the benchmark configurations use the literal formula.
+"""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2609_16389_b200 import binding as B
+from paper_2609_16389_b200 import harness, synth
+from paper_2609_16389_b200.synth import BF16, FP16, FP32, ROW_MAJOR, COL_MAJOR
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-3
+
+
+def run_gpu(p, flags=0):
+    cbuf, info = harness.gemm_host(p, flags)
+    return cbuf, oracle.logical_view(cbuf, p.M, p.N, p.c_layout, p.ldc, p.c_dtype), info
+
+
+def check_full(p, flags=0, literal=None):
+    cbuf, got, info = run_gpu(p, flags)
+    cref, den = oracle.gemm_problem(p)
+    if literal is None:
+        literal = p.c_dtype == FP32
+    if literal:
+        err = oracle.max_error(got, cref, den)
+        assert err <= TOL, (p.name, err, info)
+    else:
+        gate = TOL * den + oracle.output_rounding_slack(cref, p.c_dtype)
+        bad = np.abs(got - cref) > gate
+        assert not bad.any(), (p.name, int(bad.sum()), np.argwhere(bad)[:5], info)
+    return cbuf, got, cref, den, info
+
+
+def flags_for(g, bn, grid=0):
+    return B.flag_cta_group(g) | B.flag_tile_n(bn) | (B.flag_grid_limit(grid) if grid else 0)
+
+
+TILE_SHAPES = [(1, 64), (1, 128), (1, 256), (2, 128), (2, 256)]
+
+
+# ------------------------------------------------------------------ closed forms on the GPU
+@pytest.mark.parametrize("g,bn", TILE_SHAPES)
+def test_identity_selector_reproduces_a_exactly(g, bn):
+    M, N, K = 256, 256, 192
+    p = synth.Problem("ident", M, N, K, BF16, FP32, 0, 1, 0, 1.0, 0.0, seed=1).generate()
+    b = np.zeros((K, N), np.float32)
+    b[np.arange(K), np.arange(K)] = 1.0
+    p.B = synth.store(synth.round_to_storage(b, BF16), p.b_layout, p.ldb)
+    _, got, _ = run_gpu(p, flags_for(g, bn))
+    a = oracle.logical_view(p.A, M, K, 0, p.lda, BF16)
+    assert np.array_equal(got[:, :K], a) and np.all(got[:, K:] == 0.0)
+
+
+@pytest.mark.parametrize("K", [16, 64, 1000, 4096])
+def test_all_ones_gives_exactly_k(K):
+    M, N = 200, 136
+    p = synth.Problem("ones", M, N, K, FP16, FP32, 0, 0, 0, 0.5, 1.0, seed=1).generate()
+    one16 = np.uint16(0x3C00)
+    p.A[:] = one16
+    p.B[:] = one16
+    p.C[:] = 1.0
+    _, got, _ = run_gpu(p)
+    assert np.all(got == K / 2 + 1)
+
+
+# ------------------------------------------------------------------ small shapes, all options
+EDGE_MN = [(1, 8), (127, 129), (128, 128), (129, 72), (255, 257), (257, 40), (384, 520)]
+
+
+@pytest.mark.parametrize("M,N", EDGE_MN)
+@pytest.mark.parametrize("K", [8, 72, 1000])
+@pytest.mark.parametrize("g,bn", TILE_SHAPES)
+def test_tile_boundaries(M, N, K, g, bn):
+    ldc = -(-N // 4) * 4
+    p = synth.Problem("edge", M, N, K, BF16, FP32, 0, 1, 0, 1.0, 0.0, seed=M * 131 + N * 7 + K,
+                      ldc=ldc).generate()
+    check_full(p, flags_for(g, bn))
+
+
+@pytest.mark.parametrize("la", [0, 1])
+@pytest.mark.parametrize("lb", [0, 1])
+@pytest.mark.parametrize("lc", [0, 1])
+@pytest.mark.parametrize("ab,cd", [(BF16, FP32), (FP16, FP32), (BF16, BF16), (FP16, FP16)])
+@pytest.mark.parametrize("g,bn", [(1, 128), (2, 256)])
+def test_layouts_dtypes_alpha_beta(la, lb, lc, ab, cd, g, bn):
+    M, N, K = 264, 328, 200
+    p = synth.Problem("lay", M, N, K, ab, cd, la, lb, lc, -1.5, 0.75, seed=la + 2 * lb + 4 * lc + 8 * ab,
+                      dist="normal" if ab == FP16 else "uniform")
+    p.generate()
+    check_full(p, flags_for(g, bn))
+
+
+@pytest.mark.parametrize("g,bn", TILE_SHAPES)
+def test_padding_is_untouched_and_nan_c_does_not_leak(g, bn):
+    M, N, K = 300, 200, 136
+    p = synth.Problem("pad", M, N, K, BF16, FP32, 0, 1, 0, 1.0, 0.0, seed=3, lda=K + 24, ldb=K + 8,
+                      ldc=N + 12)
+    nan16 = np.uint16(0x7FC0)
+    p.generate(pad_a=nan16, pad_b=nan16)
+    p.C[:] = np.nan                                   # beta == 0: C_in must never be read
+    cbuf, got, cref, den, _ = check_full(p, flags_for(g, bn))
+    assert np.isfinite(got).all()
+    pad = cbuf.reshape(M, N + 12)[:, N:]
+    assert np.isnan(pad).all(), "padding columns of C were written"
+
+
+def test_bf16_padding_untouched_with_beta():
+    M, N, K = 200, 136, 64
+    p = synth.Problem("pad16", M, N, K, FP16, FP16, 1, 0, 1, 2.0, -1.0, seed=4, lda=M + 8, ldb=N + 16,
+                      ldc=M + 24).generate(pad_c=np.uint16(0x1234))
+    cbuf, *_ = check_full(p, flags_for(2, 128))
+    pad = cbuf.reshape(N, M + 24)[:, M:]
+    assert np.all(pad == 0x1234)
+
+
+def test_degenerate_sizes_and_scalars():
+    # alpha == 0: A and B are not read; C = beta * C
+    p = synth.Problem("a0", 130, 72, 64, BF16, FP32, 0, 1, 0, 0.0, 2.0, seed=5).generate()
+    p.A[:] = np.uint16(0x7FC0)
+    _, got, _ = run_gpu(p)
+    assert np.array_equal(got, 2.0 * oracle.logical_view(p.C, 130, 72, 0, p.ldc, FP32))
+    # alpha == 0 and beta == 0: zeros, whatever C held
+    p = synth.Problem("a0b0", 130, 72, 64, BF16, BF16, 0, 1, 0, 0.0, 0.0, seed=5).generate()
+    p.C[:] = np.uint16(0x7FC0)
+    _, got, _ = run_gpu(p)
+    assert np.all(got == 0.0)
+    # K == 0 behaves like alpha == 0
+    p = synth.Problem("k0", 40, 24, 0, FP16, FP32, 0, 0, 0, 1.0, -1.0, seed=6).generate()
+    _, got, _ = run_gpu(p)
+    assert np.array_equal(got, -oracle.logical_view(p.C, 40, 24, 0, p.ldc, FP32))
+    # M == 0: nothing is launched, OK is returned
+    d = B.make_desc(0, 64, 64, BF16, FP32, 0, 1, 0)
+    with B.Plan(d) as plan:
+        assert plan.info()["kernel_launches_per_run"] == 0
+        plan.run(0, 0, 0, 1.0, 0.0, 0)
+
+
+def test_run_rejects_bad_pointers_before_launch():
+    import torch
+    d = B.make_desc(128, 128, 64, BF16, FP32, 0, 1, 0)
+    buf = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
+    with B.Plan(d) as plan:
+        ptr = buf.data_ptr()
+        assert B.exo_gemm_run(plan.handle, ptr + 2, ptr + 65536, ptr + 131072, 1.0, 0.0, 0) == B.ERR_ALIGNMENT
+        assert B.exo_gemm_run(plan.handle, ptr, ptr + 65536, ptr + 131072 + 4, 1.0, 0.0, 0) == B.ERR_ALIGNMENT
+        assert B.exo_gemm_run(plan.handle, 0, ptr, ptr + 131072, 1.0, 0.0, 0) == B.ERR_NULL
+        assert B.exo_gemm_run(plan.handle, 0, 0, ptr + 131072, 0.0, 0.0, 0) == B.OK   # alpha == 0: A, B unused
+        torch.cuda.synchronize()
+        plan.check()
+
+
+def test_bitwise_determinism_across_runs_and_grid_sizes():
+    p = synth.Problem("det", 1000, 1000, 520, BF16, FP32, 0, 1, 0, 1.0, 0.0, seed=8).generate()
+    ref = None
+    for grid in (0, 2, 14, 148):
+        for rep in range(3):
+            cbuf, _, _ = run_gpu(p, flags_for(2, 256, grid))
+            if ref is None:
+                ref = cbuf.copy()
+            assert np.array_equal(cbuf.view(np.uint32), ref.view(np.uint32)), (grid, rep)
+
+
+def test_persistent_loop_many_tiles_on_few_ctas():
+    # 96 tiles on 4 CTAs: every ring / accumulator barrier wraps many times
+    p = synth.Problem("few", 1536, 1024, 328, FP16, FP16, 0, 0, 0, 1.0, 1.0, seed=9, dist="normal").generate()
+    check_full(p, flags_for(1, 128, 4))
+    check_full(p, flags_for(2, 128, 4))
+
+
+def test_bounded_wait_reports_timeout_and_the_plan_stays_usable():
+    import torch
+    p = synth.Problem("tmo", 512, 512, 1024, BF16, FP32, 0, 1, 0, 1.0, 0.0, seed=10).generate()
+    dp = harness.DeviceProblem(p, flags_for(1, 128))
+    try:
+        # the producer of CTA 0 leaves out the loads of its k-block 5: the MMA issuer's wait runs
+        # out after 20 ms, every role leaves its loop, TMEM is freed, the kernel returns
+        assert B.exo_gemm_debug_set(dp.plan.handle, 20, 5) == B.OK
+        dp.run()
+        torch.cuda.synchronize()
+        st, detail = B.exo_gemm_check(dp.plan.handle)
+        assert st == B.ERR_DEVICE_TIMEOUT
+        assert detail[0] == 1 and detail[1] in (1, 2, 3) and detail[5] == 0, detail
+        # the context is intact and the same plan computes correctly afterwards
+        dp.reset_c()
+        dp.run()
+        torch.cuda.synchronize()
+        dp.plan.check()
+        got = oracle.logical_view(dp.result_buffer(), p.M, p.N, 0, p.ldc, FP32)
+        cref, den = oracle.gemm_problem(p)
+        assert oracle.max_error(got, cref, den) <= TOL
+    finally:
+        dp.close()
+
+
+# ------------------------------------------------------------------ the benchmark configurations
+def structured_sample(M, N, rng, n_random=1 << 14):
+    """Rows/columns next to every 128/256 tile boundary crossed with random partners, plus random entries."""
+    def edges(n):
+        e = set()
+        for t in range(0, n + 1, 128):
+            for d in (-1, 0, 1):
+                if 0 <= t + d < n:
+                    e.add(t + d)
+        return np.array(sorted(e))
+    er, ec = edges(M), edges(N)
+    rows = [np.repeat(er, 8), rng.integers(0, M, 8 * ec.size), rng.integers(0, M, n_random)]
+    cols = [rng.integers(0, N, 8 * er.size), np.repeat(ec, 8), rng.integers(0, N, n_random)]
+    return np.concatenate(rows), np.concatenate(cols)
+
+
+def check_sampled(p, flags=0):
+    cbuf, got, info = run_gpu(p, flags)
+    rng = np.random.default_rng(p.seed)
+    r, c = structured_sample(p.M, p.N, rng)
+    cref, den = oracle.gemm_problem_entries(p, r, c)
+    err = oracle.max_error(got[r, c], cref, den)
+    assert err <= TOL, (p.name, err, info)
+    assert oracle.freivalds(p, got) <= TOL, (p.name, info)
+    return err, info
+
+
+def test_config1_256_full():
+    check_full(synth.config(0).generate(), literal=True)
+
+
+def test_config2_4096_full_matrix_literal_metric():
+    check_full(synth.config(1).generate(), literal=True)
+
+
+def test_config3_8192_fp16_beta_sampled_and_freivalds():
+    check_sampled(synth.config(2).generate())
+
+
+@pytest.mark.parametrize("variant", ["a", "b"])
+def test_config4_skinny_sampled_and_freivalds(variant):
+    check_sampled(synth.config(3, variant).generate())
+
+
+SWEEP_SUBSET = [(512, 512, 512), (1000, 1000, 1000), (512, 12288, 1000), (3072, 1000, 2048),
+                (1000, 512, 12288), (6144, 2048, 512), (2048, 3072, 6144)]
+
+
+@pytest.mark.parametrize("M,N,K", SWEEP_SUBSET)
+def test_shape_sweep_subset(M, N, K):
+    p = synth.sweep_problem(M, N, K).generate()
+    if M * N * K <= 2 ** 32:
+        check_full(p, literal=True)
+    else:
+        check_sampled(p)
