@@ -62,7 +62,7 @@ def lib():
     """Loads (building first if needed) the CUDA library; raises if that fails."""
     global _lib
     if _lib is None:
-        path = _build.build()
+        path = os.environ.get("EXO_GEMM_LIBRARY") or _build.build()   # override: a development build
         if not os.path.exists(path):
             raise RuntimeError("libexo_gemm.so is missing: the CUDA path cannot run")
         L = ctypes.CDLL(path)

@@ -34,6 +34,12 @@ static KernelFn pick_kernel(int cta_group, int bn, int out) {
 
 static thread_local int g_last_cuda_error = 0;
 
+#ifdef EXO_GEMM_TRACE
+constexpr size_t kStatusBytes = 32 + 3 * 4096 * 2 * 8;  // status block + clock stamps of CTA 0
+#else
+constexpr size_t kStatusBytes = 32;
+#endif
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
@@ -246,9 +252,9 @@ exo_gemm_status_t exo_gemm_create(exo_gemm_handle_t* out, const exo_gemm_desc_t*
   p->smem_bytes = smem_bytes_for(p->cfg.cta_group, p->cfg.tile_n);
   e = cudaFuncSetAttribute((const void*)p->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, p->smem_bytes);
   if (e != cudaSuccess) { delete p; return cuda_fail(e); }
-  e = cudaMalloc((void**)&p->d_status, 32);
+  e = cudaMalloc((void**)&p->d_status, kStatusBytes);
   if (e != cudaSuccess) { delete p; return cuda_fail(e); }
-  e = cudaMemset(p->d_status, 0, 32);
+  e = cudaMemset(p->d_status, 0, kStatusBytes);
   if (e != cudaSuccess) { cudaFree(p->d_status); delete p; return cuda_fail(e); }
   *out = p;
   return EXO_GEMM_OK;
@@ -348,6 +354,15 @@ exo_gemm_status_t exo_gemm_check(exo_gemm_handle_t plan, uint32_t* detail) {
   if (e != cudaSuccess) return cuda_fail(e);
   return EXO_GEMM_ERR_DEVICE_TIMEOUT;
 }
+
+#ifdef EXO_GEMM_TRACE
+// Development aid: copies the clock stamps of CTA 0 (3 roles x 4096 x 2 int64) to the host.
+exo_gemm_status_t exo_gemm_debug_read_trace(exo_gemm_handle_t plan, long long* out) {
+  if (!plan || !out) return EXO_GEMM_ERR_NULL;
+  cudaError_t e = cudaMemcpy(out, plan->d_status + 8, kStatusBytes - 32, cudaMemcpyDeviceToHost);
+  return e == cudaSuccess ? EXO_GEMM_OK : cuda_fail(e);
+}
+#endif
 
 exo_gemm_status_t exo_gemm_destroy(exo_gemm_handle_t plan) {
   if (!plan) return EXO_GEMM_OK;

@@ -40,6 +40,18 @@ namespace exo {
 
 enum OutKind : int { kOutBf16 = 0, kOutFp16 = 1, kOutFp32 = 2 };
 
+// Development aid, compiled only with -DEXO_GEMM_TRACE: CTA 0 stamps clock64() at
+// points of its three roles into the words that follow the status block.
+#ifdef EXO_GEMM_TRACE
+#define EXO_TRACE(role, idx, field, cap)                                                        \
+  do {                                                                                          \
+    if (blockIdx.x == 0 && (idx) < (cap))                                                       \
+      reinterpret_cast<long long*>(p.status + 8)[((role) * 4096 + (idx)) * 2 + (field)] = clock64(); \
+  } while (0)
+#else
+#define EXO_TRACE(role, idx, field, cap) do {} while (0)
+#endif
+
 struct WaitSite {
   uint32_t role, barrier, tile, k_block;
 };
@@ -174,22 +186,23 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
 
   if (warp == 0) {
     // ============================================================ producer
-    if (lane == 0) {
-      uint32_t s = 0, ph = 0;
-      int64_t issued = 0;
-      // in a pair, both CTAs' loads are counted on the leader's full barrier
-      const uint32_t full0 = PAIR ? ptx::map_to_cta(full_bar(0), 0) : full_bar(0);
-      for (int64_t t = worker; t < total_tiles && ok; t += num_workers) {
-        const TileCoord tc = raster_decode(p.raster, t);
-        const int32_t a_mn0 = tc.m * (kBlockM * CTA_GROUP) + (int32_t)cta_rank * kBlockM;
-        const int32_t b_mn0 = tc.n * BN + (int32_t)cta_rank * B_ROWS;
-        for (int32_t kb = 0; kb < nkb; ++kb) {
-          ok = wait_barrier<PAIR>(empty_bar(s), ph ^ 1u, p,
-                                  WaitSite{kRoleProducer, s, (uint32_t)t, (uint32_t)kb});
-          if (!ok) break;
+    // The whole warp runs the loop (uniform control flow); one elected lane issues.
+    uint32_t s = 0, ph = 0;
+    int64_t issued = 0;
+    // in a pair, both CTAs' loads are counted on the leader's full barrier
+    const uint32_t full0 = PAIR ? ptx::map_to_cta(full_bar(0), 0) : full_bar(0);
+    for (int64_t t = worker; t < total_tiles && ok; t += num_workers) {
+      const TileCoord tc = raster_decode(p.raster, t);
+      const int32_t a_mn0 = tc.m * (kBlockM * CTA_GROUP) + (int32_t)cta_rank * kBlockM;
+      const int32_t b_mn0 = tc.n * BN + (int32_t)cta_rank * B_ROWS;
+      for (int32_t kb = 0; kb < nkb; ++kb) {
+        ok = wait_barrier<PAIR>(empty_bar(s), ph ^ 1u, p, WaitSite{kRoleProducer, s, (uint32_t)t, (uint32_t)kb});
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        const bool skip = (p.debug_skip_k_block == issued) && blockIdx.x == 0;
+        if (ptx::elect_one()) {
+          EXO_TRACE(0, issued, 0, 4096);
           if (cta_rank == 0) ptx::mbar_arrive_expect_tx(full_bar(s), STAGE_BYTES * CTA_GROUP);
-          const bool skip = (p.debug_skip_k_block == issued) && blockIdx.x == 0;
-          ++issued;
           if (!skip) {
             const uint32_t a_dst = stage0 + s * STAGE_BYTES;
             const uint32_t b_dst = a_dst + kATileBytes;
@@ -212,50 +225,66 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
               for (int b = 0; b < B_ROWS / 64; ++b) load(b_dst + b * 8192, &tm_b, b_mn0 + 64 * b, k0);
             }
           }
-          if (++s == STAGES) { s = 0; ph ^= 1u; }
+          EXO_TRACE(0, issued, 1, 4096);
         }
-      }
-      // Tail: do not leave while stage releases addressed to this CTA are still in flight.
-      for (uint32_t i = 0; i < STAGES && ok; ++i) {
-        ok = wait_barrier<PAIR>(empty_bar(s), ph ^ 1u, p, WaitSite{kRoleProducerTail, s, 0, 0});
+        ++issued;
         if (++s == STAGES) { s = 0; ph ^= 1u; }
       }
     }
-    __syncwarp();
+    // Tail: do not leave while stage releases addressed to this CTA are still in flight.
+    for (uint32_t i = 0; i < STAGES && ok; ++i) {
+      ok = wait_barrier<PAIR>(empty_bar(s), ph ^ 1u, p, WaitSite{kRoleProducerTail, s, 0, 0});
+      ok = __all_sync(0xffffffffu, ok);
+      if (++s == STAGES) { s = 0; ph ^= 1u; }
+    }
   } else if (warp == 1) {
     // ============================================================ MMA issuer
-    if (lane == 0 && cta_rank == 0 && nkb > 0) {
+    if (cta_rank == 0 && nkb > 0) {
       uint32_t s = 0, ph = 0, acc = 0, acc_ph = 0;
       constexpr uint16_t kMask = PAIR ? 3 : 1;
+      [[maybe_unused]] int64_t consumed = 0;
+      const uint32_t a_step = p.a.k_step_enc, b_step = p.b.k_step_enc;
+      const uint32_t idesc = p.idesc;
       for (int64_t t = worker; t < total_tiles && ok; t += num_workers) {
         // the epilogue (of both CTAs) must have drained this accumulator
         ok = wait_barrier<PAIR>(tempty_bar(acc), acc_ph ^ 1u, p, WaitSite{kRoleMma, 100 + acc, (uint32_t)t, 0});
+        ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         ptx::tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + acc * BN;
         for (int32_t kb = 0; kb < nkb; ++kb) {
           ok = wait_barrier<PAIR>(full_bar(s), ph, p, WaitSite{kRoleMma, s, (uint32_t)t, (uint32_t)kb});
+          ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           ptx::tc_fence_after_sync();
           const uint32_t a_addr = stage0 + s * STAGE_BYTES;
           const uint64_t a_desc = make_smem_desc(a_addr, p.a);
           const uint64_t b_desc = make_smem_desc(a_addr + kATileBytes, p.b);
           const int32_t k_left = p.K - kb * kBlockK;
-          const int32_t n_mma = k_left >= kBlockK ? kBlockK / kUmmaK : (k_left + kUmmaK - 1) / kUmmaK;
-          for (int32_t k = 0; k < n_mma; ++k) {
-            ptx::umma_f16<CTA_GROUP>(d_tmem, a_desc + (uint64_t)(k * p.a.k_step_enc),
-                                     b_desc + (uint64_t)(k * p.b.k_step_enc), p.idesc,
-                                     (kb | k) != 0 ? 1u : 0u);
+          if (ptx::elect_one()) {  // the same lane every time: commits track this thread's MMAs
+            EXO_TRACE(1, consumed, 0, 4096);
+            if (k_left >= kBlockK) {
+#pragma unroll
+              for (int32_t k = 0; k < kBlockK / kUmmaK; ++k)
+                ptx::umma_f16<CTA_GROUP>(d_tmem, a_desc + (uint64_t)(k * a_step), b_desc + (uint64_t)(k * b_step),
+                                         idesc, (kb | k) != 0 ? 1u : 0u);
+            } else {  // ragged last k-block: skip the MMAs that would only read zero fill
+              const int32_t n_mma = (k_left + kUmmaK - 1) / kUmmaK;
+              for (int32_t k = 0; k < n_mma; ++k)
+                ptx::umma_f16<CTA_GROUP>(d_tmem, a_desc + (uint64_t)(k * a_step), b_desc + (uint64_t)(k * b_step),
+                                         idesc, (kb | k) != 0 ? 1u : 0u);
+            }
+            ptx::umma_commit<CTA_GROUP>(empty_bar(s), kMask);  // stage free once these MMAs completed
+            if (kb == nkb - 1) ptx::umma_commit<CTA_GROUP>(tfull_bar(acc), kMask);  // accumulator complete
+            EXO_TRACE(1, consumed, 1, 4096);
           }
-          ptx::umma_commit<CTA_GROUP>(empty_bar(s), kMask);  // stage free once these MMAs completed
+          ++consumed;
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
         if (!ok) break;
-        ptx::umma_commit<CTA_GROUP>(tfull_bar(acc), kMask);  // accumulator complete
         if ((acc ^= 1u) == 0u) acc_ph ^= 1u;
       }
     }
-    __syncwarp();
   } else {
     // ============================================================ epilogue
     const uint32_t quad = warp & 3u;  // TMEM lanes 32*quad .. 32*quad+31 belong to this warp
@@ -285,6 +314,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         if (!ok) break;
         ptx::tc_fence_after_sync();
       }
+      if (warp == 2 && lane == 0) EXO_TRACE(2, (t - worker) / num_workers, 0, 4096);
       auto release_acc = [&]() {
         ptx::tc_fence_before_sync();
         __syncwarp();
@@ -379,6 +409,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         ++g;
       }
       if (!ok) break;
+      if (warp == 2 && lane == 0) EXO_TRACE(2, (t - worker) / num_workers, 1, 4096);
       if ((acc ^= 1u) == 0u) acc_ph ^= 1u;
     }
     if (lane == 0) ptx::bulk_wait<0>();  // all stores of this warp have completed

@@ -18,10 +18,17 @@ __device__ __forceinline__ uint32_t lane_id() {
   return v;
 }
 
-__device__ __forceinline__ uint64_t globaltimer_ns() {
-  uint64_t v;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(v));
-  return v;
+// True in exactly one lane of a fully converged warp.  Code guarded by it stays on
+// the warp-uniform path, which the single-thread instructions (TMA, tcgen05.mma,
+// tcgen05.commit) need to issue quickly; a plain `lane == 0` test makes them slow.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred = 0;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
 }
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
