@@ -45,12 +45,14 @@ typedef enum { EXO_GEMM_ROW_MAJOR = 0, EXO_GEMM_COL_MAJOR = 1 } exo_gemm_layout_
  *   bits 6..9   raster band width in tiles (1..15)
  *   bit  10     raster direction: 0 = library choice, set = bands along M instead of N
  *   bits 12..19 grid limit: launch at most this many CTAs (multiple of cta_group), 0 = all SMs
+ *   bits 20..21 k sub-blocks (of 64 elements) per pipeline stage: 1 or 2
  */
 #define EXO_GEMM_FLAG_CTA_GROUP(g)  ((uint32_t)(g) & 3u)
 #define EXO_GEMM_FLAG_TILE_N(n)     ((((uint32_t)(n) / 64u) & 15u) << 2)
 #define EXO_GEMM_FLAG_BAND(b)       (((uint32_t)(b) & 15u) << 6)
 #define EXO_GEMM_FLAG_BANDS_ALONG_M (1u << 10)
 #define EXO_GEMM_FLAG_GRID_LIMIT(c) (((uint32_t)(c) & 255u) << 12)
+#define EXO_GEMM_FLAG_K_SUBBLOCKS(k) (((uint32_t)(k) & 3u) << 20)
 
 /*
  * Problem descriptor.  Logical shapes: A is M x K, B is K x N, C is M x N.
@@ -79,7 +81,7 @@ typedef struct {
 typedef struct {
   int32_t cta_group;      /* 1 or 2 SMs per tile                                               */
   int32_t tile_m, tile_n; /* output tile of one CTA group (tile_m = 128 * cta_group)           */
-  int32_t tile_k;         /* k-block staged per pipeline stage (64 elements = 128 bytes)       */
+  int32_t tile_k;         /* k-elements staged per pipeline stage (64 or 128)                  */
   int32_t stages;         /* depth of the shared-memory operand ring                           */
   int32_t grid;           /* CTAs launched (persistent)                                        */
   int32_t smem_bytes;     /* dynamic shared memory per CTA                                     */

@@ -16,20 +16,25 @@ namespace exo {
 
 using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const GemmParams);
 
-template <int G, int BN>
+template <int G, int BN, int KSUB>
 static KernelFn pick_out(int out) {
   switch (out) {
-    case EXO_GEMM_BF16: return exo_gemm_kernel<G, BN, kOutBf16>;
-    case EXO_GEMM_FP16: return exo_gemm_kernel<G, BN, kOutFp16>;
-    default:            return exo_gemm_kernel<G, BN, kOutFp32>;
+    case EXO_GEMM_BF16: return exo_gemm_kernel<G, BN, kOutBf16, KSUB>;
+    case EXO_GEMM_FP16: return exo_gemm_kernel<G, BN, kOutFp16, KSUB>;
+    default:            return exo_gemm_kernel<G, BN, kOutFp32, KSUB>;
   }
 }
 
-static KernelFn pick_kernel(int cta_group, int bn, int out) {
-  if (cta_group == 2) return bn == 256 ? pick_out<2, 256>(out) : pick_out<2, 128>(out);
-  if (bn == 256) return pick_out<1, 256>(out);
-  if (bn == 128) return pick_out<1, 128>(out);
-  return pick_out<1, 64>(out);
+template <int KSUB>
+static KernelFn pick_shape(int cta_group, int bn, int out) {
+  if (cta_group == 2) return bn == 256 ? pick_out<2, 256, KSUB>(out) : pick_out<2, 128, KSUB>(out);
+  if (bn == 256) return pick_out<1, 256, KSUB>(out);
+  if (bn == 128) return pick_out<1, 128, KSUB>(out);
+  return pick_out<1, 64, KSUB>(out);
+}
+
+static KernelFn pick_kernel(int cta_group, int bn, int ksub, int out) {
+  return ksub == 2 ? pick_shape<2>(cta_group, bn, out) : pick_shape<1>(cta_group, bn, out);
 }
 
 static thread_local int g_last_cuda_error = 0;
@@ -123,7 +128,7 @@ void fill_info(const exo_gemm_plan* p, exo_gemm_info_t* info) {
   info->cta_group = p->cfg.cta_group;
   info->tile_m = 128 * p->cfg.cta_group;
   info->tile_n = p->cfg.tile_n;
-  info->tile_k = kBlockK;
+  info->tile_k = kBlockK * p->cfg.ksub;
   info->stages = p->cfg.stages;
   info->grid = p->cfg.workers * p->cfg.cta_group;
   info->smem_bytes = p->smem_bytes;
@@ -187,7 +192,7 @@ exo_gemm_status_t exo_gemm_plan_preview(const exo_gemm_desc_t* desc, int32_t sm_
   p.canon = canonicalize(*desc);
   p.sm_count = sm_count;
   p.cfg = choose_config(p.canon, decode_flags(desc->flags), sm_count, sm_count / 2);
-  p.smem_bytes = smem_bytes_for(p.cfg.cta_group, p.cfg.tile_n);
+  p.smem_bytes = smem_bytes_for(p.cfg.cta_group, p.cfg.tile_n, p.cfg.ksub);
   fill_info(&p, info);
   return EXO_GEMM_OK;
 }
@@ -226,8 +231,8 @@ exo_gemm_status_t exo_gemm_create(exo_gemm_handle_t* out, const exo_gemm_desc_t*
   // How many 2-CTA clusters can be resident at once (GPC shapes may leave SMs unpaired).
   int max_pairs = 0;
   if (ov.cta_group != 1) {
-    KernelFn probe = pick_kernel(2, 256, desc->c_dtype);
-    const int smem = smem_bytes_for(2, 256);
+    KernelFn probe = pick_kernel(2, 256, 2, desc->c_dtype);
+    const int smem = smem_bytes_for(2, 256, 2);
     e = cudaFuncSetAttribute((const void*)probe, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) { delete p; return cuda_fail(e); }
     cudaLaunchConfig_t lc{};
@@ -248,8 +253,8 @@ exo_gemm_status_t exo_gemm_create(exo_gemm_handle_t* out, const exo_gemm_desc_t*
   }
 
   p->cfg = choose_config(p->canon, ov, sms, max_pairs);
-  p->kernel = pick_kernel(p->cfg.cta_group, p->cfg.tile_n, desc->c_dtype);
-  p->smem_bytes = smem_bytes_for(p->cfg.cta_group, p->cfg.tile_n);
+  p->kernel = pick_kernel(p->cfg.cta_group, p->cfg.tile_n, p->cfg.ksub, desc->c_dtype);
+  p->smem_bytes = smem_bytes_for(p->cfg.cta_group, p->cfg.tile_n, p->cfg.ksub);
   e = cudaFuncSetAttribute((const void*)p->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, p->smem_bytes);
   if (e != cudaSuccess) { delete p; return cuda_fail(e); }
   e = cudaMalloc((void**)&p->d_status, kStatusBytes);
@@ -292,13 +297,14 @@ exo_gemm_status_t exo_gemm_run(exo_gemm_handle_t plan, const void* A, const void
   prm.M = (int32_t)cn.M;
   prm.N = (int32_t)cn.N;
   prm.K = (int32_t)cn.K;
-  prm.num_k_blocks = read_ab ? (int32_t)((cn.K + kBlockK - 1) / kBlockK) : 0;
+  const int stage_k = kBlockK * cfg.ksub;
+  prm.num_k_blocks = read_ab ? (int32_t)((cn.K + stage_k - 1) / stage_k) : 0;
   prm.raster = Raster{cfg.tiles_m, cfg.tiles_n, cfg.band, cfg.along_m};
   prm.alpha = read_ab ? alpha : 0.f;
   prm.beta = beta;
   prm.idesc = make_idesc(d.ab_dtype, cn.a_mn_major, cn.b_mn_major, 128 * cfg.cta_group, cfg.tile_n);
-  prm.a = make_staging(cn.a_mn_major);
-  prm.b = make_staging(cn.b_mn_major);
+  prm.a = make_staging(cn.a_mn_major, kBlockM, cfg.ksub);
+  prm.b = make_staging(cn.b_mn_major, cfg.tile_n / cfg.cta_group, cfg.ksub);
   prm.status = plan->d_status;
   const int32_t dbg_ms = plan->dbg_timeout_ms.exchange(0);
   // SM clocks, converted at 2 GHz (an upper bound of the SM clock, so the real limit is not shorter)
@@ -311,10 +317,10 @@ exo_gemm_status_t exo_gemm_run(exo_gemm_handle_t plan, const void* A, const void
   CUresult r;
   const int b_rows = cfg.tile_n / cfg.cta_group;
   if (read_ab) {
-    r = cn.a_mn_major ? encode_2d(&tm_a, d.ab_dtype, opA, cn.M, cn.K, cn.lda, 64, kBlockK, true)
+    r = cn.a_mn_major ? encode_2d(&tm_a, d.ab_dtype, opA, cn.M, cn.K, cn.lda, 64, stage_k, true)
                       : encode_2d(&tm_a, d.ab_dtype, opA, cn.K, cn.M, cn.lda, kBlockK, kBlockM, true);
     if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return EXO_GEMM_ERR_CUDA; }
-    r = cn.b_mn_major ? encode_2d(&tm_b, d.ab_dtype, opB, cn.N, cn.K, cn.ldb, 64, kBlockK, true)
+    r = cn.b_mn_major ? encode_2d(&tm_b, d.ab_dtype, opB, cn.N, cn.K, cn.ldb, 64, stage_k, true)
                       : encode_2d(&tm_b, d.ab_dtype, opB, cn.K, cn.N, cn.ldb, kBlockK, b_rows, true);
     if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return EXO_GEMM_ERR_CUDA; }
   }

@@ -117,13 +117,15 @@ __device__ __forceinline__ float2 unpack2(uint32_t w) {
   }
 }
 
-template <int CTA_GROUP, int BN, int OUT>
+template <int CTA_GROUP, int BN, int OUT, int KSUB>
 __global__ void __launch_bounds__(kNumThreads, 1)
 exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                 const __grid_constant__ CUtensorMap tm_c, const GemmParams p) {
-  constexpr int STAGES = max_stages(CTA_GROUP, BN);
+  constexpr int STAGES = max_stages(CTA_GROUP, BN, KSUB);
+  constexpr int STAGE_K = kBlockK * KSUB;            // k-elements per stage
   constexpr int B_ROWS = BN / CTA_GROUP;             // rows of the B tile this CTA stages
-  constexpr int STAGE_BYTES = stage_bytes(CTA_GROUP, BN);
+  constexpr int STAGE_BYTES = stage_bytes(CTA_GROUP, BN, KSUB);
+  constexpr int A_BYTES = KSUB * kATileBytes;        // the A part of a stage
   constexpr uint32_t TMEM_COLS = 2 * BN;             // two accumulators; 128, 256 or 512 columns
   constexpr int CW = (OUT == kOutFp32) ? 32 : 64;    // columns per epilogue chunk = 128 bytes of C
   constexpr int NCHUNK = BN / CW;
@@ -205,24 +207,28 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
           if (cta_rank == 0) ptx::mbar_arrive_expect_tx(full_bar(s), STAGE_BYTES * CTA_GROUP);
           if (!skip) {
             const uint32_t a_dst = stage0 + s * STAGE_BYTES;
-            const uint32_t b_dst = a_dst + kATileBytes;
+            const uint32_t b_dst = a_dst + A_BYTES;
             const uint32_t bar = full0 + 8u * s;
-            const int32_t k0 = kb * kBlockK;
+            const int32_t k0 = kb * STAGE_K;
             auto load = [&](uint32_t dst, const CUtensorMap* map, int32_t x, int32_t y) {
               if constexpr (PAIR) ptx::tma_load_2d_pair(dst, map, x, y, bar);
               else ptx::tma_load_2d(dst, map, x, y, bar);
             };
             if (!p.a.mn_major) {
-              load(a_dst, &tm_a, k0, a_mn0);
+#pragma unroll
+              for (int h = 0; h < KSUB; ++h) load(a_dst + h * kATileBytes, &tm_a, k0 + h * kBlockK, a_mn0);
             } else {
 #pragma unroll
-              for (int b = 0; b < kBlockM / 64; ++b) load(a_dst + b * 8192, &tm_a, a_mn0 + 64 * b, k0);
+              for (int b = 0; b < kBlockM / 64; ++b)
+                load(a_dst + b * (KSUB * 8192), &tm_a, a_mn0 + 64 * b, k0);
             }
             if (!p.b.mn_major) {
-              load(b_dst, &tm_b, k0, b_mn0);
+#pragma unroll
+              for (int h = 0; h < KSUB; ++h) load(b_dst + h * (B_ROWS * 128), &tm_b, k0 + h * kBlockK, b_mn0);
             } else {
 #pragma unroll
-              for (int b = 0; b < B_ROWS / 64; ++b) load(b_dst + b * 8192, &tm_b, b_mn0 + 64 * b, k0);
+              for (int b = 0; b < B_ROWS / 64; ++b)
+                load(b_dst + b * (KSUB * 8192), &tm_b, b_mn0 + 64 * b, k0);
             }
           }
           EXO_TRACE(0, issued, 1, 4096);
@@ -244,6 +250,11 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       constexpr uint16_t kMask = PAIR ? 3 : 1;
       [[maybe_unused]] int64_t consumed = 0;
       const uint32_t a_step = p.a.k_step_enc, b_step = p.b.k_step_enc;
+      const uint32_t a_sub = p.a.k_sub_enc, b_sub = p.b.k_sub_enc;
+      constexpr int kMmaPerStage = STAGE_K / kUmmaK;
+      auto k_off = [](int32_t k, uint32_t step, uint32_t sub) {  // descriptor offset of the k-th MMA of a stage
+        return (uint64_t)((uint32_t)(k & 3) * step + (uint32_t)(k >> 2) * sub);
+      };
       const uint32_t idesc = p.idesc;
       for (int64_t t = worker; t < total_tiles && ok; t += num_workers) {
         // the epilogue (of both CTAs) must have drained this accumulator
@@ -259,19 +270,19 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
           ptx::tc_fence_after_sync();
           const uint32_t a_addr = stage0 + s * STAGE_BYTES;
           const uint64_t a_desc = make_smem_desc(a_addr, p.a);
-          const uint64_t b_desc = make_smem_desc(a_addr + kATileBytes, p.b);
-          const int32_t k_left = p.K - kb * kBlockK;
+          const uint64_t b_desc = make_smem_desc(a_addr + A_BYTES, p.b);
+          const int32_t k_left = p.K - kb * STAGE_K;
           if (ptx::elect_one()) {  // the same lane every time: commits track this thread's MMAs
             EXO_TRACE(1, consumed, 0, 4096);
-            if (k_left >= kBlockK) {
+            if (k_left >= STAGE_K) {
 #pragma unroll
-              for (int32_t k = 0; k < kBlockK / kUmmaK; ++k)
-                ptx::umma_f16<CTA_GROUP>(d_tmem, a_desc + (uint64_t)(k * a_step), b_desc + (uint64_t)(k * b_step),
+              for (int32_t k = 0; k < kMmaPerStage; ++k)
+                ptx::umma_f16<CTA_GROUP>(d_tmem, a_desc + k_off(k, a_step, a_sub), b_desc + k_off(k, b_step, b_sub),
                                          idesc, (kb | k) != 0 ? 1u : 0u);
             } else {  // ragged last k-block: skip the MMAs that would only read zero fill
               const int32_t n_mma = (k_left + kUmmaK - 1) / kUmmaK;
               for (int32_t k = 0; k < n_mma; ++k)
-                ptx::umma_f16<CTA_GROUP>(d_tmem, a_desc + (uint64_t)(k * a_step), b_desc + (uint64_t)(k * b_step),
+                ptx::umma_f16<CTA_GROUP>(d_tmem, a_desc + k_off(k, a_step, a_sub), b_desc + k_off(k, b_step, b_sub),
                                          idesc, (kb | k) != 0 ? 1u : 0u);
             }
             ptx::umma_commit<CTA_GROUP>(empty_bar(s), kMask);  // stage free once these MMAs completed

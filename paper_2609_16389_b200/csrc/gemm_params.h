@@ -8,7 +8,7 @@
 namespace exo {
 
 constexpr int kBlockM = 128;        // rows of C per CTA (one TMEM lane per row)
-constexpr int kBlockK = 64;         // elements of K per stage: 128 bytes = one swizzle span
+constexpr int kBlockK = 64;         // elements of K per sub-block: 128 bytes = one swizzle span
 constexpr int kUmmaK = 16;          // K of one tcgen05.mma for 16-bit inputs
 constexpr int kNumThreads = 192;    // warp 0 producer, warp 1 MMA issuer + TMEM owner, warps 2..5 epilogue
 constexpr int kEpiWarps = 4;
@@ -24,21 +24,26 @@ constexpr int kATileBytes = kBlockM * kBlockK * 2;  // 16 KB
 #else
 #define EXO_CX constexpr
 #endif
-EXO_CX int stage_bytes(int cta_group, int bn) { return kATileBytes + (bn / cta_group) * kBlockK * 2; }
-
-EXO_CX int max_stages(int cta_group, int bn) {
-  return (kSmemLimit - 1024 /*alignment slack*/ - kBarrierBytes -
-          kEpiWarps * kEpiBufsPerWarp * kEpiBufBytes) /
-         stage_bytes(cta_group, bn);
+// A stage holds `ksub` sub-blocks of 64 k-elements (1 or 2): one barrier round trip per stage.
+EXO_CX int stage_bytes(int cta_group, int bn, int ksub) {
+  return ksub * (kATileBytes + (bn / cta_group) * kBlockK * 2);
 }
 
-// How one operand is staged.  K-major: one TMA box {64 k, rows}.  MN-major: rows/64
-// boxes {64 mn, 64 k}, 8 KB apart.
+EXO_CX int max_stages(int cta_group, int bn, int ksub) {
+  return (kSmemLimit - 1024 /*alignment slack*/ - kBarrierBytes -
+          kEpiWarps * kEpiBufsPerWarp * kEpiBufBytes) /
+         stage_bytes(cta_group, bn, ksub);
+}
+
+// How one operand is staged.  K-major: per 64-k sub-block one TMA box {64 k, rows},
+// sub-blocks rows*128 bytes apart.  MN-major: rows/64 boxes {64 mn, 64*ksub k}.
 struct OperandStaging {
   uint32_t mn_major;   // 0: K contiguous in memory, 1: M/N contiguous
   uint32_t desc_hi;    // upper half of the UMMA shared-memory descriptor
   uint32_t lbo_enc;    // leading byte offset >> 4
-  uint32_t k_step_enc; // descriptor start-address increment per UMMA_K (bytes >> 4)
+  uint32_t k_step_enc; // descriptor start-address increment per UMMA_K inside a sub-block (bytes >> 4)
+  uint32_t k_sub_enc;  // descriptor start-address increment per 64-k sub-block (bytes >> 4)
+  uint32_t box_bytes;  // MN-major: bytes of one TMA box in shared memory
 };
 
 enum StatusCode : uint32_t {
@@ -56,7 +61,7 @@ enum WaitRole : uint32_t {
 
 struct GemmParams {
   int32_t M, N, K;          // canonical problem (C row-major; operands possibly swapped)
-  int32_t num_k_blocks;     // ceil(K / 64), or 0 when alpha == 0 / K == 0
+  int32_t num_k_blocks;     // ceil(K / (64 * ksub)), or 0 when alpha == 0 / K == 0
   Raster raster;
   float alpha, beta;
   uint32_t idesc;           // tcgen05 instruction descriptor

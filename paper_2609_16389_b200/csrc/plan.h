@@ -12,6 +12,7 @@ namespace exo {
 inline int elem_bytes(int dtype) { return dtype == EXO_GEMM_FP32 ? 4 : 2; }
 
 struct FlagOverrides {
+  int ksub;        // 0 = auto
   int cta_group;   // 0 = auto
   int tile_n;      // 0 = auto
   int band;        // 0 = auto
@@ -26,6 +27,7 @@ inline FlagOverrides decode_flags(uint32_t f) {
   o.band = (int)((f >> 6) & 15u);
   o.along_m = (int)((f >> 10) & 1u);
   o.grid_limit = (int)((f >> 12) & 255u);
+  o.ksub = (int)((f >> 20) & 3u);
   return o;
 }
 
@@ -49,7 +51,8 @@ inline exo_gemm_status_t validate_desc(const exo_gemm_desc_t* d) {
   if (d->lda < extent(d->a_layout, d->M, d->K) || d->ldb < extent(d->b_layout, d->K, d->N) ||
       d->ldc < extent(d->c_layout, d->M, d->N) || d->lda > kMaxLd || d->ldb > kMaxLd || d->ldc > kMaxLd)
     return EXO_GEMM_ERR_INVALID_ARG;
-  if (d->flags >> 20) return EXO_GEMM_ERR_INVALID_ARG;
+  if (d->flags >> 22) return EXO_GEMM_ERR_INVALID_ARG;
+  if (((d->flags >> 20) & 3u) == 3u) return EXO_GEMM_ERR_INVALID_ARG;
   if (d->flags & (1u << 11)) return EXO_GEMM_ERR_INVALID_ARG;
   const FlagOverrides o = decode_flags(d->flags);
   if (o.cta_group == 3) return EXO_GEMM_ERR_INVALID_ARG;
@@ -97,17 +100,24 @@ inline Canonical canonicalize(const exo_gemm_desc_t& d) {
 }
 
 struct TileConfig {
-  int cta_group, tile_n, stages;
+  int cta_group, tile_n, ksub, stages;
   int tiles_m, tiles_n;
   int band, along_m;
   int workers;  // CTA groups launched
 };
 
-// Relative tensor-pipe efficiency of a tile shape in the main loop (1 = the MMA
-// rate): smaller N per CTA re-reads A from shared memory more often per flop.
+// Sub-blocks of 64 k-elements per pipeline stage.  Two per stage halves the number of
+// barrier round trips per MMA, which is what bounds the issuing thread when a tile's
+// MMAs are short (N <= 128); with N = 256 on one CTA two would leave only two stages.
+inline int default_ksub(int cta_group, int bn) { (void)cta_group; return bn == 256 ? 1 : 2; }
+
+// Main-loop throughput of a tile shape relative to the 2-CTA 256x256 tile, measured on
+// a B200 at 4096^3 with the wave-quantisation factor divided out: smaller N per CTA
+// moves more operand bytes through shared memory per flop and leaves the issuing
+// thread less time per MMA.
 inline double shape_efficiency(int cta_group, int bn) {
-  if (cta_group == 2) return bn == 256 ? 1.0 : 0.9;
-  return bn == 256 ? 0.93 : (bn == 128 ? 0.8 : 0.55);
+  if (cta_group == 2) return bn == 256 ? 1.0 : 0.81;
+  return bn == 256 ? 0.86 : (bn == 128 ? 0.66 : 0.40);
 }
 
 // Estimated time of the whole problem in SM clocks for one candidate shape.
@@ -120,8 +130,9 @@ inline double estimate_clocks(int64_t M, int64_t N, int64_t K, int cta_group, in
   const int64_t waves = (tiles + workers - 1) / workers;
   const int64_t nkb = (K + kBlockK - 1) / kBlockK;
   const double mainloop = (double)nkb * 2.0 * bn / shape_efficiency(cta_group, bn);  // clocks per tile
-  const double epilogue = 6.0 * bn + 1500.0;  // drain of one accumulator: exposed once, plus fill latency
-  const double per_tile = mainloop > 4.0 * bn ? mainloop : 4.0 * bn;  // epilogue-bound tiles
+  const double drain = 22.0 * bn;             // draining one accumulator (measured ~5.9k clocks at N = 256)
+  const double epilogue = drain + 1500.0;     // exposed once at the end, plus pipeline fill latency
+  const double per_tile = mainloop > drain ? mainloop : drain;  // small K: the epilogue bounds a tile
   return (double)waves * per_tile + epilogue;
 }
 
@@ -143,7 +154,8 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
   TileConfig cfg;
   cfg.cta_group = best_g;
   cfg.tile_n = best_n;
-  cfg.stages = max_stages(best_g, best_n);
+  cfg.ksub = o.ksub ? o.ksub : default_ksub(best_g, best_n);
+  cfg.stages = max_stages(best_g, best_n, cfg.ksub);
   cfg.tiles_m = (int)((c.M + 128 * best_g - 1) / (128 * best_g));
   cfg.tiles_n = (int)((c.N + best_n - 1) / best_n);
   int64_t workers = best_g == 2 ? max_pairs : sm_count;
@@ -166,8 +178,8 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
   return cfg;
 }
 
-inline int smem_bytes_for(int cta_group, int bn) {
-  return 1024 + max_stages(cta_group, bn) * stage_bytes(cta_group, bn) +
+inline int smem_bytes_for(int cta_group, int bn, int ksub) {
+  return 1024 + max_stages(cta_group, bn, ksub) * stage_bytes(cta_group, bn, ksub) +
          kEpiWarps * kEpiBufsPerWarp * kEpiBufBytes + kBarrierBytes;
 }
 
@@ -186,7 +198,7 @@ inline uint32_t make_idesc(int ab_dtype, int a_mn_major, int b_mn_major, int umm
 }
 
 // How an operand tile sits in shared memory (128-byte swizzle, 8-row atoms of 1 KB).
-inline OperandStaging make_staging(int mn_major) {
+inline OperandStaging make_staging(int mn_major, int rows, int ksub) {
   OperandStaging s;
   s.mn_major = (uint32_t)mn_major;
   const uint32_t sbo = 1024u >> 4;       // between 8-row groups of a swizzle atom column
@@ -196,9 +208,13 @@ inline OperandStaging make_staging(int mn_major) {
   if (!mn_major) {
     s.lbo_enc = 1;                                   // unused for swizzled K-major tiles
     s.k_step_enc = (kUmmaK * 2) >> 4;                // 32 bytes along the 128-byte row
+    s.k_sub_enc = ((uint32_t)rows * 128u) >> 4;      // next sub-block: next box of `rows` rows
+    s.box_bytes = (uint32_t)rows * 128u;
   } else {
-    s.lbo_enc = (kBlockK * 128u) >> 4;               // next 64 M/N elements: next 8 KB box
+    s.box_bytes = (uint32_t)ksub * kBlockK * 128u;   // one box: 64*ksub k-rows of 128 bytes
+    s.lbo_enc = s.box_bytes >> 4;                    // next 64 M/N elements: next box
     s.k_step_enc = (kUmmaK * 128u) >> 4;             // 16 k-rows of 128 bytes
+    s.k_sub_enc = (kBlockK * 128u) >> 4;             // k-rows continue inside the same box
   }
   return s;
 }

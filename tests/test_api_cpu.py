@@ -102,7 +102,7 @@ def test_plan_preview_geometry_and_overrides():
     st, info = B.exo_gemm_plan_preview(good(M=4096, N=4096, K=4096, c_dtype=B.BF16), 148)
     assert st == B.OK
     i = info.as_dict()
-    assert i["tile_m"] == 128 * i["cta_group"] and i["tile_k"] == 64
+    assert i["tile_m"] == 128 * i["cta_group"] and i["tile_k"] in (64, 128)
     assert i["tiles_m"] * i["tile_m"] >= 4096 and i["tiles_n"] * i["tile_n"] >= 4096
     assert i["grid"] <= 148 and i["grid"] % i["cta_group"] == 0
     assert i["smem_bytes"] <= 232448 and i["tmem_columns"] == 2 * i["tile_n"] <= 512
@@ -114,7 +114,8 @@ def test_plan_preview_geometry_and_overrides():
         assert (i["cta_group"], i["tile_n"]) == (g, bn)
         assert i["tiles_m"] == -(-1000 // (128 * g)) and i["tiles_n"] == -(-520 // bn)
         assert i["grid"] == min(148 // g, i["tiles_m"] * i["tiles_n"]) * g
-        assert i["stages"] * (16384 + bn // g * 128) + 32768 + 1536 <= 232448
+        assert i["tile_k"] in (64, 128) and i["stages"] >= 2
+        assert i["stages"] * (i["tile_k"] // 64) * (16384 + bn // g * 128) + 32768 + 1536 <= 232448
     # column-major C is computed as the transposed product
     st, info = B.exo_gemm_plan_preview(good(M=512, N=2048, K=64, c_layout=1, ldc=512), 148)
     i = info.as_dict()

@@ -40,8 +40,9 @@ def check_full(p, flags=0, literal=None):
     return cbuf, got, cref, den, info
 
 
-def flags_for(g, bn, grid=0):
-    return B.flag_cta_group(g) | B.flag_tile_n(bn) | (B.flag_grid_limit(grid) if grid else 0)
+def flags_for(g, bn, grid=0, ksub=0):
+    return (B.flag_cta_group(g) | B.flag_tile_n(bn) | (B.flag_grid_limit(grid) if grid else 0)
+            | B.flag_k_subblocks(ksub))
 
 
 TILE_SHAPES = [(1, 64), (1, 128), (1, 256), (2, 128), (2, 256)]
@@ -79,24 +80,25 @@ EDGE_MN = [(1, 8), (127, 129), (128, 128), (129, 72), (255, 257), (257, 40), (38
 @pytest.mark.parametrize("M,N", EDGE_MN)
 @pytest.mark.parametrize("K", [8, 72, 1000])
 @pytest.mark.parametrize("g,bn", TILE_SHAPES)
-def test_tile_boundaries(M, N, K, g, bn):
+@pytest.mark.parametrize("ksub", [1, 2])
+def test_tile_boundaries(M, N, K, g, bn, ksub):
     ldc = -(-N // 4) * 4
     p = synth.Problem("edge", M, N, K, BF16, FP32, 0, 1, 0, 1.0, 0.0, seed=M * 131 + N * 7 + K,
                       ldc=ldc).generate()
-    check_full(p, flags_for(g, bn))
+    check_full(p, flags_for(g, bn, ksub=ksub))
 
 
 @pytest.mark.parametrize("la", [0, 1])
 @pytest.mark.parametrize("lb", [0, 1])
 @pytest.mark.parametrize("lc", [0, 1])
 @pytest.mark.parametrize("ab,cd", [(BF16, FP32), (FP16, FP32), (BF16, BF16), (FP16, FP16)])
-@pytest.mark.parametrize("g,bn", [(1, 128), (2, 256)])
-def test_layouts_dtypes_alpha_beta(la, lb, lc, ab, cd, g, bn):
+@pytest.mark.parametrize("g,bn,ksub", [(1, 128, 2), (2, 256, 2), (2, 128, 1), (1, 256, 1)])
+def test_layouts_dtypes_alpha_beta(la, lb, lc, ab, cd, g, bn, ksub):
     M, N, K = 264, 328, 200
     p = synth.Problem("lay", M, N, K, ab, cd, la, lb, lc, -1.5, 0.75, seed=la + 2 * lb + 4 * lc + 8 * ab,
                       dist="normal" if ab == FP16 else "uniform")
     p.generate()
-    check_full(p, flags_for(g, bn))
+    check_full(p, flags_for(g, bn, ksub=ksub))
 
 
 @pytest.mark.parametrize("g,bn", TILE_SHAPES)
