@@ -156,6 +156,41 @@ exo_gemm_status_t exo_gemm_plan_preview(const exo_gemm_desc_t* desc, int32_t sm_
 /* Reports what the plan chose. */
 exo_gemm_status_t exo_gemm_get_info(exo_gemm_handle_t plan, exo_gemm_info_t* info);
 
+/*
+ * The same GEMM for callers that must not allocate device memory.  (The paper has
+ * no counterpart; this is a library convenience.)  Who needs it: code running
+ * where cudaMalloc is off limits or fails by design -- a process whose device
+ * memory is entirely owned by a framework's pool, a real-time loop that may not
+ * take the allocator's lock or its latency, a plug-in that is forbidden to
+ * allocate after initialisation.  exo_gemm_create calls cudaMalloc for the plan's
+ * 32-byte status block; this entry point needs no plan and calls no cudaMalloc,
+ * cudaFree or other allocating routine: it plans on the host stack and keeps the
+ * status block in a 256-byte device array that is part of the library image
+ * (every GPU that loads the library holds those 256 bytes until exit).
+ *
+ *   desc, A, B, C, alpha, beta, cuda_stream   as for exo_gemm_create + exo_gemm_run;
+ *             the caller still owns and passes all inputs and outputs.
+ *   detail    NULL: asynchronous, like exo_gemm_run.  Not NULL (host pointer to 8
+ *             words): the call waits for the stream, copies the status words there
+ *             and returns EXO_GEMM_ERR_DEVICE_TIMEOUT if a device-side wait gave up.
+ *
+ * Limit: the scratch a launch needs must fit the 256-byte array.  The status block
+ * is 32 bytes for every problem size, so every supported problem fits; a build
+ * whose status block is larger (the development trace build) is refused with
+ * EXO_GEMM_ERR_UNSUPPORTED.  Devices with ordinal >= 64 are refused the same way.
+ *
+ * The first call on a device looks up the array's device address
+ * (cudaGetSymbolAddress, once per device); make that first call before any
+ * stream capture.  All calls on a device share the one array, which keeps the last
+ * call's contents: each call clears the status words on cuda_stream before its
+ * kernel, so calls must not overlap on the GPU (two streams, or a plan-less call
+ * racing another) -- overlapping calls race on the status words.  Each call repeats
+ * the planning work of exo_gemm_create (a few attribute queries), so it costs a few
+ * microseconds more of host time than exo_gemm_run on a kept plan.
+ */
+exo_gemm_status_t exo_gemm_run_static(const exo_gemm_desc_t* desc, const void* A, const void* B, void* C,
+                                      float alpha, float beta, void* cuda_stream, uint32_t* detail);
+
 /* Frees the plan and its device status block.  NULL is a no-op returning OK. */
 exo_gemm_status_t exo_gemm_destroy(exo_gemm_handle_t plan);
 

@@ -18,7 +18,7 @@ ROW_MAJOR, COL_MAJOR = 0, 1
 EXPORTED_SYMBOLS = (
     "exo_gemm_validate", "exo_gemm_create", "exo_gemm_run", "exo_gemm_check", "exo_gemm_plan_preview",
     "exo_gemm_get_info", "exo_gemm_destroy", "exo_gemm_status_string", "exo_gemm_last_cuda_error",
-    "exo_gemm_schedule_enumerate", "exo_gemm_debug_set",
+    "exo_gemm_schedule_enumerate", "exo_gemm_debug_set", "exo_gemm_run_static",
 )
 
 
@@ -82,6 +82,9 @@ def lib():
                                                   ctypes.POINTER(i32), i64]
         L.exo_gemm_schedule_enumerate.restype = i64
         L.exo_gemm_debug_set.argtypes = [vp, i32, i64]
+        L.exo_gemm_run_static.argtypes = [ctypes.POINTER(Desc), vp, vp, vp, ctypes.c_float, ctypes.c_float, vp,
+                                          ctypes.POINTER(ctypes.c_uint32)]
+        L.exo_gemm_run_static.restype = ctypes.c_int
         for name in ("exo_gemm_validate", "exo_gemm_create", "exo_gemm_run", "exo_gemm_check",
                      "exo_gemm_plan_preview", "exo_gemm_get_info", "exo_gemm_destroy", "exo_gemm_debug_set"):
             getattr(L, name).restype = ctypes.c_int
@@ -148,6 +151,17 @@ def exo_gemm_last_cuda_error() -> int:
 
 def exo_gemm_debug_set(handle, timeout_ms: int, skip_k_block: int) -> int:
     return lib().exo_gemm_debug_set(handle, timeout_ms, skip_k_block)
+
+
+def exo_gemm_run_static(desc: Desc, a_ptr: int, b_ptr: int, c_ptr: int, alpha: float, beta: float,
+                        stream: int = 0, blocking: bool = False):
+    """The allocation-free GEMM entry point: no plan, no cudaMalloc (for callers that may not
+    allocate device memory).  Returns (status, detail words or None)."""
+    if blocking:
+        detail = (ctypes.c_uint32 * 8)()
+        st = lib().exo_gemm_run_static(ctypes.byref(desc), a_ptr, b_ptr, c_ptr, alpha, beta, stream, detail)
+        return st, list(detail)
+    return lib().exo_gemm_run_static(ctypes.byref(desc), a_ptr, b_ptr, c_ptr, alpha, beta, stream, None), None
 
 
 def exo_gemm_schedule_enumerate(tiles_m, tiles_n, band, along_m, num_workers, worker):

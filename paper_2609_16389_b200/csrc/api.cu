@@ -361,6 +361,112 @@ exo_gemm_status_t exo_gemm_check(exo_gemm_handle_t plan, uint32_t* detail) {
   return EXO_GEMM_ERR_DEVICE_TIMEOUT;
 }
 
+// ---------------------------------------------------------------------------------------
+// Allocation-free entry point.  The only global memory the kernel needs beyond A, B and C
+// is its status block; here that block lives in a file-scope device array instead of a
+// cudaMalloc'ed one.  In host code the array's name is only a host-side stand-in for the
+// device object: its device address comes from cudaGetSymbolAddress, once per device.
+constexpr size_t kStaticScratchBytes = 256;  // stated maximum; the status block needs kStatusBytes
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+uint32_t* g_static_ptr[kMaxDevices] = {};  // device address of g_static_scratch, per device
+
+// Set-up, once per device, with that device current.
+cudaError_t static_scratch_for_current_device(int device, uint32_t** out) {
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (!g_static_ptr[device]) {
+    void* ptr = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+    if (e != cudaSuccess) return e;
+    g_static_ptr[device] = static_cast<uint32_t*>(ptr);
+  }
+  *out = g_static_ptr[device];
+  return cudaSuccess;
+}
+}  // namespace
+
+exo_gemm_status_t exo_gemm_run_static(const exo_gemm_desc_t* desc, const void* A, const void* B, void* C,
+                                      float alpha, float beta, void* cuda_stream, uint32_t* detail) {
+  exo_gemm_status_t st = validate_desc(desc);
+  if (st != EXO_GEMM_OK) return st;
+  if (kStatusBytes > kStaticScratchBytes) return EXO_GEMM_ERR_UNSUPPORTED;  // scratch need beyond the static array
+
+  int device = desc->device;
+  cudaError_t e;
+  if (device < 0) {
+    e = cudaGetDevice(&device);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
+  if (device >= kMaxDevices) return EXO_GEMM_ERR_UNSUPPORTED;
+  DeviceGuard guard(device);
+  if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+  int major = 0, sms = 0;
+  e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (major != 10) return EXO_GEMM_ERR_ARCH;
+  e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (!get_encode_fn()) return EXO_GEMM_ERR_CUDA;
+
+  // a plan on the stack: same choices as exo_gemm_create, nothing allocated
+  exo_gemm_plan plan{};
+  plan.desc = *desc;
+  plan.canon = canonicalize(*desc);
+  plan.device = device;
+  plan.sm_count = sms;
+  plan.dbg_timeout_ms = 0;
+  plan.dbg_skip_k_block = -1;
+  const FlagOverrides ov = decode_flags(desc->flags);
+  int max_pairs = 0;
+  if (ov.cta_group != 1) {
+    KernelFn probe = pick_kernel(2, 256, 2, desc->c_dtype);
+    const int smem = smem_bytes_for(2, 256, 2);
+    e = cudaFuncSetAttribute((const void*)probe, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return cuda_fail(e);
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3((unsigned)sms & ~1u, 1, 1);
+    lc.blockDim = dim3(kNumThreads, 1, 1);
+    lc.dynamicSmemBytes = smem;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    lc.attrs = at;
+    lc.numAttrs = 1;
+    int n = 0;
+    e = cudaOccupancyMaxActiveClusters(&n, (const void*)probe, &lc);
+    if (e != cudaSuccess) return cuda_fail(e);
+    max_pairs = n < sms / 2 ? n : sms / 2;
+  }
+  plan.cfg = choose_config(plan.canon, ov, sms, max_pairs);
+  plan.kernel = pick_kernel(plan.cfg.cta_group, plan.cfg.tile_n, plan.cfg.ksub, desc->c_dtype);
+  plan.smem_bytes = smem_bytes_for(plan.cfg.cta_group, plan.cfg.tile_n, plan.cfg.ksub);
+  e = cudaFuncSetAttribute((const void*)plan.kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem_bytes);
+  if (e != cudaSuccess) return cuda_fail(e);
+
+  e = static_scratch_for_current_device(device, &plan.d_status);
+  if (e != cudaSuccess) return cuda_fail(e);
+  // the array keeps the last call's contents: the status words must start at zero
+  e = cudaMemsetAsync(plan.d_status, 0, kStatusBytes, (cudaStream_t)cuda_stream);
+  if (e != cudaSuccess) return cuda_fail(e);
+
+  st = exo_gemm_run(&plan, A, B, C, alpha, beta, cuda_stream);
+  if (st != EXO_GEMM_OK || !detail) return st;
+
+  // blocking mode: wait for the kernel and report what it recorded
+  e = cudaStreamSynchronize((cudaStream_t)cuda_stream);
+  if (e != cudaSuccess) return cuda_fail(e);
+  uint32_t h[8];
+  e = cudaMemcpy(h, plan.d_status, 32, cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return cuda_fail(e);
+  memcpy(detail, h, 32);
+  return h[0] == kStatusOk ? EXO_GEMM_OK : EXO_GEMM_ERR_DEVICE_TIMEOUT;
+}
+
 #ifdef EXO_GEMM_TRACE
 // Development aid: copies the clock stamps of CTA 0 (3 roles x 4096 x 2 int64) to the host.
 exo_gemm_status_t exo_gemm_debug_read_trace(exo_gemm_handle_t plan, long long* out) {
