@@ -46,6 +46,8 @@ typedef enum { EXO_GEMM_ROW_MAJOR = 0, EXO_GEMM_COL_MAJOR = 1 } exo_gemm_layout_
  *   bit  10     raster direction: 0 = library choice, set = bands along M instead of N
  *   bits 12..19 grid limit: launch at most this many CTAs (multiple of cta_group), 0 = all SMs
  *   bits 20..21 k sub-blocks (of 64 elements) per pipeline stage: 1 or 2
+ *   bits 22..23 staging buffers per epilogue warp: 1 or 2
+ *   bits 24..27 upper limit on the pipeline depth (2..8)
  */
 #define EXO_GEMM_FLAG_CTA_GROUP(g)  ((uint32_t)(g) & 3u)
 #define EXO_GEMM_FLAG_TILE_N(n)     ((((uint32_t)(n) / 64u) & 15u) << 2)
@@ -53,6 +55,8 @@ typedef enum { EXO_GEMM_ROW_MAJOR = 0, EXO_GEMM_COL_MAJOR = 1 } exo_gemm_layout_
 #define EXO_GEMM_FLAG_BANDS_ALONG_M (1u << 10)
 #define EXO_GEMM_FLAG_GRID_LIMIT(c) (((uint32_t)(c) & 255u) << 12)
 #define EXO_GEMM_FLAG_K_SUBBLOCKS(k) (((uint32_t)(k) & 3u) << 20)
+#define EXO_GEMM_FLAG_EPI_BUFFERS(b) (((uint32_t)(b) & 3u) << 22)
+#define EXO_GEMM_FLAG_MAX_STAGES(s) (((uint32_t)(s) & 15u) << 24)
 
 /*
  * Problem descriptor.  Logical shapes: A is M x K, B is K x N, C is M x N.
@@ -92,7 +96,8 @@ typedef struct {
   int32_t swapped;        /* 1: column-major C computed as C^T = B^T A^T                       */
   int32_t sm_count;
   int32_t kernel_launches_per_run; /* 1, or 0 for an empty problem                             */
-  int32_t reserved[5];
+  int32_t epilogue_buffers; /* staging buffers per epilogue warp (1 or 2)                      */
+  int32_t reserved[4];
 } exo_gemm_info_t;
 
 /*

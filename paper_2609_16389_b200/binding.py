@@ -28,6 +28,8 @@ def flag_band(b): return (b & 15) << 6
 FLAG_BANDS_ALONG_M = 1 << 10
 def flag_grid_limit(c): return (c & 255) << 12
 def flag_k_subblocks(k): return (k & 3) << 20
+def flag_epi_buffers(b): return (b & 3) << 22
+def flag_max_stages(s): return (s & 15) << 24
 
 
 class Desc(ctypes.Structure):
@@ -43,7 +45,7 @@ class Info(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "cta_group", "tile_m", "tile_n", "tile_k", "stages", "grid", "smem_bytes", "tmem_columns",
         "tiles_m", "tiles_n", "raster_along_m", "raster_band", "swapped", "sm_count",
-        "kernel_launches_per_run")] + [("reserved", ctypes.c_int32 * 5)]
+        "kernel_launches_per_run", "epilogue_buffers")] + [("reserved", ctypes.c_int32 * 4)]
 
     def as_dict(self):
         return {n: getattr(self, n) for n, _ in self._fields_ if n != "reserved"}

@@ -140,6 +140,7 @@ void fill_info(const exo_gemm_plan* p, exo_gemm_info_t* info) {
   info->swapped = p->canon.swapped;
   info->sm_count = p->sm_count;
   info->kernel_launches_per_run = (p->canon.M == 0 || p->canon.N == 0) ? 0 : 1;
+  info->epilogue_buffers = p->cfg.epi_bufs;
 }
 
 }  // namespace
@@ -192,7 +193,7 @@ exo_gemm_status_t exo_gemm_plan_preview(const exo_gemm_desc_t* desc, int32_t sm_
   p.canon = canonicalize(*desc);
   p.sm_count = sm_count;
   p.cfg = choose_config(p.canon, decode_flags(desc->flags), sm_count, sm_count / 2);
-  p.smem_bytes = smem_bytes_for(p.cfg.cta_group, p.cfg.tile_n, p.cfg.ksub);
+  p.smem_bytes = smem_bytes_for(p.cfg.cta_group, p.cfg.tile_n, p.cfg.ksub, p.cfg.stages, p.cfg.epi_bufs);
   fill_info(&p, info);
   return EXO_GEMM_OK;
 }
@@ -232,7 +233,7 @@ exo_gemm_status_t exo_gemm_create(exo_gemm_handle_t* out, const exo_gemm_desc_t*
   int max_pairs = 0;
   if (ov.cta_group != 1) {
     KernelFn probe = pick_kernel(2, 256, 2, desc->c_dtype);
-    const int smem = smem_bytes_for(2, 256, 2);
+    const int smem = kSmemLimit - 1024;  // every plan's shared-memory request is close to the limit
     e = cudaFuncSetAttribute((const void*)probe, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) { delete p; return cuda_fail(e); }
     cudaLaunchConfig_t lc{};
@@ -254,7 +255,7 @@ exo_gemm_status_t exo_gemm_create(exo_gemm_handle_t* out, const exo_gemm_desc_t*
 
   p->cfg = choose_config(p->canon, ov, sms, max_pairs);
   p->kernel = pick_kernel(p->cfg.cta_group, p->cfg.tile_n, p->cfg.ksub, desc->c_dtype);
-  p->smem_bytes = smem_bytes_for(p->cfg.cta_group, p->cfg.tile_n, p->cfg.ksub);
+  p->smem_bytes = smem_bytes_for(p->cfg.cta_group, p->cfg.tile_n, p->cfg.ksub, p->cfg.stages, p->cfg.epi_bufs);
   e = cudaFuncSetAttribute((const void*)p->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, p->smem_bytes);
   if (e != cudaSuccess) { delete p; return cuda_fail(e); }
   e = cudaMalloc((void**)&p->d_status, kStatusBytes);
@@ -300,6 +301,8 @@ exo_gemm_status_t exo_gemm_run(exo_gemm_handle_t plan, const void* A, const void
   const int stage_k = kBlockK * cfg.ksub;
   prm.num_k_blocks = read_ab ? (int32_t)((cn.K + stage_k - 1) / stage_k) : 0;
   prm.raster = Raster{cfg.tiles_m, cfg.tiles_n, cfg.band, cfg.along_m};
+  prm.stages = cfg.stages;
+  prm.epi_bufs = cfg.epi_bufs;
   prm.alpha = read_ab ? alpha : 0.f;
   prm.beta = beta;
   prm.idesc = make_idesc(d.ab_dtype, cn.a_mn_major, cn.b_mn_major, 128 * cfg.cta_group, cfg.tile_n);
@@ -423,7 +426,7 @@ exo_gemm_status_t exo_gemm_run_static(const exo_gemm_desc_t* desc, const void* A
   int max_pairs = 0;
   if (ov.cta_group != 1) {
     KernelFn probe = pick_kernel(2, 256, 2, desc->c_dtype);
-    const int smem = smem_bytes_for(2, 256, 2);
+    const int smem = kSmemLimit - 1024;  // every plan's shared-memory request is close to the limit
     e = cudaFuncSetAttribute((const void*)probe, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return cuda_fail(e);
     cudaLaunchConfig_t lc{};
@@ -444,7 +447,7 @@ exo_gemm_status_t exo_gemm_run_static(const exo_gemm_desc_t* desc, const void* A
   }
   plan.cfg = choose_config(plan.canon, ov, sms, max_pairs);
   plan.kernel = pick_kernel(plan.cfg.cta_group, plan.cfg.tile_n, plan.cfg.ksub, desc->c_dtype);
-  plan.smem_bytes = smem_bytes_for(plan.cfg.cta_group, plan.cfg.tile_n, plan.cfg.ksub);
+  plan.smem_bytes = smem_bytes_for(plan.cfg.cta_group, plan.cfg.tile_n, plan.cfg.ksub, plan.cfg.stages, plan.cfg.epi_bufs);
   e = cudaFuncSetAttribute((const void*)plan.kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem_bytes);
   if (e != cudaSuccess) return cuda_fail(e);
 

@@ -10,9 +10,10 @@
 //                      memory into one of two TMEM accumulators; tcgen05.commit
 //                      releases stages and publishes finished accumulators
 //   warp 1             owns the TMEM allocation
-//   warps 2..5         epilogue: tcgen05.ld the accumulator (warp w reads TMEM
-//                      lanes 32*(w%4)..), alpha*acc + beta*C_in in fp32, convert,
-//                      write a 128B-swizzled staging buffer, TMA store
+//   warps 2..9         epilogue: tcgen05.ld the accumulator (warp w reads TMEM
+//                      lanes 32*(w%4).. and every other 128-byte column chunk),
+//                      alpha*acc + beta*C_in in fp32, convert, write a 128B-swizzled
+//                      staging buffer, TMA store
 //
 // The structure follows the kernel class of the paper's Section 6 (persistent,
 // warp-specialised, TMA + swizzled shared memory + asynchronous tensor-core
@@ -121,7 +122,6 @@ template <int CTA_GROUP, int BN, int OUT, int KSUB>
 __global__ void __launch_bounds__(kNumThreads, 1)
 exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                 const __grid_constant__ CUtensorMap tm_c, const GemmParams p) {
-  constexpr int STAGES = max_stages(CTA_GROUP, BN, KSUB);
   constexpr int STAGE_K = kBlockK * KSUB;            // k-elements per stage
   constexpr int B_ROWS = BN / CTA_GROUP;             // rows of the B tile this CTA stages
   constexpr int STAGE_BYTES = stage_bytes(CTA_GROUP, BN, KSUB);
@@ -131,19 +131,21 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   constexpr int NCHUNK = BN / CW;
   constexpr bool PAIR = CTA_GROUP == 2;
   static_assert(BN == 64 || BN == 128 || BN == 256, "tile N");
-  static_assert(STAGES >= 2, "ring too shallow");
+  const uint32_t STAGES = (uint32_t)p.stages;         // ring depth, chosen by the host plan
+  const uint32_t EPI_BUFS = (uint32_t)p.epi_bufs;     // staging buffers per epilogue warp (1 or 2)
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;  // swizzle atoms are 1 KB
   const uint32_t stage0 = smem_base;
   const uint32_t epi0 = smem_base + STAGES * STAGE_BYTES;
-  const uint32_t bar0 = epi0 + kEpiWarps * kEpiBufsPerWarp * kEpiBufBytes;
+  const uint32_t bar0 = epi0 + kEpiWarps * EPI_BUFS * kEpiBufBytes;
   auto full_bar = [&](uint32_t s) { return bar0 + 8u * s; };
-  auto empty_bar = [&](uint32_t s) { return bar0 + 8u * (STAGES + s); };
-  auto tfull_bar = [&](uint32_t a) { return bar0 + 8u * (2 * STAGES + a); };
-  auto tempty_bar = [&](uint32_t a) { return bar0 + 8u * (2 * STAGES + 2 + a); };
-  auto cin_bar = [&](uint32_t w, uint32_t b) { return bar0 + 8u * (2 * STAGES + 4 + 2 * w + b); };
-  const uint32_t tmem_slot = bar0 + 8u * (2 * STAGES + 12);
+  auto empty_bar = [&](uint32_t s) { return bar0 + 8u * (kMaxStages + s); };
+  auto tfull_bar = [&](uint32_t a) { return bar0 + 8u * (2 * kMaxStages + a); };
+  auto tempty_bar = [&](uint32_t a) { return bar0 + 8u * (2 * kMaxStages + 2 + a); };
+  auto cin_bar = [&](uint32_t w, uint32_t b) { return bar0 + 8u * (2 * kMaxStages + 4 + kMaxEpiBufs * w + b); };
+  const uint32_t tmem_slot = bar0 + 8u * (2 * kMaxStages + 4 + kMaxEpiBufs * kEpiWarps);
+  static_assert(8 * (2 * kMaxStages + 4 + kMaxEpiBufs * kEpiWarps) + 4 <= kBarrierBytes, "barrier area");
 
   const uint32_t warp = threadIdx.x >> 5;
   const uint32_t lane = threadIdx.x & 31u;
@@ -153,6 +155,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   const int64_t total_tiles = raster_total(p.raster);
   const int32_t nkb = p.num_k_blocks;
 
+  if (threadIdx.x == 0) EXO_TRACE(2, 4095, 0, 4096);
   // ---------------------------------------------------------------- setup
   if (threadIdx.x == 0) {
     for (uint32_t s = 0; s < STAGES; ++s) {
@@ -164,7 +167,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       ptx::mbar_init(tempty_bar(a), kEpiWarps * CTA_GROUP);
     }
     for (uint32_t w = 0; w < kEpiWarps; ++w)
-      for (uint32_t b = 0; b < 2; ++b) ptx::mbar_init(cin_bar(w, b), 1);
+      for (uint32_t b = 0; b < kMaxEpiBufs; ++b) ptx::mbar_init(cin_bar(w, b), 1);
     ptx::fence_mbar_init();
     ptx::prefetch_tensormap(&tm_a);
     ptx::prefetch_tensormap(&tm_b);
@@ -185,6 +188,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot) : "memory");
 
   bool ok = true;
+  if (threadIdx.x == 0) EXO_TRACE(2, 4094, 0, 4096);
 
   if (warp == 0) {
     // ============================================================ producer
@@ -298,27 +302,36 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     }
   } else {
     // ============================================================ epilogue
-    const uint32_t quad = warp & 3u;  // TMEM lanes 32*quad .. 32*quad+31 belong to this warp
+    // Warp w reads TMEM lanes 32*(w%4)..+31 (a hardware rule) and, of the tile's column
+    // chunks (128 bytes of C per row each), those with index == half (mod 2).
+    constexpr int UPC = CW / 32;                       // 32-column TMEM loads per chunk
+    const uint32_t quad = warp & 3u;
     const uint32_t ew = warp - 2u;
-    const uint32_t buf0 = epi0 + ew * (kEpiBufsPerWarp * kEpiBufBytes);
+    const int32_t half = (int32_t)(ew >> 2);
+    const uint32_t buf0 = epi0 + ew * EPI_BUFS * kEpiBufBytes;
     const uint32_t tempty0 = PAIR ? ptx::map_to_cta(tempty_bar(0), 0) : tempty_bar(0);
     const bool has_beta = p.beta != 0.f;
     const bool has_acc = nkb > 0;
+    const bool scale = p.alpha != 1.f;
     const float alpha = p.alpha, beta = p.beta;
-    const uint32_t row_off = lane * 128u;
-    const uint32_t sw = lane & 7u;
-    uint32_t g = 0;  // running chunk counter: staging buffer g & 1, its C_in barrier phase (g >> 1) & 1
+    uint32_t piece[8];  // where this thread's eight 16-byte pieces of a 128-byte row go (swizzled)
+#pragma unroll
+    for (int j = 0; j < 8; ++j) piece[j] = buf0 + lane * 128u + (((uint32_t)j ^ (lane & 7u)) << 4);
+    // running chunk counter: staging buffer g % EPI_BUFS, its C_in barrier phase (g / EPI_BUFS) & 1
+    uint32_t g = 0;
+    const bool two_bufs = EPI_BUFS == 2;
     uint32_t acc = 0, acc_ph = 0;
 
     for (int64_t t = worker; t < total_tiles; t += num_workers) {
       const TileCoord tc = raster_decode(p.raster, t);
       const int32_t row0 = tc.m * (kBlockM * CTA_GROUP) + (int32_t)cta_rank * kBlockM + (int32_t)quad * 32;
       const int32_t col0 = tc.n * BN;
-      int32_t nch = 0;
+      int32_t nch = 0;  // chunks of this tile that hold any valid column, if this warp's rows exist
       if (row0 < p.M) {
         nch = (p.N - col0 + CW - 1) / CW;
         if (nch > NCHUNK) nch = NCHUNK;
       }
+      const int32_t mine = nch > half ? (nch - half + 1) / 2 : 0;  // how many of them are this warp's
       if (has_acc) {
         ok = wait_barrier<PAIR>(tfull_bar(acc), acc_ph, p, WaitSite{kRoleEpilogue, 200 + acc, (uint32_t)t, 0});
         ok = __all_sync(0xffffffffu, ok);
@@ -329,101 +342,132 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       auto release_acc = [&]() {
         ptx::tc_fence_before_sync();
         __syncwarp();
-        if (lane == 0) {
+        if (ptx::elect_one()) {
           if constexpr (PAIR) ptx::mbar_arrive_cluster(tempty0 + 8u * acc);
           else ptx::mbar_arrive(tempty0 + 8u * acc);
         }
       };
-      auto issue_cin = [&](uint32_t gg, int32_t chunk) {  // lane 0 only
-        const uint32_t b = gg & 1u;
-        ptx::mbar_arrive_expect_tx(cin_bar(ew, b), kEpiBufBytes);
-        ptx::tma_load_2d(buf0 + b * kEpiBufBytes, &tm_c, col0 + chunk * CW, row0, cin_bar(ew, b));
+      const uint32_t tacc = tmem_base + ((quad * 32u) << 16) + acc * BN;
+      // unit q of this warp's i-th chunk: 32 accumulator columns
+      auto tmem_load = [&](uint32_t (&dst)[32], int32_t i, int32_t q) {  // asynchronous until tmem_ld_wait()
+        ptx::tmem_ld_32x32(tacc + (uint32_t)((half + 2 * i) * CW + q * 32), dst);
       };
-      if (nch == 0) {
-        if (has_acc) release_acc();
-      } else if (has_beta) {
-        if (lane == 0) {
+      if (mine == 0 && has_acc) release_acc();
+      auto issue_cin = [&](uint32_t gg, int32_t i) {  // elected lane only: C_in of this warp's i-th chunk
+        const uint32_t b = two_bufs ? (gg & 1u) : 0u;
+        ptx::mbar_arrive_expect_tx(cin_bar(ew, b), kEpiBufBytes);
+        ptx::tma_load_2d(buf0 + b * kEpiBufBytes, &tm_c, col0 + (half + 2 * i) * CW, row0, cin_bar(ew, b));
+      };
+      if (mine > 0 && has_beta && two_bufs) {
+        if (ptx::elect_one()) {
           ptx::bulk_wait_read<0>();
           issue_cin(g, 0);
         }
       }
-      for (int32_t c = 0; c < nch; ++c) {
-        const uint32_t buf = buf0 + (g & 1u) * kEpiBufBytes;
-        if (has_beta) {
-          if (c + 1 < nch && lane == 0) {
-            ptx::bulk_wait_read<0>();  // the other buffer's last store has been read out
-            issue_cin(g + 1, c + 1);
-          }
-          ok = wait_barrier<false>(cin_bar(ew, g & 1u), (g >> 1) & 1u, p,
-                                   WaitSite{kRoleEpilogueCin, 300 + (g & 1u), (uint32_t)t, (uint32_t)c});
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
-        } else {
-          if (lane == 0) ptx::bulk_wait_read<1>();  // this buffer's last store (two chunks ago) is read out
-          __syncwarp();
-        }
-
-        uint32_t v[CW];
-        if (has_acc) {
-          const uint32_t taddr = tmem_base + ((quad * 32u) << 16) + acc * BN + c * CW;
-          ptx::tmem_ld_32x32(taddr, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
-          if constexpr (CW == 64) ptx::tmem_ld_32x32(taddr + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
-          ptx::tmem_ld_wait();
-          if (c == nch - 1) release_acc();  // last read of this accumulator: hand it back early
-        } else {
-#pragma unroll
-          for (int i = 0; i < CW; ++i) v[i] = 0u;
-        }
-
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {  // eight 16-byte pieces of this thread's 128-byte row segment
-          const uint32_t addr = buf + row_off + ((j ^ sw) << 4);
-          if constexpr (OUT == kOutFp32) {
-            float x0 = alpha * __uint_as_float(v[4 * j + 0]);
-            float x1 = alpha * __uint_as_float(v[4 * j + 1]);
-            float x2 = alpha * __uint_as_float(v[4 * j + 2]);
-            float x3 = alpha * __uint_as_float(v[4 * j + 3]);
+      // The chunk loop stays rolled: eight warps interleave, which hides the TMEM load
+      // latency as well as a software pipeline did, at a fraction of the code size.
+      uint32_t v[UPC][32];
+#pragma unroll 1
+      for (int32_t i = 0; i < mine; ++i) {
+        if (ok) {
+          const int32_t col = col0 + (half + 2 * i) * CW;
+          const uint32_t b = two_bufs ? (g & 1u) : 0u;
+          const uint32_t boff = b * kEpiBufBytes;
+          // A staging buffer is free once the store that last used it has read it out.
+          if (ptx::elect_one()) {
             if (has_beta) {
-              uint32_t c0, c1, c2, c3;
-              ptx::ld_shared_v4(addr, c0, c1, c2, c3);
-              x0 = fmaf(beta, __uint_as_float(c0), x0);
-              x1 = fmaf(beta, __uint_as_float(c1), x1);
-              x2 = fmaf(beta, __uint_as_float(c2), x2);
-              x3 = fmaf(beta, __uint_as_float(c3), x3);
+              if (two_bufs) {  // prefetch the next chunk's C_in into the other buffer
+                if (i + 1 < mine) {
+                  ptx::bulk_wait_read<0>();
+                  issue_cin(g + 1, i + 1);
+                }
+              } else {
+                ptx::bulk_wait_read<0>();
+                issue_cin(g, i);
+              }
+            } else {
+              if (two_bufs) ptx::bulk_wait_read<1>();
+              else ptx::bulk_wait_read<0>();
             }
-            ptx::st_shared_v4(addr, __float_as_uint(x0), __float_as_uint(x1), __float_as_uint(x2),
-                              __float_as_uint(x3));
-          } else {
-            float x[8];
+          }
+          __syncwarp();
+          if (has_beta) {
+            ok = wait_barrier<false>(cin_bar(ew, b), (two_bufs ? (g >> 1) : g) & 1u, p,
+                                     WaitSite{kRoleEpilogueCin, 300 + b, (uint32_t)t, (uint32_t)i});
+            ok = __all_sync(0xffffffffu, ok);
+          }
 #pragma unroll
-            for (int i = 0; i < 8; ++i) x[i] = alpha * __uint_as_float(v[8 * j + i]);
-            if (has_beta) {
-              uint32_t cw[4];
-              ptx::ld_shared_v4(addr, cw[0], cw[1], cw[2], cw[3]);
+          for (int32_t q = 0; q < UPC; ++q) {
+            uint32_t(&cur)[32] = v[q];
+            if (has_acc) {
+              if (q == 0) {
 #pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                const float2 cc = unpack2<OUT>(cw[i]);
-                x[2 * i] = fmaf(beta, cc.x, x[2 * i]);
-                x[2 * i + 1] = fmaf(beta, cc.y, x[2 * i + 1]);
+                for (int32_t qq = 0; qq < UPC; ++qq) tmem_load(v[qq], i, qq);
+                ptx::tmem_ld_wait();
+                if (i + 1 == mine) release_acc();  // this warp's last read of the accumulator: hand it back early
+              }
+            } else {
+#pragma unroll
+              for (int k = 0; k < 32; ++k) cur[k] = 0u;
+            }
+            if (scale) {
+#pragma unroll
+              for (int k = 0; k < 32; ++k) cur[k] = __float_as_uint(alpha * __uint_as_float(cur[k]));
+            }
+            if (ok) {
+              if constexpr (OUT == kOutFp32) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                  if (has_beta) {
+                    uint32_t c0, c1, c2, c3;
+                    ptx::ld_shared_v4(piece[j] + boff, c0, c1, c2, c3);
+                    cur[4 * j + 0] = __float_as_uint(fmaf(beta, __uint_as_float(c0), __uint_as_float(cur[4 * j + 0])));
+                    cur[4 * j + 1] = __float_as_uint(fmaf(beta, __uint_as_float(c1), __uint_as_float(cur[4 * j + 1])));
+                    cur[4 * j + 2] = __float_as_uint(fmaf(beta, __uint_as_float(c2), __uint_as_float(cur[4 * j + 2])));
+                    cur[4 * j + 3] = __float_as_uint(fmaf(beta, __uint_as_float(c3), __uint_as_float(cur[4 * j + 3])));
+                  }
+                  ptx::st_shared_v4(piece[j] + boff, cur[4 * j + 0], cur[4 * j + 1], cur[4 * j + 2], cur[4 * j + 3]);
+                }
+              } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {  // 32 columns = four 16-byte pieces of 8 halves
+                  const uint32_t addr = piece[4 * q + j] + boff;
+                  float x[8];
+#pragma unroll
+                  for (int k = 0; k < 8; ++k) x[k] = __uint_as_float(cur[8 * j + k]);
+                  if (has_beta) {
+                    uint32_t cw[4];
+                    ptx::ld_shared_v4(addr, cw[0], cw[1], cw[2], cw[3]);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                      const float2 cc = unpack2<OUT>(cw[k]);
+                      x[2 * k] = fmaf(beta, cc.x, x[2 * k]);
+                      x[2 * k + 1] = fmaf(beta, cc.y, x[2 * k + 1]);
+                    }
+                  }
+                  ptx::st_shared_v4(addr, pack2<OUT>(x[0], x[1]), pack2<OUT>(x[2], x[3]), pack2<OUT>(x[4], x[5]),
+                                    pack2<OUT>(x[6], x[7]));
+                }
               }
             }
-            ptx::st_shared_v4(addr, pack2<OUT>(x[0], x[1]), pack2<OUT>(x[2], x[3]), pack2<OUT>(x[4], x[5]),
-                              pack2<OUT>(x[6], x[7]));
+          }
+          if (ok) {
+            ptx::fence_proxy_async_smem();  // generic-proxy writes -> visible to the TMA store
+            __syncwarp();
+            if (ptx::elect_one()) {
+              ptx::tma_store_2d(&tm_c, col, row0, buf0 + boff);
+              ptx::bulk_commit();
+            }
+            ++g;
           }
         }
-        ptx::fence_proxy_async_smem();  // generic-proxy writes -> visible to the TMA store
-        __syncwarp();
-        if (lane == 0) {
-          ptx::tma_store_2d(&tm_c, col0 + c * CW, row0, buf);
-          ptx::bulk_commit();
-        }
-        ++g;
       }
       if (!ok) break;
       if (warp == 2 && lane == 0) EXO_TRACE(2, (t - worker) / num_workers, 1, 4096);
       if ((acc ^= 1u) == 0u) acc_ph ^= 1u;
     }
-    if (lane == 0) ptx::bulk_wait<0>();  // all stores of this warp have completed
+    __syncwarp();
+    if (ptx::elect_one()) ptx::bulk_wait<0>();  // all stores of this warp have completed
     __syncwarp();
   }
 
@@ -443,6 +487,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     ptx::tc_fence_after_sync();
     ptx::tmem_dealloc<CTA_GROUP>(tmem_base, TMEM_COLS);
   }
+  if (threadIdx.x == 0) EXO_TRACE(2, 4095, 1, 4096);
 }
 
 }  // namespace exo

@@ -10,10 +10,11 @@ namespace exo {
 constexpr int kBlockM = 128;        // rows of C per CTA (one TMEM lane per row)
 constexpr int kBlockK = 64;         // elements of K per sub-block: 128 bytes = one swizzle span
 constexpr int kUmmaK = 16;          // K of one tcgen05.mma for 16-bit inputs
-constexpr int kNumThreads = 192;    // warp 0 producer, warp 1 MMA issuer + TMEM owner, warps 2..5 epilogue
-constexpr int kEpiWarps = 4;
+constexpr int kNumThreads = 320;    // warp 0 producer, warp 1 MMA issuer + TMEM owner, warps 2..9 epilogue
+constexpr int kEpiWarps = 8;        // two per TMEM lane quadrant, each taking every other column chunk
 constexpr int kEpiBufBytes = 4096;  // one staging buffer: 32 rows x 128 bytes
-constexpr int kEpiBufsPerWarp = 2;
+constexpr int kMaxEpiBufs = 2;      // staging buffers per epilogue warp: 1 or 2 (chosen per plan)
+constexpr int kMaxStages = 8;
 constexpr int kSmemLimit = 232448;  // 227 KB opt-in limit per CTA
 constexpr int kBarrierBytes = 512;
 constexpr int kATileBytes = kBlockM * kBlockK * 2;  // 16 KB
@@ -29,10 +30,11 @@ EXO_CX int stage_bytes(int cta_group, int bn, int ksub) {
   return ksub * (kATileBytes + (bn / cta_group) * kBlockK * 2);
 }
 
-EXO_CX int max_stages(int cta_group, int bn, int ksub) {
-  return (kSmemLimit - 1024 /*alignment slack*/ - kBarrierBytes -
-          kEpiWarps * kEpiBufsPerWarp * kEpiBufBytes) /
-         stage_bytes(cta_group, bn, ksub);
+// Stages that fit beside `epi_bufs` staging buffers per epilogue warp.
+EXO_CX int max_stages(int cta_group, int bn, int ksub, int epi_bufs) {
+  const int n = (kSmemLimit - 1024 /*alignment slack*/ - kBarrierBytes - kEpiWarps * epi_bufs * kEpiBufBytes) /
+                stage_bytes(cta_group, bn, ksub);
+  return n > kMaxStages ? kMaxStages : n;
 }
 
 // How one operand is staged.  K-major: per 64-k sub-block one TMA box {64 k, rows},
@@ -62,6 +64,8 @@ enum WaitRole : uint32_t {
 struct GemmParams {
   int32_t M, N, K;          // canonical problem (C row-major; operands possibly swapped)
   int32_t num_k_blocks;     // ceil(K / (64 * ksub)), or 0 when alpha == 0 / K == 0
+  int32_t stages;           // depth of the operand ring (2 .. kMaxStages)
+  int32_t epi_bufs;         // staging buffers per epilogue warp (1 or 2)
   Raster raster;
   float alpha, beta;
   uint32_t idesc;           // tcgen05 instruction descriptor

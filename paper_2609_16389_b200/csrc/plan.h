@@ -12,6 +12,8 @@ namespace exo {
 inline int elem_bytes(int dtype) { return dtype == EXO_GEMM_FP32 ? 4 : 2; }
 
 struct FlagOverrides {
+  int epi_bufs;    // 0 = auto
+  int stages;      // 0 = as many as fit, else an upper limit
   int ksub;        // 0 = auto
   int cta_group;   // 0 = auto
   int tile_n;      // 0 = auto
@@ -28,6 +30,8 @@ inline FlagOverrides decode_flags(uint32_t f) {
   o.along_m = (int)((f >> 10) & 1u);
   o.grid_limit = (int)((f >> 12) & 255u);
   o.ksub = (int)((f >> 20) & 3u);
+  o.epi_bufs = (int)((f >> 22) & 3u);
+  o.stages = (int)((f >> 24) & 15u);
   return o;
 }
 
@@ -51,8 +55,9 @@ inline exo_gemm_status_t validate_desc(const exo_gemm_desc_t* d) {
   if (d->lda < extent(d->a_layout, d->M, d->K) || d->ldb < extent(d->b_layout, d->K, d->N) ||
       d->ldc < extent(d->c_layout, d->M, d->N) || d->lda > kMaxLd || d->ldb > kMaxLd || d->ldc > kMaxLd)
     return EXO_GEMM_ERR_INVALID_ARG;
-  if (d->flags >> 22) return EXO_GEMM_ERR_INVALID_ARG;
-  if (((d->flags >> 20) & 3u) == 3u) return EXO_GEMM_ERR_INVALID_ARG;
+  if (d->flags >> 28) return EXO_GEMM_ERR_INVALID_ARG;
+  if (((d->flags >> 20) & 3u) == 3u || ((d->flags >> 22) & 3u) == 3u) return EXO_GEMM_ERR_INVALID_ARG;
+  if (((d->flags >> 24) & 15u) == 1u || ((d->flags >> 24) & 15u) > (uint32_t)kMaxStages) return EXO_GEMM_ERR_INVALID_ARG;
   if (d->flags & (1u << 11)) return EXO_GEMM_ERR_INVALID_ARG;
   const FlagOverrides o = decode_flags(d->flags);
   if (o.cta_group == 3) return EXO_GEMM_ERR_INVALID_ARG;
@@ -100,7 +105,7 @@ inline Canonical canonicalize(const exo_gemm_desc_t& d) {
 }
 
 struct TileConfig {
-  int cta_group, tile_n, ksub, stages;
+  int cta_group, tile_n, ksub, stages, epi_bufs;
   int tiles_m, tiles_n;
   int band, along_m;
   int workers;  // CTA groups launched
@@ -155,7 +160,14 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
   cfg.cta_group = best_g;
   cfg.tile_n = best_n;
   cfg.ksub = o.ksub ? o.ksub : default_ksub(best_g, best_n);
-  cfg.stages = max_stages(best_g, best_n, cfg.ksub);
+  // Two staging buffers per epilogue warp let a warp fill one while the TMA store still
+  // reads the other; they cost 32 KB of ring.  Take them when at least 3 stages remain.
+  // Short K: the epilogue bounds a tile, so staging depth matters more than ring depth.
+  const bool want_two = max_stages(best_g, best_n, cfg.ksub, 2) >= 5 ||
+                        (c.K <= 1024 && max_stages(best_g, best_n, cfg.ksub, 2) >= 3);
+  cfg.epi_bufs = o.epi_bufs ? o.epi_bufs : (want_two ? 2 : 1);
+  cfg.stages = max_stages(best_g, best_n, cfg.ksub, cfg.epi_bufs);
+  if (o.stages && o.stages < cfg.stages) cfg.stages = o.stages < 2 ? 2 : o.stages;
   cfg.tiles_m = (int)((c.M + 128 * best_g - 1) / (128 * best_g));
   cfg.tiles_n = (int)((c.N + best_n - 1) / best_n);
   int64_t workers = best_g == 2 ? max_pairs : sm_count;
@@ -178,9 +190,8 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
   return cfg;
 }
 
-inline int smem_bytes_for(int cta_group, int bn, int ksub) {
-  return 1024 + max_stages(cta_group, bn, ksub) * stage_bytes(cta_group, bn, ksub) +
-         kEpiWarps * kEpiBufsPerWarp * kEpiBufBytes + kBarrierBytes;
+inline int smem_bytes_for(int cta_group, int bn, int ksub, int stages, int epi_bufs) {
+  return 1024 + stages * stage_bytes(cta_group, bn, ksub) + kEpiWarps * epi_bufs * kEpiBufBytes + kBarrierBytes;
 }
 
 // tcgen05 instruction descriptor for kind::f16 with fp32 accumulation.

@@ -72,7 +72,10 @@ def test_validate_rejects_bad_arguments():
     assert B.exo_gemm_validate(good(flags=3)) == B.ERR_INVALID_ARG                       # cta_group 3
     assert B.exo_gemm_validate(good(flags=B.flag_tile_n(192))) == B.ERR_INVALID_ARG
     assert B.exo_gemm_validate(good(flags=B.flag_cta_group(2) | B.flag_tile_n(64))) == B.ERR_INVALID_ARG
-    assert B.exo_gemm_validate(good(flags=1 << 25)) == B.ERR_INVALID_ARG
+    assert B.exo_gemm_validate(good(flags=1 << 28)) == B.ERR_INVALID_ARG
+    assert B.exo_gemm_validate(good(flags=B.flag_max_stages(1))) == B.ERR_INVALID_ARG
+    assert B.exo_gemm_validate(good(flags=B.flag_max_stages(9))) == B.ERR_INVALID_ARG
+    assert B.exo_gemm_validate(good(flags=B.flag_epi_buffers(3))) == B.ERR_INVALID_ARG
 
 
 def test_validate_unsupported_but_legal_blas_calls():
@@ -114,8 +117,9 @@ def test_plan_preview_geometry_and_overrides():
         assert (i["cta_group"], i["tile_n"]) == (g, bn)
         assert i["tiles_m"] == -(-1000 // (128 * g)) and i["tiles_n"] == -(-520 // bn)
         assert i["grid"] == min(148 // g, i["tiles_m"] * i["tiles_n"]) * g
-        assert i["tile_k"] in (64, 128) and i["stages"] >= 2
-        assert i["stages"] * (i["tile_k"] // 64) * (16384 + bn // g * 128) + 32768 + 1536 <= 232448
+        assert i["tile_k"] in (64, 128) and i["stages"] >= 2 and i["epilogue_buffers"] in (1, 2)
+        assert (i["stages"] * (i["tile_k"] // 64) * (16384 + bn // g * 128) + 32768 * i["epilogue_buffers"] + 1536
+                == i["smem_bytes"] <= 232448)
     # column-major C is computed as the transposed product
     st, info = B.exo_gemm_plan_preview(good(M=512, N=2048, K=64, c_layout=1, ldc=512), 148)
     i = info.as_dict()
@@ -124,6 +128,8 @@ def test_plan_preview_geometry_and_overrides():
     st, info = B.exo_gemm_plan_preview(good(M=4096, N=4096, K=512, flags=B.flag_grid_limit(8) | B.flag_band(3)
                                             | B.flag_cta_group(2) | B.flag_tile_n(256)), 148)
     assert info.grid == 8 and info.raster_band == 3
+    st, info = B.exo_gemm_plan_preview(good(flags=B.flag_max_stages(2) | B.flag_epi_buffers(1)), 148)
+    assert info.stages == 2 and info.epilogue_buffers == 1
     st, info = B.exo_gemm_plan_preview(good(M=0), 148)
     assert st == B.OK and info.kernel_launches_per_run == 0
     assert B.exo_gemm_plan_preview(good(), 0)[0] == B.ERR_INVALID_ARG

@@ -40,9 +40,9 @@ def check_full(p, flags=0, literal=None):
     return cbuf, got, cref, den, info
 
 
-def flags_for(g, bn, grid=0, ksub=0):
+def flags_for(g, bn, grid=0, ksub=0, epi=0, stages=0):
     return (B.flag_cta_group(g) | B.flag_tile_n(bn) | (B.flag_grid_limit(grid) if grid else 0)
-            | B.flag_k_subblocks(ksub))
+            | B.flag_k_subblocks(ksub) | B.flag_epi_buffers(epi) | B.flag_max_stages(stages))
 
 
 TILE_SHAPES = [(1, 64), (1, 128), (1, 256), (2, 128), (2, 256)]
@@ -92,13 +92,13 @@ def test_tile_boundaries(M, N, K, g, bn, ksub):
 @pytest.mark.parametrize("lb", [0, 1])
 @pytest.mark.parametrize("lc", [0, 1])
 @pytest.mark.parametrize("ab,cd", [(BF16, FP32), (FP16, FP32), (BF16, BF16), (FP16, FP16)])
-@pytest.mark.parametrize("g,bn,ksub", [(1, 128, 2), (2, 256, 2), (2, 128, 1), (1, 256, 1)])
-def test_layouts_dtypes_alpha_beta(la, lb, lc, ab, cd, g, bn, ksub):
+@pytest.mark.parametrize("g,bn,ksub,epi", [(1, 128, 2, 1), (2, 256, 2, 1), (2, 128, 1, 2), (1, 256, 1, 2)])
+def test_layouts_dtypes_alpha_beta(la, lb, lc, ab, cd, g, bn, ksub, epi):
     M, N, K = 264, 328, 200
     p = synth.Problem("lay", M, N, K, ab, cd, la, lb, lc, -1.5, 0.75, seed=la + 2 * lb + 4 * lc + 8 * ab,
                       dist="normal" if ab == FP16 else "uniform")
     p.generate()
-    check_full(p, flags_for(g, bn, ksub=ksub))
+    check_full(p, flags_for(g, bn, ksub=ksub, epi=epi))
 
 
 @pytest.mark.parametrize("g,bn", TILE_SHAPES)
@@ -176,6 +176,8 @@ def test_persistent_loop_many_tiles_on_few_ctas():
     p = synth.Problem("few", 1536, 1024, 328, FP16, FP16, 0, 0, 0, 1.0, 1.0, seed=9, dist="normal").generate()
     check_full(p, flags_for(1, 128, 4))
     check_full(p, flags_for(2, 128, 4))
+    check_full(p, flags_for(2, 256, 4, ksub=1, epi=1, stages=2))   # shallowest ring, single staging buffer
+    check_full(p, flags_for(1, 64, 4, ksub=2, epi=2, stages=3))
 
 
 def test_bounded_wait_reports_timeout_and_the_plan_stays_usable():
