@@ -48,6 +48,7 @@ typedef enum { EXO_GEMM_ROW_MAJOR = 0, EXO_GEMM_COL_MAJOR = 1 } exo_gemm_layout_
  *   bits 20..21 k sub-blocks (of 64 elements) per pipeline stage: 1 or 2
  *   bits 22..23 staging buffers per epilogue warp: 1 or 2
  *   bits 24..27 upper limit on the pipeline depth (2..8)
+ *   bits 28..31 K-slices per tile of the partial last wave: 1 = never split, 2..8 = at most this many
  */
 #define EXO_GEMM_FLAG_CTA_GROUP(g)  ((uint32_t)(g) & 3u)
 #define EXO_GEMM_FLAG_TILE_N(n)     ((((uint32_t)(n) / 64u) & 15u) << 2)
@@ -57,6 +58,7 @@ typedef enum { EXO_GEMM_ROW_MAJOR = 0, EXO_GEMM_COL_MAJOR = 1 } exo_gemm_layout_
 #define EXO_GEMM_FLAG_K_SUBBLOCKS(k) (((uint32_t)(k) & 3u) << 20)
 #define EXO_GEMM_FLAG_EPI_BUFFERS(b) (((uint32_t)(b) & 3u) << 22)
 #define EXO_GEMM_FLAG_MAX_STAGES(s) (((uint32_t)(s) & 15u) << 24)
+#define EXO_GEMM_FLAG_SPLIT_K(f) (((uint32_t)(f) & 15u) << 28)
 
 /*
  * Problem descriptor.  Logical shapes: A is M x K, B is K x N, C is M x N.
@@ -97,7 +99,10 @@ typedef struct {
   int32_t sm_count;
   int32_t kernel_launches_per_run; /* 1, or 0 for an empty problem                             */
   int32_t epilogue_buffers; /* staging buffers per epilogue warp (1 or 2)                      */
-  int32_t reserved[4];
+  int32_t split_k;         /* K-slices per tile of the partial last wave (1 = none)            */
+  int32_t tail_tiles;      /* tiles in that partial last wave                                  */
+  int32_t workspace_bytes; /* device scratch the plan owns for the slices' partial sums        */
+  int32_t reserved[1];
 } exo_gemm_info_t;
 
 /*
@@ -112,7 +117,9 @@ exo_gemm_status_t exo_gemm_validate(const exo_gemm_desc_t* desc);
  * cta_group, the pipeline depth and the raster, and sizes the persistent grid
  * (the paper's counterpart is the device-function configuration of Section 3.2,
  * clusterDim and warp configuration, and the persistent task loop of
- * Section 4.2).  Allocates host state and one 32-byte device status block;
+ * Section 4.2).  Allocates host state, one 32-byte device status block and, if the
+ * tiles of a partial last wave are to be cut along K (exo_gemm_info_t.split_k > 1),
+ * a device workspace of exo_gemm_info_t.workspace_bytes for their partial sums;
  * touches no user matrix.  *out is written only on success.
  */
 exo_gemm_status_t exo_gemm_create(exo_gemm_handle_t* out, const exo_gemm_desc_t* desc);
@@ -136,7 +143,9 @@ exo_gemm_status_t exo_gemm_create(exo_gemm_handle_t* out, const exo_gemm_desc_t*
  *
  * All checks happen before the launch; on any error nothing is enqueued.  A
  * handle may be used from several host threads (tensor maps are built on the
- * caller's stack).  Device-side waits are bounded: if one gives up, the kernel
+ * caller's stack), but runs of ONE plan whose exo_gemm_info_t.split_k > 1 must not
+ * overlap on the GPU (enqueue them on one stream, or order the streams): they
+ * share the plan's partial-sum workspace and arrival counters.  Device-side waits are bounded: if one gives up, the kernel
  * records where in the plan's status block and exits cleanly; a later
  * exo_gemm_check reports EXO_GEMM_ERR_DEVICE_TIMEOUT.
  */
@@ -217,6 +226,19 @@ int exo_gemm_last_cuda_error(void);
 int64_t exo_gemm_schedule_enumerate(int32_t tiles_m, int32_t tiles_n, int32_t band, int32_t along_m,
                                     int32_t num_workers, int32_t worker, int32_t* out_m,
                                     int32_t* out_n, int64_t cap);
+
+/*
+ * Host-side enumeration of one worker's work list including the K-slicing of the
+ * tail tiles (the paper's Section 6 measures split-K variants of its GEMM against
+ * wave quantisation; here only the tiles of the partial last wave are cut, into
+ * `split` slices each, slice 0 owning the output and taking `owner_extra` k-blocks
+ * more than an even share).  `tiles` tiles, `num_workers` workers; writes tile index, slice and k-block range [begin, end) of
+ * `num_k_blocks` per item (capacity `cap`); returns the item count, or -1 on bad
+ * arguments (including tail_tiles * split > num_workers).  Needs no GPU.
+ */
+int64_t exo_gemm_schedule_work(int64_t tiles, int32_t num_workers, int32_t split, int32_t owner_extra,
+                               int32_t num_k_blocks, int32_t worker, int64_t* out_tile, int32_t* out_slice, int32_t* out_kb_begin,
+                               int32_t* out_kb_end, int64_t cap);
 
 /*
  * Test hook for the bounded waits: the next exo_gemm_run on this plan uses

@@ -18,7 +18,7 @@ ROW_MAJOR, COL_MAJOR = 0, 1
 EXPORTED_SYMBOLS = (
     "exo_gemm_validate", "exo_gemm_create", "exo_gemm_run", "exo_gemm_check", "exo_gemm_plan_preview",
     "exo_gemm_get_info", "exo_gemm_destroy", "exo_gemm_status_string", "exo_gemm_last_cuda_error",
-    "exo_gemm_schedule_enumerate", "exo_gemm_debug_set", "exo_gemm_run_static",
+    "exo_gemm_schedule_enumerate", "exo_gemm_debug_set", "exo_gemm_run_static", "exo_gemm_schedule_work",
 )
 
 
@@ -30,6 +30,7 @@ def flag_grid_limit(c): return (c & 255) << 12
 def flag_k_subblocks(k): return (k & 3) << 20
 def flag_epi_buffers(b): return (b & 3) << 22
 def flag_max_stages(s): return (s & 15) << 24
+def flag_split_k(f): return (f & 15) << 28
 
 
 class Desc(ctypes.Structure):
@@ -45,7 +46,8 @@ class Info(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "cta_group", "tile_m", "tile_n", "tile_k", "stages", "grid", "smem_bytes", "tmem_columns",
         "tiles_m", "tiles_n", "raster_along_m", "raster_band", "swapped", "sm_count",
-        "kernel_launches_per_run", "epilogue_buffers")] + [("reserved", ctypes.c_int32 * 4)]
+        "kernel_launches_per_run", "epilogue_buffers", "split_k", "tail_tiles", "workspace_bytes")] + [
+        ("reserved", ctypes.c_int32 * 1)]
 
     def as_dict(self):
         return {n: getattr(self, n) for n, _ in self._fields_ if n != "reserved"}
@@ -84,6 +86,9 @@ def lib():
                                                   ctypes.POINTER(i32), i64]
         L.exo_gemm_schedule_enumerate.restype = i64
         L.exo_gemm_debug_set.argtypes = [vp, i32, i64]
+        L.exo_gemm_schedule_work.argtypes = [i64, i32, i32, i32, i32, i32, ctypes.POINTER(i64), ctypes.POINTER(i32),
+                                             ctypes.POINTER(i32), ctypes.POINTER(i32), i64]
+        L.exo_gemm_schedule_work.restype = i64
         L.exo_gemm_run_static.argtypes = [ctypes.POINTER(Desc), vp, vp, vp, ctypes.c_float, ctypes.c_float, vp,
                                           ctypes.POINTER(ctypes.c_uint32)]
         L.exo_gemm_run_static.restype = ctypes.c_int
@@ -174,6 +179,20 @@ def exo_gemm_schedule_enumerate(tiles_m, tiles_n, band, along_m, num_workers, wo
     on = (ctypes.c_int32 * max(n, 1))()
     lib().exo_gemm_schedule_enumerate(tiles_m, tiles_n, band, along_m, num_workers, worker, om, on, n)
     return [(om[i], on[i]) for i in range(n)]
+
+
+def exo_gemm_schedule_work(tiles, num_workers, split, num_k_blocks, worker, owner_extra=0):
+    """[(tile, slice, kb_begin, kb_end), ...] for one worker, tail tiles cut into `split` K-slices."""
+    n = lib().exo_gemm_schedule_work(tiles, num_workers, split, owner_extra, num_k_blocks, worker,
+                                     None, None, None, None, 0)
+    if n < 0:
+        raise ValueError("bad work-schedule arguments")
+    t = (ctypes.c_int64 * max(n, 1))()
+    s = (ctypes.c_int32 * max(n, 1))()
+    b = (ctypes.c_int32 * max(n, 1))()
+    e = (ctypes.c_int32 * max(n, 1))()
+    lib().exo_gemm_schedule_work(tiles, num_workers, split, owner_extra, num_k_blocks, worker, t, s, b, e, n)
+    return [(t[i], s[i], b[i], e[i]) for i in range(n)]
 
 
 # ---- thin convenience wrapper ---------------------------------------------------------

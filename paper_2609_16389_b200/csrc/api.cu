@@ -93,6 +93,9 @@ struct exo_gemm_plan {
   int sm_count;
   int smem_bytes;
   uint32_t* d_status;
+  float* d_split_ws;                   // fp32 partials of the tail tiles' K-slices (NULL if none)
+  uint32_t* d_split_flags;             // one arrival counter per tail tile
+  std::atomic<uint32_t> split_epoch;   // runs that used the counters so far
   std::atomic<int32_t> dbg_timeout_ms;
   std::atomic<int64_t> dbg_skip_k_block;
 };
@@ -141,6 +144,9 @@ void fill_info(const exo_gemm_plan* p, exo_gemm_info_t* info) {
   info->sm_count = p->sm_count;
   info->kernel_launches_per_run = (p->canon.M == 0 || p->canon.N == 0) ? 0 : 1;
   info->epilogue_buffers = p->cfg.epi_bufs;
+  info->split_k = p->cfg.split;
+  info->tail_tiles = p->cfg.tail_tiles;
+  info->workspace_bytes = (int32_t)(p->cfg.workspace_bytes > 2147483647LL ? 2147483647LL : p->cfg.workspace_bytes);
 }
 
 }  // namespace
@@ -183,6 +189,31 @@ int64_t exo_gemm_schedule_enumerate(int32_t tiles_m, int32_t tiles_n, int32_t ba
   return n;
 }
 
+int64_t exo_gemm_schedule_work(int64_t tiles, int32_t num_workers, int32_t split, int32_t owner_extra,
+                               int32_t num_k_blocks, int32_t worker, int64_t* out_tile, int32_t* out_slice, int32_t* out_kb_begin,
+                               int32_t* out_kb_end, int64_t cap) {
+  if (tiles < 0 || num_workers < 1 || split < 1 || owner_extra < 0 || num_k_blocks < 0 || worker < 0 || worker >= num_workers || cap < 0 ||
+      (cap > 0 && (!out_tile || !out_slice || !out_kb_begin || !out_kb_end)))
+    return -1;
+  WorkPlan w;
+  w.full_tiles = (tiles / num_workers) * num_workers;
+  w.tail_tiles = (int32_t)(tiles - w.full_tiles);
+  w.split = split;
+  w.owner_extra = owner_extra;
+  if ((int64_t)w.tail_tiles * split > num_workers) return -1;
+  int64_t n = 0;
+  WorkItem wi;
+  for (int64_t i = 0; work_item(w, worker, num_workers, i, num_k_blocks, &wi); ++i, ++n) {
+    if (n < cap) {
+      out_tile[n] = wi.tile;
+      out_slice[n] = wi.slice;
+      out_kb_begin[n] = wi.kb_begin;
+      out_kb_end[n] = wi.kb_end;
+    }
+  }
+  return n;
+}
+
 exo_gemm_status_t exo_gemm_plan_preview(const exo_gemm_desc_t* desc, int32_t sm_count, exo_gemm_info_t* info) {
   if (!info) return EXO_GEMM_ERR_NULL;
   exo_gemm_status_t st = validate_desc(desc);
@@ -193,6 +224,7 @@ exo_gemm_status_t exo_gemm_plan_preview(const exo_gemm_desc_t* desc, int32_t sm_
   p.canon = canonicalize(*desc);
   p.sm_count = sm_count;
   p.cfg = choose_config(p.canon, decode_flags(desc->flags), sm_count, sm_count / 2);
+  p.cfg.workspace_bytes = split_workspace_bytes(p.cfg, desc->c_dtype);
   p.smem_bytes = smem_bytes_for(p.cfg.cta_group, p.cfg.tile_n, p.cfg.ksub, p.cfg.stages, p.cfg.epi_bufs);
   fill_info(&p, info);
   return EXO_GEMM_OK;
@@ -254,6 +286,8 @@ exo_gemm_status_t exo_gemm_create(exo_gemm_handle_t* out, const exo_gemm_desc_t*
   }
 
   p->cfg = choose_config(p->canon, ov, sms, max_pairs);
+  p->cfg.workspace_bytes = split_workspace_bytes(p->cfg, desc->c_dtype);
+  p->split_epoch = 0;
   p->kernel = pick_kernel(p->cfg.cta_group, p->cfg.tile_n, p->cfg.ksub, desc->c_dtype);
   p->smem_bytes = smem_bytes_for(p->cfg.cta_group, p->cfg.tile_n, p->cfg.ksub, p->cfg.stages, p->cfg.epi_bufs);
   e = cudaFuncSetAttribute((const void*)p->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, p->smem_bytes);
@@ -262,6 +296,18 @@ exo_gemm_status_t exo_gemm_create(exo_gemm_handle_t* out, const exo_gemm_desc_t*
   if (e != cudaSuccess) { delete p; return cuda_fail(e); }
   e = cudaMemset(p->d_status, 0, kStatusBytes);
   if (e != cudaSuccess) { cudaFree(p->d_status); delete p; return cuda_fail(e); }
+  if (p->cfg.split > 1) {  // scratch for the K-slices of the tail tiles
+    e = cudaMalloc((void**)&p->d_split_ws, (size_t)p->cfg.workspace_bytes);
+    if (e == cudaSuccess) e = cudaMalloc((void**)&p->d_split_flags, sizeof(uint32_t) * (size_t)p->cfg.tail_tiles);
+    if (e == cudaSuccess) e = cudaMemset(p->d_split_flags, 0, sizeof(uint32_t) * (size_t)p->cfg.tail_tiles);
+    if (e != cudaSuccess) {
+      cudaFree(p->d_split_ws);
+      cudaFree(p->d_split_flags);
+      cudaFree(p->d_status);
+      delete p;
+      return cuda_fail(e);
+    }
+  }
   *out = p;
   return EXO_GEMM_OK;
 }
@@ -303,6 +349,12 @@ exo_gemm_status_t exo_gemm_run(exo_gemm_handle_t plan, const void* A, const void
   prm.raster = Raster{cfg.tiles_m, cfg.tiles_n, cfg.band, cfg.along_m};
   prm.stages = cfg.stages;
   prm.epi_bufs = cfg.epi_bufs;
+  // the tail tiles are cut along K only when there is a K loop to cut and scratch to reduce through
+  const bool split_now = cfg.split > 1 && read_ab && plan->d_split_ws != nullptr;
+  prm.work = WorkPlan{cfg.full_tiles, cfg.tail_tiles, split_now ? cfg.split : 1, split_now ? cfg.owner_extra : 0};
+  prm.split_ws = plan->d_split_ws;
+  prm.split_flags = plan->d_split_flags;
+  prm.split_target = 0;
   prm.alpha = read_ab ? alpha : 0.f;
   prm.beta = beta;
   prm.idesc = make_idesc(d.ab_dtype, cn.a_mn_major, cn.b_mn_major, 128 * cfg.cta_group, cfg.tile_n);
@@ -345,6 +397,10 @@ exo_gemm_status_t exo_gemm_run(exo_gemm_handle_t plan, const void* A, const void
   at[0].val.clusterDim.z = 1;
   lc.attrs = at;
   lc.numAttrs = 1;
+  if (split_now) {  // arrival counters only grow: this run is complete at epoch * arrivals-per-run
+    const uint32_t epoch = plan->split_epoch.fetch_add(1) + 1;
+    prm.split_target = epoch * (uint32_t)((cfg.split - 1) * kEpiWarps * cfg.cta_group);
+  }
   cudaError_t e = cudaLaunchKernelEx(&lc, plan->kernel, tm_a, tm_b, tm_c, prm);
   if (e != cudaSuccess) return cuda_fail(e);
   return EXO_GEMM_OK;
@@ -361,6 +417,11 @@ exo_gemm_status_t exo_gemm_check(exo_gemm_handle_t plan, uint32_t* detail) {
   if (h[0] == kStatusOk) return EXO_GEMM_OK;
   e = cudaMemset(plan->d_status, 0, 32);
   if (e != cudaSuccess) return cuda_fail(e);
+  if (plan->d_split_flags) {  // an abandoned run may have left the arrival counters short
+    e = cudaMemset(plan->d_split_flags, 0, sizeof(uint32_t) * (size_t)plan->cfg.tail_tiles);
+    if (e != cudaSuccess) return cuda_fail(e);
+    plan->split_epoch = 0;
+  }
   return EXO_GEMM_ERR_DEVICE_TIMEOUT;
 }
 
@@ -422,7 +483,8 @@ exo_gemm_status_t exo_gemm_run_static(const exo_gemm_desc_t* desc, const void* A
   plan.sm_count = sms;
   plan.dbg_timeout_ms = 0;
   plan.dbg_skip_k_block = -1;
-  const FlagOverrides ov = decode_flags(desc->flags);
+  FlagOverrides ov = decode_flags(desc->flags);
+  ov.no_workspace = true;  // K-slicing of the tail tiles needs device scratch this entry point may not allocate
   int max_pairs = 0;
   if (ov.cta_group != 1) {
     KernelFn probe = pick_kernel(2, 256, 2, desc->c_dtype);
@@ -488,6 +550,8 @@ exo_gemm_status_t exo_gemm_destroy(exo_gemm_handle_t plan) {
       cudaError_t e = cudaFree(plan->d_status);
       if (e != cudaSuccess) st = cuda_fail(e);
     }
+    if (plan->d_split_ws) cudaFree(plan->d_split_ws);
+    if (plan->d_split_flags) cudaFree(plan->d_split_flags);
   }
   delete plan;
   return st;

@@ -152,7 +152,6 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   const uint32_t cta_rank = PAIR ? ptx::cluster_ctarank() : 0u;
   const int64_t worker = blockIdx.x / CTA_GROUP;
   const int64_t num_workers = gridDim.x / CTA_GROUP;
-  const int64_t total_tiles = raster_total(p.raster);
   const int32_t nkb = p.num_k_blocks;
 
   if (threadIdx.x == 0) EXO_TRACE(2, 4095, 0, 4096);
@@ -197,11 +196,14 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     int64_t issued = 0;
     // in a pair, both CTAs' loads are counted on the leader's full barrier
     const uint32_t full0 = PAIR ? ptx::map_to_cta(full_bar(0), 0) : full_bar(0);
-    for (int64_t t = worker; t < total_tiles && ok; t += num_workers) {
+    for (int64_t it = 0; ok; ++it) {
+      WorkItem wi;
+      if (!work_item(p.work, worker, num_workers, it, nkb, &wi)) break;
+      const int64_t t = wi.tile;
       const TileCoord tc = raster_decode(p.raster, t);
       const int32_t a_mn0 = tc.m * (kBlockM * CTA_GROUP) + (int32_t)cta_rank * kBlockM;
       const int32_t b_mn0 = tc.n * BN + (int32_t)cta_rank * B_ROWS;
-      for (int32_t kb = 0; kb < nkb; ++kb) {
+      for (int32_t kb = wi.kb_begin; kb < wi.kb_end; ++kb) {
         ok = wait_barrier<PAIR>(empty_bar(s), ph ^ 1u, p, WaitSite{kRoleProducer, s, (uint32_t)t, (uint32_t)kb});
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
@@ -260,14 +262,17 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         return (uint64_t)((uint32_t)(k & 3) * step + (uint32_t)(k >> 2) * sub);
       };
       const uint32_t idesc = p.idesc;
-      for (int64_t t = worker; t < total_tiles && ok; t += num_workers) {
+      for (int64_t it = 0; ok; ++it) {
+        WorkItem wi;
+        if (!work_item(p.work, worker, num_workers, it, nkb, &wi)) break;
+        const int64_t t = wi.tile;
         // the epilogue (of both CTAs) must have drained this accumulator
         ok = wait_barrier<PAIR>(tempty_bar(acc), acc_ph ^ 1u, p, WaitSite{kRoleMma, 100 + acc, (uint32_t)t, 0});
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         ptx::tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + acc * BN;
-        for (int32_t kb = 0; kb < nkb; ++kb) {
+        for (int32_t kb = wi.kb_begin; kb < wi.kb_end; ++kb) {
           ok = wait_barrier<PAIR>(full_bar(s), ph, p, WaitSite{kRoleMma, s, (uint32_t)t, (uint32_t)kb});
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
@@ -282,15 +287,15 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
 #pragma unroll
               for (int32_t k = 0; k < kMmaPerStage; ++k)
                 ptx::umma_f16<CTA_GROUP>(d_tmem, a_desc + k_off(k, a_step, a_sub), b_desc + k_off(k, b_step, b_sub),
-                                         idesc, (kb | k) != 0 ? 1u : 0u);
+                                         idesc, (kb != wi.kb_begin || k != 0) ? 1u : 0u);
             } else {  // ragged last k-block: skip the MMAs that would only read zero fill
               const int32_t n_mma = (k_left + kUmmaK - 1) / kUmmaK;
               for (int32_t k = 0; k < n_mma; ++k)
                 ptx::umma_f16<CTA_GROUP>(d_tmem, a_desc + k_off(k, a_step, a_sub), b_desc + k_off(k, b_step, b_sub),
-                                         idesc, (kb | k) != 0 ? 1u : 0u);
+                                         idesc, (kb != wi.kb_begin || k != 0) ? 1u : 0u);
             }
             ptx::umma_commit<CTA_GROUP>(empty_bar(s), kMask);  // stage free once these MMAs completed
-            if (kb == nkb - 1) ptx::umma_commit<CTA_GROUP>(tfull_bar(acc), kMask);  // accumulator complete
+            if (kb == wi.kb_end - 1) ptx::umma_commit<CTA_GROUP>(tfull_bar(acc), kMask);  // accumulator complete
             EXO_TRACE(1, consumed, 1, 4096);
           }
           ++consumed;
@@ -322,7 +327,10 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     const bool two_bufs = EPI_BUFS == 2;
     uint32_t acc = 0, acc_ph = 0;
 
-    for (int64_t t = worker; t < total_tiles; t += num_workers) {
+    for (int64_t it = 0;; ++it) {
+      WorkItem wi;
+      if (!work_item(p.work, worker, num_workers, it, nkb, &wi)) break;
+      const int64_t t = wi.tile;
       const TileCoord tc = raster_decode(p.raster, t);
       const int32_t row0 = tc.m * (kBlockM * CTA_GROUP) + (int32_t)cta_rank * kBlockM + (int32_t)quad * 32;
       const int32_t col0 = tc.n * BN;
@@ -338,7 +346,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         if (!ok) break;
         ptx::tc_fence_after_sync();
       }
-      if (warp == 2 && lane == 0) EXO_TRACE(2, (t - worker) / num_workers, 0, 4096);
+      if (warp == 2 && lane == 0) EXO_TRACE(2, it, 0, 4096);
       auto release_acc = [&]() {
         ptx::tc_fence_before_sync();
         __syncwarp();
@@ -353,6 +361,67 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         ptx::tmem_ld_32x32(tacc + (uint32_t)((half + 2 * i) * CW + q * 32), dst);
       };
       if (mine == 0 && has_acc) release_acc();
+
+      // ---- a slice of a tail tile (the tile's K range is cut into wi.slices parts)
+      // Partial accumulators travel through a private fp32 workspace in a layout where a warp's
+      // 16-byte pieces are contiguous (coalesced both ways): [tail tile][slice-1][cta][warp][chunk]
+      // [unit][piece][lane].
+      constexpr uint32_t kUnitBytes = 8u * 512u;  // 32 lanes x 32 columns x 4 bytes
+      const bool contributor = wi.slices > 1 && wi.slice != 0;
+      const bool owner = wi.slices > 1 && wi.slice == 0;
+      auto ws_unit = [&](int32_t slice_m1, int32_t i, int32_t q) {
+        const uint64_t idx = ((((uint64_t)wi.tail_index * (uint32_t)(wi.slices - 1) + (uint32_t)slice_m1) * CTA_GROUP +
+                               cta_rank) * kEpiWarps + ew) * (uint32_t)(((NCHUNK + 1) / 2) * UPC) +
+                             (uint32_t)(i * UPC + q);
+        return reinterpret_cast<char*>(p.split_ws) + idx * kUnitBytes + lane * 16u;
+      };
+      if (contributor) {
+        // raw accumulators out, then one arrival per warp on the tile's counter
+        for (int32_t i = 0; i < mine; ++i) {
+#pragma unroll
+          for (int32_t q = 0; q < UPC; ++q) {
+            uint32_t r[32];
+            tmem_load(r, i, q);
+            ptx::tmem_ld_wait();
+            if (i + 1 == mine && q == UPC - 1) release_acc();
+            char* dst = ws_unit(wi.slice - 1, i, q);
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              ptx::st_global_v4(dst + j * 512, r[4 * j + 0], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+          }
+        }
+        __threadfence();  // each lane's partials are visible GPU-wide before the arrival below
+        __syncwarp();
+        if (ptx::elect_one()) ptx::red_release_gpu_add(p.split_flags + wi.tail_index, 1u);
+        if ((acc ^= 1u) == 0u) acc_ph ^= 1u;
+        continue;
+      }
+      if (owner && mine > 0) {
+        // wait (bounded) until every warp of every other slice has delivered its partials
+        const uint32_t* flag = p.split_flags + wi.tail_index;
+        const long long t_start = clock64();
+        uint32_t spins = 0;
+        for (;;) {
+          const bool ready = (int32_t)(ptx::ld_acquire_gpu(flag) - p.split_target) >= 0;
+          if (__all_sync(0xffffffffu, ready)) break;
+          if ((++spins & 63u) == 0u) {
+            bool give_up = *(volatile uint32_t*)p.status != kStatusOk;
+            if (!give_up && (uint64_t)(clock64() - t_start) > p.timeout_cycles) {
+              if (atomicCAS(p.status, (uint32_t)kStatusOk, (uint32_t)kStatusTimeout) == kStatusOk) {
+                p.status[1] = kRoleEpiloguePartials;
+                p.status[2] = (uint32_t)wi.tail_index;
+                p.status[3] = (uint32_t)t;
+                p.status[4] = 0;
+                p.status[5] = blockIdx.x;
+                __threadfence();
+              }
+              give_up = true;
+            }
+            if (__any_sync(0xffffffffu, give_up)) { ok = false; break; }
+          }
+        }
+        if (!ok) break;
+      }
       auto issue_cin = [&](uint32_t gg, int32_t i) {  // elected lane only: C_in of this warp's i-th chunk
         const uint32_t b = two_bufs ? (gg & 1u) : 0u;
         ptx::mbar_arrive_expect_tx(cin_bar(ew, b), kEpiBufBytes);
@@ -410,6 +479,20 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
 #pragma unroll
               for (int k = 0; k < 32; ++k) cur[k] = 0u;
             }
+            if (owner) {  // add the other slices' partial sums, in slice order
+              for (int32_t sm1 = 0; sm1 < wi.slices - 1; ++sm1) {
+                const char* src = ws_unit(sm1, i, q);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                  uint32_t a0, a1, a2, a3;
+                  ptx::ld_global_cg_v4(src + j * 512, a0, a1, a2, a3);
+                  cur[4 * j + 0] = __float_as_uint(__uint_as_float(cur[4 * j + 0]) + __uint_as_float(a0));
+                  cur[4 * j + 1] = __float_as_uint(__uint_as_float(cur[4 * j + 1]) + __uint_as_float(a1));
+                  cur[4 * j + 2] = __float_as_uint(__uint_as_float(cur[4 * j + 2]) + __uint_as_float(a2));
+                  cur[4 * j + 3] = __float_as_uint(__uint_as_float(cur[4 * j + 3]) + __uint_as_float(a3));
+                }
+              }
+            }
             if (scale) {
 #pragma unroll
               for (int k = 0; k < 32; ++k) cur[k] = __float_as_uint(alpha * __uint_as_float(cur[k]));
@@ -463,7 +546,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         }
       }
       if (!ok) break;
-      if (warp == 2 && lane == 0) EXO_TRACE(2, (t - worker) / num_workers, 1, 4096);
+      if (warp == 2 && lane == 0) EXO_TRACE(2, it, 1, 4096);
       if ((acc ^= 1u) == 0u) acc_ph ^= 1u;
     }
     __syncwarp();

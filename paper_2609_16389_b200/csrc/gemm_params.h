@@ -59,6 +59,7 @@ enum WaitRole : uint32_t {
   kRoleEpilogue = 3,
   kRoleProducerTail = 4,
   kRoleEpilogueCin = 5,
+  kRoleEpiloguePartials = 6,
 };
 
 struct GemmParams {
@@ -70,6 +71,10 @@ struct GemmParams {
   float alpha, beta;
   uint32_t idesc;           // tcgen05 instruction descriptor
   OperandStaging a, b;
+  WorkPlan work;            // whole-K tiles round-robin, then the tail tiles cut along K
+  float* split_ws;          // device: fp32 partial accumulators of the slices 1.. of every tail tile
+  uint32_t* split_flags;    // device: one arrival counter per tail tile, never reset, only grows
+  uint32_t split_target;    // counter value that means "all partials of this run have landed"
   uint32_t* status;         // device: 8 words {code, role, barrier, tile, k_block, cta, -, -}
   uint64_t timeout_cycles;  // bound of every device-side wait, in SM clocks
   int64_t debug_skip_k_block;  // -1, or the producer k-block of CTA 0 whose loads are skipped

@@ -12,6 +12,8 @@ namespace exo {
 inline int elem_bytes(int dtype) { return dtype == EXO_GEMM_FP32 ? 4 : 2; }
 
 struct FlagOverrides {
+  int split;       // 0 = auto, 1 = never split, 2..8 = slices per tail tile (if they fit)
+  bool no_workspace;  // set by the allocation-free entry point: nothing that needs device scratch
   int epi_bufs;    // 0 = auto
   int stages;      // 0 = as many as fit, else an upper limit
   int ksub;        // 0 = auto
@@ -32,6 +34,8 @@ inline FlagOverrides decode_flags(uint32_t f) {
   o.ksub = (int)((f >> 20) & 3u);
   o.epi_bufs = (int)((f >> 22) & 3u);
   o.stages = (int)((f >> 24) & 15u);
+  o.split = (int)((f >> 28) & 15u);
+  o.no_workspace = false;
   return o;
 }
 
@@ -55,7 +59,7 @@ inline exo_gemm_status_t validate_desc(const exo_gemm_desc_t* d) {
   if (d->lda < extent(d->a_layout, d->M, d->K) || d->ldb < extent(d->b_layout, d->K, d->N) ||
       d->ldc < extent(d->c_layout, d->M, d->N) || d->lda > kMaxLd || d->ldb > kMaxLd || d->ldc > kMaxLd)
     return EXO_GEMM_ERR_INVALID_ARG;
-  if (d->flags >> 28) return EXO_GEMM_ERR_INVALID_ARG;
+  if (((d->flags >> 28) & 15u) > 8u) return EXO_GEMM_ERR_INVALID_ARG;
   if (((d->flags >> 20) & 3u) == 3u || ((d->flags >> 22) & 3u) == 3u) return EXO_GEMM_ERR_INVALID_ARG;
   if (((d->flags >> 24) & 15u) == 1u || ((d->flags >> 24) & 15u) > (uint32_t)kMaxStages) return EXO_GEMM_ERR_INVALID_ARG;
   if (d->flags & (1u << 11)) return EXO_GEMM_ERR_INVALID_ARG;
@@ -105,6 +109,10 @@ inline Canonical canonicalize(const exo_gemm_desc_t& d) {
 }
 
 struct TileConfig {
+  int64_t full_tiles;      // tiles dealt round-robin as whole-K work items
+  int tail_tiles, split;   // the tiles of the partial last wave, each cut into `split` K-slices
+  int owner_extra;         // k-blocks the owning slice takes beyond an even share
+  int64_t workspace_bytes; // fp32 partials of slices 1.. of the tail tiles
   int cta_group, tile_n, ksub, stages, epi_bufs;
   int tiles_m, tiles_n;
   int band, along_m;
@@ -174,7 +182,41 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
   if (o.grid_limit && o.grid_limit / best_g < workers) workers = o.grid_limit / best_g;
   if (workers < 1) workers = 1;
   const int64_t tiles = (int64_t)cfg.tiles_m * cfg.tiles_n;
-  if (tiles < workers) workers = tiles < 1 ? 1 : tiles;
+  // Wave quantisation: the tiles that do not fill a whole wave are cut along K so that the
+  // last wave takes 1/split of a tile's time (split-K applied to the tail only; for a problem
+  // smaller than one wave that is plain split-K).
+  {
+    const int64_t full_waves = tiles / workers;
+    cfg.full_tiles = full_waves * workers;
+    cfg.tail_tiles = (int)(tiles - cfg.full_tiles);
+    cfg.split = 1;
+    const int64_t k_blocks = (c.K + kBlockK * cfg.ksub - 1) / (kBlockK * cfg.ksub);
+    if (cfg.tail_tiles > 0 && o.split != 1 && !o.no_workspace) {
+      int64_t f = workers / cfg.tail_tiles;
+      const int64_t by_k = (c.K / kBlockK) / 4;   // every slice keeps at least 256 k-elements
+      if (f > by_k) f = by_k;
+      if (f > 8) f = 8;
+      if (o.split >= 2 && o.split < f) f = o.split;
+      if (f > k_blocks) f = k_blocks;
+      if (f >= 2) cfg.split = (int)f;
+    }
+    // Publishing a 128 x N fp32 partial takes a contributor about as long as 8 k-blocks of 64
+    // (128*N*4 bytes at ~30 B/clk against 2*N clocks of MMA per k-block); let the owner compute that
+    // much longer, so that the partials are there when it finishes.
+    cfg.owner_extra = 0;
+    if (cfg.split > 1) {
+      int64_t extra = 8 / cfg.ksub;
+      const int64_t room = k_blocks / cfg.split - 1;   // every other slice keeps at least one k-block
+      if (extra > room / 2) extra = room / 2;
+      if (extra < 0) extra = 0;
+      cfg.owner_extra = (int)extra;
+    }
+    cfg.workspace_bytes = 0;  // filled in by split_workspace_bytes() once the output type is known
+  }
+  if (tiles < workers) {  // less than one wave: launch only the CTA groups that get a work item
+    workers = tiles * cfg.split;
+    if (workers < 1) workers = 1;
+  }
   cfg.workers = (int)workers;
   cfg.along_m = o.along_m;
   // Tiles that run together should cover a square patch of C: band width G along
@@ -188,6 +230,16 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
   if (band < 1) band = 1;
   cfg.band = band;
   return cfg;
+}
+
+// Bytes of fp32 partials: per tail tile and slice beyond the first, every epilogue warp of every
+// CTA of the group stores its chunks as 4 KB units (32 rows x 32 fp32 columns).
+inline int64_t split_workspace_bytes(const TileConfig& cfg, int c_dtype) {
+  if (cfg.split <= 1) return 0;
+  const int cw = c_dtype == EXO_GEMM_FP32 ? 32 : 64;        // columns per epilogue chunk
+  const int nchunk = cfg.tile_n / cw;
+  const int units_per_warp = ((nchunk + 1) / 2) * (cw / 32);
+  return (int64_t)cfg.tail_tiles * (cfg.split - 1) * cfg.cta_group * kEpiWarps * units_per_warp * 4096;
 }
 
 inline int smem_bytes_for(int cta_group, int bn, int ksub, int stages, int epi_bufs) {

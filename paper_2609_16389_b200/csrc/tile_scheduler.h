@@ -53,4 +53,67 @@ EXO_HD TileCoord raster_decode(const Raster& r, int64_t t) {
   return c;
 }
 
+// ---------------------------------------------------------------------------
+// Work list of one worker.  Tiles are dealt round-robin for as long as whole
+// waves can be filled (`full_tiles` = the largest multiple of the worker count
+// not above the tile count).  The `tail_tiles` tiles left over would occupy only
+// part of a last wave, so each of them is cut along K into `split` slices and
+// the tail_tiles * split <= num_workers units are dealt one per worker: the
+// last wave then takes about 1/split of a tile's time.  (The paper's Section 6
+// kernels use split-K for the same wave-quantisation problem; here the split is
+// applied only where it pays, and the reduction order is fixed.)  split == 1
+// degenerates to plain round-robin.
+struct WorkPlan {
+  int64_t full_tiles;   // tiles [0, full_tiles) are whole-K work items
+  int32_t tail_tiles;   // tiles [full_tiles, full_tiles + tail_tiles) are cut into slices
+  int32_t split;        // slices per tail tile, >= 1
+  int32_t owner_extra;  // k-blocks slice 0 takes beyond an even share: the other slices finish
+                        // earlier by about the time it takes them to publish their partial sums
+};
+
+struct WorkItem {
+  int64_t tile;         // linear tile index (to be decoded by raster_decode)
+  int32_t tail_index;   // index among the tail tiles, or -1 for a whole-K item
+  int32_t slice;        // 0 .. slices - 1; slice 0 owns the output tile
+  int32_t slices;
+  int32_t kb_begin, kb_end;  // k-blocks [kb_begin, kb_end) of num_k_blocks
+};
+
+// The i-th work item of `worker`; returns false when the worker has no i-th item.
+EXO_HD bool work_item(const WorkPlan& w, int64_t worker, int64_t num_workers, int64_t i, int32_t num_k_blocks,
+                      WorkItem* out) {
+  const int64_t t = worker + i * num_workers;
+  if (t < w.full_tiles) {
+    out->tile = t;
+    out->tail_index = -1;
+    out->slice = 0;
+    out->slices = 1;
+    out->kb_begin = 0;
+    out->kb_end = num_k_blocks;
+    return true;
+  }
+  if (t - w.full_tiles != worker) return false;             // only the wave right after the full ones
+  if (worker >= (int64_t)w.tail_tiles * w.split) return false;
+  const int32_t ti = (int32_t)(worker / w.split);
+  const int32_t sl = (int32_t)(worker - (int64_t)ti * w.split);
+  out->tile = w.full_tiles + ti;
+  out->tail_index = w.split > 1 ? ti : -1;
+  out->slice = sl;
+  out->slices = w.split;
+  // slice 0: an even share plus owner_extra; slices 1.. share the rest evenly, in K order
+  int32_t own = (num_k_blocks + w.split - 1) / w.split + (w.split > 1 ? w.owner_extra : 0);
+  if (own > num_k_blocks - (w.split - 1)) own = num_k_blocks - (w.split - 1);
+  if (own < 1) own = 1;
+  if (w.split == 1) own = num_k_blocks;
+  if (sl == 0) {
+    out->kb_begin = 0;
+    out->kb_end = own;
+  } else {
+    const int64_t rest = num_k_blocks - own;
+    out->kb_begin = own + (int32_t)((rest * (sl - 1)) / (w.split - 1));
+    out->kb_end = own + (int32_t)((rest * sl) / (w.split - 1));
+  }
+  return true;
+}
+
 }  // namespace exo

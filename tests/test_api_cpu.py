@@ -72,7 +72,7 @@ def test_validate_rejects_bad_arguments():
     assert B.exo_gemm_validate(good(flags=3)) == B.ERR_INVALID_ARG                       # cta_group 3
     assert B.exo_gemm_validate(good(flags=B.flag_tile_n(192))) == B.ERR_INVALID_ARG
     assert B.exo_gemm_validate(good(flags=B.flag_cta_group(2) | B.flag_tile_n(64))) == B.ERR_INVALID_ARG
-    assert B.exo_gemm_validate(good(flags=1 << 28)) == B.ERR_INVALID_ARG
+    assert B.exo_gemm_validate(good(flags=15 << 28)) == B.ERR_INVALID_ARG
     assert B.exo_gemm_validate(good(flags=B.flag_max_stages(1))) == B.ERR_INVALID_ARG
     assert B.exo_gemm_validate(good(flags=B.flag_max_stages(9))) == B.ERR_INVALID_ARG
     assert B.exo_gemm_validate(good(flags=B.flag_epi_buffers(3))) == B.ERR_INVALID_ARG
@@ -179,3 +179,58 @@ def test_create_fails_cleanly_without_a_gpu():
         B.Plan(good())
     assert B.exo_gemm_destroy(None) == B.OK
     assert B.exo_gemm_run(None, 0, 0, 0, 1.0, 0.0, 0) == B.ERR_NULL
+
+
+@pytest.mark.parametrize("tiles,workers,split", [(256, 74, 2), (256, 74, 1), (32, 148, 4), (5, 148, 8), (300, 148, 3),
+                                                  (148, 148, 1), (149, 148, 8), (1, 1, 1), (0, 4, 1)])
+@pytest.mark.parametrize("nkb", [64, 7, 1000])
+@pytest.mark.parametrize("extra", [0, 3])
+def test_work_schedule_covers_every_tile_and_k_block_exactly_once(tiles, workers, split, nkb, extra):
+    tail = tiles % workers
+    if tail * split > workers or split > nkb:
+        pytest.skip("not a plan the library would make")
+    cover = {}
+    longest = 0
+    for w in range(workers):
+        items = B.exo_gemm_schedule_work(tiles, workers, split, nkb, w, extra)
+        longest = max(longest, len(items))
+        for tile, sl, b, e in items:
+            assert 0 <= tile < tiles and 0 <= b < e <= nkb
+            cover.setdefault(tile, []).append((b, e, sl))
+    assert sorted(cover) == list(range(tiles))
+    for tile, parts in cover.items():
+        parts.sort()
+        assert parts[0][0] == 0 and parts[-1][1] == nkb
+        assert all(parts[i][1] == parts[i + 1][0] for i in range(len(parts) - 1))      # a partition of K
+        assert [p[2] for p in parts] == list(range(len(parts)))                         # slice order = K order
+        is_tail = tile >= tiles - tail
+        assert len(parts) == (split if is_tail else 1)
+        sizes = [e - b for b, e, _ in parts]
+        if len(sizes) > 1:
+            assert max(sizes[1:]) - min(sizes[1:]) <= 1                                 # contributors balanced
+            assert sizes[0] >= min(sizes[1:])                                           # the owner takes no less
+    assert longest == -(-tiles // workers)      # nobody does more items than the wave count
+
+
+def test_work_schedule_rejects_impossible_splits():
+    with pytest.raises(ValueError):
+        B.exo_gemm_schedule_work(256, 74, 3, 64, 0)      # 34 tail tiles x 3 slices > 74 workers
+    with pytest.raises(ValueError):
+        B.exo_gemm_schedule_work(10, 4, 0, 8, 0)
+
+
+def test_plan_preview_splits_the_partial_last_wave():
+    # 4096^3 with 256x256 pair tiles: 256 tiles on 74 pairs = 3 whole waves + 34 tiles, cut in two
+    st, info = B.exo_gemm_plan_preview(good(M=4096, N=4096, K=4096, c_dtype=B.BF16), 148)
+    i = info.as_dict()
+    assert (i["cta_group"], i["tile_n"]) == (2, 256) and i["tail_tiles"] == 34 and i["split_k"] == 2
+    assert i["workspace_bytes"] == 34 * 1 * 256 * 256 * 4
+    # never split when told not to, and never more slices than fit the workers or the K loop
+    st, info = B.exo_gemm_plan_preview(good(M=4096, N=4096, K=4096, flags=B.flag_split_k(1)), 148)
+    assert info.split_k == 1 and info.workspace_bytes == 0
+    st, info = B.exo_gemm_plan_preview(good(M=512, N=512, K=256), 148)
+    assert info.split_k == 1                           # 256 k-elements: nothing to cut
+    st, info = B.exo_gemm_plan_preview(good(M=512, N=512, K=12288), 148)
+    i = info.as_dict()
+    assert i["split_k"] >= 2 and i["tail_tiles"] * i["split_k"] <= i["grid"] // i["cta_group"]
+    assert B.exo_gemm_validate(good(flags=B.flag_split_k(9))) == B.ERR_INVALID_ARG

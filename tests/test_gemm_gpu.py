@@ -40,9 +40,10 @@ def check_full(p, flags=0, literal=None):
     return cbuf, got, cref, den, info
 
 
-def flags_for(g, bn, grid=0, ksub=0, epi=0, stages=0):
+def flags_for(g, bn, grid=0, ksub=0, epi=0, stages=0, split=0):
     return (B.flag_cta_group(g) | B.flag_tile_n(bn) | (B.flag_grid_limit(grid) if grid else 0)
-            | B.flag_k_subblocks(ksub) | B.flag_epi_buffers(epi) | B.flag_max_stages(stages))
+            | B.flag_k_subblocks(ksub) | B.flag_epi_buffers(epi) | B.flag_max_stages(stages)
+            | B.flag_split_k(split))
 
 
 TILE_SHAPES = [(1, 64), (1, 128), (1, 256), (2, 128), (2, 256)]
@@ -163,9 +164,11 @@ def test_run_rejects_bad_pointers_before_launch():
 def test_bitwise_determinism_across_runs_and_grid_sizes():
     p = synth.Problem("det", 1000, 1000, 520, BF16, FP32, 0, 1, 0, 1.0, 0.0, seed=8).generate()
     ref = None
+    # with whole-K tiles only, the k order inside every tile is fixed: which CTA computes a tile, and
+    # when, cannot change a bit (K-slicing of tail tiles depends on the grid, so it is switched off here)
     for grid in (0, 2, 14, 148):
         for rep in range(3):
-            cbuf, _, _ = run_gpu(p, flags_for(2, 256, grid))
+            cbuf, _, _ = run_gpu(p, flags_for(2, 256, grid, split=1))
             if ref is None:
                 ref = cbuf.copy()
             assert np.array_equal(cbuf.view(np.uint32), ref.view(np.uint32)), (grid, rep)
@@ -180,10 +183,71 @@ def test_persistent_loop_many_tiles_on_few_ctas():
     check_full(p, flags_for(1, 64, 4, ksub=2, epi=2, stages=3))
 
 
+# ------------------------------------------------------------------ K-slices of the tail tiles
+SPLIT_CASES = [
+    # (M, N, K, ab, cd, alpha, beta, g, bn, grid): tiles vs workers chosen so that a tail exists
+    (1280, 1280, 1024, BF16, FP32, 1.0, 0.0, 2, 256, 16),    # 25 tiles on 8 pairs: 1 tail tile, up to 4 slices
+    (1280, 1000, 2048, FP16, FP16, -0.5, 1.5, 2, 256, 24),   # 20 tiles on 12 pairs: 8 tail tiles -> no room: 1 slice
+    (1000, 1160, 1544, BF16, BF16, 1.0, 1.0, 1, 128, 36),    # 80 tiles on 36 CTAs: 8 tail tiles, 4 slices, ragged K
+    (640, 520, 4096, FP16, FP32, 2.0, 0.0, 2, 128, 0),       # 15 tiles on 74 pairs: split-K of a small problem
+    (512, 512, 12288, BF16, FP32, 1.0, 0.0, 1, 64, 0),       # 32 tiles on 148 CTAs, long K
+    (300, 200, 5000, BF16, BF16, 1.0, -1.0, 1, 256, 0),      # 3 tiles, ragged everywhere
+]
+
+
+@pytest.mark.parametrize("case", SPLIT_CASES, ids=lambda c: "x".join(str(v) for v in c[:3]))
+@pytest.mark.parametrize("split", [0, 2, 8])
+def test_tail_tiles_cut_along_k(case, split):
+    M, N, K, ab, cd, alpha, beta, g, bn, grid = case
+    p = synth.Problem("split", M, N, K, ab, cd, 0, 1, 0, alpha, beta, seed=M + N + K,
+                      dist="normal" if ab == FP16 else "uniform").generate()
+    flags = flags_for(g, bn, grid, split=split)
+    cbuf, got, cref, den, info = check_full(p, flags)
+    assert info["tail_tiles"] * info["split_k"] <= info["grid"] // info["cta_group"]
+    if split == 0 and case in SPLIT_CASES[3:5]:
+        assert info["split_k"] >= 2 and info["workspace_bytes"] > 0
+    # the slices are reduced in a fixed order: bitwise reproducible, also across repeated runs of one plan
+    dp = harness.DeviceProblem(p, flags)
+    try:
+        for _ in range(3):
+            dp.reset_c()
+            dp.run()
+            assert np.array_equal(dp.result_buffer(), cbuf)
+        dp.plan.check()
+    finally:
+        dp.close()
+
+
+def test_split_plan_recovers_after_a_timed_out_run():
+    import torch
+    p = synth.Problem("split_tmo", 640, 520, 4096, BF16, FP32, 0, 1, 0, 1.0, 0.0, seed=77).generate()
+    dp = harness.DeviceProblem(p, flags_for(2, 128, split=4))
+    try:
+        assert dp.plan.info()["split_k"] >= 2
+        dp.run()
+        torch.cuda.synchronize()
+        dp.plan.check()
+        good_bits = dp.result_buffer().copy()
+        # CTA 0's producer leaves out one k-block: its MMA issuer gives up after 20 ms, the slice never
+        # arrives, the owner of that tile gives up too, every role returns
+        assert B.exo_gemm_debug_set(dp.plan.handle, 20, 3) == B.OK
+        dp.run()
+        torch.cuda.synchronize()
+        st, detail = B.exo_gemm_check(dp.plan.handle)
+        assert st == B.ERR_DEVICE_TIMEOUT, detail
+        dp.reset_c()
+        dp.run()
+        torch.cuda.synchronize()
+        dp.plan.check()
+        assert np.array_equal(dp.result_buffer(), good_bits)
+    finally:
+        dp.close()
+
+
 def test_bounded_wait_reports_timeout_and_the_plan_stays_usable():
     import torch
     p = synth.Problem("tmo", 512, 512, 1024, BF16, FP32, 0, 1, 0, 1.0, 0.0, seed=10).generate()
-    dp = harness.DeviceProblem(p, flags_for(1, 128))
+    dp = harness.DeviceProblem(p, flags_for(1, 128, split=1))
     try:
         # the producer of CTA 0 leaves out the loads of its k-block 5: the MMA issuer's wait runs
         # out after 20 ms, every role leaves its loop, TMEM is freed, the kernel returns

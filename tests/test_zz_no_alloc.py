@@ -31,7 +31,10 @@ CASES = [
 def test_static_entry_point_matches_the_plan_based_one_twice_in_a_row(p):
     import torch
     p.generate()
-    want_buf, _ = harness.gemm_host(p)                       # exo_gemm_create + exo_gemm_run
+    # exo_gemm_create + exo_gemm_run.  K-slicing of tail tiles needs a device workspace, which the
+    # allocation-free entry point never uses, so the reference plan is told not to slice either:
+    # then both run the same kernel with the same work list.
+    want_buf, _ = harness.gemm_host(p, B.flag_split_k(1))
     want = oracle.logical_view(want_buf, p.M, p.N, p.c_layout, p.ldc, p.c_dtype)
     cref, den = oracle.gemm_problem(p)
     slack = oracle.output_rounding_slack(cref, p.c_dtype)
@@ -53,7 +56,11 @@ def test_static_entry_point_matches_the_plan_based_one_twice_in_a_row(p):
         buf = dC.cpu().numpy().view(synth.storage_np_dtype(p.c_dtype))
         got = oracle.logical_view(buf, p.M, p.N, p.c_layout, p.ldc, p.c_dtype)
         assert oracle.max_error(got, want, den) <= TOL       # against the existing entry point
-        assert np.array_equal(buf, want_buf)                 # same kernel, same plan: same bits
+        assert np.array_equal(buf, want_buf)                 # same kernel, same work list: same bits
+    # and against the library's default plan for this problem (which may slice K), within tolerance
+    auto_buf, _ = harness.gemm_host(p)
+    auto = oracle.logical_view(auto_buf, p.M, p.N, p.c_layout, p.ldc, p.c_dtype)
+    assert (np.abs(got - auto) <= TOL * den + 2 * slack).all()
 
 
 def test_static_entry_point_checks_its_arguments_like_the_others():
