@@ -397,11 +397,94 @@ def cpu_baseline(p, workload):
             "sample": f"rows 0..{rows} of C ({rows}x{p.N}x{p.K}) of {workload}, {dt:.1f} s wall"}
 
 
+def run_sweep(args, rank, world, local_rank):
+    """The shape sweep: M, N, K each in {512, 1000, 2048, 3072, 6144, 12288}, bf16 in, fp32 out.
+
+    Timing only (parity of sweep shapes is covered by the GPU tests on host-generated inputs):
+    operands are drawn on the device, uniform[-1, 1) rounded to bf16.  Every shape gets its own plan,
+    3 warm-up and `--steps` timed launches; the line reports whole-sweep throughput and, per shape,
+    TFLOP/s and the fraction of roofline(shape) = min(tensor peak, AI x HBM bandwidth).
+    """
+    import itertools
+    import torch
+    from paper_2609_16389_b200 import binding as B
+    from paper_2609_16389_b200 import synth
+    if rank != 0:
+        return
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    pk = peaks()
+    stream = torch.cuda.current_stream(dev)
+    steps = max(3, min(args.steps, 20))
+    rows, tot_flop, tot_ms, launches = [], 0.0, 0.0, 0
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    for (M, N, K) in itertools.product(synth.SWEEP_DIMS, repeat=3):
+        set_bytes = 2 * (M * K + K * N) + 4 * M * N
+        n_sets = int(min(8, max(1, np.ceil(2.0 * L2_BYTES / set_bytes))))
+        sets = [((torch.rand(M, K, device=dev) * 2 - 1).to(torch.bfloat16),
+                 (torch.rand(N, K, device=dev) * 2 - 1).to(torch.bfloat16),
+                 torch.empty(M, N, device=dev, dtype=torch.float32)) for _ in range(n_sets)]
+        plan = B.Plan(B.make_desc(M, N, K, B.BF16, B.FP32, B.ROW_MAJOR, B.COL_MAJOR, B.ROW_MAJOR,
+                                  device=local_rank, flags=args.flags))
+
+        def step(i):
+            a, b, c = sets[i % n_sets]
+            plan.run(a.data_ptr(), b.data_ptr(), c.data_ptr(), 1.0, 0.0, stream.cuda_stream)
+
+        for i in range(3):
+            step(i)
+        torch.cuda.synchronize(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(steps):
+            step(i)
+        e1.record(stream)
+        torch.cuda.synchronize(dev)
+        plan.check()
+        ms = e0.elapsed_time(e1) / steps
+        info = plan.info()
+        plan.close()
+        flop = 2.0 * M * N * K
+        ai = flop / set_bytes
+        roof = min(pk["tflops_burst"], ai * pk["hbm_gbs"] / 1e3)
+        tf = flop / (ms * 1e-3) / 1e12
+        rows.append({"M": M, "N": N, "K": K, "us": round(ms * 1e3, 2), "tflops": round(tf, 1),
+                     "roofline_tflops": round(roof, 1), "frac": round(tf / roof, 3),
+                     "plan": [info["cta_group"], info["tile_n"], info["tile_k"], info["split_k"]],
+                     "l2_sets": n_sets})
+        tot_flop += flop * steps
+        tot_ms += ms * steps
+        launches += steps
+        del sets
+    clocks = sampler.stop()
+    fr = np.array([r["frac"] for r in rows])
+    line = {
+        "metric": METRIC, "value": tot_flop / (tot_ms * 1e-3) / 1e12, "unit": UNIT, "n_gpus": 1, "steps": steps,
+        "warmup": 3, "ms_per_step": tot_ms / launches, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16 in, fp32 accumulate", "data": "synthetic (device-generated, timing only)",
+        "config": {"workload": "sweep_216", "shapes": len(rows), "dims": list(synth.SWEEP_DIMS),
+                   "layouts": "Ar Bc Cr", "c_dtype": "fp32",
+                   "l2": "operand sets rotated to exceed 2x L2 where 8 sets suffice, else L2-warm (l2_sets per shape)"},
+        "roofline": {"bound": "mixed", "achieved": float(np.exp(np.log(fr).mean())), "peak": 1.0, "unit": "fraction",
+                     "frac": float(np.exp(np.log(fr).mean())), "traffic": None,
+                     "note": "geometric mean over shapes of TFLOP/s / min(measured tensor peak, AI x measured HBM GB/s)",
+                     "min_frac": float(fr.min()), "max_frac": float(fr.max())},
+        "gpu_launches": launches, "clocks": clocks, "sweep": rows,
+    }
+    print(json.dumps(line), flush=True)
+
+
 def main():
     args = parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.workload == "sweep":
+        if args.impl == "reference":
+            raise SystemExit("the reference arm times one workload; pick e.g. --workload sweep_1000x1000x1000")
+        run_sweep(args, rank, world, local_rank)
+        return
     if args.workload not in WORKLOADS and not args.workload.startswith("sweep_"):
         raise SystemExit(f"unknown workload {args.workload}")
     if args.impl == "reference":

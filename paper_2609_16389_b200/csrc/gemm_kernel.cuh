@@ -550,7 +550,9 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       if ((acc ^= 1u) == 0u) acc_ph ^= 1u;
     }
     __syncwarp();
-    if (ptx::elect_one()) ptx::bulk_wait<0>();  // all stores of this warp have completed
+    // The stores must have read their staging buffers before this CTA's shared memory goes away;
+    // their global writes complete on their own and are visible when the kernel has ended.
+    if (ptx::elect_one()) ptx::bulk_wait_read<0>();
     __syncwarp();
   }
 

@@ -71,6 +71,8 @@ inline exo_gemm_status_t validate_desc(const exo_gemm_desc_t* d) {
   // beyond here the call is a legal BLAS call; what follows is this library's supported set
   if (d->ab_dtype == EXO_GEMM_FP32) return EXO_GEMM_ERR_UNSUPPORTED;
   if (d->c_dtype != EXO_GEMM_FP32 && d->c_dtype != d->ab_dtype) return EXO_GEMM_ERR_UNSUPPORTED;
+  // the persistent scheduler indexes tiles (at least 128 x 64 each) and k-blocks with 32 bits
+  if (((d->M + 127) / 128) * ((d->N + 63) / 64) >= (1LL << 31)) return EXO_GEMM_ERR_UNSUPPORTED;
   // a matrix that is never touched (empty problem, K == 0) has no stride rule
   const bool c_used = d->M > 0 && d->N > 0;
   const bool ab_used = c_used && d->K > 0;

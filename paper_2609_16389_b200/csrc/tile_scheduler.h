@@ -35,21 +35,23 @@ struct Raster {
 
 EXO_HD int64_t raster_total(const Raster& r) { return (int64_t)r.tiles_m * r.tiles_n; }
 
-// linear index -> tile coordinate
-EXO_HD TileCoord raster_decode(const Raster& r, int64_t t) {
+// linear index -> tile coordinate.  Tile counts stay below 2^31 (checked by the host plan), so
+// the arithmetic is 32-bit: these divisions sit on the critical path of every tile.
+EXO_HD TileCoord raster_decode(const Raster& r, int64_t t64) {
+  const uint32_t t = (uint32_t)t64;
   // "major" = the banded dimension, "minor" = the other one
-  const int32_t major = r.along_m ? r.tiles_m : r.tiles_n;
-  const int32_t minor = r.along_m ? r.tiles_n : r.tiles_m;
-  const int64_t per_band = (int64_t)r.band * minor;
-  const int32_t b = (int32_t)(t / per_band);
-  const int64_t in_band = t - (int64_t)b * per_band;
-  const int32_t first = b * r.band;
-  const int32_t width = (major - first) < r.band ? (major - first) : r.band;  // last band may be narrower
-  const int32_t i_minor = (int32_t)(in_band / width);
-  const int32_t i_major = first + (int32_t)(in_band - (int64_t)i_minor * width);
+  const uint32_t major = (uint32_t)(r.along_m ? r.tiles_m : r.tiles_n);
+  const uint32_t minor = (uint32_t)(r.along_m ? r.tiles_n : r.tiles_m);
+  const uint32_t per_band = (uint32_t)r.band * minor;
+  const uint32_t b = t / per_band;
+  const uint32_t in_band = t - b * per_band;
+  const uint32_t first = b * (uint32_t)r.band;
+  const uint32_t width = (major - first) < (uint32_t)r.band ? (major - first) : (uint32_t)r.band;  // last band may be narrower
+  const uint32_t i_minor = in_band / width;
+  const uint32_t i_major = first + (in_band - i_minor * width);
   TileCoord c;
-  c.m = r.along_m ? i_major : i_minor;
-  c.n = r.along_m ? i_minor : i_major;
+  c.m = (int32_t)(r.along_m ? i_major : i_minor);
+  c.n = (int32_t)(r.along_m ? i_minor : i_major);
   return c;
 }
 
@@ -94,8 +96,8 @@ EXO_HD bool work_item(const WorkPlan& w, int64_t worker, int64_t num_workers, in
   }
   if (t - w.full_tiles != worker) return false;             // only the wave right after the full ones
   if (worker >= (int64_t)w.tail_tiles * w.split) return false;
-  const int32_t ti = (int32_t)(worker / w.split);
-  const int32_t sl = (int32_t)(worker - (int64_t)ti * w.split);
+  const int32_t ti = (int32_t)((uint32_t)worker / (uint32_t)w.split);
+  const int32_t sl = (int32_t)((uint32_t)worker - (uint32_t)ti * (uint32_t)w.split);
   out->tile = w.full_tiles + ti;
   out->tail_index = w.split > 1 ? ti : -1;
   out->slice = sl;
@@ -109,9 +111,9 @@ EXO_HD bool work_item(const WorkPlan& w, int64_t worker, int64_t num_workers, in
     out->kb_begin = 0;
     out->kb_end = own;
   } else {
-    const int64_t rest = num_k_blocks - own;
-    out->kb_begin = own + (int32_t)((rest * (sl - 1)) / (w.split - 1));
-    out->kb_end = own + (int32_t)((rest * sl) / (w.split - 1));
+    const uint32_t rest = (uint32_t)(num_k_blocks - own);   // rest * slice < 2^31: both are small
+    out->kb_begin = own + (int32_t)((rest * (uint32_t)(sl - 1)) / (uint32_t)(w.split - 1));
+    out->kb_end = own + (int32_t)((rest * (uint32_t)sl) / (uint32_t)(w.split - 1));
   }
   return true;
 }
