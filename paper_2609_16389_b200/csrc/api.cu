@@ -390,13 +390,18 @@ exo_gemm_status_t exo_gemm_run(exo_gemm_handle_t plan, const void* A, const void
   lc.blockDim = dim3(kNumThreads, 1, 1);
   lc.dynamicSmemBytes = plan->smem_bytes;
   lc.stream = (cudaStream_t)cuda_stream;
-  cudaLaunchAttribute at[1];
+  cudaLaunchAttribute at[2];
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = cfg.cta_group;
   at[0].val.clusterDim.y = 1;
   at[0].val.clusterDim.z = 1;
+  // Programmatic dependent launch: this kernel's CTAs may start (barrier set-up, TMEM allocation)
+  // while the previous kernel in the stream drains; the kernel waits for that kernel before it
+  // touches global memory, so stream order is kept for data.
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
   lc.attrs = at;
-  lc.numAttrs = 1;
+  lc.numAttrs = 2;
   if (split_now) {  // arrival counters only grow: this run is complete at epoch * arrivals-per-run
     const uint32_t epoch = plan->split_epoch.fetch_add(1) + 1;
     prm.split_target = epoch * (uint32_t)((cfg.split - 1) * kEpiWarps * cfg.cta_group);

@@ -186,6 +186,12 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   uint32_t tmem_base;
   asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot) : "memory");
 
+  // Everything above touched only this CTA's shared and tensor memory, so with programmatic
+  // dependent launch it overlaps the tail of the previous kernel in the stream.  From here on global
+  // memory is read and written: wait for that kernel, then let our own successor start likewise.
+  ptx::grid_dependency_wait();
+  ptx::grid_launch_dependents();
+
   bool ok = true;
   if (threadIdx.x == 0) EXO_TRACE(2, 4094, 0, 4096);
 

@@ -269,6 +269,37 @@ def test_bounded_wait_reports_timeout_and_the_plan_stays_usable():
         dp.close()
 
 
+def test_back_to_back_dependent_gemms_keep_stream_order():
+    """D = (A B) E enqueued as two GEMMs on one stream without a host sync in between: the second
+    kernel may start early (programmatic dependent launch) but must not read C before it is written."""
+    import torch
+    M, K, N, N2 = 1000, 520, 776, 392
+    p1 = synth.Problem("chain1", M, N, K, BF16, BF16, 0, 1, 0, 1.0, 0.0, seed=31).generate()
+    p2 = synth.Problem("chain2", M, N2, N, BF16, FP32, 0, 1, 0, 1.0, 0.0, seed=32).generate()
+    dev = torch.device("cuda:0")
+    dA, dB = harness._to_device(p1.A, dev), harness._to_device(p1.B, dev)
+    dE = harness._to_device(p2.B, dev)
+    stream = torch.cuda.current_stream(dev).cuda_stream
+    with B.Plan(harness.desc_of(p1)) as g1, B.Plan(harness.desc_of(p2)) as g2:
+        ref = None
+        for rep in range(5):
+            dC = torch.full((M * N * 2,), 0xFF, dtype=torch.uint8, device=dev)      # NaN patterns until GEMM 1 writes
+            dD = torch.zeros(M * N2 * 4, dtype=torch.uint8, device=dev)
+            g1.run(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), 1.0, 0.0, stream)
+            g2.run(dC.data_ptr(), dE.data_ptr(), dD.data_ptr(), 1.0, 0.0, stream)
+            torch.cuda.synchronize(dev)
+            g1.check(); g2.check()
+            c_host = dC.cpu().numpy().view(np.uint16)
+            d_host = dD.cpu().numpy().view(np.float32)
+            # oracle for the second GEMM on the first one's actual (bf16-rounded) output
+            p2.A = c_host.copy()
+            cref, den = oracle.gemm_problem(p2)
+            got = d_host.reshape(M, N2).astype(np.float64)
+            assert oracle.max_error(got, cref, den) <= TOL, rep
+            ref = d_host.copy() if ref is None else ref
+            assert np.array_equal(d_host, ref)
+
+
 # ------------------------------------------------------------------ the benchmark configurations
 def structured_sample(M, N, rng, n_random=1 << 14):
     """Rows/columns next to every 128/256 tile boundary crossed with random partners, plus random entries."""
