@@ -135,20 +135,42 @@ inline double shape_efficiency(int cta_group, int bn) {
   return bn == 256 ? 0.86 : (bn == 128 ? 0.66 : 0.40);
 }
 
-// Estimated time of the whole problem in SM clocks for one candidate shape.
-inline double estimate_clocks(int64_t M, int64_t N, int64_t K, int cta_group, int bn, int max_workers) {
+// How many K-slices each tile of the partial last wave is cut into (1 = not cut).
+inline int split_factor(int64_t tiles, int64_t workers, int64_t K, int ksub, const FlagOverrides& o) {
+  const int64_t tail = tiles % workers;
+  if (tail == 0 || o.split == 1 || o.no_workspace) return 1;
+  const int64_t k_blocks = (K + kBlockK * ksub - 1) / (kBlockK * ksub);
+  int64_t f = workers / tail;
+  const int64_t by_k = (K / kBlockK) / 4;   // every slice keeps at least 256 k-elements
+  if (f > by_k) f = by_k;
+  if (f > 8) f = 8;
+  if (o.split >= 2 && o.split < f) f = o.split;
+  if (f > k_blocks) f = k_blocks;
+  return f >= 2 ? (int)f : 1;
+}
+
+// Estimated time of the whole problem in SM clocks for one candidate tile shape: whole waves of
+// tiles, then the partial last wave (cut along K if that pays), plus what is exposed once per launch.
+inline double estimate_clocks(int64_t M, int64_t N, int64_t K, int cta_group, int bn, int max_workers,
+                              const FlagOverrides& o) {
   const int64_t tm = (M + 128 * cta_group - 1) / (128 * cta_group);
   const int64_t tn = (N + bn - 1) / bn;
   const int64_t tiles = tm * tn;
   if (tiles == 0) return 0.0;
-  const int64_t workers = tiles < max_workers ? tiles : max_workers;
-  const int64_t waves = (tiles + workers - 1) / workers;
+  const int ksub = o.ksub ? o.ksub : (bn == 256 ? 1 : 2);
   const int64_t nkb = (K + kBlockK - 1) / kBlockK;
-  const double mainloop = (double)nkb * 2.0 * bn / shape_efficiency(cta_group, bn);  // clocks per tile
-  const double drain = 22.0 * bn;             // draining one accumulator (measured ~5.9k clocks at N = 256)
-  const double epilogue = drain + 1500.0;     // exposed once at the end, plus pipeline fill latency
+  const double mainloop = (double)nkb * 2.0 * bn / shape_efficiency(cta_group, bn);  // clocks per whole tile
+  const double drain = 22.0 * bn;             // draining one accumulator (measured 5-7k clocks at N = 256)
   const double per_tile = mainloop > drain ? mainloop : drain;  // small K: the epilogue bounds a tile
-  return (double)waves * per_tile + epilogue;
+  const int64_t full_waves = tiles / max_workers;
+  const int64_t tail = tiles % max_workers;
+  double t = (double)full_waves * per_tile;
+  if (tail > 0) {
+    const int f = split_factor(tiles, max_workers, K, ksub, o);
+    if (f > 1) t += mainloop / f + (30.0 + 8.0 * (f - 1)) * bn;  // slice + exchange of partial sums
+    else t += per_tile;
+  }
+  return t + drain + 3000.0;  // the last epilogue and the pipeline fill are exposed once
 }
 
 inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int sm_count,
@@ -162,7 +184,10 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
     if (o.tile_n && o.tile_n != n) continue;
     if (g == 2 && max_pairs < 1) continue;
     const int workers = g == 2 ? max_pairs : sm_count;
-    const double t = estimate_clocks(c.M, c.N, c.K, g, n, workers);
+    int w_eff = workers;
+    if (o.grid_limit && o.grid_limit / g < w_eff) w_eff = o.grid_limit / g;
+    if (w_eff < 1) w_eff = 1;
+    const double t = estimate_clocks(c.M, c.N, c.K, g, n, w_eff, o);
     if (best_g == 0 || t < best * 0.999) { best = t; best_g = g; best_n = n; }
   }
   if (best_g == 0) { best_g = o.cta_group ? o.cta_group : 1; best_n = o.tile_n ? o.tile_n : 128; }
@@ -191,17 +216,8 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
     const int64_t full_waves = tiles / workers;
     cfg.full_tiles = full_waves * workers;
     cfg.tail_tiles = (int)(tiles - cfg.full_tiles);
-    cfg.split = 1;
     const int64_t k_blocks = (c.K + kBlockK * cfg.ksub - 1) / (kBlockK * cfg.ksub);
-    if (cfg.tail_tiles > 0 && o.split != 1 && !o.no_workspace) {
-      int64_t f = workers / cfg.tail_tiles;
-      const int64_t by_k = (c.K / kBlockK) / 4;   // every slice keeps at least 256 k-elements
-      if (f > by_k) f = by_k;
-      if (f > 8) f = 8;
-      if (o.split >= 2 && o.split < f) f = o.split;
-      if (f > k_blocks) f = k_blocks;
-      if (f >= 2) cfg.split = (int)f;
-    }
+    cfg.split = split_factor(tiles, workers, c.K, cfg.ksub, o);
     // Publishing a 128 x N fp32 partial takes a contributor about as long as 8 k-blocks of 64
     // (128*N*4 bytes at ~30 B/clk against 2*N clocks of MMA per k-block); let the owner compute that
     // much longer, so that the partials are there when it finishes.
