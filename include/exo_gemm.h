@@ -102,7 +102,7 @@ typedef struct {
   int32_t split_k;         /* K-slices per tile of the partial last wave (1 = none)            */
   int32_t tail_tiles;      /* tiles in that partial last wave                                  */
   int32_t workspace_bytes; /* device scratch the plan owns for the slices' partial sums        */
-  int32_t reserved[1];
+  int32_t batch_count;     /* matrices per launch (1 unless created by exo_gemm_create_batched) */
 } exo_gemm_info_t;
 
 /*
@@ -123,6 +123,22 @@ exo_gemm_status_t exo_gemm_validate(const exo_gemm_desc_t* desc);
  * touches no user matrix.  *out is written only on success.
  */
 exo_gemm_status_t exo_gemm_create(exo_gemm_handle_t* out, const exo_gemm_desc_t* desc);
+
+/*
+ * Strided-batched variant (the paper's Section 6 also measures batched GEMM, against
+ * cublasSgemmStridedBatched): `batch_count` independent products
+ * C_i = alpha*A_i*B_i + beta*C_i, i = 0 .. batch_count-1, where matrix i of each operand
+ * starts stride_x ELEMENTS after matrix i-1 and every matrix has the descriptor's
+ * shape, layout and leading dimension.  One persistent launch covers the whole
+ * batch (the batch index is the third coordinate of the TMA tensor maps and part of
+ * the tile index).  stride_a or stride_b may be 0 (that operand is shared by all
+ * products); the C matrices must not overlap (stride_c >= the extent of one C,
+ * else ERR_INVALID_ARG); each stride times its element size must be a multiple of
+ * 16 bytes (else ERR_UNSUPPORTED); 1 <= batch_count <= 65535.  exo_gemm_run then
+ * takes the base pointers of matrix 0.  batch_count == 1 is exo_gemm_create.
+ */
+exo_gemm_status_t exo_gemm_create_batched(exo_gemm_handle_t* out, const exo_gemm_desc_t* desc, int64_t batch_count,
+                                          int64_t stride_a, int64_t stride_b, int64_t stride_c);
 
 /*
  * Enqueues C = alpha*A*B + beta*C on cuda_stream (a cudaStream_t; NULL = the

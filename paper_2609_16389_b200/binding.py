@@ -19,6 +19,7 @@ EXPORTED_SYMBOLS = (
     "exo_gemm_validate", "exo_gemm_create", "exo_gemm_run", "exo_gemm_check", "exo_gemm_plan_preview",
     "exo_gemm_get_info", "exo_gemm_destroy", "exo_gemm_status_string", "exo_gemm_last_cuda_error",
     "exo_gemm_schedule_enumerate", "exo_gemm_debug_set", "exo_gemm_run_static", "exo_gemm_schedule_work",
+    "exo_gemm_create_batched",
 )
 
 
@@ -46,11 +47,11 @@ class Info(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "cta_group", "tile_m", "tile_n", "tile_k", "stages", "grid", "smem_bytes", "tmem_columns",
         "tiles_m", "tiles_n", "raster_along_m", "raster_band", "swapped", "sm_count",
-        "kernel_launches_per_run", "epilogue_buffers", "split_k", "tail_tiles", "workspace_bytes")] + [
-        ("reserved", ctypes.c_int32 * 1)]
+        "kernel_launches_per_run", "epilogue_buffers", "split_k", "tail_tiles", "workspace_bytes",
+        "batch_count")]
 
     def as_dict(self):
-        return {n: getattr(self, n) for n, _ in self._fields_ if n != "reserved"}
+        return {n: getattr(self, n) for n, _ in self._fields_}
 
 
 class ExoGemmError(RuntimeError):
@@ -75,6 +76,8 @@ def lib():
         L.exo_gemm_validate.argtypes = [ctypes.POINTER(Desc)]
         L.exo_gemm_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(Desc)]
         L.exo_gemm_run.argtypes = [vp, vp, vp, vp, ctypes.c_float, ctypes.c_float, vp]
+        L.exo_gemm_create_batched.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(Desc), i64, i64, i64, i64]
+        L.exo_gemm_create_batched.restype = ctypes.c_int
         L.exo_gemm_check.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
         L.exo_gemm_plan_preview.argtypes = [ctypes.POINTER(Desc), i32, ctypes.POINTER(Info)]
         L.exo_gemm_get_info.argtypes = [vp, ctypes.POINTER(Info)]
@@ -117,6 +120,12 @@ def exo_gemm_validate(desc: Desc) -> int:
 def exo_gemm_create(desc: Desc):
     h = ctypes.c_void_p()
     st = lib().exo_gemm_create(ctypes.byref(h), ctypes.byref(desc))
+    return st, (h if st == OK else None)
+
+
+def exo_gemm_create_batched(desc: Desc, batch_count: int, stride_a: int, stride_b: int, stride_c: int):
+    h = ctypes.c_void_p()
+    st = lib().exo_gemm_create_batched(ctypes.byref(h), ctypes.byref(desc), batch_count, stride_a, stride_b, stride_c)
     return st, (h if st == OK else None)
 
 
@@ -199,8 +208,12 @@ def exo_gemm_schedule_work(tiles, num_workers, split, num_k_blocks, worker, owne
 class Plan:
     """Owns one handle.  ``run`` takes raw device pointers (ints) and a stream handle."""
 
-    def __init__(self, desc: Desc):
-        st, h = exo_gemm_create(desc)
+    def __init__(self, desc: Desc, batch=None):
+        """``batch`` = (count, stride_a, stride_b, stride_c) in elements for a strided batch."""
+        if batch is None:
+            st, h = exo_gemm_create(desc)
+        else:
+            st, h = exo_gemm_create_batched(desc, *batch)
         if st != OK:
             raise ExoGemmError(st, "exo_gemm_create")
         self.handle = h

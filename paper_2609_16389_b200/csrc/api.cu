@@ -82,6 +82,27 @@ static CUresult encode_2d(CUtensorMap* map, int dtype, const void* base, uint64_
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
 }
 
+// The same with a third dimension: `batch` matrices `batch_stride` elements apart, boxes one matrix deep.
+static CUresult encode_3d(CUtensorMap* map, int dtype, const void* base, uint64_t inner, uint64_t outer,
+                          uint64_t ld, uint64_t batch, uint64_t batch_stride, uint32_t box_inner,
+                          uint32_t box_outer, bool operand) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return CUDA_ERROR_NOT_FOUND;
+  const CUtensorMapDataType dt = dtype == EXO_GEMM_FP32   ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                                 : dtype == EXO_GEMM_FP16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
+                                                          : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+  const uint64_t es = (uint64_t)elem_bytes(dtype);
+  // A repeated operand (stride 0) is described as a batch of one; the kernel then always asks for z = 0.
+  cuuint64_t dims[3] = {inner, outer, batch_stride ? batch : 1};
+  cuuint64_t strides[2] = {ld * es, batch_stride ? batch_stride * es : ld * es * (outer ? outer : 1)};
+  cuuint32_t box[3] = {box_inner, box_outer, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, dt, 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B,
+            operand ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_NONE,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+}
+
 }  // namespace exo
 
 struct exo_gemm_plan {
@@ -146,6 +167,7 @@ void fill_info(const exo_gemm_plan* p, exo_gemm_info_t* info) {
   info->epilogue_buffers = p->cfg.epi_bufs;
   info->split_k = p->cfg.split;
   info->tail_tiles = p->cfg.tail_tiles;
+  info->batch_count = (int32_t)p->canon.batch;
   info->workspace_bytes = (int32_t)(p->cfg.workspace_bytes > 2147483647LL ? 2147483647LL : p->cfg.workspace_bytes);
 }
 
@@ -230,9 +252,17 @@ exo_gemm_status_t exo_gemm_plan_preview(const exo_gemm_desc_t* desc, int32_t sm_
   return EXO_GEMM_OK;
 }
 
+exo_gemm_status_t exo_gemm_create_batched(exo_gemm_handle_t* out, const exo_gemm_desc_t* desc, int64_t batch_count,
+                                          int64_t stride_a, int64_t stride_b, int64_t stride_c);
+
 exo_gemm_status_t exo_gemm_create(exo_gemm_handle_t* out, const exo_gemm_desc_t* desc) {
+  return exo_gemm_create_batched(out, desc, 1, 0, 0, 0);
+}
+
+exo_gemm_status_t exo_gemm_create_batched(exo_gemm_handle_t* out, const exo_gemm_desc_t* desc, int64_t batch_count,
+                                          int64_t stride_a, int64_t stride_b, int64_t stride_c) {
   if (!out) return EXO_GEMM_ERR_NULL;
-  exo_gemm_status_t st = validate_desc(desc);
+  exo_gemm_status_t st = validate_batch(desc, batch_count, stride_a, stride_b, stride_c);
   if (st != EXO_GEMM_OK) return st;
 
   int device = desc->device;
@@ -254,7 +284,7 @@ exo_gemm_status_t exo_gemm_create(exo_gemm_handle_t* out, const exo_gemm_desc_t*
   exo_gemm_plan* p = new (std::nothrow) exo_gemm_plan{};
   if (!p) return EXO_GEMM_ERR_CUDA;
   p->desc = *desc;
-  p->canon = canonicalize(*desc);
+  p->canon = canonicalize(*desc, batch_count, stride_a, stride_b, stride_c);
   p->device = device;
   p->sm_count = sms;
   p->dbg_timeout_ms = 0;
@@ -347,6 +377,10 @@ exo_gemm_status_t exo_gemm_run(exo_gemm_handle_t plan, const void* A, const void
   const int stage_k = kBlockK * cfg.ksub;
   prm.num_k_blocks = read_ab ? (int32_t)((cn.K + stage_k - 1) / stage_k) : 0;
   prm.raster = Raster{cfg.tiles_m, cfg.tiles_n, cfg.band, cfg.along_m};
+  prm.batch = (uint32_t)cn.batch;
+  prm.tiles_per_batch = (uint32_t)cfg.tiles_m * (uint32_t)cfg.tiles_n;
+  prm.a_z_mask = cn.stride_a ? 0xFFFFFFFFu : 0u;
+  prm.b_z_mask = cn.stride_b ? 0xFFFFFFFFu : 0u;
   prm.stages = cfg.stages;
   prm.epi_bufs = cfg.epi_bufs;
   // the tail tiles are cut along K only when there is a K loop to cut and scratch to reduce through
@@ -371,16 +405,32 @@ exo_gemm_status_t exo_gemm_run(exo_gemm_handle_t plan, const void* A, const void
   memset(&tm_b, 0, sizeof tm_b);
   CUresult r;
   const int b_rows = cfg.tile_n / cfg.cta_group;
-  if (read_ab) {
-    r = cn.a_mn_major ? encode_2d(&tm_a, d.ab_dtype, opA, cn.M, cn.K, cn.lda, 64, stage_k, true)
-                      : encode_2d(&tm_a, d.ab_dtype, opA, cn.K, cn.M, cn.lda, kBlockK, kBlockM, true);
+  const uint32_t c_box = d.c_dtype == EXO_GEMM_FP32 ? 32 : 64;
+  if (cn.batch <= 1) {
+    if (read_ab) {
+      r = cn.a_mn_major ? encode_2d(&tm_a, d.ab_dtype, opA, cn.M, cn.K, cn.lda, 64, stage_k, true)
+                        : encode_2d(&tm_a, d.ab_dtype, opA, cn.K, cn.M, cn.lda, kBlockK, kBlockM, true);
+      if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return EXO_GEMM_ERR_CUDA; }
+      r = cn.b_mn_major ? encode_2d(&tm_b, d.ab_dtype, opB, cn.N, cn.K, cn.ldb, 64, stage_k, true)
+                        : encode_2d(&tm_b, d.ab_dtype, opB, cn.K, cn.N, cn.ldb, kBlockK, b_rows, true);
+      if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return EXO_GEMM_ERR_CUDA; }
+    }
+    r = encode_2d(&tm_c, d.c_dtype, C, cn.N, cn.M, cn.ldc, c_box, 32, false);
     if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return EXO_GEMM_ERR_CUDA; }
-    r = cn.b_mn_major ? encode_2d(&tm_b, d.ab_dtype, opB, cn.N, cn.K, cn.ldb, 64, stage_k, true)
-                      : encode_2d(&tm_b, d.ab_dtype, opB, cn.K, cn.N, cn.ldb, kBlockK, b_rows, true);
+  } else {  // strided batch: the matrix index is the third tensor-map coordinate
+    if (read_ab) {
+      r = cn.a_mn_major
+              ? encode_3d(&tm_a, d.ab_dtype, opA, cn.M, cn.K, cn.lda, cn.batch, cn.stride_a, 64, stage_k, true)
+              : encode_3d(&tm_a, d.ab_dtype, opA, cn.K, cn.M, cn.lda, cn.batch, cn.stride_a, kBlockK, kBlockM, true);
+      if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return EXO_GEMM_ERR_CUDA; }
+      r = cn.b_mn_major
+              ? encode_3d(&tm_b, d.ab_dtype, opB, cn.N, cn.K, cn.ldb, cn.batch, cn.stride_b, 64, stage_k, true)
+              : encode_3d(&tm_b, d.ab_dtype, opB, cn.K, cn.N, cn.ldb, cn.batch, cn.stride_b, kBlockK, b_rows, true);
+      if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return EXO_GEMM_ERR_CUDA; }
+    }
+    r = encode_3d(&tm_c, d.c_dtype, C, cn.N, cn.M, cn.ldc, cn.batch, cn.stride_c, c_box, 32, false);
     if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return EXO_GEMM_ERR_CUDA; }
   }
-  r = encode_2d(&tm_c, d.c_dtype, C, cn.N, cn.M, cn.ldc, d.c_dtype == EXO_GEMM_FP32 ? 32 : 64, 32, false);
-  if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return EXO_GEMM_ERR_CUDA; }
   if (!read_ab) { tm_a = tm_c; tm_b = tm_c; }  // never dereferenced for data; keeps the prefetch valid
 
   DeviceGuard guard(plan->device);

@@ -206,7 +206,9 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       WorkItem wi;
       if (!work_item(p.work, worker, num_workers, it, nkb, &wi)) break;
       const int64_t t = wi.tile;
-      const TileCoord tc = raster_decode(p.raster, t);
+      const bool batched = p.batch > 1;
+      const uint32_t bz = batched ? (uint32_t)t / p.tiles_per_batch : 0u;  // which matrix of the batch
+      const TileCoord tc = raster_decode(p.raster, batched ? (uint32_t)t - bz * p.tiles_per_batch : t);
       const int32_t a_mn0 = tc.m * (kBlockM * CTA_GROUP) + (int32_t)cta_rank * kBlockM;
       const int32_t b_mn0 = tc.n * BN + (int32_t)cta_rank * B_ROWS;
       for (int32_t kb = wi.kb_begin; kb < wi.kb_end; ++kb) {
@@ -223,8 +225,14 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             const uint32_t bar = full0 + 8u * s;
             const int32_t k0 = kb * STAGE_K;
             auto load = [&](uint32_t dst, const CUtensorMap* map, int32_t x, int32_t y) {
-              if constexpr (PAIR) ptx::tma_load_2d_pair(dst, map, x, y, bar);
-              else ptx::tma_load_2d(dst, map, x, y, bar);
+              if (batched) {
+                const int32_t z = (int32_t)(bz & (map == &tm_a ? p.a_z_mask : p.b_z_mask));
+                if constexpr (PAIR) ptx::tma_load_3d_pair(dst, map, x, y, z, bar);
+                else ptx::tma_load_3d(dst, map, x, y, z, bar);
+              } else {
+                if constexpr (PAIR) ptx::tma_load_2d_pair(dst, map, x, y, bar);
+                else ptx::tma_load_2d(dst, map, x, y, bar);
+              }
             };
             if (!p.a.mn_major) {
 #pragma unroll
@@ -337,7 +345,9 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       WorkItem wi;
       if (!work_item(p.work, worker, num_workers, it, nkb, &wi)) break;
       const int64_t t = wi.tile;
-      const TileCoord tc = raster_decode(p.raster, t);
+      const bool batched = p.batch > 1;
+      const uint32_t bz = batched ? (uint32_t)t / p.tiles_per_batch : 0u;
+      const TileCoord tc = raster_decode(p.raster, batched ? (uint32_t)t - bz * p.tiles_per_batch : t);
       const int32_t row0 = tc.m * (kBlockM * CTA_GROUP) + (int32_t)cta_rank * kBlockM + (int32_t)quad * 32;
       const int32_t col0 = tc.n * BN;
       int32_t nch = 0;  // chunks of this tile that hold any valid column, if this warp's rows exist
@@ -431,7 +441,8 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       auto issue_cin = [&](uint32_t gg, int32_t i) {  // elected lane only: C_in of this warp's i-th chunk
         const uint32_t b = two_bufs ? (gg & 1u) : 0u;
         ptx::mbar_arrive_expect_tx(cin_bar(ew, b), kEpiBufBytes);
-        ptx::tma_load_2d(buf0 + b * kEpiBufBytes, &tm_c, col0 + (half + 2 * i) * CW, row0, cin_bar(ew, b));
+        if (batched) ptx::tma_load_3d(buf0 + b * kEpiBufBytes, &tm_c, col0 + (half + 2 * i) * CW, row0, (int32_t)bz, cin_bar(ew, b));
+        else ptx::tma_load_2d(buf0 + b * kEpiBufBytes, &tm_c, col0 + (half + 2 * i) * CW, row0, cin_bar(ew, b));
       };
       if (mine > 0 && has_beta && two_bufs) {
         if (ptx::elect_one()) {
@@ -544,7 +555,8 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             ptx::fence_proxy_async_smem();  // generic-proxy writes -> visible to the TMA store
             __syncwarp();
             if (ptx::elect_one()) {
-              ptx::tma_store_2d(&tm_c, col, row0, buf0 + boff);
+              if (batched) ptx::tma_store_3d(&tm_c, col, row0, (int32_t)bz, buf0 + boff);
+              else ptx::tma_store_2d(&tm_c, col, row0, buf0 + boff);
               ptx::bulk_commit();
             }
             ++g;

@@ -68,6 +68,9 @@ struct GemmParams {
   int32_t stages;           // depth of the operand ring (2 .. kMaxStages)
   int32_t epi_bufs;         // staging buffers per epilogue warp (1 or 2)
   Raster raster;
+  uint32_t batch;           // matrices in the strided batch (1 = a plain GEMM, 2-D tensor maps)
+  uint32_t tiles_per_batch; // raster.tiles_m * raster.tiles_n
+  uint32_t a_z_mask, b_z_mask;  // all ones, or 0 for an operand that every matrix of the batch shares
   float alpha, beta;
   uint32_t idesc;           // tcgen05 instruction descriptor
   OperandStaging a, b;

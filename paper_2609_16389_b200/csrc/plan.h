@@ -81,6 +81,23 @@ inline exo_gemm_status_t validate_desc(const exo_gemm_desc_t* d) {
   return EXO_GEMM_OK;
 }
 
+// Strided batch: `batch` matrices, consecutive ones stride_x elements apart.  A and B may repeat
+// (stride 0); C matrices must not overlap.  Strides obey the same 16-byte rule as leading dimensions.
+inline exo_gemm_status_t validate_batch(const exo_gemm_desc_t* d, int64_t batch, int64_t sa, int64_t sb, int64_t sc) {
+  exo_gemm_status_t st = validate_desc(d);
+  if (st != EXO_GEMM_OK) return st;
+  if (batch < 1 || batch > 65535 || sa < 0 || sb < 0 || sc < 0) return EXO_GEMM_ERR_INVALID_ARG;
+  const int64_t kMaxStride = 1LL << 38;
+  if (sa > kMaxStride || sb > kMaxStride || sc > kMaxStride) return EXO_GEMM_ERR_INVALID_ARG;
+  if (batch > 1) {
+    const int64_t c_extent = d->c_layout == EXO_GEMM_ROW_MAJOR ? (d->M - 1) * d->ldc + d->N : (d->N - 1) * d->ldc + d->M;
+    if (d->M > 0 && d->N > 0 && sc < c_extent) return EXO_GEMM_ERR_INVALID_ARG;  // overlapping outputs
+    if ((sa * 2) % 16 || (sb * 2) % 16 || (sc * elem_bytes(d->c_dtype)) % 16) return EXO_GEMM_ERR_UNSUPPORTED;
+    if (((d->M + 127) / 128) * ((d->N + 63) / 64) * batch >= (1LL << 31)) return EXO_GEMM_ERR_UNSUPPORTED;
+  }
+  return EXO_GEMM_OK;
+}
+
 // The problem after canonicalisation: C is always written row-major.  A
 // column-major C is computed as C^T = B^T A^T, which only swaps the operands and
 // M with N; an operand's "major-ness" (is K or M/N contiguous) carries over.
@@ -89,10 +106,17 @@ struct Canonical {
   int a_mn_major, b_mn_major;  // of the canonical operands
   int64_t lda, ldb, ldc;
   int swapped;
+  int64_t batch;                         // matrices in a strided batch (1 = plain GEMM)
+  int64_t stride_a, stride_b, stride_c;  // elements between consecutive matrices (canonical operands)
 };
 
-inline Canonical canonicalize(const exo_gemm_desc_t& d) {
+inline Canonical canonicalize(const exo_gemm_desc_t& d, int64_t batch = 1, int64_t stride_a = 0,
+                              int64_t stride_b = 0, int64_t stride_c = 0) {
   Canonical c;
+  c.batch = batch;
+  c.stride_c = stride_c;
+  c.stride_a = d.c_layout == EXO_GEMM_COL_MAJOR ? stride_b : stride_a;
+  c.stride_b = d.c_layout == EXO_GEMM_COL_MAJOR ? stride_a : stride_b;
   const int a_mn = d.a_layout == EXO_GEMM_COL_MAJOR;  // A (M x K) col-major: M contiguous
   const int b_mn = d.b_layout == EXO_GEMM_ROW_MAJOR;  // B (K x N) row-major: N contiguous
   c.swapped = d.c_layout == EXO_GEMM_COL_MAJOR;
@@ -151,11 +175,11 @@ inline int split_factor(int64_t tiles, int64_t workers, int64_t K, int ksub, con
 
 // Estimated time of the whole problem in SM clocks for one candidate tile shape: whole waves of
 // tiles, then the partial last wave (cut along K if that pays), plus what is exposed once per launch.
-inline double estimate_clocks(int64_t M, int64_t N, int64_t K, int cta_group, int bn, int max_workers,
-                              const FlagOverrides& o) {
+inline double estimate_clocks(int64_t M, int64_t N, int64_t K, int64_t batch, int cta_group, int bn,
+                              int max_workers, const FlagOverrides& o) {
   const int64_t tm = (M + 128 * cta_group - 1) / (128 * cta_group);
   const int64_t tn = (N + bn - 1) / bn;
-  const int64_t tiles = tm * tn;
+  const int64_t tiles = tm * tn * batch;
   if (tiles == 0) return 0.0;
   const int ksub = o.ksub ? o.ksub : (bn == 256 ? 1 : 2);
   const int64_t nkb = (K + kBlockK - 1) / kBlockK;
@@ -187,7 +211,7 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
     int w_eff = workers;
     if (o.grid_limit && o.grid_limit / g < w_eff) w_eff = o.grid_limit / g;
     if (w_eff < 1) w_eff = 1;
-    const double t = estimate_clocks(c.M, c.N, c.K, g, n, w_eff, o);
+    const double t = estimate_clocks(c.M, c.N, c.K, c.batch, g, n, w_eff, o);
     if (best_g == 0 || t < best * 0.999) { best = t; best_g = g; best_n = n; }
   }
   if (best_g == 0) { best_g = o.cta_group ? o.cta_group : 1; best_n = o.tile_n ? o.tile_n : 128; }
@@ -208,7 +232,7 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
   int64_t workers = best_g == 2 ? max_pairs : sm_count;
   if (o.grid_limit && o.grid_limit / best_g < workers) workers = o.grid_limit / best_g;
   if (workers < 1) workers = 1;
-  const int64_t tiles = (int64_t)cfg.tiles_m * cfg.tiles_n;
+  const int64_t tiles = (int64_t)cfg.tiles_m * cfg.tiles_n * c.batch;
   // Wave quantisation: the tiles that do not fill a whole wave are cut along K so that the
   // last wave takes 1/split of a tile's time (split-K applied to the tail only; for a problem
   // smaller than one wave that is plain split-K).

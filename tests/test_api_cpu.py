@@ -234,3 +234,17 @@ def test_plan_preview_splits_the_partial_last_wave():
     i = info.as_dict()
     assert i["split_k"] >= 2 and i["tail_tiles"] * i["split_k"] <= i["grid"] // i["cta_group"]
     assert B.exo_gemm_validate(good(flags=B.flag_split_k(9))) == B.ERR_INVALID_ARG
+
+
+def test_batched_create_checks_its_arguments_before_touching_cuda():
+    d = good(M=256, N=192, K=128)                       # C row-major fp32, ldc = 192: one C spans 256*192 elements
+    c_extent = 255 * 192 + 192
+    assert B.exo_gemm_create_batched(d, 0, 0, 0, c_extent)[0] == B.ERR_INVALID_ARG          # batch_count < 1
+    assert B.exo_gemm_create_batched(d, 70000, 0, 0, c_extent)[0] == B.ERR_INVALID_ARG
+    assert B.exo_gemm_create_batched(d, 4, -8, 0, c_extent)[0] == B.ERR_INVALID_ARG
+    assert B.exo_gemm_create_batched(d, 4, 256 * 128, 192 * 128, c_extent - 4)[0] == B.ERR_INVALID_ARG   # C overlap
+    assert B.exo_gemm_create_batched(d, 4, 256 * 128 + 4, 192 * 128, c_extent)[0] == B.ERR_UNSUPPORTED   # 8 bytes off
+    assert B.exo_gemm_create_batched(d, 4, 256 * 128, 192 * 128, c_extent + 2)[0] == B.ERR_UNSUPPORTED
+    import torch
+    if not torch.cuda.is_available():                   # well-formed: only the missing GPU stops it
+        assert B.exo_gemm_create_batched(d, 4, 256 * 128, 0, c_extent)[0] in (B.ERR_CUDA, B.ERR_ARCH)

@@ -300,6 +300,65 @@ def test_back_to_back_dependent_gemms_keep_stream_order():
             assert np.array_equal(d_host, ref)
 
 
+# ------------------------------------------------------------------ strided batch
+BATCH_CASES = [
+    # M, N, K, ab, cd, la, lb, lc, alpha, beta, batch, pad (extra elements between matrices), shared operand
+    (300, 200, 136, BF16, FP32, 0, 1, 0, 1.0, 0.0, 5, 0, None),
+    (264, 328, 200, FP16, FP16, 1, 0, 0, -1.5, 0.75, 3, 64, None),
+    (128, 520, 1024, BF16, BF16, 0, 1, 1, 1.0, 1.0, 7, 8, "b"),      # one B for the whole batch, col-major C
+    (1000, 72, 264, BF16, FP32, 0, 0, 0, 2.0, 0.0, 4, 16, "a"),      # one A for the whole batch
+    (256, 256, 4096, FP16, FP32, 0, 1, 0, 1.0, 0.0, 6, 0, None),     # few tiles, long K: batch + K-slices
+]
+
+
+@pytest.mark.parametrize("case", BATCH_CASES, ids=lambda c: f"{c[0]}x{c[1]}x{c[2]}_b{c[10]}")
+@pytest.mark.parametrize("g,bn", [(0, 0), (1, 128), (2, 256)])
+def test_strided_batched_gemm(case, g, bn):
+    import torch
+    M, N, K, ab, cd, la, lb, lc, alpha, beta, batch, pad, shared = case
+    probs = [synth.Problem(f"b{i}", M, N, K, ab, cd, la, lb, lc, alpha, beta, seed=1000 + 17 * i,
+                           dist="normal" if ab == FP16 else "uniform").generate() for i in range(batch)]
+    if shared == "a":
+        for p in probs[1:]:
+            p.A = probs[0].A
+    if shared == "b":
+        for p in probs[1:]:
+            p.B = probs[0].B
+    sa = 0 if shared == "a" else probs[0].A.size + pad
+    sb = 0 if shared == "b" else probs[0].B.size + pad
+    sc = probs[0].C.size + pad
+    canary16, canaryc = np.uint16(0x7FC0), (np.float32(np.nan) if cd == FP32 else np.uint16(0x7FC0))
+
+    def pack(bufs, stride, canary):
+        if stride == 0:
+            return bufs[0].copy()
+        out = np.full(stride * len(bufs), canary, dtype=bufs[0].dtype)
+        for i, b in enumerate(bufs):
+            out[i * stride:i * stride + b.size] = b
+        return out
+
+    hA, hB = pack([p.A for p in probs], sa, canary16), pack([p.B for p in probs], sb, canary16)
+    hC = pack([p.C for p in probs], sc, canaryc)
+    dev = torch.device("cuda:0")
+    dA, dB, dC = harness._to_device(hA, dev), harness._to_device(hB, dev), harness._to_device(hC, dev)
+    flags = flags_for(g, bn) if g else 0
+    with B.Plan(harness.desc_of(probs[0], flags), batch=(batch, sa, sb, sc)) as plan:
+        info = plan.info()
+        assert info["batch_count"] == batch and info["kernel_launches_per_run"] == 1
+        plan.run(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), alpha, beta, torch.cuda.current_stream(dev).cuda_stream)
+        torch.cuda.synchronize(dev)
+        plan.check()
+    out = dC.cpu().numpy().view(synth.storage_np_dtype(cd))
+    for i, p in enumerate(probs):
+        got = oracle.logical_view(out[i * sc:i * sc + p.C.size], M, N, lc, p.ldc, cd)
+        cref, den = oracle.gemm_problem(p)
+        gate = TOL * den + oracle.output_rounding_slack(cref, cd)
+        assert (np.abs(got - cref) <= gate).all(), (i, info)
+        if pad:                                        # the gap between consecutive C matrices is untouched
+            gap = out[i * sc + p.C.size:(i + 1) * sc]
+            assert (np.isnan(gap).all() if cd == FP32 else (gap == 0x7FC0).all())
+
+
 # ------------------------------------------------------------------ the benchmark configurations
 def structured_sample(M, N, rng, n_random=1 << 14):
     """Rows/columns next to every 128/256 tile boundary crossed with random partners, plus random entries."""
