@@ -56,7 +56,10 @@ def parse_args():
 
 def make_problem(name: str, rank: int = 0):
     from paper_2609_16389_b200 import synth
-    if name.startswith("sweep_"):
+    if name.startswith("batched_"):
+        batch, n = (int(x) for x in name[len("batched_"):].split("x"))
+        p = synth.batched(batch, n)
+    elif name.startswith("sweep_"):
         M, N, K = (int(x) for x in name[len("sweep_"):].split("x"))
         p = synth.sweep_problem(M, N, K)
     else:
@@ -160,6 +163,8 @@ def run_reference(args, rank, world):
         return
     import oracle
     p = make_problem(args.workload)
+    if getattr(p, "batch", 1) > 1:
+        p = p.matrix(0)
     cores = oracle.num_threads()
     # calibrate on a thin band, then size the per-step band so the whole run stays bounded
     cal_rows = min(p.M, 16)
@@ -218,7 +223,9 @@ def run_ours(args, rank, world, local_rank):
     sets = []
     for _ in range(n_sets):
         sets.append((harness._to_device(p.A, dev), harness._to_device(p.B, dev), harness._to_device(p.C, dev)))
-    plan = B.Plan(harness.desc_of(p, args.flags, local_rank))
+    batch = getattr(p, "batch", 1)
+    plan = B.Plan(harness.desc_of(p, args.flags, local_rank),
+                  batch=(batch, p.stride_a, p.stride_b, p.stride_c) if batch > 1 else None)
     info = plan.info()
     stream = torch.cuda.current_stream(dev)
 
@@ -322,7 +329,7 @@ def run_ours(args, rank, world, local_rank):
             "scaling": "weak", "vs_baseline": None,
             "dtype": ("bf16" if p.ab_dtype == synth.BF16 else "fp16") + " in, fp32 accumulate",
             "data": "synthetic",
-            "config": {"workload": args.workload, "M": p.M, "N": p.N, "K": p.K,
+            "config": {"workload": args.workload, "M": p.M, "N": p.N, "K": p.K, "batch": batch,
                        "ab_dtype": synth.dtype_name(p.ab_dtype), "c_dtype": synth.dtype_name(p.c_dtype),
                        "layouts": "A%s B%s C%s" % tuple("rc"[x] for x in (p.a_layout, p.b_layout, p.c_layout)),
                        "alpha": p.alpha, "beta": p.beta,
@@ -353,6 +360,22 @@ def time_cublas(p, dev, steps, n_sets):
     from paper_2609_16389_b200 import synth
     try:
         tdt = torch.bfloat16 if p.ab_dtype == synth.BF16 else torch.float16
+        batch = getattr(p, "batch", 1)
+        if batch > 1:
+            a = torch.randn(batch, p.M, p.K, device=dev).to(tdt)
+            b = torch.randn(batch, p.N, p.K, device=dev).to(tdt).transpose(1, 2)
+            c = torch.empty(batch, p.M, p.N, device=dev, dtype=tdt)
+            for _ in range(3):
+                torch.bmm(a, b, out=c)
+            torch.cuda.synchronize(dev)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(steps):
+                torch.bmm(a, b, out=c)
+            e1.record()
+            torch.cuda.synchronize(dev)
+            ms = e0.elapsed_time(e1) / steps
+            return {"tflops": p.flop / (ms * 1e-3) / 1e12, "ms_per_step": ms, "note": "torch.bmm, same shapes (L2-warm)"}
         sets = []
         for _ in range(n_sets):
             a = torch.randn(p.M, p.K, device=dev, dtype=torch.float32).to(tdt)
@@ -383,6 +406,8 @@ def time_cublas(p, dev, steps, n_sets):
 
 def cpu_baseline(p, workload):
     import oracle
+    if getattr(p, "batch", 1) > 1:
+        p = p.matrix(0)
     cores = oracle.num_threads()
     cal_rows = min(p.M, 16)
     t0 = time.perf_counter()
@@ -485,7 +510,7 @@ def main():
             raise SystemExit("the reference arm times one workload; pick e.g. --workload sweep_1000x1000x1000")
         run_sweep(args, rank, world, local_rank)
         return
-    if args.workload not in WORKLOADS and not args.workload.startswith("sweep_"):
+    if args.workload not in WORKLOADS and not args.workload.startswith(("sweep_", "batched_")):
         raise SystemExit(f"unknown workload {args.workload}")
     if args.impl == "reference":
         run_reference(args, rank, world)

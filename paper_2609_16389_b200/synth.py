@@ -222,6 +222,54 @@ class Problem:
         return n
 
 
+class BatchedProblem(Problem):
+    """`batch` independent problems of one shape, packed back to back (strides = one matrix)."""
+
+    def __init__(self, name, batch, *args, **kw):
+        super().__init__(name, *args, **kw)
+        self.batch = batch
+        self.stride_a = self.stride_b = self.stride_c = 0
+
+    def generate(self, **kw):
+        parts = []
+        base_seed = self.seed
+        for i in range(self.batch):
+            self.seed = base_seed + 7919 * i
+            super().generate(**kw)
+            parts.append((self.A, self.B, self.C))
+        self.seed = base_seed
+        self.stride_a, self.stride_b, self.stride_c = parts[0][0].size, parts[0][1].size, parts[0][2].size
+        self.A = np.concatenate([q[0] for q in parts])
+        self.B = np.concatenate([q[1] for q in parts])
+        self.C = np.concatenate([q[2] for q in parts])
+        return self
+
+    def matrix(self, i: int) -> Problem:
+        """Problem view of matrix i (shares the packed buffers)."""
+        q = Problem(f"{self.name}[{i}]", self.M, self.N, self.K, self.ab_dtype, self.c_dtype, self.a_layout,
+                    self.b_layout, self.c_layout, self.alpha, self.beta, self.seed, self.dist,
+                    self.lda, self.ldb, self.ldc)
+        q.A = self.A[i * self.stride_a:(i + 1) * self.stride_a]
+        q.B = self.B[i * self.stride_b:(i + 1) * self.stride_b]
+        q.C = self.C[i * self.stride_c:(i + 1) * self.stride_c]
+        return q
+
+    @property
+    def flop(self) -> float:
+        return self.batch * super().flop
+
+    @property
+    def algorithmic_bytes(self) -> int:
+        return self.batch * super().algorithmic_bytes
+
+
+def batched(batch: int, n: int) -> BatchedProblem:
+    """Strided batch of `batch` cubes n^3: bf16 uniform, A row / B col, bf16 C (the paper's
+    evaluation also measures a strided-batched GEMM; it gives no sizes)."""
+    return BatchedProblem(f"batched_{batch}x{n}", batch, n, n, n, BF16, BF16, ROW_MAJOR, COL_MAJOR, ROW_MAJOR,
+                          1.0, 0.0, BASE_SEED + 50)
+
+
 def config(idx: int, variant: str | None = None) -> Problem:
     """The benchmark configurations (0-based index into the configuration list).
 
