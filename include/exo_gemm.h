@@ -65,16 +65,21 @@ typedef enum { EXO_GEMM_ROW_MAJOR = 0, EXO_GEMM_COL_MAJOR = 1 } exo_gemm_layout_
  * Leading dimensions are in elements: for a row-major matrix ld >= #columns, for
  * a column-major matrix ld >= #rows.
  *
- * Supported set: ab_dtype in {BF16, FP16}; c_dtype FP32 or equal to ab_dtype; any
- * of the 8 layout combinations; 0 <= M, N, K <= 2^31 - 1.  Because operands and
+ * Supported set: ab_dtype in {BF16, FP16, FP32}; c_dtype FP32 or equal to ab_dtype;
+ * any of the 8 layout combinations; 0 <= M, N, K <= 2^31 - 1.  FP32 operands are
+ * multiplied as tf32 (the tensor core reads sign, exponent and the upper 10 fraction
+ * bits of each fp32 operand and ignores the rest; products are accumulated in fp32):
+ * this is the precision of the paper's own Section 6 kernels and of
+ * CUBLAS_TF32_TENSOR_OP_MATH.  FP32 operands must have K contiguous (A row-major,
+ * B column-major); other FP32 layouts return ERR_UNSUPPORTED.  Because operands and
  * results move by TMA, every leading dimension times its element size must be a
- * multiple of 16 bytes (16-bit: ld % 8 == 0, fp32 C: ldc % 4 == 0) and every base
+ * multiple of 16 bytes (16-bit: ld % 8 == 0, fp32: ld % 4 == 0) and every base
  * pointer passed to exo_gemm_run must be 16-byte aligned.  Legal BLAS calls
  * outside this set return EXO_GEMM_ERR_UNSUPPORTED.
  */
 typedef struct {
   int64_t M, N, K;
-  int32_t ab_dtype;                     /* exo_gemm_dtype_t: BF16 or FP16, both operands       */
+  int32_t ab_dtype;                     /* exo_gemm_dtype_t of both operands (FP32 = tf32 math) */
   int32_t c_dtype;                      /* exo_gemm_dtype_t: FP32 or the same as ab_dtype      */
   int32_t a_layout, b_layout, c_layout; /* exo_gemm_layout_t                                   */
   int32_t device;                       /* CUDA device ordinal; -1 = the current device        */
@@ -87,7 +92,7 @@ typedef struct {
 typedef struct {
   int32_t cta_group;      /* 1 or 2 SMs per tile                                               */
   int32_t tile_m, tile_n; /* output tile of one CTA group (tile_m = 128 * cta_group)           */
-  int32_t tile_k;         /* k-elements staged per pipeline stage (64 or 128)                  */
+  int32_t tile_k;         /* k-elements staged per pipeline stage (64 or 128; tf32: 32 or 64)  */
   int32_t stages;         /* depth of the shared-memory operand ring                           */
   int32_t grid;           /* CTAs launched (persistent)                                        */
   int32_t smem_bytes;     /* dynamic shared memory per CTA                                     */

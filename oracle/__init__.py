@@ -71,7 +71,7 @@ def _ptr(a):
     return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
 
 
-def _check_buf(buf, dtype, n_needed, what):
+def _check_buf(buf, dtype, n_needed, what):  # dtype FP32 also covers tf32-mode operands (stored as float32)
     want = np.float32 if dtype == FP32 else np.uint16
     if buf.dtype != want or not buf.flags.c_contiguous or buf.ndim != 1:
         raise ValueError(f"{what}: need flat contiguous {want.__name__}")

@@ -19,7 +19,11 @@
  *
  * with a, b, c the stored 16-bit / 32-bit values widened exactly to fp64.  A
  * product of two bf16 or two fp16 numbers is exact in fp64, so the only error
- * of S is fp64 summation error (<= K * 2^-53 * D_ij).  beta == 0 means C_in is
+ * of S is fp64 summation error (<= K * 2^-53 * D_ij).  fp32 operands (the tf32
+ * mode, the precision of the paper's Section 6 kernels) are widened exactly as
+ * stored: the comparison with a tf32 tensor-core result is meaningful for
+ * operands that are representable in tf32 (10 fraction bits), which is what the
+ * input generator produces; their products are exact in fp64 as well.  beta == 0 means C_in is
  * never read (BLAS convention), so NaN there cannot reach the result.
  *
  * There is no blocking, no reordering and no library call.  The only
@@ -111,7 +115,7 @@ double oracle_widen(uint32_t bits, int dtype) {
 static int bad_args(int64_t M, int64_t N, int64_t K, int ab_dtype, int c_dtype, int a_layout,
                     int b_layout, int c_layout, int64_t lda, int64_t ldb, int64_t ldc) {
     if (M < 0 || N < 0 || K < 0) return 1;
-    if (ab_dtype != ORC_BF16 && ab_dtype != ORC_FP16) return 1;
+    if (ab_dtype != ORC_BF16 && ab_dtype != ORC_FP16 && ab_dtype != ORC_FP32) return 1;
     if (c_dtype != ORC_BF16 && c_dtype != ORC_FP16 && c_dtype != ORC_FP32) return 1;
     if ((a_layout | b_layout | c_layout) & ~1) return 1;
     if (lda < (a_layout == ORC_ROW ? K : M)) return 1;

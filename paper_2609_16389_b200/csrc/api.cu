@@ -152,7 +152,7 @@ void fill_info(const exo_gemm_plan* p, exo_gemm_info_t* info) {
   info->cta_group = p->cfg.cta_group;
   info->tile_m = 128 * p->cfg.cta_group;
   info->tile_n = p->cfg.tile_n;
-  info->tile_k = kBlockK * p->cfg.ksub;
+  info->tile_k = sub_block_k(p->canon.ab_bytes) * p->cfg.ksub;
   info->stages = p->cfg.stages;
   info->grid = p->cfg.workers * p->cfg.cta_group;
   info->smem_bytes = p->smem_bytes;
@@ -374,7 +374,8 @@ exo_gemm_status_t exo_gemm_run(exo_gemm_handle_t plan, const void* A, const void
   prm.M = (int32_t)cn.M;
   prm.N = (int32_t)cn.N;
   prm.K = (int32_t)cn.K;
-  const int stage_k = kBlockK * cfg.ksub;
+  const int sub_k = sub_block_k(cn.ab_bytes);
+  const int stage_k = sub_k * cfg.ksub;
   prm.num_k_blocks = read_ab ? (int32_t)((cn.K + stage_k - 1) / stage_k) : 0;
   prm.raster = Raster{cfg.tiles_m, cfg.tiles_n, cfg.band, cfg.along_m};
   prm.batch = (uint32_t)cn.batch;
@@ -392,8 +393,11 @@ exo_gemm_status_t exo_gemm_run(exo_gemm_handle_t plan, const void* A, const void
   prm.alpha = read_ab ? alpha : 0.f;
   prm.beta = beta;
   prm.idesc = make_idesc(d.ab_dtype, cn.a_mn_major, cn.b_mn_major, 128 * cfg.cta_group, cfg.tile_n);
-  prm.a = make_staging(cn.a_mn_major, kBlockM, cfg.ksub);
-  prm.b = make_staging(cn.b_mn_major, cfg.tile_n / cfg.cta_group, cfg.ksub);
+  prm.a = make_staging(cn.a_mn_major, kBlockM, cfg.ksub, cn.ab_bytes);
+  prm.b = make_staging(cn.b_mn_major, cfg.tile_n / cfg.cta_group, cfg.ksub, cn.ab_bytes);
+  prm.sub_k = (uint32_t)sub_k;
+  prm.umma_k = (uint32_t)sub_k / 4;
+  prm.tf32 = d.ab_dtype == EXO_GEMM_FP32 ? 1u : 0u;
   prm.status = plan->d_status;
   const int32_t dbg_ms = plan->dbg_timeout_ms.exchange(0);
   // SM clocks, converted at 2 GHz (an upper bound of the SM clock, so the real limit is not shorter)
@@ -408,11 +412,11 @@ exo_gemm_status_t exo_gemm_run(exo_gemm_handle_t plan, const void* A, const void
   const uint32_t c_box = d.c_dtype == EXO_GEMM_FP32 ? 32 : 64;
   if (cn.batch <= 1) {
     if (read_ab) {
-      r = cn.a_mn_major ? encode_2d(&tm_a, d.ab_dtype, opA, cn.M, cn.K, cn.lda, 64, stage_k, true)
-                        : encode_2d(&tm_a, d.ab_dtype, opA, cn.K, cn.M, cn.lda, kBlockK, kBlockM, true);
+      r = cn.a_mn_major ? encode_2d(&tm_a, d.ab_dtype, opA, cn.M, cn.K, cn.lda, sub_k, stage_k, true)
+                        : encode_2d(&tm_a, d.ab_dtype, opA, cn.K, cn.M, cn.lda, sub_k, kBlockM, true);
       if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return EXO_GEMM_ERR_CUDA; }
-      r = cn.b_mn_major ? encode_2d(&tm_b, d.ab_dtype, opB, cn.N, cn.K, cn.ldb, 64, stage_k, true)
-                        : encode_2d(&tm_b, d.ab_dtype, opB, cn.K, cn.N, cn.ldb, kBlockK, b_rows, true);
+      r = cn.b_mn_major ? encode_2d(&tm_b, d.ab_dtype, opB, cn.N, cn.K, cn.ldb, sub_k, stage_k, true)
+                        : encode_2d(&tm_b, d.ab_dtype, opB, cn.K, cn.N, cn.ldb, sub_k, b_rows, true);
       if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return EXO_GEMM_ERR_CUDA; }
     }
     r = encode_2d(&tm_c, d.c_dtype, C, cn.N, cn.M, cn.ldc, c_box, 32, false);
@@ -420,12 +424,12 @@ exo_gemm_status_t exo_gemm_run(exo_gemm_handle_t plan, const void* A, const void
   } else {  // strided batch: the matrix index is the third tensor-map coordinate
     if (read_ab) {
       r = cn.a_mn_major
-              ? encode_3d(&tm_a, d.ab_dtype, opA, cn.M, cn.K, cn.lda, cn.batch, cn.stride_a, 64, stage_k, true)
-              : encode_3d(&tm_a, d.ab_dtype, opA, cn.K, cn.M, cn.lda, cn.batch, cn.stride_a, kBlockK, kBlockM, true);
+              ? encode_3d(&tm_a, d.ab_dtype, opA, cn.M, cn.K, cn.lda, cn.batch, cn.stride_a, sub_k, stage_k, true)
+              : encode_3d(&tm_a, d.ab_dtype, opA, cn.K, cn.M, cn.lda, cn.batch, cn.stride_a, sub_k, kBlockM, true);
       if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return EXO_GEMM_ERR_CUDA; }
       r = cn.b_mn_major
-              ? encode_3d(&tm_b, d.ab_dtype, opB, cn.N, cn.K, cn.ldb, cn.batch, cn.stride_b, 64, stage_k, true)
-              : encode_3d(&tm_b, d.ab_dtype, opB, cn.K, cn.N, cn.ldb, cn.batch, cn.stride_b, kBlockK, b_rows, true);
+              ? encode_3d(&tm_b, d.ab_dtype, opB, cn.N, cn.K, cn.ldb, cn.batch, cn.stride_b, sub_k, stage_k, true)
+              : encode_3d(&tm_b, d.ab_dtype, opB, cn.K, cn.N, cn.ldb, cn.batch, cn.stride_b, sub_k, b_rows, true);
       if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return EXO_GEMM_ERR_CUDA; }
     }
     r = encode_3d(&tm_c, d.c_dtype, C, cn.N, cn.M, cn.ldc, cn.batch, cn.stride_c, c_box, 32, false);

@@ -122,7 +122,7 @@ template <int CTA_GROUP, int BN, int OUT, int KSUB>
 __global__ void __launch_bounds__(kNumThreads, 1)
 exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                 const __grid_constant__ CUtensorMap tm_c, const GemmParams p) {
-  constexpr int STAGE_K = kBlockK * KSUB;            // k-elements per stage
+  const int32_t STAGE_K = (int32_t)p.sub_k * KSUB;   // k-elements per stage (64 or 32 per sub-block)
   constexpr int B_ROWS = BN / CTA_GROUP;             // rows of the B tile this CTA stages
   constexpr int STAGE_BYTES = stage_bytes(CTA_GROUP, BN, KSUB);
   constexpr int A_BYTES = KSUB * kATileBytes;        // the A part of a stage
@@ -236,19 +236,17 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             };
             if (!p.a.mn_major) {
 #pragma unroll
-              for (int h = 0; h < KSUB; ++h) load(a_dst + h * kATileBytes, &tm_a, k0 + h * kBlockK, a_mn0);
+              for (int h = 0; h < KSUB; ++h) load(a_dst + h * kATileBytes, &tm_a, k0 + h * (int32_t)p.sub_k, a_mn0);
             } else {
-#pragma unroll
-              for (int b = 0; b < kBlockM / 64; ++b)
-                load(a_dst + b * (KSUB * 8192), &tm_a, a_mn0 + 64 * b, k0);
+              for (uint32_t b = 0; b < p.a.mn_boxes; ++b)
+                load(a_dst + b * p.a.box_bytes, &tm_a, a_mn0 + (int32_t)(p.a.mn_box * b), k0);
             }
             if (!p.b.mn_major) {
 #pragma unroll
-              for (int h = 0; h < KSUB; ++h) load(b_dst + h * (B_ROWS * 128), &tm_b, k0 + h * kBlockK, b_mn0);
+              for (int h = 0; h < KSUB; ++h) load(b_dst + h * (B_ROWS * 128), &tm_b, k0 + h * (int32_t)p.sub_k, b_mn0);
             } else {
-#pragma unroll
-              for (int b = 0; b < B_ROWS / 64; ++b)
-                load(b_dst + b * (KSUB * 8192), &tm_b, b_mn0 + 64 * b, k0);
+              for (uint32_t b = 0; b < p.b.mn_boxes; ++b)
+                load(b_dst + b * p.b.box_bytes, &tm_b, b_mn0 + (int32_t)(p.b.mn_box * b), k0);
             }
           }
           EXO_TRACE(0, issued, 1, 4096);
@@ -271,7 +269,9 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       [[maybe_unused]] int64_t consumed = 0;
       const uint32_t a_step = p.a.k_step_enc, b_step = p.b.k_step_enc;
       const uint32_t a_sub = p.a.k_sub_enc, b_sub = p.b.k_sub_enc;
-      constexpr int kMmaPerStage = STAGE_K / kUmmaK;
+      constexpr int kMmaPerStage = 4 * KSUB;  // an MMA consumes 32 bytes of K whatever the element size
+      const bool tf32 = p.tf32 != 0;
+      const int32_t umma_k = (int32_t)p.umma_k;
       auto k_off = [](int32_t k, uint32_t step, uint32_t sub) {  // descriptor offset of the k-th MMA of a stage
         return (uint64_t)((uint32_t)(k & 3) * step + (uint32_t)(k >> 2) * sub);
       };
@@ -297,16 +297,27 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
           const int32_t k_left = p.K - kb * STAGE_K;
           if (ptx::elect_one()) {  // the same lane every time: commits track this thread's MMAs
             EXO_TRACE(1, consumed, 0, 4096);
-            if (k_left >= STAGE_K) {
+            if (k_left >= STAGE_K && !tf32) {
 #pragma unroll
               for (int32_t k = 0; k < kMmaPerStage; ++k)
                 ptx::umma_f16<CTA_GROUP>(d_tmem, a_desc + k_off(k, a_step, a_sub), b_desc + k_off(k, b_step, b_sub),
                                          idesc, (kb != wi.kb_begin || k != 0) ? 1u : 0u);
+            } else if (k_left >= STAGE_K) {
+#pragma unroll
+              for (int32_t k = 0; k < kMmaPerStage; ++k)
+                ptx::umma_tf32<CTA_GROUP>(d_tmem, a_desc + k_off(k, a_step, a_sub), b_desc + k_off(k, b_step, b_sub),
+                                          idesc, (kb != wi.kb_begin || k != 0) ? 1u : 0u);
             } else {  // ragged last k-block: skip the MMAs that would only read zero fill
-              const int32_t n_mma = (k_left + kUmmaK - 1) / kUmmaK;
-              for (int32_t k = 0; k < n_mma; ++k)
-                ptx::umma_f16<CTA_GROUP>(d_tmem, a_desc + k_off(k, a_step, a_sub), b_desc + k_off(k, b_step, b_sub),
-                                         idesc, (kb != wi.kb_begin || k != 0) ? 1u : 0u);
+              const int32_t n_mma = (k_left + umma_k - 1) / umma_k;
+              for (int32_t k = 0; k < n_mma; ++k) {
+                const uint32_t accumulate = (kb != wi.kb_begin || k != 0) ? 1u : 0u;
+                if (tf32)
+                  ptx::umma_tf32<CTA_GROUP>(d_tmem, a_desc + k_off(k, a_step, a_sub), b_desc + k_off(k, b_step, b_sub),
+                                            idesc, accumulate);
+                else
+                  ptx::umma_f16<CTA_GROUP>(d_tmem, a_desc + k_off(k, a_step, a_sub), b_desc + k_off(k, b_step, b_sub),
+                                           idesc, accumulate);
+              }
             }
             ptx::umma_commit<CTA_GROUP>(empty_bar(s), kMask);  // stage free once these MMAs completed
             if (kb == wi.kb_end - 1) ptx::umma_commit<CTA_GROUP>(tfull_bar(acc), kMask);  // accumulator complete

@@ -8,8 +8,8 @@
 namespace exo {
 
 constexpr int kBlockM = 128;        // rows of C per CTA (one TMEM lane per row)
-constexpr int kBlockK = 64;         // elements of K per sub-block: 128 bytes = one swizzle span
-constexpr int kUmmaK = 16;          // K of one tcgen05.mma for 16-bit inputs
+constexpr int kBlockK = 64;         // 16-bit elements of K per sub-block: 128 bytes = one swizzle span
+constexpr int kUmmaK = 16;          // K of one tcgen05.mma for 16-bit inputs (32 bytes; 8 for tf32)
 constexpr int kNumThreads = 320;    // warp 0 producer, warp 1 MMA issuer + TMEM owner, warps 2..9 epilogue
 constexpr int kEpiWarps = 8;        // two per TMEM lane quadrant, each taking every other column chunk
 constexpr int kEpiBufBytes = 4096;  // one staging buffer: 32 rows x 128 bytes
@@ -46,6 +46,8 @@ struct OperandStaging {
   uint32_t k_step_enc; // descriptor start-address increment per UMMA_K inside a sub-block (bytes >> 4)
   uint32_t k_sub_enc;  // descriptor start-address increment per 64-k sub-block (bytes >> 4)
   uint32_t box_bytes;  // MN-major: bytes of one TMA box in shared memory
+  uint32_t mn_boxes;   // MN-major: boxes per operand tile (rows / elements per 128 bytes)
+  uint32_t mn_box;     // MN-major: M/N elements per box (64 for 16-bit, 32 for tf32)
 };
 
 enum StatusCode : uint32_t {
@@ -65,6 +67,9 @@ enum WaitRole : uint32_t {
 struct GemmParams {
   int32_t M, N, K;          // canonical problem (C row-major; operands possibly swapped)
   int32_t num_k_blocks;     // ceil(K / (64 * ksub)), or 0 when alpha == 0 / K == 0
+  uint32_t sub_k;           // k-elements per sub-block: 64 (16-bit operands) or 32 (fp32 storage, tf32 math)
+  uint32_t umma_k;          // k-elements per MMA: 16 or 8
+  uint32_t tf32;            // 1: operands are fp32 in memory and multiplied as tf32
   int32_t stages;           // depth of the operand ring (2 .. kMaxStages)
   int32_t epi_bufs;         // staging buffers per epilogue warp (1 or 2)
   Raster raster;

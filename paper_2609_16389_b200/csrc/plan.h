@@ -69,14 +69,19 @@ inline exo_gemm_status_t validate_desc(const exo_gemm_desc_t* d) {
   if (o.cta_group == 2 && o.tile_n == 64) return EXO_GEMM_ERR_INVALID_ARG;
   if (o.grid_limit != 0 && o.cta_group == 2 && (o.grid_limit & 1)) return EXO_GEMM_ERR_INVALID_ARG;
   // beyond here the call is a legal BLAS call; what follows is this library's supported set
-  if (d->ab_dtype == EXO_GEMM_FP32) return EXO_GEMM_ERR_UNSUPPORTED;
+  // fp32 operands are multiplied as tf32 (the precision of the paper's own kernels) into an fp32 C
   if (d->c_dtype != EXO_GEMM_FP32 && d->c_dtype != d->ab_dtype) return EXO_GEMM_ERR_UNSUPPORTED;
+  // tf32 operands must have K contiguous (A row-major, B column-major): the M/N-contiguous form
+  // needs a different shared-memory swizzle (32-byte atoms) that this library does not stage
+  if (d->ab_dtype == EXO_GEMM_FP32 && (d->a_layout != EXO_GEMM_ROW_MAJOR || d->b_layout != EXO_GEMM_COL_MAJOR))
+    return EXO_GEMM_ERR_UNSUPPORTED;
   // the persistent scheduler indexes tiles (at least 128 x 64 each) and k-blocks with 32 bits
   if (((d->M + 127) / 128) * ((d->N + 63) / 64) >= (1LL << 31)) return EXO_GEMM_ERR_UNSUPPORTED;
   // a matrix that is never touched (empty problem, K == 0) has no stride rule
   const bool c_used = d->M > 0 && d->N > 0;
   const bool ab_used = c_used && d->K > 0;
-  if (ab_used && ((d->lda * 2) % 16 || (d->ldb * 2) % 16)) return EXO_GEMM_ERR_UNSUPPORTED;
+  if (ab_used && ((d->lda * elem_bytes(d->ab_dtype)) % 16 || (d->ldb * elem_bytes(d->ab_dtype)) % 16))
+    return EXO_GEMM_ERR_UNSUPPORTED;
   if (c_used && (d->ldc * elem_bytes(d->c_dtype)) % 16) return EXO_GEMM_ERR_UNSUPPORTED;
   return EXO_GEMM_OK;
 }
@@ -92,7 +97,9 @@ inline exo_gemm_status_t validate_batch(const exo_gemm_desc_t* d, int64_t batch,
   if (batch > 1) {
     const int64_t c_extent = d->c_layout == EXO_GEMM_ROW_MAJOR ? (d->M - 1) * d->ldc + d->N : (d->N - 1) * d->ldc + d->M;
     if (d->M > 0 && d->N > 0 && sc < c_extent) return EXO_GEMM_ERR_INVALID_ARG;  // overlapping outputs
-    if ((sa * 2) % 16 || (sb * 2) % 16 || (sc * elem_bytes(d->c_dtype)) % 16) return EXO_GEMM_ERR_UNSUPPORTED;
+    if ((sa * elem_bytes(d->ab_dtype)) % 16 || (sb * elem_bytes(d->ab_dtype)) % 16 ||
+        (sc * elem_bytes(d->c_dtype)) % 16)
+      return EXO_GEMM_ERR_UNSUPPORTED;
     if (((d->M + 127) / 128) * ((d->N + 63) / 64) * batch >= (1LL << 31)) return EXO_GEMM_ERR_UNSUPPORTED;
   }
   return EXO_GEMM_OK;
@@ -106,6 +113,7 @@ struct Canonical {
   int a_mn_major, b_mn_major;  // of the canonical operands
   int64_t lda, ldb, ldc;
   int swapped;
+  int ab_bytes;                          // 2 (bf16/fp16) or 4 (fp32 storage, tf32 math)
   int64_t batch;                         // matrices in a strided batch (1 = plain GEMM)
   int64_t stride_a, stride_b, stride_c;  // elements between consecutive matrices (canonical operands)
 };
@@ -113,6 +121,7 @@ struct Canonical {
 inline Canonical canonicalize(const exo_gemm_desc_t& d, int64_t batch = 1, int64_t stride_a = 0,
                               int64_t stride_b = 0, int64_t stride_c = 0) {
   Canonical c;
+  c.ab_bytes = elem_bytes(d.ab_dtype);
   c.batch = batch;
   c.stride_c = stride_c;
   c.stride_a = d.c_layout == EXO_GEMM_COL_MAJOR ? stride_b : stride_a;
@@ -159,7 +168,11 @@ inline double shape_efficiency(int cta_group, int bn) {
   return bn == 256 ? 0.86 : (bn == 128 ? 0.66 : 0.40);
 }
 
+// k-elements in one 128-byte sub-block row: 64 for 16-bit operands, 32 for fp32 storage.
+inline int sub_block_k(int ab_bytes) { return 128 / ab_bytes; }
+
 // How many K-slices each tile of the partial last wave is cut into (1 = not cut).
+// (K is given in units of 128-byte sub-block rows x 64, i.e. already scaled by the element size.)
 inline int split_factor(int64_t tiles, int64_t workers, int64_t K, int ksub, const FlagOverrides& o) {
   const int64_t tail = tiles % workers;
   if (tail == 0 || o.split == 1 || o.no_workspace) return 1;
@@ -211,7 +224,7 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
     int w_eff = workers;
     if (o.grid_limit && o.grid_limit / g < w_eff) w_eff = o.grid_limit / g;
     if (w_eff < 1) w_eff = 1;
-    const double t = estimate_clocks(c.M, c.N, c.K, c.batch, g, n, w_eff, o);
+    const double t = estimate_clocks(c.M, c.N, c.K * (c.ab_bytes / 2), c.batch, g, n, w_eff, o);
     if (best_g == 0 || t < best * 0.999) { best = t; best_g = g; best_n = n; }
   }
   if (best_g == 0) { best_g = o.cta_group ? o.cta_group : 1; best_n = o.tile_n ? o.tile_n : 128; }
@@ -223,7 +236,7 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
   // reads the other; they cost 32 KB of ring.  Take them when at least 3 stages remain.
   // Short K: the epilogue bounds a tile, so staging depth matters more than ring depth.
   const bool want_two = max_stages(best_g, best_n, cfg.ksub, 2) >= 5 ||
-                        (c.K <= 1024 && max_stages(best_g, best_n, cfg.ksub, 2) >= 3);
+                        (c.K * (c.ab_bytes / 2) <= 1024 && max_stages(best_g, best_n, cfg.ksub, 2) >= 3);
   cfg.epi_bufs = o.epi_bufs ? o.epi_bufs : (want_two ? 2 : 1);
   cfg.stages = max_stages(best_g, best_n, cfg.ksub, cfg.epi_bufs);
   if (o.stages && o.stages < cfg.stages) cfg.stages = o.stages < 2 ? 2 : o.stages;
@@ -240,8 +253,9 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
     const int64_t full_waves = tiles / workers;
     cfg.full_tiles = full_waves * workers;
     cfg.tail_tiles = (int)(tiles - cfg.full_tiles);
-    const int64_t k_blocks = (c.K + kBlockK * cfg.ksub - 1) / (kBlockK * cfg.ksub);
-    cfg.split = split_factor(tiles, workers, c.K, cfg.ksub, o);
+    const int64_t k_scaled = c.K * (c.ab_bytes / 2);  // in 16-bit-element units: 64 per sub-block
+    const int64_t k_blocks = (k_scaled + kBlockK * cfg.ksub - 1) / (kBlockK * cfg.ksub);
+    cfg.split = split_factor(tiles, workers, k_scaled, cfg.ksub, o);
     // Publishing a 128 x N fp32 partial takes a contributor about as long as 8 k-blocks of 64
     // (128*N*4 bytes at ~30 B/clk against 2*N clocks of MMA per k-block); let the owner compute that
     // much longer, so that the partials are there when it finishes.
@@ -290,7 +304,8 @@ inline int smem_bytes_for(int cta_group, int bn, int ksub, int stages, int epi_b
 
 // tcgen05 instruction descriptor for kind::f16 with fp32 accumulation.
 inline uint32_t make_idesc(int ab_dtype, int a_mn_major, int b_mn_major, int umma_m, int umma_n) {
-  const uint32_t fmt = ab_dtype == EXO_GEMM_BF16 ? 1u : 0u;  // 0 = fp16, 1 = bf16
+  // kind::f16: 0 = fp16, 1 = bf16; kind::tf32: 2 = tf32
+  const uint32_t fmt = ab_dtype == EXO_GEMM_BF16 ? 1u : (ab_dtype == EXO_GEMM_FP32 ? 2u : 0u);
   uint32_t d = 0;
   d |= 1u << 4;                        // D format: fp32
   d |= fmt << 7;                       // A format
@@ -303,7 +318,7 @@ inline uint32_t make_idesc(int ab_dtype, int a_mn_major, int b_mn_major, int umm
 }
 
 // How an operand tile sits in shared memory (128-byte swizzle, 8-row atoms of 1 KB).
-inline OperandStaging make_staging(int mn_major, int rows, int ksub) {
+inline OperandStaging make_staging(int mn_major, int rows, int ksub, int ab_bytes) {
   OperandStaging s;
   s.mn_major = (uint32_t)mn_major;
   const uint32_t sbo = 1024u >> 4;       // between 8-row groups of a swizzle atom column
@@ -315,11 +330,17 @@ inline OperandStaging make_staging(int mn_major, int rows, int ksub) {
     s.k_step_enc = (kUmmaK * 2) >> 4;                // 32 bytes along the 128-byte row
     s.k_sub_enc = ((uint32_t)rows * 128u) >> 4;      // next sub-block: next box of `rows` rows
     s.box_bytes = (uint32_t)rows * 128u;
+    s.mn_boxes = 1;
+    s.mn_box = (uint32_t)rows;
   } else {
-    s.box_bytes = (uint32_t)ksub * kBlockK * 128u;   // one box: 64*ksub k-rows of 128 bytes
-    s.lbo_enc = s.box_bytes >> 4;                    // next 64 M/N elements: next box
-    s.k_step_enc = (kUmmaK * 128u) >> 4;             // 16 k-rows of 128 bytes
-    s.k_sub_enc = (kBlockK * 128u) >> 4;             // k-rows continue inside the same box
+    const uint32_t sub_k = (uint32_t)sub_block_k(ab_bytes);   // k-rows per sub-block: 64 or 32
+    const uint32_t umma_k = sub_k / 4;                        // k-rows per MMA: 16 or 8
+    s.mn_box = sub_k;                                         // M/N elements in 128 bytes: also 64 or 32
+    s.mn_boxes = (uint32_t)rows / s.mn_box;
+    s.box_bytes = (uint32_t)ksub * sub_k * 128u;     // one box: sub_k*ksub k-rows of 128 bytes
+    s.lbo_enc = s.box_bytes >> 4;                    // next group of M/N elements: next box
+    s.k_step_enc = (umma_k * 128u) >> 4;             // the k-rows of one MMA
+    s.k_sub_enc = (sub_k * 128u) >> 4;               // k-rows continue inside the same box
   }
   return s;
 }

@@ -102,8 +102,23 @@ def to_fp16_bits(x: np.ndarray) -> np.ndarray:
     return np.ascontiguousarray(x).astype(np.float16).view(np.uint16)
 
 
-def round_to_storage(x: np.ndarray, dtype: int) -> np.ndarray:
-    """Round a real array to the storage type; returns uint16 bits or float32."""
+def f32_round_to_tf32(x: np.ndarray) -> np.ndarray:
+    """fp32 values rounded to nearest-even onto the tf32 grid (10 fraction bits), still stored as fp32."""
+    b = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    lsb = (b >> np.uint32(13)) & np.uint32(1)
+    r = (b + np.uint32(0x0FFF) + lsb) & np.uint32(0xFFFFE000)
+    return r.view(np.float32)
+
+
+def round_to_storage(x: np.ndarray, dtype: int, operand: bool = False) -> np.ndarray:
+    """Round a real array to the storage type; returns uint16 bits or float32.
+
+    ``operand=True`` with FP32 means an A or B matrix of the tf32 mode: stored as fp32, with values
+    on the tf32 grid, so that the tensor core (which ignores the low 13 fraction bits) and the oracle
+    (which widens the stored value exactly) see the same numbers.
+    """
+    if dtype == FP32 and operand:
+        return f32_round_to_tf32(x.astype(np.float32))
     if dtype == BF16:
         return f32_to_bf16_bits(x.astype(np.float32))
     if dtype == FP16:
@@ -158,7 +173,7 @@ def load(buf: np.ndarray, rows: int, cols: int, layout: int, ld: int) -> np.ndar
 # matrices and workloads
 # ----------------------------------------------------------------------------
 def matrix(seed: int, tag: int, rows: int, cols: int, dtype: int, dist: str = "uniform",
-           chunk_rows: int = 2048) -> np.ndarray:
+           chunk_rows: int = 2048, operand: bool = False) -> np.ndarray:
     """Logical rows x cols matrix in storage type (uint16 bits, or float32)."""
     out = np.empty((rows, cols), dtype=storage_np_dtype(dtype))
     cj = np.arange(cols, dtype=np.int64)
@@ -170,7 +185,7 @@ def matrix(seed: int, tag: int, rows: int, cols: int, dtype: int, dist: str = "u
             x = normal_01(seed, tag, ri, cj)
         else:
             raise ValueError(dist)
-        out[r0:r0 + len(ri)] = round_to_storage(x, dtype)
+        out[r0:r0 + len(ri)] = round_to_storage(x, dtype, operand)
     return out
 
 
@@ -199,8 +214,8 @@ class Problem:
     def generate(self, pad_a=None, pad_b=None, pad_c=None):
         """Fill A, B and C_in.  C_in is drawn uniform[-1,1] in every case (it is
         only read when beta != 0)."""
-        a = matrix(self.seed, TAG_A, self.M, self.K, self.ab_dtype, self.dist)
-        b = matrix(self.seed, TAG_B, self.K, self.N, self.ab_dtype, self.dist)
+        a = matrix(self.seed, TAG_A, self.M, self.K, self.ab_dtype, self.dist, operand=True)
+        b = matrix(self.seed, TAG_B, self.K, self.N, self.ab_dtype, self.dist, operand=True)
         c = matrix(self.seed, TAG_C, self.M, self.N, self.c_dtype, "uniform")
         self.A = store(a, self.a_layout, self.lda, pad_a)
         self.B = store(b, self.b_layout, self.ldb, pad_b)

@@ -79,7 +79,10 @@ def test_validate_rejects_bad_arguments():
 
 
 def test_validate_unsupported_but_legal_blas_calls():
-    assert B.exo_gemm_validate(good(ab_dtype=B.FP32)) == B.ERR_UNSUPPORTED
+    assert B.exo_gemm_validate(good(ab_dtype=B.FP32, c_dtype=B.FP32)) == B.OK        # tf32 mode
+    assert B.exo_gemm_validate(good(ab_dtype=B.FP32, c_dtype=B.BF16)) == B.ERR_UNSUPPORTED
+    assert B.exo_gemm_validate(good(ab_dtype=B.FP32, K=130)) == B.ERR_UNSUPPORTED     # 520 bytes per row
+    assert B.exo_gemm_validate(good(ab_dtype=B.FP32, K=132)) == B.OK
     assert B.exo_gemm_validate(good(ab_dtype=B.BF16, c_dtype=B.FP16)) == B.ERR_UNSUPPORTED
     assert B.exo_gemm_validate(good(K=100)) == B.ERR_UNSUPPORTED            # lda = 100: 200 bytes, not 16 | it
     assert B.exo_gemm_validate(good(K=100, lda=104, ldb=104)) == B.OK
@@ -106,6 +109,8 @@ def test_plan_preview_geometry_and_overrides():
     assert st == B.OK
     i = info.as_dict()
     assert i["tile_m"] == 128 * i["cta_group"] and i["tile_k"] in (64, 128)
+    st, t32 = B.exo_gemm_plan_preview(good(M=4096, N=4096, K=4096, ab_dtype=B.FP32), 148)
+    assert st == B.OK and t32.tile_k in (32, 64)
     assert i["tiles_m"] * i["tile_m"] >= 4096 and i["tiles_n"] * i["tile_n"] >= 4096
     assert i["grid"] <= 148 and i["grid"] % i["cta_group"] == 0
     assert i["smem_bytes"] <= 232448 and i["tmem_columns"] == 2 * i["tile_n"] <= 512

@@ -300,6 +300,29 @@ def test_back_to_back_dependent_gemms_keep_stream_order():
             assert np.array_equal(d_host, ref)
 
 
+# ------------------------------------------------------------------ fp32 storage, tf32 math
+@pytest.mark.parametrize("lc", [0, 1])
+@pytest.mark.parametrize("shape", [(128, 64, 32), (264, 328, 200), (1000, 520, 1028), (129, 257, 36), (72, 40, 4)])
+@pytest.mark.parametrize("g,bn,ksub", [(0, 0, 0), (1, 64, 1), (1, 128, 2), (1, 256, 1), (2, 128, 2), (2, 256, 1), (2, 256, 2)])
+def test_tf32_operands(lc, shape, g, bn, ksub):
+    M, N, K = shape
+    ldc = -(-(N if lc == 0 else M) // 4) * 4
+    p = synth.Problem("tf32", M, N, K, FP32, FP32, 0, 1, lc, 1.25, -0.5, seed=M + 3 * N + 7 * K + lc,
+                      ldc=ldc, lda=-(-K // 4) * 4, ldb=-(-K // 4) * 4)
+    p.generate()
+    check_full(p, flags_for(g, bn, ksub=ksub) if g else 0, literal=True)
+
+
+def test_tf32_other_layouts_are_refused():
+    for la, lb in ((1, 1), (0, 0), (1, 0)):
+        assert B.exo_gemm_validate(B.make_desc(128, 128, 64, FP32, FP32, la, lb, 0)) == B.ERR_UNSUPPORTED
+
+
+def test_tf32_large_sampled():
+    p = synth.Problem("tf32_big", 4096, 2048, 4096, FP32, FP32, 0, 1, 0, 1.0, 0.0, seed=4242).generate()
+    check_sampled(p)
+
+
 # ------------------------------------------------------------------ strided batch
 BATCH_CASES = [
     # M, N, K, ab, cd, la, lb, lc, alpha, beta, batch, pad (extra elements between matrices), shared operand

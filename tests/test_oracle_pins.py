@@ -323,3 +323,26 @@ def test_bf16_rounding_is_nearest_even():
     got = oracle.widen(synth.f32_to_bf16_bits(x), BF16)
     want = np.array([1.0, 1.0, 1.0 + 2 ** -6, 1.0 + 2 ** -7, 1.0 + 2 ** -7, -1.0, 0.0, 2.0 ** -20])
     assert np.array_equal(got, want)
+
+
+def test_tf32_grid_rounding_and_fp32_operands_in_the_oracle():
+    x = np.array([1.0, 1.0 + 2 ** -11, 1.0 + 3 * 2 ** -11, 1.0 + 2 ** -10, -1.0 - 2 ** -11 - 2 ** -20, 3.14159265, 0.0],
+                 dtype=np.float32)
+    got = synth.f32_round_to_tf32(x)
+    want = np.array([1.0, 1.0, 1.0 + 2 ** -9, 1.0 + 2 ** -10, -1.0 - 2 ** -10, 3.140625, 0.0], dtype=np.float32)
+    assert np.array_equal(got, want)                       # ties to even, 10 fraction bits kept
+    assert np.all(got.view(np.uint32) & 0x1FFF == 0)
+    # fp32 operands go through the same definition: an all-ones product gives exactly K
+    M, N, K = 5, 4, 300
+    A = np.ones(M * K, np.float32)
+    Bm = np.ones(K * N, np.float32)
+    C = np.zeros(M * N, np.float32)
+    cref, den = oracle.gemm(M, N, K, A, Bm, C, FP32, FP32, 0, 0, 0, K, N, N, 1.0, 0.0)
+    assert np.all(cref == K) and np.all(den == K)
+    p = synth.Problem("t32", 40, 24, 64, FP32, FP32, 0, 1, 0, 0.5, 1.0, seed=9).generate()
+    assert np.all(p.A.view(np.uint32) & 0x1FFF == 0) and np.any(p.C.view(np.uint32) & 0x1FFF != 0)
+    cref, den = oracle.gemm_problem(p)
+    A64 = oracle.logical_view(p.A, 40, 64, 0, p.lda, FP32)
+    B64 = oracle.logical_view(p.B, 64, 24, 1, p.ldb, FP32)
+    C64 = oracle.logical_view(p.C, 40, 24, 0, p.ldc, FP32)
+    assert np.max(np.abs(cref - (0.5 * (A64 @ B64) + C64))) < 1e-12
