@@ -59,6 +59,8 @@ def make_problem(name: str, rank: int = 0):
     if name.startswith("batched_"):
         batch, n = (int(x) for x in name[len("batched_"):].split("x"))
         p = synth.batched(batch, n)
+    elif name.startswith("tf32_"):
+        p = synth.tf32_square(int(name[len("tf32_"):]))
     elif name.startswith("sweep_"):
         M, N, K = (int(x) for x in name[len("sweep_"):].split("x"))
         p = synth.sweep_problem(M, N, K)
@@ -304,6 +306,8 @@ def run_ours(args, rank, world, local_rank):
         achieved = flop / (avg_kernel_ms * 1e-3) / 1e12
         timed_region_s = total_ms * 1e-3
         peak = pk["tflops_burst"] if timed_region_s < 1.0 else pk["tflops_sustained"]
+        if p.ab_dtype == synth.FP32:   # tf32: the bf16 measurement times the nominal tf32/bf16 ratio (1.1 / 2.25)
+            peak *= 1.1 / 2.25
         ai = flop / p.algorithmic_bytes
         hbm_bound_tflops = ai * pk["hbm_gbs"] / 1e3
         tensor_bound = hbm_bound_tflops >= peak
@@ -327,7 +331,7 @@ def run_ours(args, rank, world, local_rank):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None,
-            "dtype": ("bf16" if p.ab_dtype == synth.BF16 else "fp16") + " in, fp32 accumulate",
+            "dtype": {synth.BF16: "bf16", synth.FP16: "fp16", synth.FP32: "tf32"}[p.ab_dtype] + " in, fp32 accumulate",
             "data": "synthetic",
             "config": {"workload": args.workload, "M": p.M, "N": p.N, "K": p.K, "batch": batch,
                        "ab_dtype": synth.dtype_name(p.ab_dtype), "c_dtype": synth.dtype_name(p.c_dtype),
@@ -359,7 +363,10 @@ def time_cublas(p, dev, steps, n_sets):
     import torch
     from paper_2609_16389_b200 import synth
     try:
-        tdt = torch.bfloat16 if p.ab_dtype == synth.BF16 else torch.float16
+        tdt = {synth.BF16: torch.bfloat16, synth.FP16: torch.float16, synth.FP32: torch.float32}[p.ab_dtype]
+        prev_tf32 = torch.backends.cuda.matmul.allow_tf32
+        if p.ab_dtype == synth.FP32:
+            torch.backends.cuda.matmul.allow_tf32 = True     # cuBLAS in tf32 tensor-op mode, as in the paper
         batch = getattr(p, "batch", 1)
         if batch > 1:
             a = torch.randn(batch, p.M, p.K, device=dev).to(tdt)
@@ -510,7 +517,7 @@ def main():
             raise SystemExit("the reference arm times one workload; pick e.g. --workload sweep_1000x1000x1000")
         run_sweep(args, rank, world, local_rank)
         return
-    if args.workload not in WORKLOADS and not args.workload.startswith(("sweep_", "batched_")):
+    if args.workload not in WORKLOADS and not args.workload.startswith(("sweep_", "batched_", "tf32_")):
         raise SystemExit(f"unknown workload {args.workload}")
     if args.impl == "reference":
         run_reference(args, rank, world)

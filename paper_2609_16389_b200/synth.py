@@ -285,6 +285,11 @@ def batched(batch: int, n: int) -> BatchedProblem:
                           1.0, 0.0, BASE_SEED + 50)
 
 
+def tf32_square(n: int) -> Problem:
+    """n^3 GEMM in the precision the paper measured (Section 6): fp32 storage, tf32 math, fp32 C."""
+    return Problem(f"tf32_{n}", n, n, n, FP32, FP32, ROW_MAJOR, COL_MAJOR, ROW_MAJOR, 1.0, 0.0, BASE_SEED + 60)
+
+
 def config(idx: int, variant: str | None = None) -> Problem:
     """The benchmark configurations (0-based index into the configuration list).
 
