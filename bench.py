@@ -507,11 +507,110 @@ def run_sweep(args, rank, world, local_rank):
     print(json.dumps(line), flush=True)
 
 
+def run_gemv(args, rank, world, local_rank):
+    """fp32 GEMV y = A x (row-major A), the paper's memory-bound companion workload (Section 6).
+    Workload name gemv_<M>x<N>.  A step = one exo_gemv_run; the matrices rotate through several copies
+    so that every step streams A from HBM.  Roofline: HBM (algorithmic bytes = 4*M*N + 4*N + 4*M)."""
+    import torch
+    from paper_2609_16389_b200 import binding as B
+    if rank != 0:
+        return
+    M, N = (int(v) for v in args.workload[len("gemv_"):].split("x"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    pk = peaks()
+    rng = np.random.default_rng(260916389 + 70)
+    hA = rng.uniform(-1, 1, size=M * N).astype(np.float32)
+    hx = rng.uniform(-1, 1, size=N).astype(np.float32)
+    n_sets = int(max(2, min(16, np.ceil(2.0 * L2_BYTES / hA.nbytes))))
+    dAs = [torch.from_numpy(hA).to(dev) for _ in range(n_sets)]
+    dx = torch.from_numpy(hx).to(dev)
+    dy = torch.zeros(M, dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream(dev)
+
+    def step(i):
+        st = B.exo_gemv_run(M, N, dAs[i % n_sets].data_ptr(), N, dx.data_ptr(), dy.data_ptr(), 1.0, 0.0, stream.cuda_stream)
+        if st != B.OK:
+            raise B.ExoGemmError(st, "exo_gemv_run")
+
+    for i in range(max(3, args.warmup)):
+        step(i)
+    torch.cuda.synchronize(dev)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    e1.record(stream)
+    torch.cuda.synchronize(dev)
+    ms = e0.elapsed_time(e1) / args.steps
+    # end to end: A, x from pinned host memory, y back
+    pA, px = torch.from_numpy(hA).pin_memory(), torch.from_numpy(hx).pin_memory()
+    py = torch.empty(M, dtype=torch.float32).pin_memory()
+    k = max(3, min(10, args.steps))
+    torch.cuda.synchronize(dev)
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record(stream)
+    for _ in range(k):
+        dAs[0].copy_(pA, non_blocking=True)
+        dx.copy_(px, non_blocking=True)
+        step(0)
+        py.copy_(dy, non_blocking=True)
+    f1.record(stream)
+    torch.cuda.synchronize(dev)
+    e2e_ms = f0.elapsed_time(f1) / k
+    clocks = sampler.stop()
+    flop = 2.0 * M * N
+    abytes = 4.0 * (M * N + N + M)
+    gbs = abytes / (ms * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": flop / (ms * 1e-3) / 1e12, "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": args.workload, "M": M, "N": N, "layout": "A row-major",
+                   "l2": f"rotating {n_sets} copies of A ({n_sets * hA.nbytes >> 20} MiB > 126 MiB L2)"},
+        "roofline": {"bound": "hbm", "achieved": gbs, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": gbs / pk["hbm_gbs"],
+                     "traffic": None, "peak_source": f"{pk['source']} (copy bandwidth)", "kernel": "exo_gemv_rowmajor_kernel",
+                     "algorithmic_bytes": abytes, "flop": flop},
+        "e2e": {"value": flop / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": int(hA.nbytes + hx.nbytes),
+                "d2h_bytes_per_step": int(4 * M), "ms_per_step": e2e_ms, "steps": k},
+        "gpu_launches": args.steps, "clocks": clocks,
+    }
+    if not args.no_cublas:
+        xs = dx
+        for _ in range(3):
+            torch.mv(dAs[0].view(M, N), xs, out=dy)
+        torch.cuda.synchronize(dev)
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record(stream)
+        for i in range(args.steps):
+            torch.mv(dAs[i % n_sets].view(M, N), xs, out=dy)
+        g1.record(stream)
+        torch.cuda.synchronize(dev)
+        cms = g0.elapsed_time(g1) / args.steps
+        line["cublas"] = {"gbs": abytes / (cms * 1e-3) / 1e9, "ms_per_step": cms, "note": "torch.mv (cublasSgemv)"}
+    if not args.no_cpu_baseline:
+        import oracle
+        rows = min(M, max(1, int(2e9 / max(N, 1))))
+        t0 = time.perf_counter()
+        oracle.gemv(rows, N, hA, N, hx, np.zeros(rows, np.float32), 1.0, 0.0)
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": 2.0 * rows * N / dt / 1e12, "unit": UNIT, "cores": oracle.num_threads(),
+                                "kind": "oracle", "sample": f"rows 0..{rows} of {args.workload}, {dt:.2f} s wall"}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     args = parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.workload.startswith("gemv_"):
+        if args.impl == "reference":
+            raise SystemExit("the reference arm times GEMM workloads")
+        run_gemv(args, rank, world, local_rank)
+        return
     if args.workload == "sweep":
         if args.impl == "reference":
             raise SystemExit("the reference arm times one workload; pick e.g. --workload sweep_1000x1000x1000")

@@ -226,6 +226,22 @@ exo_gemm_status_t exo_gemm_get_info(exo_gemm_handle_t plan, exo_gemm_info_t* inf
 exo_gemm_status_t exo_gemm_run_static(const exo_gemm_desc_t* desc, const void* A, const void* B, void* C,
                                       float alpha, float beta, void* cuda_stream, uint32_t* detail);
 
+/*
+ * fp32 matrix-vector product y = alpha*A*x + beta*y, A an M x N row-major matrix with
+ * leading dimension lda >= N (elements): the paper's second workload (Section 6: a
+ * full-precision GEMV from warp shuffles and scalar math, memory-bound, roofline
+ * 2 FLOP per 4 bytes of A).  A, x, y are DEVICE pointers owned by the caller; y is
+ * updated in place; x and A must not overlap y.  beta == 0: y is not read;
+ * alpha == 0: A and x are not read.  Enqueued on cuda_stream (current device),
+ * returns without synchronising; nothing is allocated.  128-bit loads are used when
+ * A and x are 16-byte aligned and lda % 4 == 0, scalar loads otherwise.  Products
+ * are accumulated in fp32 (one warp per row, lanes interleaved over the row, then a
+ * shuffle tree).  Errors: ERR_INVALID_ARG (negative size, lda < N), ERR_NULL,
+ * ERR_ARCH, ERR_CUDA.
+ */
+exo_gemm_status_t exo_gemv_run(int64_t M, int64_t N, const float* A, int64_t lda, const float* x, float* y,
+                               float alpha, float beta, void* cuda_stream);
+
 /* Frees the plan and its device status block.  NULL is a no-op returning OK. */
 exo_gemm_status_t exo_gemm_destroy(exo_gemm_handle_t plan);
 

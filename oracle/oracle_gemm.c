@@ -231,3 +231,29 @@ int oracle_gemm_entries(int64_t M, int64_t N, int64_t K,
     }
     return 0;
 }
+
+/*
+ * y_ref = alpha * A x + beta * y for a row-major fp32 A (the paper's Section 6 GEMV workload), by the
+ * definition, in fp64, j ascending; den_i = sum_j |a_ij x_j| + |beta y_i|.  beta == 0: y is not read.
+ */
+int oracle_gemv(int64_t M, int64_t N, const float* A, int64_t lda, const float* x, const float* y,
+                double alpha, double beta, double* yref, double* den) {
+    if (M < 0 || N < 0 || lda < N) return 1;
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < M; ++i) {
+        double s = 0.0, d = 0.0;
+        for (int64_t j = 0; j < N; ++j) {
+            double p = (double)A[i * lda + j] * (double)x[j];
+            s += p;
+            d += fabs(p);
+        }
+        double r = alpha * s;
+        if (beta != 0.0) {
+            r += beta * (double)y[i];
+            d += fabs(beta * (double)y[i]);
+        }
+        yref[i] = r;
+        den[i] = d;
+    }
+    return 0;
+}

@@ -9,8 +9,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libexo_gemm.so")
-SOURCES = ["api.cu"]
-DEPS = ["api.cu", "gemm_kernel.cuh", "gemm_params.h", "plan.h", "ptx.cuh", "tile_scheduler.h",
+SOURCES = ["api.cu", "gemv.cu"]
+DEPS = ["api.cu", "gemv.cu", "gemm_kernel.cuh", "gemm_params.h", "plan.h", "ptx.cuh", "tile_scheduler.h",
         os.path.join("..", "..", "include", "exo_gemm.h")]
 
 

@@ -323,6 +323,49 @@ def test_tf32_large_sampled():
     check_sampled(p)
 
 
+# ------------------------------------------------------------------ fp32 GEMV
+@pytest.mark.parametrize("M,N,lda", [(1, 1, 1), (37, 53, 60), (300, 1000, 1000), (4096, 4099, 4100), (5000, 520, 520),
+                                     (2, 70000, 70000), (20000, 128, 132)])
+@pytest.mark.parametrize("alpha,beta", [(1.0, 0.0), (-0.75, 1.5), (0.0, 2.0)])
+def test_gemv_against_the_oracle(M, N, lda, alpha, beta):
+    import torch
+    rng = np.random.default_rng(M * 7 + N)
+    A = rng.uniform(-1, 1, size=M * lda).astype(np.float32)
+    x = rng.uniform(-1, 1, size=N).astype(np.float32)
+    y = rng.uniform(-1, 1, size=M).astype(np.float32)
+    if beta == 0.0:
+        y[:] = np.nan
+    dev = torch.device("cuda:0")
+    dA, dx, dy = harness._to_device(A, dev), harness._to_device(x, dev), harness._to_device(y, dev)
+    st = B.exo_gemv_run(M, N, dA.data_ptr(), lda, dx.data_ptr(), dy.data_ptr(), alpha, beta,
+                        torch.cuda.current_stream(dev).cuda_stream)
+    assert st == B.OK
+    torch.cuda.synchronize(dev)
+    got = dy.cpu().numpy().view(np.float32).astype(np.float64)
+    yref, den = oracle.gemv(M, N, A, lda, x, np.nan_to_num(y), alpha, beta)
+    assert oracle.max_error(got, yref, den) <= TOL
+
+
+def test_gemv_unaligned_operands_take_the_scalar_path_and_bad_arguments_are_refused():
+    import torch
+    M, N, lda = 200, 333, 335                       # lda % 4 != 0
+    rng = np.random.default_rng(3)
+    A = rng.uniform(-1, 1, size=M * lda + 1).astype(np.float32)
+    x = rng.uniform(-1, 1, size=N + 1).astype(np.float32)
+    y = np.zeros(M, np.float32)
+    dev = torch.device("cuda:0")
+    dA, dx, dy = harness._to_device(A, dev), harness._to_device(x, dev), harness._to_device(y, dev)
+    st = B.exo_gemv_run(M, N, dA.data_ptr() + 4, lda, dx.data_ptr() + 4, dy.data_ptr(), 1.0, 0.0)   # 4-byte offsets
+    assert st == B.OK
+    torch.cuda.synchronize(dev)
+    got = dy.cpu().numpy().view(np.float32).astype(np.float64)
+    yref, den = oracle.gemv(M, N, A[1:].copy(), lda, x[1:].copy(), y, 1.0, 0.0)
+    assert oracle.max_error(got, yref, den) <= TOL
+    assert B.exo_gemv_run(-1, 4, dA.data_ptr(), 4, dx.data_ptr(), dy.data_ptr(), 1.0, 0.0) == B.ERR_INVALID_ARG
+    assert B.exo_gemv_run(4, 8, dA.data_ptr(), 4, dx.data_ptr(), dy.data_ptr(), 1.0, 0.0) == B.ERR_INVALID_ARG
+    assert B.exo_gemv_run(4, 8, 0, 8, dx.data_ptr(), dy.data_ptr(), 1.0, 0.0) == B.ERR_NULL
+
+
 # ------------------------------------------------------------------ strided batch
 BATCH_CASES = [
     # M, N, K, ab, cd, la, lb, lc, alpha, beta, batch, pad (extra elements between matrices), shared operand

@@ -346,3 +346,29 @@ def test_tf32_grid_rounding_and_fp32_operands_in_the_oracle():
     B64 = oracle.logical_view(p.B, 64, 24, 1, p.ldb, FP32)
     C64 = oracle.logical_view(p.C, 40, 24, 0, p.ldc, FP32)
     assert np.max(np.abs(cref - (0.5 * (A64 @ B64) + C64))) < 1e-12
+
+
+def test_gemv_oracle_against_closed_forms_and_a_library_product():
+    rng = np.random.default_rng(12)
+    M, N, lda = 37, 53, 60
+    A = np.full(M * lda, np.nan, dtype=np.float32)                # padding must never be read
+    Al = rng.integers(-8, 9, size=(M, N)).astype(np.float32) / 4
+    A.reshape(M, lda)[:, :N] = Al
+    x = (rng.integers(-8, 9, size=N) / 8).astype(np.float32)
+    y = rng.integers(-8, 9, size=M).astype(np.float32)
+    yref, den = oracle.gemv(M, N, A, lda, x, y, 2.0, -0.5)
+    want = 2.0 * (Al.astype(np.float64) @ x.astype(np.float64)) - 0.5 * y
+    assert np.array_equal(yref, want)                              # small dyadic values: exact either way
+    assert np.array_equal(den, np.abs(Al.astype(np.float64)) @ np.abs(x.astype(np.float64)) + np.abs(0.5 * y))
+    ones = np.ones(M * lda, np.float32)
+    yref, den = oracle.gemv(M, N, ones, lda, np.ones(N, np.float32), np.full(M, np.nan, np.float32), 1.0, 0.0)
+    assert np.all(yref == N) and np.all(den == N)                  # beta == 0 ignores y
+    e = np.zeros(N, np.float32); e[7] = 1.0                        # unit vector picks a column
+    yref, _ = oracle.gemv(M, N, A, lda, e, y, 1.0, 0.0)
+    assert np.array_equal(yref, Al[:, 7].astype(np.float64))
+    # as a one-column GEMM the fp16 oracle gives the same numbers on fp16-exact data
+    A16 = synth.round_to_storage(Al, FP16); x16 = synth.round_to_storage(x.reshape(N, 1), FP16)
+    cref, cden = oracle.gemm(M, 1, N, synth.store(A16, 0), synth.store(x16, 0), np.zeros(M, np.float32),
+                             FP16, FP32, 0, 0, 0, N, 1, 1, 1.0, 0.0)
+    g, gd = oracle.gemv(M, N, A, lda, x, y, 1.0, 0.0)
+    assert np.array_equal(cref[:, 0], g) and np.array_equal(cden[:, 0], gd)
