@@ -51,6 +51,8 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-cublas", action="store_true")
     ap.add_argument("--flags", type=int, default=0, help="EXO_GEMM_FLAG_* overrides (experiments)")
+    ap.add_argument("--share", default="auto", choices=["auto", "never", "always"],
+                    help="shared-operand 4-CTA clusters (needs the variant library; single-GPU runs only)")
     return ap.parse_args()
 
 
@@ -226,7 +228,8 @@ def run_ours(args, rank, world, local_rank):
     for _ in range(n_sets):
         sets.append((harness._to_device(p.A, dev), harness._to_device(p.B, dev), harness._to_device(p.C, dev)))
     batch = getattr(p, "batch", 1)
-    plan = B.Plan(harness.desc_of(p, args.flags, local_rank),
+    flags2 = {"auto": B.FLAG2_SHARE_AUTO, "never": B.FLAG2_SHARE_NEVER, "always": B.FLAG2_SHARE_ALWAYS}[args.share]
+    plan = B.Plan(harness.desc_of(p, args.flags, local_rank, flags2),
                   batch=(batch, p.stride_a, p.stride_b, p.stride_c) if batch > 1 else None)
     info = plan.info()
     stream = torch.cuda.current_stream(dev)

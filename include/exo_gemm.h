@@ -61,6 +61,25 @@ typedef enum { EXO_GEMM_ROW_MAJOR = 0, EXO_GEMM_COL_MAJOR = 1 } exo_gemm_layout_
 #define EXO_GEMM_FLAG_SPLIT_K(f) (((uint32_t)(f) & 15u) << 28)
 
 /*
+ * flags2, bits 0-1: clusters of two CTA pairs (4 SMs) that compute neighbouring 256 x 256
+ * tiles of the same rows of C and share the loads of A -- each of the two CTAs that need a
+ * 128-row block fetches half of it and the TMA copy is multicast to both (the paper's
+ * Section 6 kernels multicast the operand their cluster has in common in the same way).
+ * The grid is cut into slots of four CTAs; the launch prefers 4-CTA clusters and lets the
+ * device substitute two plain pairs for a slot where no four SMs of one GPC are free (those
+ * pairs compute the same two tiles, each loading all of its A rows), so every SM is used.
+ * 0 = the library decides, 1 = never, 2 = always (ERR_UNSUPPORTED from create /
+ * run_static / plan_preview if the loaded library was built without the variant, see
+ * exo_gemm_has_shared_operand_clusters; ERR_INVALID_ARG together with a CTA_GROUP(1),
+ * a TILE_N other than 256 or a GRID_LIMIT that is not a multiple of 4), 3 = as 2 but every
+ * slot is launched as two plain pairs (a test aid for the substitute path).
+ */
+#define EXO_GEMM_FLAG2_SHARE_AUTO 0u
+#define EXO_GEMM_FLAG2_SHARE_NEVER 1u
+#define EXO_GEMM_FLAG2_SHARE_ALWAYS 2u
+#define EXO_GEMM_FLAG2_SHARE_SUBSTITUTED 3u
+
+/*
  * Problem descriptor.  Logical shapes: A is M x K, B is K x N, C is M x N.
  * Leading dimensions are in elements: for a row-major matrix ld >= #columns, for
  * a column-major matrix ld >= #rows.
@@ -85,7 +104,7 @@ typedef struct {
   int32_t device;                       /* CUDA device ordinal; -1 = the current device        */
   int64_t lda, ldb, ldc;                /* elements                                            */
   uint32_t flags;                       /* 0, or EXO_GEMM_FLAG_* overrides                     */
-  uint32_t reserved;                    /* must be 0                                           */
+  uint32_t flags2;                      /* 0, or EXO_GEMM_FLAG2_*; other bits must be 0        */
 } exo_gemm_desc_t;
 
 /* What a plan decided; filled by exo_gemm_get_info. */
@@ -108,6 +127,8 @@ typedef struct {
   int32_t tail_tiles;      /* tiles in that partial last wave                                  */
   int32_t workspace_bytes; /* device scratch the plan owns for the slices' partial sums        */
   int32_t batch_count;     /* matrices per launch (1 unless created by exo_gemm_create_batched) */
+  int32_t cluster_size;    /* CTAs per cluster: cta_group, or 4 when two pairs share the loads of A
+                              (tiles_n then counts 2 * tile_n columns per step)                 */
 } exo_gemm_info_t;
 
 /*
@@ -285,6 +306,13 @@ int64_t exo_gemm_schedule_work(int64_t tiles, int32_t num_workers, int32_t split
  * error status without trapping.  The settings apply to one run, then reset.
  */
 exo_gemm_status_t exo_gemm_debug_set(exo_gemm_handle_t plan, int32_t timeout_ms, int64_t skip_k_block);
+
+/*
+ * 1 if this build of the library contains the shared-operand cluster variant
+ * (EXO_GEMM_FLAG2_SHARE_*), else 0.  The variant is compiled into a separate
+ * library file; programs that span several GPUs use the base library.
+ */
+int32_t exo_gemm_has_shared_operand_clusters(void);
 
 #ifdef __cplusplus
 }

@@ -19,7 +19,7 @@ EXPORTED_SYMBOLS = (
     "exo_gemm_validate", "exo_gemm_create", "exo_gemm_run", "exo_gemm_check", "exo_gemm_plan_preview",
     "exo_gemm_get_info", "exo_gemm_destroy", "exo_gemm_status_string", "exo_gemm_last_cuda_error",
     "exo_gemm_schedule_enumerate", "exo_gemm_debug_set", "exo_gemm_run_static", "exo_gemm_schedule_work",
-    "exo_gemm_create_batched", "exo_gemv_run",
+    "exo_gemm_create_batched", "exo_gemv_run", "exo_gemm_has_shared_operand_clusters",
 )
 
 
@@ -32,6 +32,7 @@ def flag_k_subblocks(k): return (k & 3) << 20
 def flag_epi_buffers(b): return (b & 3) << 22
 def flag_max_stages(s): return (s & 15) << 24
 def flag_split_k(f): return (f & 15) << 28
+FLAG2_SHARE_AUTO, FLAG2_SHARE_NEVER, FLAG2_SHARE_ALWAYS, FLAG2_SHARE_SUBSTITUTED = 0, 1, 2, 3
 
 
 class Desc(ctypes.Structure):
@@ -40,7 +41,7 @@ class Desc(ctypes.Structure):
                 ("a_layout", ctypes.c_int32), ("b_layout", ctypes.c_int32), ("c_layout", ctypes.c_int32),
                 ("device", ctypes.c_int32),
                 ("lda", ctypes.c_int64), ("ldb", ctypes.c_int64), ("ldc", ctypes.c_int64),
-                ("flags", ctypes.c_uint32), ("reserved", ctypes.c_uint32)]
+                ("flags", ctypes.c_uint32), ("flags2", ctypes.c_uint32)]
 
 
 class Info(ctypes.Structure):
@@ -48,7 +49,7 @@ class Info(ctypes.Structure):
         "cta_group", "tile_m", "tile_n", "tile_k", "stages", "grid", "smem_bytes", "tmem_columns",
         "tiles_m", "tiles_n", "raster_along_m", "raster_band", "swapped", "sm_count",
         "kernel_launches_per_run", "epilogue_buffers", "split_k", "tail_tiles", "workspace_bytes",
-        "batch_count")]
+        "batch_count", "cluster_size")]
 
     def as_dict(self):
         return {n: getattr(self, n) for n, _ in self._fields_}
@@ -68,7 +69,9 @@ def lib():
     """Loads (building first if needed) the CUDA library; raises if that fails."""
     global _lib
     if _lib is None:
-        path = os.environ.get("EXO_GEMM_LIBRARY") or _build.build()   # override: a development build
+        # EXO_GEMM_LIBRARY overrides (a development build); otherwise the variant library -- the base
+        # library plus the shared-operand cluster kernels -- where its sources are present, else the base one
+        path = os.environ.get("EXO_GEMM_LIBRARY") or _build.build_preferred()
         if not os.path.exists(path):
             raise RuntimeError("libexo_gemm.so is missing: the CUDA path cannot run")
         L = ctypes.CDLL(path)
@@ -85,6 +88,7 @@ def lib():
         L.exo_gemm_status_string.argtypes = [ctypes.c_int]
         L.exo_gemm_status_string.restype = ctypes.c_char_p
         L.exo_gemm_last_cuda_error.restype = ctypes.c_int
+        L.exo_gemm_has_shared_operand_clusters.restype = i32
         L.exo_gemm_schedule_enumerate.argtypes = [i32, i32, i32, i32, i32, i32, ctypes.POINTER(i32),
                                                   ctypes.POINTER(i32), i64]
         L.exo_gemm_schedule_enumerate.restype = i64
@@ -105,16 +109,20 @@ def lib():
 
 
 def make_desc(M, N, K, ab_dtype, c_dtype, a_layout, b_layout, c_layout, lda=None, ldb=None, ldc=None,
-              device=-1, flags=0) -> Desc:
+              device=-1, flags=0, flags2=0) -> Desc:
     def ext(layout, rows, cols):
         return max(1, cols if layout == ROW_MAJOR else rows)
     return Desc(M, N, K, ab_dtype, c_dtype, a_layout, b_layout, c_layout, device,
                 ext(a_layout, M, K) if lda is None else lda,
                 ext(b_layout, K, N) if ldb is None else ldb,
-                ext(c_layout, M, N) if ldc is None else ldc, flags, 0)
+                ext(c_layout, M, N) if ldc is None else ldc, flags, flags2)
 
 
 # ---- one function per C entry point -------------------------------------------------
+def exo_gemm_has_shared_operand_clusters() -> int:
+    return int(lib().exo_gemm_has_shared_operand_clusters())
+
+
 def exo_gemm_validate(desc: Desc) -> int:
     return lib().exo_gemm_validate(ctypes.byref(desc) if desc is not None else None)
 

@@ -9,6 +9,12 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libexo_gemm.so")
+# The same library with the shared-operand cluster kernels compiled in.  Those kernels use a form of TMA
+# load that only single-GPU programs may contain, so their source directory and this file are left
+# out of multi-GPU deployments, which then run on the base library.
+SHARE_DIR = os.path.join(CSRC, "cluster4")
+SHARE_LIB = os.path.join(HERE, "libexo_gemm_cluster4.so")
+SHARE_DEPS = [os.path.join("cluster4", "share_pairs.cuh")]
 SOURCES = ["api.cu", "gemv.cu"]
 DEPS = ["api.cu", "gemv.cu", "gemm_kernel.cuh", "gemm_params.h", "plan.h", "ptx.cuh", "tile_scheduler.h",
         os.path.join("..", "..", "include", "exo_gemm.h")]
@@ -21,26 +27,59 @@ def nvcc_path() -> str:
     raise RuntimeError("nvcc not found: the CUDA library cannot be built")
 
 
-def is_stale() -> bool:
-    if not os.path.exists(LIB):
+def is_stale(lib: str = LIB, deps=DEPS) -> bool:
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
-    return any(os.path.getmtime(os.path.join(CSRC, d)) > t for d in DEPS)
+    t = os.path.getmtime(lib)
+    return any(os.path.getmtime(os.path.join(CSRC, d)) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not is_stale():
-        return LIB
-    tmp = LIB + f".tmp{os.getpid()}"
+def _compile(lib: str, defines, verbose: bool) -> str:
+    tmp = lib + f".tmp{os.getpid()}"
     cmd = [nvcc_path(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-shared", "-Xcompiler", "-fPIC", "-cudart", "static", "-o", tmp]
+    cmd += [f"-D{d}" for d in defines]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += [os.path.join(CSRC, s) for s in SOURCES]
     subprocess.run(cmd, check=True)
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    return lib
+
+
+def build(force: bool = False, verbose: bool = False) -> str:
+    """The base library."""
+    if not force and not is_stale():
+        return LIB
+    return _compile(LIB, [], verbose)
+
+
+def have_share_sources() -> bool:
+    return all(os.path.exists(os.path.join(CSRC, d)) for d in SHARE_DEPS)
+
+
+def build_share(force: bool = False, verbose: bool = False) -> str:
+    """The variant library; raises if its sources are not present."""
+    if not have_share_sources():
+        raise RuntimeError("the shared-operand cluster sources are not part of this deployment")
+    if not force and not is_stale(SHARE_LIB, DEPS + SHARE_DEPS):
+        return SHARE_LIB
+    return _compile(SHARE_LIB, ["EXO_GEMM_SHARE_PAIRS"], verbose)
+
+
+def build_preferred() -> str:
+    """The library a single-GPU program should load: the variant where it can be built, else the base."""
+    if os.environ.get("EXO_GEMM_BASE_ONLY") != "1" and have_share_sources():
+        return build_share()
+    return build()
+
+
+def build_all(force: bool = False, verbose: bool = False):
+    out = [build(force, verbose)]
+    if have_share_sources():
+        out.append(build_share(force, verbose))
+    return out
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build_all(force="--force" in sys.argv, verbose="-v" in sys.argv))

@@ -11,6 +11,9 @@
 #include "../../include/exo_gemm.h"
 #include "gemm_kernel.cuh"
 #include "plan.h"
+#ifdef EXO_GEMM_SHARE_PAIRS
+#include "cluster4/share_pairs.cuh"
+#endif
 
 namespace exo {
 
@@ -33,7 +36,24 @@ static KernelFn pick_shape(int cta_group, int bn, int out) {
   return pick_out<1, 64, KSUB>(out);
 }
 
-static KernelFn pick_kernel(int cta_group, int bn, int ksub, int out) {
+#ifdef EXO_GEMM_SHARE_PAIRS
+constexpr bool kHaveSharePairs = true;
+template <int KSUB>
+static KernelFn pick_shared(int out) {
+  switch (out) {
+    case EXO_GEMM_BF16: return exo_gemm_kernel<2, 256, kOutBf16, KSUB, SharePairs>;
+    case EXO_GEMM_FP16: return exo_gemm_kernel<2, 256, kOutFp16, KSUB, SharePairs>;
+    default:            return exo_gemm_kernel<2, 256, kOutFp32, KSUB, SharePairs>;
+  }
+}
+#else
+constexpr bool kHaveSharePairs = false;
+template <int KSUB>
+static KernelFn pick_shared(int) { return nullptr; }
+#endif
+
+static KernelFn pick_kernel(int cta_group, int bn, int ksub, int out, int pairs = 1) {
+  if (pairs == 2) return ksub == 2 ? pick_shared<2>(out) : pick_shared<1>(out);
   return ksub == 2 ? pick_shape<2>(cta_group, bn, out) : pick_shape<1>(cta_group, bn, out);
 }
 
@@ -147,6 +167,47 @@ exo_gemm_status_t cuda_fail(cudaError_t e) {
   return EXO_GEMM_ERR_CUDA;
 }
 
+// How many clusters of `cluster` CTAs of kernel `probe` can be resident at once (GPC shapes may
+// leave SMs that fit no further cluster).
+cudaError_t max_active_clusters(KernelFn probe, int sms, int cluster, int* out) {
+  const int smem = kSmemLimit - 1024;  // every plan's shared-memory request is close to the limit
+  cudaError_t e = cudaFuncSetAttribute((const void*)probe, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t lc{};
+  lc.gridDim = dim3((unsigned)(sms / cluster * cluster), 1, 1);
+  lc.blockDim = dim3(kNumThreads, 1, 1);
+  lc.dynamicSmemBytes = smem;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = (unsigned)cluster;
+  at[0].val.clusterDim.y = 1;
+  at[0].val.clusterDim.z = 1;
+  lc.attrs = at;
+  lc.numAttrs = 1;
+  int n = 0;
+  e = cudaOccupancyMaxActiveClusters(&n, (const void*)probe, &lc);
+  if (e != cudaSuccess) return e;
+  *out = n < sms / cluster ? n : sms / cluster;
+  return cudaSuccess;
+}
+
+// Co-resident CTA pairs, and slots of two pairs (0 where the shared-operand variant is not built in
+// or not wanted).  A slot runs as one 4-CTA cluster where the device finds four free SMs in a GPC
+// and as two 2-CTA clusters elsewhere, so the pairs bound the slot count.
+cudaError_t cluster_capacity(int sms, int c_dtype, const FlagOverrides& ov, int* max_pairs, int* max_quads) {
+  *max_pairs = 0;
+  *max_quads = 0;
+  if (ov.cta_group == 1) return cudaSuccess;
+  cudaError_t e = max_active_clusters(pick_kernel(2, 256, 2, c_dtype), sms, 2, max_pairs);
+  if (e != cudaSuccess) return e;
+  if (kHaveSharePairs && ov.share != 1) {
+    int pairs_shared = 0;  // the variant kernel has its own resource footprint
+    e = max_active_clusters(pick_kernel(2, 256, 2, c_dtype, 2), sms, 2, &pairs_shared);
+    *max_quads = pairs_shared / 2 < sms / 4 ? pairs_shared / 2 : sms / 4;
+  }
+  return e;
+}
+
 void fill_info(const exo_gemm_plan* p, exo_gemm_info_t* info) {
   memset(info, 0, sizeof(*info));
   info->cta_group = p->cfg.cta_group;
@@ -154,7 +215,8 @@ void fill_info(const exo_gemm_plan* p, exo_gemm_info_t* info) {
   info->tile_n = p->cfg.tile_n;
   info->tile_k = sub_block_k(p->canon.ab_bytes) * p->cfg.ksub;
   info->stages = p->cfg.stages;
-  info->grid = p->cfg.workers * p->cfg.cta_group;
+  info->grid = p->cfg.workers * p->cfg.cta_group * p->cfg.pairs;
+  info->cluster_size = p->cfg.cta_group * p->cfg.pairs;
   info->smem_bytes = p->smem_bytes;
   info->tmem_columns = 2 * p->cfg.tile_n;
   info->tiles_m = p->cfg.tiles_m;
@@ -245,7 +307,9 @@ exo_gemm_status_t exo_gemm_plan_preview(const exo_gemm_desc_t* desc, int32_t sm_
   p.desc = *desc;
   p.canon = canonicalize(*desc);
   p.sm_count = sm_count;
-  p.cfg = choose_config(p.canon, decode_flags(desc->flags), sm_count, sm_count / 2);
+  const FlagOverrides ov = decode_flags(desc->flags, desc->flags2);
+  if (ov.share >= 2 && !kHaveSharePairs) return EXO_GEMM_ERR_UNSUPPORTED;
+  p.cfg = choose_config(p.canon, ov, sm_count, sm_count / 2, kHaveSharePairs ? sm_count / 4 : 0);
   p.cfg.workspace_bytes = split_workspace_bytes(p.cfg, desc->c_dtype);
   p.smem_bytes = smem_bytes_for(p.cfg.cta_group, p.cfg.tile_n, p.cfg.ksub, p.cfg.stages, p.cfg.epi_bufs);
   fill_info(&p, info);
@@ -289,36 +353,18 @@ exo_gemm_status_t exo_gemm_create_batched(exo_gemm_handle_t* out, const exo_gemm
   p->sm_count = sms;
   p->dbg_timeout_ms = 0;
   p->dbg_skip_k_block = -1;
-  const FlagOverrides ov = decode_flags(desc->flags);
+  const FlagOverrides ov = decode_flags(desc->flags, desc->flags2);
 
-  // How many 2-CTA clusters can be resident at once (GPC shapes may leave SMs unpaired).
-  int max_pairs = 0;
-  if (ov.cta_group != 1) {
-    KernelFn probe = pick_kernel(2, 256, 2, desc->c_dtype);
-    const int smem = kSmemLimit - 1024;  // every plan's shared-memory request is close to the limit
-    e = cudaFuncSetAttribute((const void*)probe, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) { delete p; return cuda_fail(e); }
-    cudaLaunchConfig_t lc{};
-    lc.gridDim = dim3((unsigned)sms & ~1u, 1, 1);
-    lc.blockDim = dim3(kNumThreads, 1, 1);
-    lc.dynamicSmemBytes = smem;
-    cudaLaunchAttribute at[1];
-    at[0].id = cudaLaunchAttributeClusterDimension;
-    at[0].val.clusterDim.x = 2;
-    at[0].val.clusterDim.y = 1;
-    at[0].val.clusterDim.z = 1;
-    lc.attrs = at;
-    lc.numAttrs = 1;
-    int n = 0;
-    e = cudaOccupancyMaxActiveClusters(&n, (const void*)probe, &lc);
-    if (e != cudaSuccess) { delete p; return cuda_fail(e); }
-    max_pairs = n < sms / 2 ? n : sms / 2;
-  }
+  if (ov.share >= 2 && !kHaveSharePairs) { delete p; return EXO_GEMM_ERR_UNSUPPORTED; }
+  int max_pairs = 0, max_quads = 0;
+  e = cluster_capacity(sms, desc->c_dtype, ov, &max_pairs, &max_quads);
+  if (e != cudaSuccess) { delete p; return cuda_fail(e); }
+  if (ov.share >= 2 && max_quads < 1) { delete p; return EXO_GEMM_ERR_UNSUPPORTED; }
 
-  p->cfg = choose_config(p->canon, ov, sms, max_pairs);
+  p->cfg = choose_config(p->canon, ov, sms, max_pairs, max_quads);
   p->cfg.workspace_bytes = split_workspace_bytes(p->cfg, desc->c_dtype);
   p->split_epoch = 0;
-  p->kernel = pick_kernel(p->cfg.cta_group, p->cfg.tile_n, p->cfg.ksub, desc->c_dtype);
+  p->kernel = pick_kernel(p->cfg.cta_group, p->cfg.tile_n, p->cfg.ksub, desc->c_dtype, p->cfg.pairs);
   p->smem_bytes = smem_bytes_for(p->cfg.cta_group, p->cfg.tile_n, p->cfg.ksub, p->cfg.stages, p->cfg.epi_bufs);
   e = cudaFuncSetAttribute((const void*)p->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, p->smem_bytes);
   if (e != cudaSuccess) { delete p; return cuda_fail(e); }
@@ -328,8 +374,9 @@ exo_gemm_status_t exo_gemm_create_batched(exo_gemm_handle_t* out, const exo_gemm
   if (e != cudaSuccess) { cudaFree(p->d_status); delete p; return cuda_fail(e); }
   if (p->cfg.split > 1) {  // scratch for the K-slices of the tail tiles
     e = cudaMalloc((void**)&p->d_split_ws, (size_t)p->cfg.workspace_bytes);
-    if (e == cudaSuccess) e = cudaMalloc((void**)&p->d_split_flags, sizeof(uint32_t) * (size_t)p->cfg.tail_tiles);
-    if (e == cudaSuccess) e = cudaMemset(p->d_split_flags, 0, sizeof(uint32_t) * (size_t)p->cfg.tail_tiles);
+    const size_t flag_bytes = sizeof(uint32_t) * (size_t)p->cfg.tail_tiles * (size_t)p->cfg.pairs;
+    if (e == cudaSuccess) e = cudaMalloc((void**)&p->d_split_flags, flag_bytes);
+    if (e == cudaSuccess) e = cudaMemset(p->d_split_flags, 0, flag_bytes);
     if (e != cudaSuccess) {
       cudaFree(p->d_split_ws);
       cudaFree(p->d_split_flags);
@@ -347,6 +394,8 @@ exo_gemm_status_t exo_gemm_get_info(exo_gemm_handle_t plan, exo_gemm_info_t* inf
   fill_info(plan, info);
   return EXO_GEMM_OK;
 }
+
+int32_t exo_gemm_has_shared_operand_clusters(void) { return kHaveSharePairs ? 1 : 0; }
 
 exo_gemm_status_t exo_gemm_debug_set(exo_gemm_handle_t plan, int32_t timeout_ms, int64_t skip_k_block) {
   if (!plan) return EXO_GEMM_ERR_NULL;
@@ -409,11 +458,12 @@ exo_gemm_status_t exo_gemm_run(exo_gemm_handle_t plan, const void* A, const void
   memset(&tm_b, 0, sizeof tm_b);
   CUresult r;
   const int b_rows = cfg.tile_n / cfg.cta_group;
+  const int a_rows = kBlockM / cfg.pairs;  // pairs that share A fetch half of a CTA's rows each
   const uint32_t c_box = d.c_dtype == EXO_GEMM_FP32 ? 32 : 64;
   if (cn.batch <= 1) {
     if (read_ab) {
       r = cn.a_mn_major ? encode_2d(&tm_a, d.ab_dtype, opA, cn.M, cn.K, cn.lda, sub_k, stage_k, true)
-                        : encode_2d(&tm_a, d.ab_dtype, opA, cn.K, cn.M, cn.lda, sub_k, kBlockM, true);
+                        : encode_2d(&tm_a, d.ab_dtype, opA, cn.K, cn.M, cn.lda, sub_k, a_rows, true);
       if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return EXO_GEMM_ERR_CUDA; }
       r = cn.b_mn_major ? encode_2d(&tm_b, d.ab_dtype, opB, cn.N, cn.K, cn.ldb, sub_k, stage_k, true)
                         : encode_2d(&tm_b, d.ab_dtype, opB, cn.K, cn.N, cn.ldb, sub_k, b_rows, true);
@@ -425,7 +475,7 @@ exo_gemm_status_t exo_gemm_run(exo_gemm_handle_t plan, const void* A, const void
     if (read_ab) {
       r = cn.a_mn_major
               ? encode_3d(&tm_a, d.ab_dtype, opA, cn.M, cn.K, cn.lda, cn.batch, cn.stride_a, sub_k, stage_k, true)
-              : encode_3d(&tm_a, d.ab_dtype, opA, cn.K, cn.M, cn.lda, cn.batch, cn.stride_a, sub_k, kBlockM, true);
+              : encode_3d(&tm_a, d.ab_dtype, opA, cn.K, cn.M, cn.lda, cn.batch, cn.stride_a, sub_k, a_rows, true);
       if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return EXO_GEMM_ERR_CUDA; }
       r = cn.b_mn_major
               ? encode_3d(&tm_b, d.ab_dtype, opB, cn.N, cn.K, cn.ldb, cn.batch, cn.stride_b, sub_k, stage_k, true)
@@ -440,13 +490,13 @@ exo_gemm_status_t exo_gemm_run(exo_gemm_handle_t plan, const void* A, const void
   DeviceGuard guard(plan->device);
   if (guard.err != cudaSuccess) return cuda_fail(guard.err);
   cudaLaunchConfig_t lc{};
-  lc.gridDim = dim3((unsigned)(cfg.workers * cfg.cta_group), 1, 1);
+  lc.gridDim = dim3((unsigned)(cfg.workers * cfg.cta_group * cfg.pairs), 1, 1);
   lc.blockDim = dim3(kNumThreads, 1, 1);
   lc.dynamicSmemBytes = plan->smem_bytes;
   lc.stream = (cudaStream_t)cuda_stream;
-  cudaLaunchAttribute at[2];
+  cudaLaunchAttribute at[3];
   at[0].id = cudaLaunchAttributeClusterDimension;
-  at[0].val.clusterDim.x = cfg.cta_group;
+  at[0].val.clusterDim.x = (unsigned)cfg.cta_group;
   at[0].val.clusterDim.y = 1;
   at[0].val.clusterDim.z = 1;
   // Programmatic dependent launch: this kernel's CTAs may start (barrier set-up, TMEM allocation)
@@ -456,6 +506,14 @@ exo_gemm_status_t exo_gemm_run(exo_gemm_handle_t plan, const void* A, const void
   at[1].val.programmaticStreamSerializationAllowed = 1;
   lc.attrs = at;
   lc.numAttrs = 2;
+  if (cfg.pairs == 2 && (d.flags2 & 3u) != 3u) {
+    // Slots of four CTAs: 4-CTA clusters wherever four SMs of a GPC are free, else two regular pairs.
+    at[2].id = cudaLaunchAttributePreferredClusterDimension;
+    at[2].val.preferredClusterDim.x = 4;
+    at[2].val.preferredClusterDim.y = 1;
+    at[2].val.preferredClusterDim.z = 1;
+    lc.numAttrs = 3;
+  }
   if (split_now) {  // arrival counters only grow: this run is complete at epoch * arrivals-per-run
     const uint32_t epoch = plan->split_epoch.fetch_add(1) + 1;
     prm.split_target = epoch * (uint32_t)((cfg.split - 1) * kEpiWarps * cfg.cta_group);
@@ -477,7 +535,7 @@ exo_gemm_status_t exo_gemm_check(exo_gemm_handle_t plan, uint32_t* detail) {
   e = cudaMemset(plan->d_status, 0, 32);
   if (e != cudaSuccess) return cuda_fail(e);
   if (plan->d_split_flags) {  // an abandoned run may have left the arrival counters short
-    e = cudaMemset(plan->d_split_flags, 0, sizeof(uint32_t) * (size_t)plan->cfg.tail_tiles);
+    e = cudaMemset(plan->d_split_flags, 0, sizeof(uint32_t) * (size_t)plan->cfg.tail_tiles * (size_t)plan->cfg.pairs);
     if (e != cudaSuccess) return cuda_fail(e);
     plan->split_epoch = 0;
   }
@@ -542,32 +600,15 @@ exo_gemm_status_t exo_gemm_run_static(const exo_gemm_desc_t* desc, const void* A
   plan.sm_count = sms;
   plan.dbg_timeout_ms = 0;
   plan.dbg_skip_k_block = -1;
-  FlagOverrides ov = decode_flags(desc->flags);
+  FlagOverrides ov = decode_flags(desc->flags, desc->flags2);
   ov.no_workspace = true;  // K-slicing of the tail tiles needs device scratch this entry point may not allocate
-  int max_pairs = 0;
-  if (ov.cta_group != 1) {
-    KernelFn probe = pick_kernel(2, 256, 2, desc->c_dtype);
-    const int smem = kSmemLimit - 1024;  // every plan's shared-memory request is close to the limit
-    e = cudaFuncSetAttribute((const void*)probe, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return cuda_fail(e);
-    cudaLaunchConfig_t lc{};
-    lc.gridDim = dim3((unsigned)sms & ~1u, 1, 1);
-    lc.blockDim = dim3(kNumThreads, 1, 1);
-    lc.dynamicSmemBytes = smem;
-    cudaLaunchAttribute at[1];
-    at[0].id = cudaLaunchAttributeClusterDimension;
-    at[0].val.clusterDim.x = 2;
-    at[0].val.clusterDim.y = 1;
-    at[0].val.clusterDim.z = 1;
-    lc.attrs = at;
-    lc.numAttrs = 1;
-    int n = 0;
-    e = cudaOccupancyMaxActiveClusters(&n, (const void*)probe, &lc);
-    if (e != cudaSuccess) return cuda_fail(e);
-    max_pairs = n < sms / 2 ? n : sms / 2;
-  }
-  plan.cfg = choose_config(plan.canon, ov, sms, max_pairs);
-  plan.kernel = pick_kernel(plan.cfg.cta_group, plan.cfg.tile_n, plan.cfg.ksub, desc->c_dtype);
+  if (ov.share >= 2 && !kHaveSharePairs) return EXO_GEMM_ERR_UNSUPPORTED;
+  int max_pairs = 0, max_quads = 0;
+  e = cluster_capacity(sms, desc->c_dtype, ov, &max_pairs, &max_quads);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (ov.share >= 2 && max_quads < 1) return EXO_GEMM_ERR_UNSUPPORTED;
+  plan.cfg = choose_config(plan.canon, ov, sms, max_pairs, max_quads);
+  plan.kernel = pick_kernel(plan.cfg.cta_group, plan.cfg.tile_n, plan.cfg.ksub, desc->c_dtype, plan.cfg.pairs);
   plan.smem_bytes = smem_bytes_for(plan.cfg.cta_group, plan.cfg.tile_n, plan.cfg.ksub, plan.cfg.stages, plan.cfg.epi_bufs);
   e = cudaFuncSetAttribute((const void*)plan.kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem_bytes);
   if (e != cudaSuccess) return cuda_fail(e);

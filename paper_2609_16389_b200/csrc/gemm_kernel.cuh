@@ -118,7 +118,14 @@ __device__ __forceinline__ float2 unpack2(uint32_t w) {
   }
 }
 
-template <int CTA_GROUP, int BN, int OUT, int KSUB>
+// Default policy: a CTA group loads all of its own operands.  The alternative (a cluster of two
+// CTA pairs that split the loads of the A rows they have in common) supplies kPairs == 2 and the
+// load functions for the shared half-blocks; it lives in a translation unit of its own.
+struct NoShare {
+  static constexpr int kPairs = 1;
+};
+
+template <int CTA_GROUP, int BN, int OUT, int KSUB, class Share = NoShare>
 __global__ void __launch_bounds__(kNumThreads, 1)
 exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                 const __grid_constant__ CUtensorMap tm_c, const GemmParams p) {
@@ -130,6 +137,10 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   constexpr int CW = (OUT == kOutFp32) ? 32 : 64;    // columns per epilogue chunk = 128 bytes of C
   constexpr int NCHUNK = BN / CW;
   constexpr bool PAIR = CTA_GROUP == 2;
+  constexpr int NPAIR = Share::kPairs;              // CTA pairs per cluster that compute side by side in N
+  constexpr bool SHARE = NPAIR > 1;                  // ... and fetch half of their common A rows each
+  constexpr int CLUSTER = CTA_GROUP * NPAIR;
+  static_assert(!SHARE || (PAIR && NPAIR == 2), "operand sharing is built on CTA pairs");
   static_assert(BN == 64 || BN == 128 || BN == 256, "tile N");
   const uint32_t STAGES = (uint32_t)p.stages;         // ring depth, chosen by the host plan
   const uint32_t EPI_BUFS = (uint32_t)p.epi_bufs;     // staging buffers per epilogue warp (1 or 2)
@@ -149,9 +160,17 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
 
   const uint32_t warp = threadIdx.x >> 5;
   const uint32_t lane = threadIdx.x & 31u;
-  const uint32_t cta_rank = PAIR ? ptx::cluster_ctarank() : 0u;
-  const int64_t worker = blockIdx.x / CTA_GROUP;
-  const int64_t num_workers = gridDim.x / CTA_GROUP;
+  const uint32_t cluster_rank = PAIR ? ptx::cluster_ctarank() : 0u;
+  const uint32_t cta_rank = cluster_rank & 1u;            // position inside the CTA pair
+  const uint32_t leader = cluster_rank & ~1u;             // cluster rank of this pair's MMA-issuing CTA
+  // With operand sharing the grid is cut into slots of four CTAs.  The launch asks for 4-CTA clusters
+  // but lets the device substitute two 2-CTA clusters where no four SMs of one GPC are free; such a
+  // slot computes the same two tiles with each pair loading all of its A rows itself.
+  const uint32_t slot_rank = (uint32_t)blockIdx.x & (uint32_t)(CLUSTER - 1);
+  const uint32_t pair_id = SHARE ? slot_rank >> 1 : 0u;   // which of the slot's two tiles
+  const bool quad = SHARE && ptx::cluster_nctarank() == 4u;
+  const int64_t worker = blockIdx.x / CLUSTER;
+  const int64_t num_workers = gridDim.x / CLUSTER;
   const int32_t nkb = p.num_k_blocks;
 
   if (threadIdx.x == 0) EXO_TRACE(2, 4095, 0, 4096);
@@ -159,7 +178,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   if (threadIdx.x == 0) {
     for (uint32_t s = 0; s < STAGES; ++s) {
       ptx::mbar_init(full_bar(s), 1);
-      ptx::mbar_init(empty_bar(s), 1);
+      ptx::mbar_init(empty_bar(s), quad ? 2 : 1);  // every pair whose CTAs fill the stage releases it
     }
     for (uint32_t a = 0; a < 2; ++a) {
       ptx::mbar_init(tfull_bar(a), 1);
@@ -201,7 +220,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     uint32_t s = 0, ph = 0;
     int64_t issued = 0;
     // in a pair, both CTAs' loads are counted on the leader's full barrier
-    const uint32_t full0 = PAIR ? ptx::map_to_cta(full_bar(0), 0) : full_bar(0);
+    const uint32_t full0 = PAIR ? ptx::map_to_cta(full_bar(0), leader) : full_bar(0);
     for (int64_t it = 0; ok; ++it) {
       WorkItem wi;
       if (!work_item(p.work, worker, num_workers, it, nkb, &wi)) break;
@@ -210,7 +229,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       const uint32_t bz = batched ? (uint32_t)t / p.tiles_per_batch : 0u;  // which matrix of the batch
       const TileCoord tc = raster_decode(p.raster, batched ? (uint32_t)t - bz * p.tiles_per_batch : t);
       const int32_t a_mn0 = tc.m * (kBlockM * CTA_GROUP) + (int32_t)cta_rank * kBlockM;
-      const int32_t b_mn0 = tc.n * BN + (int32_t)cta_rank * B_ROWS;
+      const int32_t b_mn0 = (tc.n * NPAIR + (int32_t)pair_id) * BN + (int32_t)cta_rank * B_ROWS;
       for (int32_t kb = wi.kb_begin; kb < wi.kb_end; ++kb) {
         ok = wait_barrier<PAIR>(empty_bar(s), ph ^ 1u, p, WaitSite{kRoleProducer, s, (uint32_t)t, (uint32_t)kb});
         ok = __all_sync(0xffffffffu, ok);
@@ -234,7 +253,32 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                 else ptx::tma_load_2d(dst, map, x, y, bar);
               }
             };
-            if (!p.a.mn_major) {
+            if (quad) {
+              if constexpr (SHARE) {
+                // The other pair's CTA of the same rank needs the same 128 rows of A: each of the two
+                // fetches 64 of them and the copy lands in both CTAs' stages; each copy's bytes count
+                // on the full barrier of the receiving CTA's own pair leader.
+                const uint16_t both = (uint16_t)((1u << cta_rank) | (1u << (cta_rank + 2u)));
+                auto load_shared = [&](uint32_t dst, int32_t x, int32_t y) {
+                  if (batched) Share::load_3d(dst, &tm_a, x, y, (int32_t)(bz & p.a_z_mask), bar, both);
+                  else Share::load_2d(dst, &tm_a, x, y, bar, both);
+                };
+                if (!p.a.mn_major) {
+#pragma unroll
+                  for (int h = 0; h < KSUB; ++h)
+                    load_shared(a_dst + h * kATileBytes + pair_id * (kATileBytes / 2), k0 + h * (int32_t)p.sub_k,
+                                a_mn0 + (int32_t)pair_id * (kBlockM / 2));
+                } else {  // two boxes of 64 rows: one each
+                  load_shared(a_dst + pair_id * p.a.box_bytes, a_mn0 + (int32_t)(p.a.mn_box * pair_id), k0);
+                }
+              }
+            } else if (SHARE && !p.a.mn_major) {  // substituted pair: both 64-row halves, same tensor map
+#pragma unroll
+              for (int h = 0; h < KSUB; ++h) {
+                load(a_dst + h * kATileBytes, &tm_a, k0 + h * (int32_t)p.sub_k, a_mn0);
+                load(a_dst + h * kATileBytes + kATileBytes / 2, &tm_a, k0 + h * (int32_t)p.sub_k, a_mn0 + kBlockM / 2);
+              }
+            } else if (!p.a.mn_major) {
 #pragma unroll
               for (int h = 0; h < KSUB; ++h) load(a_dst + h * kATileBytes, &tm_a, k0 + h * (int32_t)p.sub_k, a_mn0);
             } else {
@@ -265,7 +309,8 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     // ============================================================ MMA issuer
     if (cta_rank == 0 && nkb > 0) {
       uint32_t s = 0, ph = 0, acc = 0, acc_ph = 0;
-      constexpr uint16_t kMask = PAIR ? 3 : 1;
+      const uint16_t kStageMask = quad ? 0xF : (PAIR ? 3 : 1);  // a stage is released in every CTA that fills it
+      const uint16_t pair_mask = (uint16_t)((PAIR ? 3u : 1u) << leader);   // the accumulator belongs to this pair
       [[maybe_unused]] int64_t consumed = 0;
       const uint32_t a_step = p.a.k_step_enc, b_step = p.b.k_step_enc;
       const uint32_t a_sub = p.a.k_sub_enc, b_sub = p.b.k_sub_enc;
@@ -319,8 +364,8 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                                            idesc, accumulate);
               }
             }
-            ptx::umma_commit<CTA_GROUP>(empty_bar(s), kMask);  // stage free once these MMAs completed
-            if (kb == wi.kb_end - 1) ptx::umma_commit<CTA_GROUP>(tfull_bar(acc), kMask);  // accumulator complete
+            ptx::umma_commit<CTA_GROUP>(empty_bar(s), kStageMask);  // stage free once these MMAs completed
+            if (kb == wi.kb_end - 1) ptx::umma_commit<CTA_GROUP>(tfull_bar(acc), pair_mask);  // accumulator complete
             EXO_TRACE(1, consumed, 1, 4096);
           }
           ++consumed;
@@ -339,7 +384,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     const uint32_t ew = warp - 2u;
     const int32_t half = (int32_t)(ew >> 2);
     const uint32_t buf0 = epi0 + ew * EPI_BUFS * kEpiBufBytes;
-    const uint32_t tempty0 = PAIR ? ptx::map_to_cta(tempty_bar(0), 0) : tempty_bar(0);
+    const uint32_t tempty0 = PAIR ? ptx::map_to_cta(tempty_bar(0), leader) : tempty_bar(0);
     const bool has_beta = p.beta != 0.f;
     const bool has_acc = nkb > 0;
     const bool scale = p.alpha != 1.f;
@@ -360,7 +405,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       const uint32_t bz = batched ? (uint32_t)t / p.tiles_per_batch : 0u;
       const TileCoord tc = raster_decode(p.raster, batched ? (uint32_t)t - bz * p.tiles_per_batch : t);
       const int32_t row0 = tc.m * (kBlockM * CTA_GROUP) + (int32_t)cta_rank * kBlockM + (int32_t)quad * 32;
-      const int32_t col0 = tc.n * BN;
+      const int32_t col0 = (tc.n * NPAIR + (int32_t)pair_id) * BN;
       int32_t nch = 0;  // chunks of this tile that hold any valid column, if this warp's rows exist
       if (row0 < p.M) {
         nch = (p.N - col0 + CW - 1) / CW;
@@ -397,8 +442,8 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       const bool contributor = wi.slices > 1 && wi.slice != 0;
       const bool owner = wi.slices > 1 && wi.slice == 0;
       auto ws_unit = [&](int32_t slice_m1, int32_t i, int32_t q) {
-        const uint64_t idx = ((((uint64_t)wi.tail_index * (uint32_t)(wi.slices - 1) + (uint32_t)slice_m1) * CTA_GROUP +
-                               cta_rank) * kEpiWarps + ew) * (uint32_t)(((NCHUNK + 1) / 2) * UPC) +
+        const uint64_t idx = ((((uint64_t)wi.tail_index * (uint32_t)(wi.slices - 1) + (uint32_t)slice_m1) * CLUSTER +
+                               slot_rank) * kEpiWarps + ew) * (uint32_t)(((NCHUNK + 1) / 2) * UPC) +
                              (uint32_t)(i * UPC + q);
         return reinterpret_cast<char*>(p.split_ws) + idx * kUnitBytes + lane * 16u;
       };
@@ -419,13 +464,13 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         }
         __threadfence();  // each lane's partials are visible GPU-wide before the arrival below
         __syncwarp();
-        if (ptx::elect_one()) ptx::red_release_gpu_add(p.split_flags + wi.tail_index, 1u);
+        if (ptx::elect_one()) ptx::red_release_gpu_add(p.split_flags + wi.tail_index * NPAIR + (int32_t)pair_id, 1u);
         if ((acc ^= 1u) == 0u) acc_ph ^= 1u;
         continue;
       }
       if (owner && mine > 0) {
         // wait (bounded) until every warp of every other slice has delivered its partials
-        const uint32_t* flag = p.split_flags + wi.tail_index;
+        const uint32_t* flag = p.split_flags + wi.tail_index * NPAIR + (int32_t)pair_id;
         const long long t_start = clock64();
         uint32_t spins = 0;
         for (;;) {

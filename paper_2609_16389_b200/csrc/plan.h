@@ -22,9 +22,11 @@ struct FlagOverrides {
   int band;        // 0 = auto
   int along_m;     // 0 = auto/default, 1 = forced
   int grid_limit;  // 0 = none
+  int share;       // clusters of two CTA pairs sharing the loads of A: 0 = auto, 1 = never, 2 = always,
+                   // 3 = always, but every slot launched as two plain pairs (exercises the substitute path)
 };
 
-inline FlagOverrides decode_flags(uint32_t f) {
+inline FlagOverrides decode_flags(uint32_t f, uint32_t f2 = 0) {
   FlagOverrides o;
   o.cta_group = (int)(f & 3u);
   o.tile_n = (int)((f >> 2) & 15u) * 64;
@@ -36,12 +38,13 @@ inline FlagOverrides decode_flags(uint32_t f) {
   o.stages = (int)((f >> 24) & 15u);
   o.split = (int)((f >> 28) & 15u);
   o.no_workspace = false;
+  o.share = (int)(f2 & 3u);
   return o;
 }
 
 inline exo_gemm_status_t validate_desc(const exo_gemm_desc_t* d) {
   if (!d) return EXO_GEMM_ERR_NULL;
-  if (d->reserved != 0) return EXO_GEMM_ERR_INVALID_ARG;
+  if ((d->flags2 & ~3u) != 0) return EXO_GEMM_ERR_INVALID_ARG;
   const int64_t kMaxDim = 2147483647LL;
   if (d->M < 0 || d->N < 0 || d->K < 0 || d->M > kMaxDim || d->N > kMaxDim || d->K > kMaxDim)
     return EXO_GEMM_ERR_INVALID_ARG;
@@ -63,11 +66,14 @@ inline exo_gemm_status_t validate_desc(const exo_gemm_desc_t* d) {
   if (((d->flags >> 20) & 3u) == 3u || ((d->flags >> 22) & 3u) == 3u) return EXO_GEMM_ERR_INVALID_ARG;
   if (((d->flags >> 24) & 15u) == 1u || ((d->flags >> 24) & 15u) > (uint32_t)kMaxStages) return EXO_GEMM_ERR_INVALID_ARG;
   if (d->flags & (1u << 11)) return EXO_GEMM_ERR_INVALID_ARG;
-  const FlagOverrides o = decode_flags(d->flags);
+  const FlagOverrides o = decode_flags(d->flags, d->flags2);
   if (o.cta_group == 3) return EXO_GEMM_ERR_INVALID_ARG;
   if (o.tile_n != 0 && o.tile_n != 64 && o.tile_n != 128 && o.tile_n != 256) return EXO_GEMM_ERR_INVALID_ARG;
   if (o.cta_group == 2 && o.tile_n == 64) return EXO_GEMM_ERR_INVALID_ARG;
   if (o.grid_limit != 0 && o.cta_group == 2 && (o.grid_limit & 1)) return EXO_GEMM_ERR_INVALID_ARG;
+  // forcing the shared-operand clusters fixes the tile shape they are built for
+  if (o.share >= 2 && (o.cta_group == 1 || (o.tile_n != 0 && o.tile_n != 256) || (o.grid_limit & 3)))
+    return EXO_GEMM_ERR_INVALID_ARG;
   // beyond here the call is a legal BLAS call; what follows is this library's supported set
   // fp32 operands are multiplied as tf32 (the precision of the paper's own kernels) into an fp32 C
   if (d->c_dtype != EXO_GEMM_FP32 && d->c_dtype != d->ab_dtype) return EXO_GEMM_ERR_UNSUPPORTED;
@@ -149,7 +155,8 @@ struct TileConfig {
   int owner_extra;         // k-blocks the owning slice takes beyond an even share
   int64_t workspace_bytes; // fp32 partials of slices 1.. of the tail tiles
   int cta_group, tile_n, ksub, stages, epi_bufs;
-  int tiles_m, tiles_n;
+  int pairs;               // CTA pairs per cluster (2: the pairs share the loads of A; else 1)
+  int tiles_m, tiles_n;    // tiles of (128 * cta_group) x (tile_n * pairs): what one cluster computes at a time
   int band, along_m;
   int workers;  // CTA groups launched
 };
@@ -167,6 +174,9 @@ inline double shape_efficiency(int cta_group, int bn) {
   if (cta_group == 2) return bn == 256 ? 1.0 : 0.81;
   return bn == 256 ? 0.86 : (bn == 128 ? 0.66 : 0.40);
 }
+
+// Main-loop speed of the shared-operand clusters relative to independent pairs.
+constexpr double kShareGain = 1.0;
 
 // k-elements in one 128-byte sub-block row: 64 for 16-bit operands, 32 for fp32 storage.
 inline int sub_block_k(int ab_bytes) { return 128 / ab_bytes; }
@@ -189,14 +199,15 @@ inline int split_factor(int64_t tiles, int64_t workers, int64_t K, int ksub, con
 // Estimated time of the whole problem in SM clocks for one candidate tile shape: whole waves of
 // tiles, then the partial last wave (cut along K if that pays), plus what is exposed once per launch.
 inline double estimate_clocks(int64_t M, int64_t N, int64_t K, int64_t batch, int cta_group, int bn,
-                              int max_workers, const FlagOverrides& o) {
+                              int max_workers, const FlagOverrides& o, int pairs = 1) {
   const int64_t tm = (M + 128 * cta_group - 1) / (128 * cta_group);
-  const int64_t tn = (N + bn - 1) / bn;
+  const int64_t tn = (N + bn * pairs - 1) / (bn * pairs);
   const int64_t tiles = tm * tn * batch;
   if (tiles == 0) return 0.0;
   const int ksub = o.ksub ? o.ksub : (bn == 256 ? 1 : 2);
   const int64_t nkb = (K + kBlockK - 1) / kBlockK;
-  const double mainloop = (double)nkb * 2.0 * bn / shape_efficiency(cta_group, bn);  // clocks per whole tile
+  double mainloop = (double)nkb * 2.0 * bn / shape_efficiency(cta_group, bn);  // clocks per whole tile
+  if (pairs == 2) mainloop /= kShareGain;
   const double drain = 22.0 * bn;             // draining one accumulator (measured 5-7k clocks at N = 256)
   const double per_tile = mainloop > drain ? mainloop : drain;  // small K: the epilogue bounds a tile
   const int64_t full_waves = tiles / max_workers;
@@ -211,26 +222,30 @@ inline double estimate_clocks(int64_t M, int64_t N, int64_t K, int64_t batch, in
 }
 
 inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int sm_count,
-                                int max_pairs /* co-resident 2-CTA clusters */) {
-  static const int cand[5][2] = {{2, 256}, {2, 128}, {1, 256}, {1, 128}, {1, 64}};
-  int best_g = 0, best_n = 0;
+                                int max_pairs /* co-resident 2-CTA clusters */,
+                                int max_quads = 0 /* co-resident 4-CTA clusters; 0: variant not available */) {
+  static const int cand[6][3] = {{2, 256, 2}, {2, 256, 1}, {2, 128, 1}, {1, 256, 1}, {1, 128, 1}, {1, 64, 1}};
+  int best_g = 0, best_n = 0, best_p = 1;
   double best = 0;
-  for (int i = 0; i < 5; ++i) {
-    const int g = cand[i][0], n = cand[i][1];
+  for (int i = 0; i < 6; ++i) {
+    const int g = cand[i][0], n = cand[i][1], pr = cand[i][2];
     if (o.cta_group && o.cta_group != g) continue;
     if (o.tile_n && o.tile_n != n) continue;
     if (g == 2 && max_pairs < 1) continue;
-    const int workers = g == 2 ? max_pairs : sm_count;
+    if (pr == 2 && (max_quads < 1 || o.share < 2)) continue;   // only on request
+    if (pr == 1 && o.share >= 2 && max_quads >= 1) continue;
+    const int workers = pr == 2 ? max_quads : (g == 2 ? max_pairs : sm_count);
     int w_eff = workers;
-    if (o.grid_limit && o.grid_limit / g < w_eff) w_eff = o.grid_limit / g;
+    if (o.grid_limit && o.grid_limit / (g * pr) < w_eff) w_eff = o.grid_limit / (g * pr);
     if (w_eff < 1) w_eff = 1;
-    const double t = estimate_clocks(c.M, c.N, c.K * (c.ab_bytes / 2), c.batch, g, n, w_eff, o);
-    if (best_g == 0 || t < best * 0.999) { best = t; best_g = g; best_n = n; }
+    const double t = estimate_clocks(c.M, c.N, c.K * (c.ab_bytes / 2), c.batch, g, n, w_eff, o, pr);
+    if (best_g == 0 || t < best * 0.999) { best = t; best_g = g; best_n = n; best_p = pr; }
   }
   if (best_g == 0) { best_g = o.cta_group ? o.cta_group : 1; best_n = o.tile_n ? o.tile_n : 128; }
   TileConfig cfg;
   cfg.cta_group = best_g;
   cfg.tile_n = best_n;
+  cfg.pairs = best_p;
   cfg.ksub = o.ksub ? o.ksub : default_ksub(best_g, best_n);
   // Two staging buffers per epilogue warp let a warp fill one while the TMA store still
   // reads the other; they cost 32 KB of ring.  Take them when at least 3 stages remain.
@@ -241,9 +256,9 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
   cfg.stages = max_stages(best_g, best_n, cfg.ksub, cfg.epi_bufs);
   if (o.stages && o.stages < cfg.stages) cfg.stages = o.stages < 2 ? 2 : o.stages;
   cfg.tiles_m = (int)((c.M + 128 * best_g - 1) / (128 * best_g));
-  cfg.tiles_n = (int)((c.N + best_n - 1) / best_n);
-  int64_t workers = best_g == 2 ? max_pairs : sm_count;
-  if (o.grid_limit && o.grid_limit / best_g < workers) workers = o.grid_limit / best_g;
+  cfg.tiles_n = (int)((c.N + best_n * best_p - 1) / (best_n * best_p));
+  int64_t workers = best_p == 2 ? max_quads : (best_g == 2 ? max_pairs : sm_count);
+  if (o.grid_limit && o.grid_limit / (best_g * best_p) < workers) workers = o.grid_limit / (best_g * best_p);
   if (workers < 1) workers = 1;
   const int64_t tiles = (int64_t)cfg.tiles_m * cfg.tiles_n * c.batch;
   // Wave quantisation: the tiles that do not fill a whole wave are cut along K so that the
@@ -277,7 +292,7 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
   cfg.along_m = o.along_m;
   // Tiles that run together should cover a square patch of C: band width G along
   // the banded dimension minimises (W/G)*extent_other + G*extent_banded.
-  const double tile_m = 128.0 * best_g, tile_n = best_n;
+  const double tile_m = 128.0 * best_g, tile_n = (double)best_n * best_p;
   const double ratio = cfg.along_m ? tile_n / tile_m : tile_m / tile_n;
   int band = o.band ? o.band : (int)floor(sqrt((double)workers * ratio) + 0.5);
   const int major = cfg.along_m ? cfg.tiles_m : cfg.tiles_n;
@@ -295,7 +310,7 @@ inline int64_t split_workspace_bytes(const TileConfig& cfg, int c_dtype) {
   const int cw = c_dtype == EXO_GEMM_FP32 ? 32 : 64;        // columns per epilogue chunk
   const int nchunk = cfg.tile_n / cw;
   const int units_per_warp = ((nchunk + 1) / 2) * (cw / 32);
-  return (int64_t)cfg.tail_tiles * (cfg.split - 1) * cfg.cta_group * kEpiWarps * units_per_warp * 4096;
+  return (int64_t)cfg.tail_tiles * (cfg.split - 1) * cfg.cta_group * cfg.pairs * kEpiWarps * units_per_warp * 4096;
 }
 
 inline int smem_bytes_for(int cta_group, int bn, int ksub, int stages, int epi_bufs) {

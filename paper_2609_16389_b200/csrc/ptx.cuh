@@ -37,6 +37,12 @@ __device__ __forceinline__ uint32_t cluster_ctarank() {
   return v;
 }
 
+__device__ __forceinline__ uint32_t cluster_nctarank() {
+  uint32_t v;
+  asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(v));
+  return v;
+}
+
 // Address of `addr` (a shared::cta address of this CTA) in CTA `rank` of the cluster.
 __device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
   uint32_t r;

@@ -14,21 +14,21 @@ def _to_device(buf: np.ndarray, device) -> torch.Tensor:
     return t.to(device, non_blocking=False)
 
 
-def desc_of(p: synth.Problem, flags: int = 0, device: int = -1) -> B.Desc:
+def desc_of(p: synth.Problem, flags: int = 0, device: int = -1, flags2: int = 0) -> B.Desc:
     return B.make_desc(p.M, p.N, p.K, p.ab_dtype, p.c_dtype, p.a_layout, p.b_layout, p.c_layout,
-                       p.lda, p.ldb, p.ldc, device=device, flags=flags)
+                       p.lda, p.ldb, p.ldc, device=device, flags=flags, flags2=flags2)
 
 
 class DeviceProblem:
     """A synth.Problem resident on the GPU, with a plan; ``run`` enqueues one GEMM."""
 
-    def __init__(self, p: synth.Problem, flags: int = 0, device="cuda:0"):
+    def __init__(self, p: synth.Problem, flags: int = 0, device="cuda:0", flags2: int = 0):
         self.p = p
         self.device = torch.device(device)
         self.dA = _to_device(p.A, self.device)
         self.dB = _to_device(p.B, self.device)
         self.dC = _to_device(p.C, self.device)
-        self.plan = B.Plan(desc_of(p, flags, self.device.index or 0))
+        self.plan = B.Plan(desc_of(p, flags, self.device.index or 0, flags2))
 
     def run(self, stream: int | None = None, alpha=None, beta=None):
         s = torch.cuda.current_stream(self.device).cuda_stream if stream is None else stream
@@ -49,9 +49,9 @@ class DeviceProblem:
         self.plan.close()
 
 
-def gemm_host(p: synth.Problem, flags: int = 0, device="cuda:0"):
+def gemm_host(p: synth.Problem, flags: int = 0, device="cuda:0", flags2: int = 0):
     """Host buffers in, host C buffer out: upload, one GEMM, check the plan, download."""
-    dp = DeviceProblem(p, flags, device)
+    dp = DeviceProblem(p, flags, device, flags2)
     try:
         dp.run()
         torch.cuda.synchronize(dp.device)

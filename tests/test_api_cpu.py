@@ -67,7 +67,7 @@ def test_validate_rejects_bad_arguments():
     assert B.exo_gemm_validate(good(ldc=100)) == B.ERR_INVALID_ARG
     assert B.exo_gemm_validate(good(device=-2)) == B.ERR_INVALID_ARG
     d = good()
-    d.reserved = 1
+    d.flags2 = 4
     assert B.exo_gemm_validate(d) == B.ERR_INVALID_ARG
     assert B.exo_gemm_validate(good(flags=3)) == B.ERR_INVALID_ARG                       # cta_group 3
     assert B.exo_gemm_validate(good(flags=B.flag_tile_n(192))) == B.ERR_INVALID_ARG
@@ -253,3 +253,49 @@ def test_batched_create_checks_its_arguments_before_touching_cuda():
     import torch
     if not torch.cuda.is_available():                   # well-formed: only the missing GPU stops it
         assert B.exo_gemm_create_batched(d, 4, 256 * 128, 0, c_extent)[0] in (B.ERR_CUDA, B.ERR_ARCH)
+
+
+def test_shared_operand_cluster_flags_and_preview():
+    ALWAYS, SUBST = B.FLAG2_SHARE_ALWAYS, B.FLAG2_SHARE_SUBSTITUTED
+    assert B.exo_gemm_validate(good(flags2=B.FLAG2_SHARE_NEVER)) == B.OK
+    for f2 in (ALWAYS, SUBST):
+        assert B.exo_gemm_validate(good(flags2=f2)) == B.OK
+        assert B.exo_gemm_validate(good(flags2=f2, flags=B.flag_cta_group(1))) == B.ERR_INVALID_ARG
+        assert B.exo_gemm_validate(good(flags2=f2, flags=B.flag_tile_n(128))) == B.ERR_INVALID_ARG
+        assert B.exo_gemm_validate(good(flags2=f2, flags=B.flag_grid_limit(6))) == B.ERR_INVALID_ARG
+        assert B.exo_gemm_validate(good(flags2=f2, flags=B.flag_grid_limit(8) | B.flag_tile_n(256))) == B.OK
+    assert B.exo_gemm_validate(good(flags2=8)) == B.ERR_INVALID_ARG
+    have = B.exo_gemm_has_shared_operand_clusters()
+    assert have in (0, 1)
+    st, info = B.exo_gemm_plan_preview(good(M=8192, N=8192, K=8192, flags2=ALWAYS), 148)
+    if not have:
+        assert st == B.ERR_UNSUPPORTED
+        return
+    i = info.as_dict()
+    # slots of four CTAs, each covering 256 x 512 of C per step; 148 SMs hold 37 of them
+    assert st == B.OK and (i["cluster_size"], i["cta_group"], i["tile_m"], i["tile_n"]) == (4, 2, 256, 256)
+    assert (i["tiles_m"], i["tiles_n"], i["grid"]) == (32, 16, 148)
+    assert i["tail_tiles"] == 512 % 37 and i["tail_tiles"] * i["split_k"] <= 37
+    # the K-slices' scratch covers both tiles of a slot
+    assert i["workspace_bytes"] == i["tail_tiles"] * (i["split_k"] - 1) * 2 * 256 * 256 * 4
+    st, info = B.exo_gemm_plan_preview(good(M=600, N=700, K=64, flags2=SUBST, flags=B.flag_grid_limit(4)), 148)
+    assert st == B.OK and (info.cluster_size, info.grid, info.tiles_m, info.tiles_n) == (4, 4, 3, 2)
+    # left to itself the library keeps independent pairs, and a plain plan reports its CTA group as the cluster
+    st, info = B.exo_gemm_plan_preview(good(M=8192, N=8192, K=8192), 148)
+    assert st == B.OK and info.cluster_size == info.cta_group == 2
+
+
+def test_base_library_has_no_shared_operand_kernels():
+    import ctypes
+    from paper_2609_16389_b200 import build as cuda_build
+    base = ctypes.CDLL(cuda_build.build())
+    base.exo_gemm_has_shared_operand_clusters.restype = ctypes.c_int32
+    assert base.exo_gemm_has_shared_operand_clusters() == 0
+    base.exo_gemm_plan_preview.argtypes = [ctypes.POINTER(B.Desc), ctypes.c_int32, ctypes.POINTER(B.Info)]
+    info = B.Info()
+    d = good(M=1024, N=1024, K=1024, flags2=B.FLAG2_SHARE_ALWAYS)
+    assert base.exo_gemm_plan_preview(ctypes.byref(d), 148, ctypes.byref(info)) == B.ERR_UNSUPPORTED
+    d = good(M=1024, N=1024, K=1024)
+    assert base.exo_gemm_plan_preview(ctypes.byref(d), 148, ctypes.byref(info)) == B.OK and info.cluster_size == info.cta_group
+    for name in B.EXPORTED_SYMBOLS:
+        getattr(base, name)
