@@ -80,6 +80,17 @@ typedef enum { EXO_GEMM_ROW_MAJOR = 0, EXO_GEMM_COL_MAJOR = 1 } exo_gemm_layout_
 #define EXO_GEMM_FLAG2_SHARE_SUBSTITUTED 3u
 
 /*
+ * flags2, bits 2-3: rows of C per CTA.  0 = the library decides, 1 = 128 (one TMEM accumulator
+ * per tile, the other one belongs to the next tile, so epilogue and main loop overlap),
+ * 2 = 256, the "tall" tile: a CTA pair computes 512 x 256, both accumulators of a CTA belong to
+ * one tile and share each B block, which moves a quarter less operand data into shared memory
+ * per flop at the price of an exposed epilogue.  2 needs the 2-CTA 256-column tile with one
+ * 64-wide k-block per stage: ERR_INVALID_ARG together with CTA_GROUP(1), another TILE_N,
+ * K_SUBBLOCKS(2) or a SHARE_ALWAYS / SHARE_SUBSTITUTED request.  3 is invalid.
+ */
+#define EXO_GEMM_FLAG2_CTA_ROWS(r) ((((uint32_t)(r) / 128u) & 3u) << 2)
+
+/*
  * Problem descriptor.  Logical shapes: A is M x K, B is K x N, C is M x N.
  * Leading dimensions are in elements: for a row-major matrix ld >= #columns, for
  * a column-major matrix ld >= #rows.
@@ -104,7 +115,7 @@ typedef struct {
   int32_t device;                       /* CUDA device ordinal; -1 = the current device        */
   int64_t lda, ldb, ldc;                /* elements                                            */
   uint32_t flags;                       /* 0, or EXO_GEMM_FLAG_* overrides                     */
-  uint32_t flags2;                      /* 0, or EXO_GEMM_FLAG2_*; other bits must be 0        */
+  uint32_t flags2;                      /* 0, or EXO_GEMM_FLAG2_*; bits 4.. must be 0          */
 } exo_gemm_desc_t;
 
 /* What a plan decided; filled by exo_gemm_get_info. */

@@ -33,6 +33,7 @@ def flag_epi_buffers(b): return (b & 3) << 22
 def flag_max_stages(s): return (s & 15) << 24
 def flag_split_k(f): return (f & 15) << 28
 FLAG2_SHARE_AUTO, FLAG2_SHARE_NEVER, FLAG2_SHARE_ALWAYS, FLAG2_SHARE_SUBSTITUTED = 0, 1, 2, 3
+def flag2_cta_rows(r): return ((r // 128) & 3) << 2
 
 
 class Desc(ctypes.Structure):

@@ -52,7 +52,16 @@ template <int KSUB>
 static KernelFn pick_shared(int) { return nullptr; }
 #endif
 
-static KernelFn pick_kernel(int cta_group, int bn, int ksub, int out, int pairs = 1) {
+static KernelFn pick_tall(int out) {
+  switch (out) {
+    case EXO_GEMM_BF16: return exo_gemm_kernel<2, 256, kOutBf16, 1, NoShare, 2>;
+    case EXO_GEMM_FP16: return exo_gemm_kernel<2, 256, kOutFp16, 1, NoShare, 2>;
+    default:            return exo_gemm_kernel<2, 256, kOutFp32, 1, NoShare, 2>;
+  }
+}
+
+static KernelFn pick_kernel(int cta_group, int bn, int ksub, int out, int pairs = 1, int mrep = 1) {
+  if (mrep == 2) return pick_tall(out);
   if (pairs == 2) return ksub == 2 ? pick_shared<2>(out) : pick_shared<1>(out);
   return ksub == 2 ? pick_shape<2>(cta_group, bn, out) : pick_shape<1>(cta_group, bn, out);
 }
@@ -211,7 +220,7 @@ cudaError_t cluster_capacity(int sms, int c_dtype, const FlagOverrides& ov, int*
 void fill_info(const exo_gemm_plan* p, exo_gemm_info_t* info) {
   memset(info, 0, sizeof(*info));
   info->cta_group = p->cfg.cta_group;
-  info->tile_m = 128 * p->cfg.cta_group;
+  info->tile_m = 128 * p->cfg.cta_group * p->cfg.mrep;
   info->tile_n = p->cfg.tile_n;
   info->tile_k = sub_block_k(p->canon.ab_bytes) * p->cfg.ksub;
   info->stages = p->cfg.stages;
@@ -311,7 +320,7 @@ exo_gemm_status_t exo_gemm_plan_preview(const exo_gemm_desc_t* desc, int32_t sm_
   if (ov.share >= 2 && !kHaveSharePairs) return EXO_GEMM_ERR_UNSUPPORTED;
   p.cfg = choose_config(p.canon, ov, sm_count, sm_count / 2, kHaveSharePairs ? sm_count / 4 : 0);
   p.cfg.workspace_bytes = split_workspace_bytes(p.cfg, desc->c_dtype);
-  p.smem_bytes = smem_bytes_for(p.cfg.cta_group, p.cfg.tile_n, p.cfg.ksub, p.cfg.stages, p.cfg.epi_bufs);
+  p.smem_bytes = smem_bytes_for(p.cfg.cta_group, p.cfg.tile_n, p.cfg.ksub, p.cfg.stages, p.cfg.epi_bufs, p.cfg.mrep);
   fill_info(&p, info);
   return EXO_GEMM_OK;
 }
@@ -364,8 +373,8 @@ exo_gemm_status_t exo_gemm_create_batched(exo_gemm_handle_t* out, const exo_gemm
   p->cfg = choose_config(p->canon, ov, sms, max_pairs, max_quads);
   p->cfg.workspace_bytes = split_workspace_bytes(p->cfg, desc->c_dtype);
   p->split_epoch = 0;
-  p->kernel = pick_kernel(p->cfg.cta_group, p->cfg.tile_n, p->cfg.ksub, desc->c_dtype, p->cfg.pairs);
-  p->smem_bytes = smem_bytes_for(p->cfg.cta_group, p->cfg.tile_n, p->cfg.ksub, p->cfg.stages, p->cfg.epi_bufs);
+  p->kernel = pick_kernel(p->cfg.cta_group, p->cfg.tile_n, p->cfg.ksub, desc->c_dtype, p->cfg.pairs, p->cfg.mrep);
+  p->smem_bytes = smem_bytes_for(p->cfg.cta_group, p->cfg.tile_n, p->cfg.ksub, p->cfg.stages, p->cfg.epi_bufs, p->cfg.mrep);
   e = cudaFuncSetAttribute((const void*)p->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, p->smem_bytes);
   if (e != cudaSuccess) { delete p; return cuda_fail(e); }
   e = cudaMalloc((void**)&p->d_status, kStatusBytes);
@@ -442,7 +451,7 @@ exo_gemm_status_t exo_gemm_run(exo_gemm_handle_t plan, const void* A, const void
   prm.alpha = read_ab ? alpha : 0.f;
   prm.beta = beta;
   prm.idesc = make_idesc(d.ab_dtype, cn.a_mn_major, cn.b_mn_major, 128 * cfg.cta_group, cfg.tile_n);
-  prm.a = make_staging(cn.a_mn_major, kBlockM, cfg.ksub, cn.ab_bytes);
+  prm.a = make_staging(cn.a_mn_major, kBlockM * cfg.mrep, cfg.ksub, cn.ab_bytes);
   prm.b = make_staging(cn.b_mn_major, cfg.tile_n / cfg.cta_group, cfg.ksub, cn.ab_bytes);
   prm.sub_k = (uint32_t)sub_k;
   prm.umma_k = (uint32_t)sub_k / 4;
@@ -458,7 +467,7 @@ exo_gemm_status_t exo_gemm_run(exo_gemm_handle_t plan, const void* A, const void
   memset(&tm_b, 0, sizeof tm_b);
   CUresult r;
   const int b_rows = cfg.tile_n / cfg.cta_group;
-  const int a_rows = kBlockM / cfg.pairs;  // pairs that share A fetch half of a CTA's rows each
+  const int a_rows = kBlockM * cfg.mrep / cfg.pairs;  // pairs that share A fetch half of a CTA's rows each
   const uint32_t c_box = d.c_dtype == EXO_GEMM_FP32 ? 32 : 64;
   if (cn.batch <= 1) {
     if (read_ab) {
@@ -516,7 +525,7 @@ exo_gemm_status_t exo_gemm_run(exo_gemm_handle_t plan, const void* A, const void
   }
   if (split_now) {  // arrival counters only grow: this run is complete at epoch * arrivals-per-run
     const uint32_t epoch = plan->split_epoch.fetch_add(1) + 1;
-    prm.split_target = epoch * (uint32_t)((cfg.split - 1) * kEpiWarps * cfg.cta_group);
+    prm.split_target = epoch * (uint32_t)((cfg.split - 1) * kEpiWarps * cfg.cta_group * cfg.mrep);
   }
   cudaError_t e = cudaLaunchKernelEx(&lc, plan->kernel, tm_a, tm_b, tm_c, prm);
   if (e != cudaSuccess) return cuda_fail(e);
@@ -608,8 +617,8 @@ exo_gemm_status_t exo_gemm_run_static(const exo_gemm_desc_t* desc, const void* A
   if (e != cudaSuccess) return cuda_fail(e);
   if (ov.share >= 2 && max_quads < 1) return EXO_GEMM_ERR_UNSUPPORTED;
   plan.cfg = choose_config(plan.canon, ov, sms, max_pairs, max_quads);
-  plan.kernel = pick_kernel(plan.cfg.cta_group, plan.cfg.tile_n, plan.cfg.ksub, desc->c_dtype, plan.cfg.pairs);
-  plan.smem_bytes = smem_bytes_for(plan.cfg.cta_group, plan.cfg.tile_n, plan.cfg.ksub, plan.cfg.stages, plan.cfg.epi_bufs);
+  plan.kernel = pick_kernel(plan.cfg.cta_group, plan.cfg.tile_n, plan.cfg.ksub, desc->c_dtype, plan.cfg.pairs, plan.cfg.mrep);
+  plan.smem_bytes = smem_bytes_for(plan.cfg.cta_group, plan.cfg.tile_n, plan.cfg.ksub, plan.cfg.stages, plan.cfg.epi_bufs, plan.cfg.mrep);
   e = cudaFuncSetAttribute((const void*)plan.kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem_bytes);
   if (e != cudaSuccess) return cuda_fail(e);
 

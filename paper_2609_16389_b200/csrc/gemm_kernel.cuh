@@ -125,14 +125,21 @@ struct NoShare {
   static constexpr int kPairs = 1;
 };
 
-template <int CTA_GROUP, int BN, int OUT, int KSUB, class Share = NoShare>
+// MREP = 128-row blocks of C per CTA.  1: the two TMEM accumulators alternate between consecutive
+// tiles, so a tile's epilogue overlaps the next tile's main loop.  2 (the "tall" tile, 256 x BN per
+// CTA): both accumulators belong to one tile -- A_lo and A_hi are multiplied with the same B block, so
+// a quarter less operand data enters shared memory per flop -- and the epilogue is exposed.
+template <int CTA_GROUP, int BN, int OUT, int KSUB, class Share = NoShare, int MREP = 1>
 __global__ void __launch_bounds__(kNumThreads, 1)
 exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                 const __grid_constant__ CUtensorMap tm_c, const GemmParams p) {
   const int32_t STAGE_K = (int32_t)p.sub_k * KSUB;   // k-elements per stage (64 or 32 per sub-block)
   constexpr int B_ROWS = BN / CTA_GROUP;             // rows of the B tile this CTA stages
-  constexpr int STAGE_BYTES = stage_bytes(CTA_GROUP, BN, KSUB);
-  constexpr int A_BYTES = KSUB * kATileBytes;        // the A part of a stage
+  constexpr int STAGE_BYTES = stage_bytes(CTA_GROUP, BN, KSUB, MREP);
+  constexpr int A_BYTES = KSUB * kATileBytes * MREP; // the A part of a stage
+  constexpr int CTA_M = kBlockM * MREP;              // rows of C per CTA
+  static_assert(MREP == 1 || (MREP == 2 && CTA_GROUP == 2 && BN == 256 && KSUB == 1 && Share::kPairs == 1),
+                "the tall tile exists for 2-CTA 256-column tiles only");
   constexpr uint32_t TMEM_COLS = 2 * BN;             // two accumulators; 128, 256 or 512 columns
   constexpr int CW = (OUT == kOutFp32) ? 32 : 64;    // columns per epilogue chunk = 128 bytes of C
   constexpr int NCHUNK = BN / CW;
@@ -228,7 +235,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       const bool batched = p.batch > 1;
       const uint32_t bz = batched ? (uint32_t)t / p.tiles_per_batch : 0u;  // which matrix of the batch
       const TileCoord tc = raster_decode(p.raster, batched ? (uint32_t)t - bz * p.tiles_per_batch : t);
-      const int32_t a_mn0 = tc.m * (kBlockM * CTA_GROUP) + (int32_t)cta_rank * kBlockM;
+      const int32_t a_mn0 = tc.m * (CTA_M * CTA_GROUP) + (int32_t)cta_rank * CTA_M;
       const int32_t b_mn0 = (tc.n * NPAIR + (int32_t)pair_id) * BN + (int32_t)cta_rank * B_ROWS;
       for (int32_t kb = wi.kb_begin; kb < wi.kb_end; ++kb) {
         ok = wait_barrier<PAIR>(empty_bar(s), ph ^ 1u, p, WaitSite{kRoleProducer, s, (uint32_t)t, (uint32_t)kb});
@@ -280,7 +287,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
               }
             } else if (!p.a.mn_major) {
 #pragma unroll
-              for (int h = 0; h < KSUB; ++h) load(a_dst + h * kATileBytes, &tm_a, k0 + h * (int32_t)p.sub_k, a_mn0);
+              for (int h = 0; h < KSUB; ++h) load(a_dst + h * (kATileBytes * MREP), &tm_a, k0 + h * (int32_t)p.sub_k, a_mn0);
             } else {
               for (uint32_t b = 0; b < p.a.mn_boxes; ++b)
                 load(a_dst + b * p.a.box_bytes, &tm_a, a_mn0 + (int32_t)(p.a.mn_box * b), k0);
@@ -321,16 +328,42 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         return (uint64_t)((uint32_t)(k & 3) * step + (uint32_t)(k >> 2) * sub);
       };
       const uint32_t idesc = p.idesc;
+      // the MMAs of one 128-row block of one stage (elected lane only)
+      auto issue_stage = [&](uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, bool first_kb, int32_t k_left) {
+        if (k_left >= STAGE_K && !tf32) {
+#pragma unroll
+          for (int32_t k = 0; k < kMmaPerStage; ++k)
+            ptx::umma_f16<CTA_GROUP>(d_tmem, a_desc + k_off(k, a_step, a_sub), b_desc + k_off(k, b_step, b_sub),
+                                     idesc, (!first_kb || k != 0) ? 1u : 0u);
+        } else if (k_left >= STAGE_K) {
+#pragma unroll
+          for (int32_t k = 0; k < kMmaPerStage; ++k)
+            ptx::umma_tf32<CTA_GROUP>(d_tmem, a_desc + k_off(k, a_step, a_sub), b_desc + k_off(k, b_step, b_sub),
+                                      idesc, (!first_kb || k != 0) ? 1u : 0u);
+        } else {  // ragged last k-block: skip the MMAs that would only read zero fill
+          const int32_t n_mma = (k_left + umma_k - 1) / umma_k;
+          for (int32_t k = 0; k < n_mma; ++k) {
+            const uint32_t accumulate = (!first_kb || k != 0) ? 1u : 0u;
+            if (tf32)
+              ptx::umma_tf32<CTA_GROUP>(d_tmem, a_desc + k_off(k, a_step, a_sub), b_desc + k_off(k, b_step, b_sub),
+                                        idesc, accumulate);
+            else
+              ptx::umma_f16<CTA_GROUP>(d_tmem, a_desc + k_off(k, a_step, a_sub), b_desc + k_off(k, b_step, b_sub),
+                                       idesc, accumulate);
+          }
+        }
+      };
       for (int64_t it = 0; ok; ++it) {
         WorkItem wi;
         if (!work_item(p.work, worker, num_workers, it, nkb, &wi)) break;
         const int64_t t = wi.tile;
-        // the epilogue (of both CTAs) must have drained this accumulator
-        ok = wait_barrier<PAIR>(tempty_bar(acc), acc_ph ^ 1u, p, WaitSite{kRoleMma, 100 + acc, (uint32_t)t, 0});
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        ptx::tc_fence_after_sync();
-        const uint32_t d_tmem = tmem_base + acc * BN;
+        if constexpr (MREP == 1) {
+          // the epilogue (of both CTAs) must have drained this accumulator
+          ok = wait_barrier<PAIR>(tempty_bar(acc), acc_ph ^ 1u, p, WaitSite{kRoleMma, 100 + acc, (uint32_t)t, 0});
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          ptx::tc_fence_after_sync();
+        }
         for (int32_t kb = wi.kb_begin; kb < wi.kb_end; ++kb) {
           ok = wait_barrier<PAIR>(full_bar(s), ph, p, WaitSite{kRoleMma, s, (uint32_t)t, (uint32_t)kb});
           ok = __all_sync(0xffffffffu, ok);
@@ -340,39 +373,33 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
           const uint64_t a_desc = make_smem_desc(a_addr, p.a);
           const uint64_t b_desc = make_smem_desc(a_addr + A_BYTES, p.b);
           const int32_t k_left = p.K - kb * STAGE_K;
-          if (ptx::elect_one()) {  // the same lane every time: commits track this thread's MMAs
-            EXO_TRACE(1, consumed, 0, 4096);
-            if (k_left >= STAGE_K && !tf32) {
+          const bool first_kb = kb == wi.kb_begin, last_kb = kb == wi.kb_end - 1;
 #pragma unroll
-              for (int32_t k = 0; k < kMmaPerStage; ++k)
-                ptx::umma_f16<CTA_GROUP>(d_tmem, a_desc + k_off(k, a_step, a_sub), b_desc + k_off(k, b_step, b_sub),
-                                         idesc, (kb != wi.kb_begin || k != 0) ? 1u : 0u);
-            } else if (k_left >= STAGE_K) {
-#pragma unroll
-              for (int32_t k = 0; k < kMmaPerStage; ++k)
-                ptx::umma_tf32<CTA_GROUP>(d_tmem, a_desc + k_off(k, a_step, a_sub), b_desc + k_off(k, b_step, b_sub),
-                                          idesc, (kb != wi.kb_begin || k != 0) ? 1u : 0u);
-            } else {  // ragged last k-block: skip the MMAs that would only read zero fill
-              const int32_t n_mma = (k_left + umma_k - 1) / umma_k;
-              for (int32_t k = 0; k < n_mma; ++k) {
-                const uint32_t accumulate = (kb != wi.kb_begin || k != 0) ? 1u : 0u;
-                if (tf32)
-                  ptx::umma_tf32<CTA_GROUP>(d_tmem, a_desc + k_off(k, a_step, a_sub), b_desc + k_off(k, b_step, b_sub),
-                                            idesc, accumulate);
-                else
-                  ptx::umma_f16<CTA_GROUP>(d_tmem, a_desc + k_off(k, a_step, a_sub), b_desc + k_off(k, b_step, b_sub),
-                                           idesc, accumulate);
-              }
+          for (uint32_t r = 0; r < (uint32_t)MREP; ++r) {
+            // tall tile: accumulator r holds rows 128r.. of the CTA's block; the previous tile's epilogue
+            // drains accumulator 0 first, so this tile's first MMAs overlap the draining of accumulator 1
+            const uint32_t a_acc = MREP == 1 ? acc : r;
+            if (MREP == 2 && first_kb) {
+              ok = wait_barrier<PAIR>(tempty_bar(a_acc), acc_ph ^ 1u, p, WaitSite{kRoleMma, 100 + a_acc, (uint32_t)t, 0});
+              ok = __all_sync(0xffffffffu, ok);
+              if (!ok) break;
+              ptx::tc_fence_after_sync();
             }
-            ptx::umma_commit<CTA_GROUP>(empty_bar(s), kStageMask);  // stage free once these MMAs completed
-            if (kb == wi.kb_end - 1) ptx::umma_commit<CTA_GROUP>(tfull_bar(acc), pair_mask);  // accumulator complete
-            EXO_TRACE(1, consumed, 1, 4096);
+            if (ptx::elect_one()) {  // the same lane every time: commits track this thread's MMAs
+              if (r == 0) EXO_TRACE(1, consumed, 0, 4096);
+              // the second 128-row block of A lies 16 KB after the first in every staging layout
+              issue_stage(tmem_base + a_acc * BN, a_desc + (uint64_t)(r * (kATileBytes >> 4)), b_desc, first_kb, k_left);
+              if (r == MREP - 1) ptx::umma_commit<CTA_GROUP>(empty_bar(s), kStageMask);  // stage free once these MMAs completed
+              if (last_kb) ptx::umma_commit<CTA_GROUP>(tfull_bar(a_acc), pair_mask);      // accumulator complete
+              if (r == MREP - 1) EXO_TRACE(1, consumed, 1, 4096);
+            }
           }
+          if (!ok) break;
           ++consumed;
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
         if (!ok) break;
-        if ((acc ^= 1u) == 0u) acc_ph ^= 1u;
+        if (MREP == 2 || (acc ^= 1u) == 0u) acc_ph ^= 1u;
       }
     }
   } else {
@@ -404,8 +431,12 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       const bool batched = p.batch > 1;
       const uint32_t bz = batched ? (uint32_t)t / p.tiles_per_batch : 0u;
       const TileCoord tc = raster_decode(p.raster, batched ? (uint32_t)t - bz * p.tiles_per_batch : t);
-      const int32_t row0 = tc.m * (kBlockM * CTA_GROUP) + (int32_t)cta_rank * kBlockM + (int32_t)quad * 32;
       const int32_t col0 = (tc.n * NPAIR + (int32_t)pair_id) * BN;
+      // one pass per accumulator of the tile: a single one, or (tall tile) rows 0..127 then 128..255 of the CTA
+#pragma unroll 1
+      for (int32_t r = 0; r < MREP; ++r) {
+      const uint32_t cur = MREP == 1 ? acc : (uint32_t)r;
+      const int32_t row0 = tc.m * (CTA_M * CTA_GROUP) + (int32_t)cta_rank * CTA_M + r * kBlockM + (int32_t)quad * 32;
       int32_t nch = 0;  // chunks of this tile that hold any valid column, if this warp's rows exist
       if (row0 < p.M) {
         nch = (p.N - col0 + CW - 1) / CW;
@@ -413,7 +444,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       }
       const int32_t mine = nch > half ? (nch - half + 1) / 2 : 0;  // how many of them are this warp's
       if (has_acc) {
-        ok = wait_barrier<PAIR>(tfull_bar(acc), acc_ph, p, WaitSite{kRoleEpilogue, 200 + acc, (uint32_t)t, 0});
+        ok = wait_barrier<PAIR>(tfull_bar(cur), acc_ph, p, WaitSite{kRoleEpilogue, 200 + cur, (uint32_t)t, 0});
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         ptx::tc_fence_after_sync();
@@ -423,11 +454,11 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         ptx::tc_fence_before_sync();
         __syncwarp();
         if (ptx::elect_one()) {
-          if constexpr (PAIR) ptx::mbar_arrive_cluster(tempty0 + 8u * acc);
-          else ptx::mbar_arrive(tempty0 + 8u * acc);
+          if constexpr (PAIR) ptx::mbar_arrive_cluster(tempty0 + 8u * cur);
+          else ptx::mbar_arrive(tempty0 + 8u * cur);
         }
       };
-      const uint32_t tacc = tmem_base + ((quad * 32u) << 16) + acc * BN;
+      const uint32_t tacc = tmem_base + ((quad * 32u) << 16) + cur * BN;
       // unit q of this warp's i-th chunk: 32 accumulator columns
       auto tmem_load = [&](uint32_t (&dst)[32], int32_t i, int32_t q) {  // asynchronous until tmem_ld_wait()
         ptx::tmem_ld_32x32(tacc + (uint32_t)((half + 2 * i) * CW + q * 32), dst);
@@ -443,8 +474,8 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       const bool owner = wi.slices > 1 && wi.slice == 0;
       auto ws_unit = [&](int32_t slice_m1, int32_t i, int32_t q) {
         const uint64_t idx = ((((uint64_t)wi.tail_index * (uint32_t)(wi.slices - 1) + (uint32_t)slice_m1) * CLUSTER +
-                               slot_rank) * kEpiWarps + ew) * (uint32_t)(((NCHUNK + 1) / 2) * UPC) +
-                             (uint32_t)(i * UPC + q);
+                               slot_rank) * kEpiWarps + ew) * (uint32_t)(MREP * ((NCHUNK + 1) / 2) * UPC) +
+                             (uint32_t)((r * ((NCHUNK + 1) / 2) + i) * UPC + q);
         return reinterpret_cast<char*>(p.split_ws) + idx * kUnitBytes + lane * 16u;
       };
       if (contributor) {
@@ -465,7 +496,6 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         __threadfence();  // each lane's partials are visible GPU-wide before the arrival below
         __syncwarp();
         if (ptx::elect_one()) ptx::red_release_gpu_add(p.split_flags + wi.tail_index * NPAIR + (int32_t)pair_id, 1u);
-        if ((acc ^= 1u) == 0u) acc_ph ^= 1u;
         continue;
       }
       if (owner && mine > 0) {
@@ -620,8 +650,10 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         }
       }
       if (!ok) break;
+      }  // accumulators of the tile
+      if (!ok) break;
       if (warp == 2 && lane == 0) EXO_TRACE(2, it, 1, 4096);
-      if ((acc ^= 1u) == 0u) acc_ph ^= 1u;
+      if (MREP == 2 || (acc ^= 1u) == 0u) acc_ph ^= 1u;
     }
     __syncwarp();
     // The stores must have read their staging buffers before this CTA's shared memory goes away;

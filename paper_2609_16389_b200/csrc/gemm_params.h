@@ -26,14 +26,15 @@ constexpr int kATileBytes = kBlockM * kBlockK * 2;  // 16 KB
 #define EXO_CX constexpr
 #endif
 // A stage holds `ksub` sub-blocks of 64 k-elements (1 or 2): one barrier round trip per stage.
-EXO_CX int stage_bytes(int cta_group, int bn, int ksub) {
-  return ksub * (kATileBytes + (bn / cta_group) * kBlockK * 2);
+// `mrep` = 128-row blocks of A per CTA (1, or 2 for the tall tile whose two accumulators fill TMEM).
+EXO_CX int stage_bytes(int cta_group, int bn, int ksub, int mrep = 1) {
+  return ksub * (mrep * kATileBytes + (bn / cta_group) * kBlockK * 2);
 }
 
 // Stages that fit beside `epi_bufs` staging buffers per epilogue warp.
-EXO_CX int max_stages(int cta_group, int bn, int ksub, int epi_bufs) {
+EXO_CX int max_stages(int cta_group, int bn, int ksub, int epi_bufs, int mrep = 1) {
   const int n = (kSmemLimit - 1024 /*alignment slack*/ - kBarrierBytes - kEpiWarps * epi_bufs * kEpiBufBytes) /
-                stage_bytes(cta_group, bn, ksub);
+                stage_bytes(cta_group, bn, ksub, mrep);
   return n > kMaxStages ? kMaxStages : n;
 }
 

@@ -24,6 +24,7 @@ struct FlagOverrides {
   int grid_limit;  // 0 = none
   int share;       // clusters of two CTA pairs sharing the loads of A: 0 = auto, 1 = never, 2 = always,
                    // 3 = always, but every slot launched as two plain pairs (exercises the substitute path)
+  int mrep;        // 128-row blocks of C per CTA: 0 = auto, 1, or 2 (the tall 2-CTA tile, 512 x 256 per pair)
 };
 
 inline FlagOverrides decode_flags(uint32_t f, uint32_t f2 = 0) {
@@ -39,12 +40,13 @@ inline FlagOverrides decode_flags(uint32_t f, uint32_t f2 = 0) {
   o.split = (int)((f >> 28) & 15u);
   o.no_workspace = false;
   o.share = (int)(f2 & 3u);
+  o.mrep = (int)((f2 >> 2) & 3u);
   return o;
 }
 
 inline exo_gemm_status_t validate_desc(const exo_gemm_desc_t* d) {
   if (!d) return EXO_GEMM_ERR_NULL;
-  if ((d->flags2 & ~3u) != 0) return EXO_GEMM_ERR_INVALID_ARG;
+  if ((d->flags2 & ~15u) != 0 || ((d->flags2 >> 2) & 3u) == 3u) return EXO_GEMM_ERR_INVALID_ARG;
   const int64_t kMaxDim = 2147483647LL;
   if (d->M < 0 || d->N < 0 || d->K < 0 || d->M > kMaxDim || d->N > kMaxDim || d->K > kMaxDim)
     return EXO_GEMM_ERR_INVALID_ARG;
@@ -73,6 +75,9 @@ inline exo_gemm_status_t validate_desc(const exo_gemm_desc_t* d) {
   if (o.grid_limit != 0 && o.cta_group == 2 && (o.grid_limit & 1)) return EXO_GEMM_ERR_INVALID_ARG;
   // forcing the shared-operand clusters fixes the tile shape they are built for
   if (o.share >= 2 && (o.cta_group == 1 || (o.tile_n != 0 && o.tile_n != 256) || (o.grid_limit & 3)))
+    return EXO_GEMM_ERR_INVALID_ARG;
+  // so does forcing the tall tile, which has no shared-operand form
+  if (o.mrep == 2 && (o.cta_group == 1 || (o.tile_n != 0 && o.tile_n != 256) || o.ksub == 2 || o.share >= 2))
     return EXO_GEMM_ERR_INVALID_ARG;
   // beyond here the call is a legal BLAS call; what follows is this library's supported set
   // fp32 operands are multiplied as tf32 (the precision of the paper's own kernels) into an fp32 C
@@ -156,6 +161,7 @@ struct TileConfig {
   int64_t workspace_bytes; // fp32 partials of slices 1.. of the tail tiles
   int cta_group, tile_n, ksub, stages, epi_bufs;
   int pairs;               // CTA pairs per cluster (2: the pairs share the loads of A; else 1)
+  int mrep;                // 128-row blocks of C per CTA (2: the tall tile; else 1)
   int tiles_m, tiles_n;    // tiles of (128 * cta_group) x (tile_n * pairs): what one cluster computes at a time
   int band, along_m;
   int workers;  // CTA groups launched
@@ -177,6 +183,10 @@ inline double shape_efficiency(int cta_group, int bn) {
 
 // Main-loop speed of the shared-operand clusters relative to independent pairs.
 constexpr double kShareGain = 1.0;
+// Main-loop speed of the tall tile (256 rows per CTA) relative to the 128-row tile, and the clocks
+// per tile its exposed epilogue costs.
+constexpr double kTallGain = 1.10;
+constexpr double kTallDrain = 4000.0;
 
 // k-elements in one 128-byte sub-block row: 64 for 16-bit operands, 32 for fp32 storage.
 inline int sub_block_k(int ab_bytes) { return 128 / ab_bytes; }
@@ -199,8 +209,8 @@ inline int split_factor(int64_t tiles, int64_t workers, int64_t K, int ksub, con
 // Estimated time of the whole problem in SM clocks for one candidate tile shape: whole waves of
 // tiles, then the partial last wave (cut along K if that pays), plus what is exposed once per launch.
 inline double estimate_clocks(int64_t M, int64_t N, int64_t K, int64_t batch, int cta_group, int bn,
-                              int max_workers, const FlagOverrides& o, int pairs = 1) {
-  const int64_t tm = (M + 128 * cta_group - 1) / (128 * cta_group);
+                              int max_workers, const FlagOverrides& o, int pairs = 1, int mrep = 1) {
+  const int64_t tm = (M + 128 * cta_group * mrep - 1) / (128 * cta_group * mrep);
   const int64_t tn = (N + bn * pairs - 1) / (bn * pairs);
   const int64_t tiles = tm * tn * batch;
   if (tiles == 0) return 0.0;
@@ -209,13 +219,17 @@ inline double estimate_clocks(int64_t M, int64_t N, int64_t K, int64_t batch, in
   double mainloop = (double)nkb * 2.0 * bn / shape_efficiency(cta_group, bn);  // clocks per whole tile
   if (pairs == 2) mainloop /= kShareGain;
   const double drain = 22.0 * bn;             // draining one accumulator (measured 5-7k clocks at N = 256)
-  const double per_tile = mainloop > drain ? mainloop : drain;  // small K: the epilogue bounds a tile
+  double per_tile = mainloop > drain ? mainloop : drain;  // small K: the epilogue bounds a tile
+  if (mrep == 2) {  // two accumulators per tile, less operand traffic, but the epilogue is not hidden
+    mainloop = 2.0 * mainloop / kTallGain;
+    per_tile = mainloop + kTallDrain;
+  }
   const int64_t full_waves = tiles / max_workers;
   const int64_t tail = tiles % max_workers;
   double t = (double)full_waves * per_tile;
   if (tail > 0) {
     const int f = split_factor(tiles, max_workers, K, ksub, o);
-    if (f > 1) t += mainloop / f + (30.0 + 8.0 * (f - 1)) * bn;  // slice + exchange of partial sums
+    if (f > 1) t += mainloop / f + (30.0 + 8.0 * (f - 1)) * bn * mrep;  // slice + exchange of partial sums
     else t += per_tile;
   }
   return t + drain + 3000.0;  // the last epilogue and the pipeline fill are exposed once
@@ -224,11 +238,14 @@ inline double estimate_clocks(int64_t M, int64_t N, int64_t K, int64_t batch, in
 inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int sm_count,
                                 int max_pairs /* co-resident 2-CTA clusters */,
                                 int max_quads = 0 /* co-resident 4-CTA clusters; 0: variant not available */) {
-  static const int cand[6][3] = {{2, 256, 2}, {2, 256, 1}, {2, 128, 1}, {1, 256, 1}, {1, 128, 1}, {1, 64, 1}};
-  int best_g = 0, best_n = 0, best_p = 1;
+  static const int cand[7][4] = {{2, 256, 2, 1}, {2, 256, 1, 2}, {2, 256, 1, 1}, {2, 128, 1, 1},
+                                 {1, 256, 1, 1}, {1, 128, 1, 1}, {1, 64, 1, 1}};
+  int best_g = 0, best_n = 0, best_p = 1, best_r = 1;
   double best = 0;
-  for (int i = 0; i < 6; ++i) {
-    const int g = cand[i][0], n = cand[i][1], pr = cand[i][2];
+  for (int i = 0; i < 7; ++i) {
+    const int g = cand[i][0], n = cand[i][1], pr = cand[i][2], mr = cand[i][3];
+    if (mr == 2 && (o.mrep == 1 || o.share >= 2 || o.ksub == 2)) continue;
+    if (mr == 1 && o.mrep == 2 && max_pairs >= 1) continue;
     if (o.cta_group && o.cta_group != g) continue;
     if (o.tile_n && o.tile_n != n) continue;
     if (g == 2 && max_pairs < 1) continue;
@@ -238,24 +255,26 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
     int w_eff = workers;
     if (o.grid_limit && o.grid_limit / (g * pr) < w_eff) w_eff = o.grid_limit / (g * pr);
     if (w_eff < 1) w_eff = 1;
-    const double t = estimate_clocks(c.M, c.N, c.K * (c.ab_bytes / 2), c.batch, g, n, w_eff, o, pr);
-    if (best_g == 0 || t < best * 0.999) { best = t; best_g = g; best_n = n; best_p = pr; }
+    double t = estimate_clocks(c.M, c.N, c.K * (c.ab_bytes / 2), c.batch, g, n, w_eff, o, pr, mr);
+    if (mr == 2) t *= 1.03;  // the tall tile's exposed epilogue makes it the riskier choice: it must win clearly
+    if (best_g == 0 || t < best * 0.999) { best = t; best_g = g; best_n = n; best_p = pr; best_r = mr; }
   }
   if (best_g == 0) { best_g = o.cta_group ? o.cta_group : 1; best_n = o.tile_n ? o.tile_n : 128; }
   TileConfig cfg;
   cfg.cta_group = best_g;
   cfg.tile_n = best_n;
   cfg.pairs = best_p;
-  cfg.ksub = o.ksub ? o.ksub : default_ksub(best_g, best_n);
+  cfg.mrep = best_r;
+  cfg.ksub = best_r == 2 ? 1 : (o.ksub ? o.ksub : default_ksub(best_g, best_n));
   // Two staging buffers per epilogue warp let a warp fill one while the TMA store still
   // reads the other; they cost 32 KB of ring.  Take them when at least 3 stages remain.
   // Short K: the epilogue bounds a tile, so staging depth matters more than ring depth.
-  const bool want_two = max_stages(best_g, best_n, cfg.ksub, 2) >= 5 ||
-                        (c.K * (c.ab_bytes / 2) <= 1024 && max_stages(best_g, best_n, cfg.ksub, 2) >= 3);
+  const bool want_two = max_stages(best_g, best_n, cfg.ksub, 2, best_r) >= 5 ||
+                        (c.K * (c.ab_bytes / 2) <= 1024 && max_stages(best_g, best_n, cfg.ksub, 2, best_r) >= 3);
   cfg.epi_bufs = o.epi_bufs ? o.epi_bufs : (want_two ? 2 : 1);
-  cfg.stages = max_stages(best_g, best_n, cfg.ksub, cfg.epi_bufs);
+  cfg.stages = max_stages(best_g, best_n, cfg.ksub, cfg.epi_bufs, best_r);
   if (o.stages && o.stages < cfg.stages) cfg.stages = o.stages < 2 ? 2 : o.stages;
-  cfg.tiles_m = (int)((c.M + 128 * best_g - 1) / (128 * best_g));
+  cfg.tiles_m = (int)((c.M + 128 * best_g * best_r - 1) / (128 * best_g * best_r));
   cfg.tiles_n = (int)((c.N + best_n * best_p - 1) / (best_n * best_p));
   int64_t workers = best_p == 2 ? max_quads : (best_g == 2 ? max_pairs : sm_count);
   if (o.grid_limit && o.grid_limit / (best_g * best_p) < workers) workers = o.grid_limit / (best_g * best_p);
@@ -292,7 +311,7 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
   cfg.along_m = o.along_m;
   // Tiles that run together should cover a square patch of C: band width G along
   // the banded dimension minimises (W/G)*extent_other + G*extent_banded.
-  const double tile_m = 128.0 * best_g, tile_n = (double)best_n * best_p;
+  const double tile_m = 128.0 * best_g * best_r, tile_n = (double)best_n * best_p;
   const double ratio = cfg.along_m ? tile_n / tile_m : tile_m / tile_n;
   int band = o.band ? o.band : (int)floor(sqrt((double)workers * ratio) + 0.5);
   const int major = cfg.along_m ? cfg.tiles_m : cfg.tiles_n;
@@ -310,11 +329,11 @@ inline int64_t split_workspace_bytes(const TileConfig& cfg, int c_dtype) {
   const int cw = c_dtype == EXO_GEMM_FP32 ? 32 : 64;        // columns per epilogue chunk
   const int nchunk = cfg.tile_n / cw;
   const int units_per_warp = ((nchunk + 1) / 2) * (cw / 32);
-  return (int64_t)cfg.tail_tiles * (cfg.split - 1) * cfg.cta_group * cfg.pairs * kEpiWarps * units_per_warp * 4096;
+  return (int64_t)cfg.tail_tiles * (cfg.split - 1) * cfg.cta_group * cfg.pairs * cfg.mrep * kEpiWarps * units_per_warp * 4096;
 }
 
-inline int smem_bytes_for(int cta_group, int bn, int ksub, int stages, int epi_bufs) {
-  return 1024 + stages * stage_bytes(cta_group, bn, ksub) + kEpiWarps * epi_bufs * kEpiBufBytes + kBarrierBytes;
+inline int smem_bytes_for(int cta_group, int bn, int ksub, int stages, int epi_bufs, int mrep = 1) {
+  return 1024 + stages * stage_bytes(cta_group, bn, ksub, mrep) + kEpiWarps * epi_bufs * kEpiBufBytes + kBarrierBytes;
 }
 
 // tcgen05 instruction descriptor for kind::f16 with fp32 accumulation.

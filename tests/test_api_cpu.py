@@ -67,7 +67,7 @@ def test_validate_rejects_bad_arguments():
     assert B.exo_gemm_validate(good(ldc=100)) == B.ERR_INVALID_ARG
     assert B.exo_gemm_validate(good(device=-2)) == B.ERR_INVALID_ARG
     d = good()
-    d.flags2 = 4
+    d.flags2 = 12
     assert B.exo_gemm_validate(d) == B.ERR_INVALID_ARG
     assert B.exo_gemm_validate(good(flags=3)) == B.ERR_INVALID_ARG                       # cta_group 3
     assert B.exo_gemm_validate(good(flags=B.flag_tile_n(192))) == B.ERR_INVALID_ARG
@@ -264,7 +264,7 @@ def test_shared_operand_cluster_flags_and_preview():
         assert B.exo_gemm_validate(good(flags2=f2, flags=B.flag_tile_n(128))) == B.ERR_INVALID_ARG
         assert B.exo_gemm_validate(good(flags2=f2, flags=B.flag_grid_limit(6))) == B.ERR_INVALID_ARG
         assert B.exo_gemm_validate(good(flags2=f2, flags=B.flag_grid_limit(8) | B.flag_tile_n(256))) == B.OK
-    assert B.exo_gemm_validate(good(flags2=8)) == B.ERR_INVALID_ARG
+    assert B.exo_gemm_validate(good(flags2=16)) == B.ERR_INVALID_ARG
     have = B.exo_gemm_has_shared_operand_clusters()
     assert have in (0, 1)
     st, info = B.exo_gemm_plan_preview(good(M=8192, N=8192, K=8192, flags2=ALWAYS), 148)
@@ -299,3 +299,31 @@ def test_base_library_has_no_shared_operand_kernels():
     assert base.exo_gemm_plan_preview(ctypes.byref(d), 148, ctypes.byref(info)) == B.OK and info.cluster_size == info.cta_group
     for name in B.EXPORTED_SYMBOLS:
         getattr(base, name)
+
+
+def test_tall_tile_flags_and_preview():
+    TALL, REG = B.flag2_cta_rows(256), B.flag2_cta_rows(128)
+    assert (TALL, REG) == (8, 4)
+    assert B.exo_gemm_validate(good(flags2=TALL)) == B.OK and B.exo_gemm_validate(good(flags2=REG)) == B.OK
+    assert B.exo_gemm_validate(good(flags2=12)) == B.ERR_INVALID_ARG                      # rows field 3
+    assert B.exo_gemm_validate(good(flags2=TALL, flags=B.flag_cta_group(1))) == B.ERR_INVALID_ARG
+    assert B.exo_gemm_validate(good(flags2=TALL, flags=B.flag_tile_n(128))) == B.ERR_INVALID_ARG
+    assert B.exo_gemm_validate(good(flags2=TALL, flags=B.flag_k_subblocks(2))) == B.ERR_INVALID_ARG
+    assert B.exo_gemm_validate(good(flags2=TALL | B.FLAG2_SHARE_ALWAYS)) == B.ERR_INVALID_ARG
+    assert B.exo_gemm_validate(good(flags2=TALL | B.FLAG2_SHARE_NEVER)) == B.OK
+    st, info = B.exo_gemm_plan_preview(good(M=1000, N=520, K=264, flags2=TALL), 148)
+    i = info.as_dict()
+    assert st == B.OK and (i["cta_group"], i["tile_m"], i["tile_n"], i["tile_k"]) == (2, 512, 256, 64)
+    assert (i["tiles_m"], i["tiles_n"], i["grid"], i["tmem_columns"]) == (2, 3, 12, 512)
+    # a stage holds 256 rows of A and this CTA's 128 rows of B
+    assert i["stages"] * 49152 + 32768 * i["epilogue_buffers"] + 1536 == i["smem_bytes"] <= 232448
+    # large cubes take the tall tile on their own, 4096^3 (two uneven waves of 512 x 256 tiles) does not
+    st, info = B.exo_gemm_plan_preview(good(M=8192, N=8192, K=8192, c_dtype=B.BF16), 148)
+    assert info.tile_m == 512 and info.stages == 4 and info.split_k == 1
+    st, info = B.exo_gemm_plan_preview(good(M=4096, N=4096, K=4096, c_dtype=B.BF16), 148)
+    assert info.tile_m == 256
+    st, info = B.exo_gemm_plan_preview(good(M=8192, N=8192, K=8192, flags2=REG), 148)
+    assert info.tile_m == 256
+    # the K-slices' scratch covers both accumulators of both CTAs
+    st, info = B.exo_gemm_plan_preview(good(M=2560, N=3840, K=2048, flags2=TALL), 148)
+    assert (info.tail_tiles, info.split_k, info.workspace_bytes) == (1, 8, 7 * 512 * 256 * 4)
