@@ -37,7 +37,7 @@ def is_stale(lib: str = LIB, deps=DEPS) -> bool:
 def _compile(lib: str, defines, verbose: bool) -> str:
     tmp = lib + f".tmp{os.getpid()}"
     cmd = [nvcc_path(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-           "-shared", "-Xcompiler", "-fPIC", "-cudart", "static", "-o", tmp]
+           "-shared", "-Xcompiler", "-fPIC", "-Xcompiler", "-fno-gnu-unique", "-cudart", "static", "-o", tmp]
     cmd += [f"-D{d}" for d in defines]
     if verbose:
         cmd += ["-Xptxas", "-v"]

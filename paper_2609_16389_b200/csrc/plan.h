@@ -209,7 +209,8 @@ inline int split_factor(int64_t tiles, int64_t workers, int64_t K, int ksub, con
 // Estimated time of the whole problem in SM clocks for one candidate tile shape: whole waves of
 // tiles, then the partial last wave (cut along K if that pays), plus what is exposed once per launch.
 inline double estimate_clocks(int64_t M, int64_t N, int64_t K, int64_t batch, int cta_group, int bn,
-                              int max_workers, const FlagOverrides& o, int pairs = 1, int mrep = 1) {
+                              int max_workers, const FlagOverrides& o, int pairs = 1, int mrep = 1,
+                              bool mn_major_operand = false) {
   const int64_t tm = (M + 128 * cta_group * mrep - 1) / (128 * cta_group * mrep);
   const int64_t tn = (N + bn * pairs - 1) / (bn * pairs);
   const int64_t tiles = tm * tn * batch;
@@ -218,6 +219,10 @@ inline double estimate_clocks(int64_t M, int64_t N, int64_t K, int64_t batch, in
   const int64_t nkb = (K + kBlockK - 1) / kBlockK;
   double mainloop = (double)nkb * 2.0 * bn / shape_efficiency(cta_group, bn);  // clocks per whole tile
   if (pairs == 2) mainloop /= kShareGain;
+  // An M/N-contiguous operand costs the 128-row 2-CTA tile about 15 % of its main-loop rate (measured at
+  // 8192^3: 1175-1260 TFLOP/s against 1340-1500 with both operands K-contiguous); the tall tile, which has
+  // shared-memory bandwidth to spare, is unaffected (1430-1573).
+  if (mn_major_operand && cta_group == 2 && mrep == 1) mainloop /= 0.87;
   const double drain = 22.0 * bn;             // draining one accumulator (measured 5-7k clocks at N = 256)
   double per_tile = mainloop > drain ? mainloop : drain;  // small K: the epilogue bounds a tile
   if (mrep == 2) {  // two accumulators per tile, less operand traffic, but the epilogue is not hidden
@@ -238,7 +243,8 @@ inline double estimate_clocks(int64_t M, int64_t N, int64_t K, int64_t batch, in
 inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int sm_count,
                                 int max_pairs /* co-resident 2-CTA clusters */,
                                 int max_quads = 0 /* co-resident 4-CTA clusters; 0: variant not available */) {
-  static const int cand[7][4] = {{2, 256, 2, 1}, {2, 256, 1, 2}, {2, 256, 1, 1}, {2, 128, 1, 1},
+  // (a plain local: a static here would be one process-wide object shared by every loaded build of the library)
+  const int cand[7][4] = {{2, 256, 2, 1}, {2, 256, 1, 2}, {2, 256, 1, 1}, {2, 128, 1, 1},
                                  {1, 256, 1, 1}, {1, 128, 1, 1}, {1, 64, 1, 1}};
   int best_g = 0, best_n = 0, best_p = 1, best_r = 1;
   double best = 0;
@@ -255,7 +261,8 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
     int w_eff = workers;
     if (o.grid_limit && o.grid_limit / (g * pr) < w_eff) w_eff = o.grid_limit / (g * pr);
     if (w_eff < 1) w_eff = 1;
-    double t = estimate_clocks(c.M, c.N, c.K * (c.ab_bytes / 2), c.batch, g, n, w_eff, o, pr, mr);
+    double t = estimate_clocks(c.M, c.N, c.K * (c.ab_bytes / 2), c.batch, g, n, w_eff, o, pr, mr,
+                               c.a_mn_major || c.b_mn_major);
     if (mr == 2) t *= 1.03;  // the tall tile's exposed epilogue makes it the riskier choice: it must win clearly
     if (best_g == 0 || t < best * 0.999) { best = t; best_g = g; best_n = n; best_p = pr; best_r = mr; }
   }
