@@ -53,6 +53,8 @@ def parse_args():
     ap.add_argument("--flags", type=int, default=0, help="EXO_GEMM_FLAG_* overrides (experiments)")
     ap.add_argument("--share", default="auto", choices=["auto", "never", "always"],
                     help="shared-operand 4-CTA clusters (needs the variant library; single-GPU runs only)")
+    ap.add_argument("--cta-rows", default="auto", choices=["auto", "128", "256"],
+                    help="rows of C per CTA of the 2-CTA tile (256 = the tall tile)")
     return ap.parse_args()
 
 
@@ -229,6 +231,8 @@ def run_ours(args, rank, world, local_rank):
         sets.append((harness._to_device(p.A, dev), harness._to_device(p.B, dev), harness._to_device(p.C, dev)))
     batch = getattr(p, "batch", 1)
     flags2 = {"auto": B.FLAG2_SHARE_AUTO, "never": B.FLAG2_SHARE_NEVER, "always": B.FLAG2_SHARE_ALWAYS}[args.share]
+    if args.cta_rows != "auto":
+        flags2 |= B.flag2_cta_rows(int(args.cta_rows))
     plan = B.Plan(harness.desc_of(p, args.flags, local_rank, flags2),
                   batch=(batch, p.stride_a, p.stride_b, p.stride_c) if batch > 1 else None)
     info = plan.info()

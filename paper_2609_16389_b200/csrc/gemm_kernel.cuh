@@ -4,8 +4,8 @@
 // 2-CTA cluster) computes output tiles of (128 * CTA_GROUP) x BN, one after
 // another, taken round-robin from a band-swizzled raster.  Roles per CTA:
 //
-//   warp 0, one lane   producer: TMA loads of the A and B k-blocks into a ring
-//                      of shared-memory stages (full/empty mbarriers)
+//   warps 0 and 10,    producers: TMA loads of the A (warp 0) and B (warp 10) k-blocks
+//   one lane each      into a ring of shared-memory stages (full/empty mbarriers)
 //   warp 1, one lane   MMA issuer (leader CTA only): tcgen05.mma from shared
 //                      memory into one of two TMEM accumulators; tcgen05.commit
 //                      releases stages and publishes finished accumulators
@@ -221,8 +221,11 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   bool ok = true;
   if (threadIdx.x == 0) EXO_TRACE(2, 4094, 0, 4096);
 
-  if (warp == 0) {
+  if (warp == 0 || warp == (uint32_t)kProducerBWarp) {
     // ============================================================ producer
+    // Issuing a stage's copies from one lane takes a few hundred clocks, which is what a stage's MMAs
+    // take too: two warps share the work (A and the byte count from warp 0, B from the other warp).
+    const bool do_a = warp == 0, do_b = warp == (uint32_t)kProducerBWarp;
     // The whole warp runs the loop (uniform control flow); one elected lane issues.
     uint32_t s = 0, ph = 0;
     int64_t issued = 0;
@@ -244,60 +247,71 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         const bool skip = (p.debug_skip_k_block == issued) && blockIdx.x == 0;
         if (ptx::elect_one()) {
           EXO_TRACE(0, issued, 0, 4096);
-          if (cta_rank == 0) ptx::mbar_arrive_expect_tx(full_bar(s), STAGE_BYTES * CTA_GROUP);
+          if (cta_rank == 0 && do_a) ptx::mbar_arrive_expect_tx(full_bar(s), STAGE_BYTES * CTA_GROUP);
           if (!skip) {
             const uint32_t a_dst = stage0 + s * STAGE_BYTES;
             const uint32_t b_dst = a_dst + A_BYTES;
             const uint32_t bar = full0 + 8u * s;
             const int32_t k0 = kb * STAGE_K;
-            auto load = [&](uint32_t dst, const CUtensorMap* map, int32_t x, int32_t y) {
-              if (batched) {
+            // This loop runs once per stage in a single lane and can bound the whole pipeline when a stage's
+            // MMAs are short: box counts and offsets are compile-time constants and the batched / plain
+            // distinction is taken once per stage, not once per copy.
+            constexpr int A_BOXES = CTA_M / 64, B_BOXES = B_ROWS / 64;   // M/N-contiguous 16-bit operands: 64 per box
+            constexpr uint32_t MN_BOX_BYTES = KSUB * 8192u;             // one box: 64 * KSUB k-rows of 128 bytes
+            auto stage_loads = [&](auto&& load) {
+              if (!do_a) {
+              } else if (quad) {
+                if constexpr (SHARE) {
+                  // The other pair's CTA of the same rank needs the same 128 rows of A: each of the two
+                  // fetches 64 of them and the copy lands in both CTAs' stages; each copy's bytes count
+                  // on the full barrier of the receiving CTA's own pair leader.
+                  const uint16_t both = (uint16_t)((1u << cta_rank) | (1u << (cta_rank + 2u)));
+                  auto load_shared = [&](uint32_t dst, int32_t x, int32_t y) {
+                    if (batched) Share::load_3d(dst, &tm_a, x, y, (int32_t)(bz & p.a_z_mask), bar, both);
+                    else Share::load_2d(dst, &tm_a, x, y, bar, both);
+                  };
+                  if (!p.a.mn_major) {
+#pragma unroll
+                    for (int h = 0; h < KSUB; ++h)
+                      load_shared(a_dst + h * kATileBytes + pair_id * (kATileBytes / 2), k0 + h * (int32_t)p.sub_k,
+                                  a_mn0 + (int32_t)pair_id * (kBlockM / 2));
+                  } else {  // two boxes of 64 rows: one each
+                    load_shared(a_dst + pair_id * MN_BOX_BYTES, a_mn0 + 64 * (int32_t)pair_id, k0);
+                  }
+                }
+              } else if (SHARE && !p.a.mn_major) {  // substituted pair: both 64-row halves, same tensor map
+#pragma unroll
+                for (int h = 0; h < KSUB; ++h) {
+                  load(a_dst + h * kATileBytes, &tm_a, k0 + h * (int32_t)p.sub_k, a_mn0);
+                  load(a_dst + h * kATileBytes + kATileBytes / 2, &tm_a, k0 + h * (int32_t)p.sub_k, a_mn0 + kBlockM / 2);
+                }
+              } else if (!p.a.mn_major) {
+#pragma unroll
+                for (int h = 0; h < KSUB; ++h) load(a_dst + h * (kATileBytes * MREP), &tm_a, k0 + h * (int32_t)p.sub_k, a_mn0);
+              } else {
+#pragma unroll
+                for (int b = 0; b < A_BOXES; ++b) load(a_dst + b * MN_BOX_BYTES, &tm_a, a_mn0 + 64 * b, k0);
+              }
+              if (!do_b) {
+              } else if (!p.b.mn_major) {
+#pragma unroll
+                for (int h = 0; h < KSUB; ++h) load(b_dst + h * (B_ROWS * 128), &tm_b, k0 + h * (int32_t)p.sub_k, b_mn0);
+              } else {
+#pragma unroll
+                for (int b = 0; b < B_BOXES; ++b) load(b_dst + b * MN_BOX_BYTES, &tm_b, b_mn0 + 64 * b, k0);
+              }
+            };
+            if (!batched) {
+              stage_loads([&](uint32_t dst, const CUtensorMap* map, int32_t x, int32_t y) {
+                if constexpr (PAIR) ptx::tma_load_2d_pair(dst, map, x, y, bar);
+                else ptx::tma_load_2d(dst, map, x, y, bar);
+              });
+            } else {
+              stage_loads([&](uint32_t dst, const CUtensorMap* map, int32_t x, int32_t y) {
                 const int32_t z = (int32_t)(bz & (map == &tm_a ? p.a_z_mask : p.b_z_mask));
                 if constexpr (PAIR) ptx::tma_load_3d_pair(dst, map, x, y, z, bar);
                 else ptx::tma_load_3d(dst, map, x, y, z, bar);
-              } else {
-                if constexpr (PAIR) ptx::tma_load_2d_pair(dst, map, x, y, bar);
-                else ptx::tma_load_2d(dst, map, x, y, bar);
-              }
-            };
-            if (quad) {
-              if constexpr (SHARE) {
-                // The other pair's CTA of the same rank needs the same 128 rows of A: each of the two
-                // fetches 64 of them and the copy lands in both CTAs' stages; each copy's bytes count
-                // on the full barrier of the receiving CTA's own pair leader.
-                const uint16_t both = (uint16_t)((1u << cta_rank) | (1u << (cta_rank + 2u)));
-                auto load_shared = [&](uint32_t dst, int32_t x, int32_t y) {
-                  if (batched) Share::load_3d(dst, &tm_a, x, y, (int32_t)(bz & p.a_z_mask), bar, both);
-                  else Share::load_2d(dst, &tm_a, x, y, bar, both);
-                };
-                if (!p.a.mn_major) {
-#pragma unroll
-                  for (int h = 0; h < KSUB; ++h)
-                    load_shared(a_dst + h * kATileBytes + pair_id * (kATileBytes / 2), k0 + h * (int32_t)p.sub_k,
-                                a_mn0 + (int32_t)pair_id * (kBlockM / 2));
-                } else {  // two boxes of 64 rows: one each
-                  load_shared(a_dst + pair_id * p.a.box_bytes, a_mn0 + (int32_t)(p.a.mn_box * pair_id), k0);
-                }
-              }
-            } else if (SHARE && !p.a.mn_major) {  // substituted pair: both 64-row halves, same tensor map
-#pragma unroll
-              for (int h = 0; h < KSUB; ++h) {
-                load(a_dst + h * kATileBytes, &tm_a, k0 + h * (int32_t)p.sub_k, a_mn0);
-                load(a_dst + h * kATileBytes + kATileBytes / 2, &tm_a, k0 + h * (int32_t)p.sub_k, a_mn0 + kBlockM / 2);
-              }
-            } else if (!p.a.mn_major) {
-#pragma unroll
-              for (int h = 0; h < KSUB; ++h) load(a_dst + h * (kATileBytes * MREP), &tm_a, k0 + h * (int32_t)p.sub_k, a_mn0);
-            } else {
-              for (uint32_t b = 0; b < p.a.mn_boxes; ++b)
-                load(a_dst + b * p.a.box_bytes, &tm_a, a_mn0 + (int32_t)(p.a.mn_box * b), k0);
-            }
-            if (!p.b.mn_major) {
-#pragma unroll
-              for (int h = 0; h < KSUB; ++h) load(b_dst + h * (B_ROWS * 128), &tm_b, k0 + h * (int32_t)p.sub_k, b_mn0);
-            } else {
-              for (uint32_t b = 0; b < p.b.mn_boxes; ++b)
-                load(b_dst + b * p.b.box_bytes, &tm_b, b_mn0 + (int32_t)(p.b.mn_box * b), k0);
+              });
             }
           }
           EXO_TRACE(0, issued, 1, 4096);

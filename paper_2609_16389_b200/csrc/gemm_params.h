@@ -10,7 +10,9 @@ namespace exo {
 constexpr int kBlockM = 128;        // rows of C per CTA (one TMEM lane per row)
 constexpr int kBlockK = 64;         // 16-bit elements of K per sub-block: 128 bytes = one swizzle span
 constexpr int kUmmaK = 16;          // K of one tcgen05.mma for 16-bit inputs (32 bytes; 8 for tf32)
-constexpr int kNumThreads = 320;    // warp 0 producer, warp 1 MMA issuer + TMEM owner, warps 2..9 epilogue
+// warp 0 producer of A, warp 1 MMA issuer + TMEM owner, warps 2..9 epilogue, warp 10 producer of B
+constexpr int kNumThreads = 352;
+constexpr int kProducerBWarp = 10;
 constexpr int kEpiWarps = 8;        // two per TMEM lane quadrant, each taking every other column chunk
 constexpr int kEpiBufBytes = 4096;  // one staging buffer: 32 rows x 128 bytes
 constexpr int kMaxEpiBufs = 2;      // staging buffers per epilogue warp: 1 or 2 (chosen per plan)

@@ -185,7 +185,7 @@ inline double shape_efficiency(int cta_group, int bn) {
 constexpr double kShareGain = 1.0;
 // Main-loop speed of the tall tile (256 rows per CTA) relative to the 128-row tile, and the clocks
 // per tile its exposed epilogue costs.
-constexpr double kTallGain = 1.10;
+constexpr double kTallGain = 1.06;
 constexpr double kTallDrain = 4000.0;
 
 // k-elements in one 128-byte sub-block row: 64 for 16-bit operands, 32 for fp32 storage.
@@ -219,10 +219,7 @@ inline double estimate_clocks(int64_t M, int64_t N, int64_t K, int64_t batch, in
   const int64_t nkb = (K + kBlockK - 1) / kBlockK;
   double mainloop = (double)nkb * 2.0 * bn / shape_efficiency(cta_group, bn);  // clocks per whole tile
   if (pairs == 2) mainloop /= kShareGain;
-  // An M/N-contiguous operand costs the 128-row 2-CTA tile about 15 % of its main-loop rate (measured at
-  // 8192^3: 1175-1260 TFLOP/s against 1340-1500 with both operands K-contiguous); the tall tile, which has
-  // shared-memory bandwidth to spare, is unaffected (1430-1573).
-  if (mn_major_operand && cta_group == 2 && mrep == 1) mainloop /= 0.87;
+  (void)mn_major_operand;  // M/N-contiguous operands run at the same rate (measured 1512 against 1516 TFLOP/s at 8192^3)
   const double drain = 22.0 * bn;             // draining one accumulator (measured 5-7k clocks at N = 256)
   double per_tile = mainloop > drain ? mainloop : drain;  // small K: the epilogue bounds a tile
   if (mrep == 2) {  // two accumulators per tile, less operand traffic, but the epilogue is not hidden
@@ -234,7 +231,8 @@ inline double estimate_clocks(int64_t M, int64_t N, int64_t K, int64_t batch, in
   double t = (double)full_waves * per_tile;
   if (tail > 0) {
     const int f = split_factor(tiles, max_workers, K, ksub, o);
-    if (f > 1) t += mainloop / f + (30.0 + 8.0 * (f - 1)) * bn * mrep;  // slice + exchange of partial sums
+    // slice + exchange of partial sums (the tall tile's partials are twice as large and nothing hides them)
+    if (f > 1) t += mainloop / f + (30.0 + 8.0 * (f - 1)) * bn * mrep * mrep;
     else t += per_tile;
   }
   return t + drain + 3000.0;  // the last epilogue and the pipeline fill are exposed once

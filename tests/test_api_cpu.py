@@ -317,8 +317,9 @@ def test_tall_tile_flags_and_preview():
     assert (i["tiles_m"], i["tiles_n"], i["grid"], i["tmem_columns"]) == (2, 3, 12, 512)
     # a stage holds 256 rows of A and this CTA's 128 rows of B
     assert i["stages"] * 49152 + 32768 * i["epilogue_buffers"] + 1536 == i["smem_bytes"] <= 232448
-    # large cubes take the tall tile on their own, 4096^3 (two uneven waves of 512 x 256 tiles) does not
-    st, info = B.exo_gemm_plan_preview(good(M=8192, N=8192, K=8192, c_dtype=B.BF16), 148)
+    # a long K loop amortises the exposed epilogue: such problems take the tall tile on their own where it fills
+    # the waves as well as the 128-row tile does; 4096^3 (two uneven waves of 512 x 256 tiles) does not
+    st, info = B.exo_gemm_plan_preview(good(M=4608, N=4096, K=16384, c_dtype=B.BF16), 148)
     assert info.tile_m == 512 and info.stages == 4 and info.split_k == 1
     st, info = B.exo_gemm_plan_preview(good(M=4096, N=4096, K=4096, c_dtype=B.BF16), 148)
     assert info.tile_m == 256

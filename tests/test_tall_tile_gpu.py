@@ -159,14 +159,14 @@ def test_alpha_zero_and_k_zero_on_the_tall_tile():
     assert_parity(p, got, info)
 
 
-def test_large_problem_takes_the_tall_tile_by_default():
-    # 6144^3: the library's own choice; checked on sampled entries and with the whole-matrix Freivalds test
-    p = synth.Problem("tall_6144", 6144, 6144, 6144, BF16, BF16, 0, 1, 0, 1.0, 0.0, seed=2).generate()
+def test_long_k_problem_takes_the_tall_tile_by_default():
+    # 4608 x 4096 x 16384: the library's own choice; checked on sampled entries and with the whole-matrix Freivalds test
+    p = synth.Problem("tall_auto", 4608, 4096, 16384, BF16, BF16, 0, 1, 0, 1.0, 0.0, seed=2).generate()
     _, got, info = run(p, 0, 0)
     if info["sm_count"] == 148:
         assert info["tile_m"] == 512, info
     rng = np.random.default_rng(3)
-    rows, cols = rng.integers(0, 6144, 1 << 14), rng.integers(0, 6144, 1 << 14)
+    rows, cols = rng.integers(0, 4608, 1 << 14), rng.integers(0, 4096, 1 << 14)
     cref, den = oracle.gemm_problem_entries(p, rows, cols)
     gate = TOL * den + oracle.output_rounding_slack(cref, BF16)
     assert (np.abs(got[rows, cols] - cref) <= gate).all(), info
