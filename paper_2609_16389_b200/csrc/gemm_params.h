@@ -48,9 +48,6 @@ struct OperandStaging {
   uint32_t lbo_enc;    // leading byte offset >> 4
   uint32_t k_step_enc; // descriptor start-address increment per UMMA_K inside a sub-block (bytes >> 4)
   uint32_t k_sub_enc;  // descriptor start-address increment per 64-k sub-block (bytes >> 4)
-  uint32_t box_bytes;  // MN-major: bytes of one TMA box in shared memory
-  uint32_t mn_boxes;   // MN-major: boxes per operand tile (rows / elements per 128 bytes)
-  uint32_t mn_box;     // MN-major: M/N elements per box (64 for 16-bit, 32 for tf32)
 };
 
 enum StatusCode : uint32_t {

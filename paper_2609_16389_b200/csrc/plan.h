@@ -369,16 +369,13 @@ inline OperandStaging make_staging(int mn_major, int rows, int ksub, int ab_byte
     s.lbo_enc = 1;                                   // unused for swizzled K-major tiles
     s.k_step_enc = (kUmmaK * 2) >> 4;                // 32 bytes along the 128-byte row
     s.k_sub_enc = ((uint32_t)rows * 128u) >> 4;      // next sub-block: next box of `rows` rows
-    s.box_bytes = (uint32_t)rows * 128u;
-    s.mn_boxes = 1;
-    s.mn_box = (uint32_t)rows;
   } else {
     const uint32_t sub_k = (uint32_t)sub_block_k(ab_bytes);   // k-rows per sub-block: 64 or 32
     const uint32_t umma_k = sub_k / 4;                        // k-rows per MMA: 16 or 8
-    s.mn_box = sub_k;                                         // M/N elements in 128 bytes: also 64 or 32
-    s.mn_boxes = (uint32_t)rows / s.mn_box;
-    s.box_bytes = (uint32_t)ksub * sub_k * 128u;     // one box: sub_k*ksub k-rows of 128 bytes
-    s.lbo_enc = s.box_bytes >> 4;                    // next group of M/N elements: next box
+    // one TMA box per group of 128 bytes of M/N elements: sub_k*ksub k-rows of 128 bytes; the kernel
+    // issues rows / 64 of them per stage (16-bit operands; fp32 operands are K-contiguous only)
+    const uint32_t box_bytes = (uint32_t)ksub * sub_k * 128u;
+    s.lbo_enc = box_bytes >> 4;                      // next group of M/N elements: next box
     s.k_step_enc = (umma_k * 128u) >> 4;             // the k-rows of one MMA
     s.k_sub_enc = (sub_k * 128u) >> 4;               // k-rows continue inside the same box
   }

@@ -328,3 +328,12 @@ def test_tall_tile_flags_and_preview():
     # the K-slices' scratch covers both accumulators of both CTAs
     st, info = B.exo_gemm_plan_preview(good(M=2560, N=3840, K=2048, flags2=TALL), 148)
     assert (info.tail_tiles, info.split_k, info.workspace_bytes) == (1, 8, 7 * 512 * 256 * 4)
+
+
+def test_smoke_cases_are_in_the_supported_set():
+    import __graft_entry__ as entry
+    from paper_2609_16389_b200 import harness
+    for p in entry.smoke_cases():
+        d = harness.desc_of(p)
+        assert B.exo_gemm_validate(d) == B.OK, p.name
+        assert B.exo_gemm_plan_preview(d, 148)[0] == B.OK, p.name
