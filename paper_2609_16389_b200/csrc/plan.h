@@ -196,6 +196,9 @@ inline int sub_block_k(int ab_bytes) { return 128 / ab_bytes; }
 inline int split_factor(int64_t tiles, int64_t workers, int64_t K, int ksub, const FlagOverrides& o) {
   const int64_t tail = tiles % workers;
   if (tail == 0 || o.split == 1 || o.no_workspace) return 1;
+  // With whole waves before it and a K loop shorter than a tile's epilogue, the tail has no main-loop time
+  // to save and the exchange of partial sums only adds output traffic (measured at K = 512: 20-27 % slower).
+  if (tiles >= workers && K < 2048 && o.split == 0) return 1;
   const int64_t k_blocks = (K + kBlockK * ksub - 1) / (kBlockK * ksub);
   int64_t f = workers / tail;
   const int64_t by_k = (K / kBlockK) / 4;   // every slice keeps at least 256 k-elements
@@ -220,7 +223,10 @@ inline double estimate_clocks(int64_t M, int64_t N, int64_t K, int64_t batch, in
   double mainloop = (double)nkb * 2.0 * bn / shape_efficiency(cta_group, bn);  // clocks per whole tile
   if (pairs == 2) mainloop /= kShareGain;
   (void)mn_major_operand;  // M/N-contiguous operands run at the same rate (measured 1512 against 1516 TFLOP/s at 8192^3)
-  const double drain = 22.0 * bn;             // draining one accumulator (measured 5-7k clocks at N = 256)
+  // draining one accumulator: 5-7k clocks at N = 256, but only about a third less at N = 128 (waits, tile
+  // decode and the last store's latency do not shrink with the tile: at K = 512 the 256-column tile is
+  // 20-27 % faster than two 128-column ones)
+  const double drain = 1500.0 + 16.0 * bn;
   double per_tile = mainloop > drain ? mainloop : drain;  // small K: the epilogue bounds a tile
   if (mrep == 2) {  // two accumulators per tile, less operand traffic, but the epilogue is not hidden
     mainloop = 2.0 * mainloop / kTallGain;
@@ -262,7 +268,9 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
     double t = estimate_clocks(c.M, c.N, c.K * (c.ab_bytes / 2), c.batch, g, n, w_eff, o, pr, mr,
                                c.a_mn_major || c.b_mn_major);
     if (mr == 2) t *= 1.03;  // the tall tile's exposed epilogue makes it the riskier choice: it must win clearly
-    if (best_g == 0 || t < best * 0.999) { best = t; best_g = g; best_n = n; best_p = pr; best_r = mr; }
+    // candidates come largest tile first; a smaller one has to win by 3 %: the estimate flatters small tiles
+    // (their fixed costs per tile are only partly modelled)
+    if (best_g == 0 || t < best * 0.97) { best = t; best_g = g; best_n = n; best_p = pr; best_r = mr; }
   }
   if (best_g == 0) { best_g = o.cta_group ? o.cta_group : 1; best_n = o.tile_n ? o.tile_n : 128; }
   TileConfig cfg;
