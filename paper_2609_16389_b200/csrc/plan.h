@@ -196,9 +196,11 @@ inline int sub_block_k(int ab_bytes) { return 128 / ab_bytes; }
 inline int split_factor(int64_t tiles, int64_t workers, int64_t K, int ksub, const FlagOverrides& o) {
   const int64_t tail = tiles % workers;
   if (tail == 0 || o.split == 1 || o.no_workspace) return 1;
-  // With whole waves before it and a K loop shorter than a tile's epilogue, the tail has no main-loop time
-  // to save and the exchange of partial sums only adds output traffic (measured at K = 512: 20-27 % slower).
-  if (tiles >= workers && K < 2048 && o.split == 0) return 1;
+  // A short K loop leaves no main-loop time to save, and the exchange of partial sums (a round trip
+  // through L2 plus the extra output traffic) costs about as much as a dozen k-blocks.  Measured: behind
+  // whole waves at K = 512 the split is 20-27 % slower; for problems smaller than one wave it loses 28 % at
+  // K = 512 and 3 % at K = 1000, and wins 13-35 % from K = 2048 on.
+  if (K < 2048 && o.split == 0) return 1;
   const int64_t k_blocks = (K + kBlockK * ksub - 1) / (kBlockK * ksub);
   int64_t f = workers / tail;
   const int64_t by_k = (K / kBlockK) / 4;   // every slice keeps at least 256 k-elements
