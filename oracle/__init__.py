@@ -54,6 +54,8 @@ def lib():
         _lib.oracle_gemm_entries.restype = ci
         _lib.oracle_gemv.argtypes = [i64, i64, vp, i64, vp, vp, dbl, dbl, vp, vp]
         _lib.oracle_gemv.restype = ci
+        _lib.oracle_gemv_colmajor.argtypes = [i64, i64, vp, i64, vp, vp, dbl, dbl, vp, vp]
+        _lib.oracle_gemv_colmajor.restype = ci
         _lib.oracle_widen.argtypes = [ctypes.c_uint32, ci]
         _lib.oracle_widen.restype = dbl
         _lib.oracle_num_threads.restype = ci
@@ -125,14 +127,16 @@ def gemm_entries(M, N, K, A, B, Cin, ab_dtype, c_dtype, a_layout, b_layout, c_la
     return cref, den
 
 
-def gemv(M, N, A, lda, x, y, alpha, beta):
-    """Reference y and metric denominator (float64, length M) of the fp32 row-major GEMV."""
-    for buf, need, what in ((A, (M - 1) * lda + N if M and N else 0, "A"), (x, N, "x"), (y, M, "y")):
+def gemv(M, N, A, lda, x, y, alpha, beta, layout=ROW_MAJOR):
+    """Reference y and metric denominator (float64, length M) of the fp32 GEMV, A row- or column-major."""
+    a_need = ((M - 1) * lda + N if layout == ROW_MAJOR else (N - 1) * lda + M) if M and N else 0
+    for buf, need, what in ((A, a_need, "A"), (x, N, "x"), (y, M, "y")):
         if buf.dtype != np.float32 or not buf.flags.c_contiguous or buf.size < need:
             raise ValueError(f"{what}: need contiguous float32 of at least {need} elements")
     yref = np.empty(M, dtype=np.float64)
     den = np.empty(M, dtype=np.float64)
-    rc = lib().oracle_gemv(M, N, _ptr(A), lda, _ptr(x), _ptr(y), float(alpha), float(beta), _ptr(yref), _ptr(den))
+    fn = lib().oracle_gemv if layout == ROW_MAJOR else lib().oracle_gemv_colmajor
+    rc = fn(M, N, _ptr(A), lda, _ptr(x), _ptr(y), float(alpha), float(beta), _ptr(yref), _ptr(den))
     if rc != 0:
         raise RuntimeError(f"oracle_gemv failed with code {rc}")
     return yref, den

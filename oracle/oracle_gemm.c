@@ -257,3 +257,30 @@ int oracle_gemv(int64_t M, int64_t N, const float* A, int64_t lda, const float* 
     }
     return 0;
 }
+
+/*
+ * The same product for a column-major A (element (i, j) at A[i + j * lda], lda >= M): the other storage
+ * order of the BLAS Sgemv the paper's Section 6 GEMV is measured against.  Same definition, same
+ * summation order (j ascending), same denominator.
+ */
+int oracle_gemv_colmajor(int64_t M, int64_t N, const float* A, int64_t lda, const float* x, const float* y,
+                         double alpha, double beta, double* yref, double* den) {
+    if (M < 0 || N < 0 || lda < M) return 1;
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < M; ++i) {
+        double s = 0.0, d = 0.0;
+        for (int64_t j = 0; j < N; ++j) {
+            double p = (double)A[i + j * lda] * (double)x[j];
+            s += p;
+            d += fabs(p);
+        }
+        double r = alpha * s;
+        if (beta != 0.0) {
+            r += beta * (double)y[i];
+            d += fabs(beta * (double)y[i]);
+        }
+        yref[i] = r;
+        den[i] = d;
+    }
+    return 0;
+}

@@ -372,3 +372,40 @@ def test_gemv_oracle_against_closed_forms_and_a_library_product():
                              FP16, FP32, 0, 0, 0, N, 1, 1, 1.0, 0.0)
     g, gd = oracle.gemv(M, N, A, lda, x, y, 1.0, 0.0)
     assert np.array_equal(cref[:, 0], g) and np.array_equal(cden[:, 0], gd)
+
+
+def test_gemv_oracle_column_major_against_closed_forms_and_the_gemm_oracle():
+    # hand-checked: a_ij = i + 5j (M = 5, N = 3, stored column by column with lda = 7), x = (1, 2, 3), y = 1:
+    # row i gives i + 2(i + 5) + 3(i + 10) = 6i + 40; with alpha = 1, beta = 1/2: 6i + 40.5
+    M, N, lda = 5, 3, 7
+    A = np.full(N * lda, np.nan, dtype=np.float32)                 # padding must never be read
+    for j in range(N):
+        A[j * lda:j * lda + M] = np.arange(M) + 5 * j
+    x = np.array([1, 2, 3], np.float32)
+    yref, den = oracle.gemv(M, N, A, lda, x, np.ones(M, np.float32), 1.0, 0.5, layout=1)
+    assert np.array_equal(yref, 6.0 * np.arange(M) + 40.5) and np.array_equal(den, 6.0 * np.arange(M) + 40.5)
+    # a transposed operand must change the answer (a_ij read as a_ji would give other numbers)
+    sq = np.arange(9, dtype=np.float32)                            # 3 x 3: row-major reading vs column-major reading
+    r, _ = oracle.gemv(3, 3, sq, 3, x, np.zeros(3, np.float32), 1.0, 0.0, layout=0)
+    c, _ = oracle.gemv(3, 3, sq, 3, x, np.zeros(3, np.float32), 1.0, 0.0, layout=1)
+    assert np.array_equal(r, [8, 26, 44]) and np.array_equal(c, [24, 30, 36])
+    # random dyadic data: equals the row-major oracle on the transposed buffer, numpy in fp64, and the
+    # one-column GEMM oracle with a column-major A
+    rng = np.random.default_rng(13)
+    M, N, lda = 41, 29, 48
+    Al = rng.integers(-8, 9, size=(M, N)).astype(np.float32) / 4
+    A = np.full(N * lda, np.nan, dtype=np.float32)
+    A.reshape(N, lda)[:, :M] = Al.T
+    x = (rng.integers(-8, 9, size=N) / 8).astype(np.float32)
+    y = rng.integers(-8, 9, size=M).astype(np.float32)
+    yref, den = oracle.gemv(M, N, A, lda, x, y, -1.5, 0.25, layout=1)
+    assert np.array_equal(yref, -1.5 * (Al.astype(np.float64) @ x.astype(np.float64)) + 0.25 * y)
+    assert np.array_equal(den, np.abs(Al.astype(np.float64)) @ np.abs(x.astype(np.float64)) + np.abs(0.25 * y))
+    rowbuf = np.ascontiguousarray(Al).reshape(-1)
+    yrow, drow = oracle.gemv(M, N, rowbuf, N, x, y, -1.5, 0.25, layout=0)
+    assert np.array_equal(yref, yrow) and np.array_equal(den, drow)
+    A16 = synth.round_to_storage(Al, FP16); x16 = synth.round_to_storage(x.reshape(N, 1), FP16)
+    cref, cden = oracle.gemm(M, 1, N, synth.store(A16, 1), synth.store(x16, 0), np.zeros(M, np.float32),
+                             FP16, FP32, 1, 0, 0, M, 1, 1, 1.0, 0.0)
+    g, gd = oracle.gemv(M, N, A, lda, x, y, 1.0, 0.0, layout=1)
+    assert np.array_equal(cref[:, 0], g) and np.array_equal(cden[:, 0], gd)
