@@ -553,14 +553,17 @@ def run_sweep(args, rank, world, local_rank):
 
 
 def run_gemv(args, rank, world, local_rank):
-    """fp32 GEMV y = A x (row-major A), the paper's memory-bound companion workload (Section 6).
-    Workload name gemv_<M>x<N>.  A step = one exo_gemv_run; the matrices rotate through several copies
+    """fp32 GEMV y = A x, the paper's memory-bound companion workload (Section 6).
+    Workload name gemv_<M>x<N> (row-major A) or gemvc_<M>x<N> (column-major A).  A step = one exo_gemv_run[_colmajor]; the matrices rotate through several copies
     so that every step streams A from HBM.  Roofline: HBM (algorithmic bytes = 4*M*N + 4*N + 4*M)."""
     import torch
     from paper_2609_16389_b200 import binding as B
     if rank != 0:
         return
-    M, N = (int(v) for v in args.workload[len("gemv_"):].split("x"))
+    col = args.workload.startswith("gemvc_")
+    M, N = (int(v) for v in args.workload.split("_", 1)[1].split("x"))
+    lda = M if col else N
+    run = B.exo_gemv_run_colmajor if col else B.exo_gemv_run
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     pk = peaks()
@@ -574,7 +577,7 @@ def run_gemv(args, rank, world, local_rank):
     stream = torch.cuda.current_stream(dev)
 
     def step(i):
-        st = B.exo_gemv_run(M, N, dAs[i % n_sets].data_ptr(), N, dx.data_ptr(), dy.data_ptr(), 1.0, 0.0, stream.cuda_stream)
+        st = run(M, N, dAs[i % n_sets].data_ptr(), lda, dx.data_ptr(), dy.data_ptr(), 1.0, 0.0, stream.cuda_stream)
         if st != B.OK:
             raise B.ExoGemmError(st, "exo_gemv_run")
 
@@ -613,10 +616,10 @@ def run_gemv(args, rank, world, local_rank):
         "metric": METRIC, "value": flop / (ms * 1e-3) / 1e12, "unit": UNIT, "n_gpus": 1, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": args.workload, "M": M, "N": N, "layout": "A row-major",
+        "config": {"workload": args.workload, "M": M, "N": N, "layout": "A column-major" if col else "A row-major",
                    "l2": f"rotating {n_sets} copies of A ({n_sets * hA.nbytes >> 20} MiB > 126 MiB L2)"},
         "roofline": {"bound": "hbm", "achieved": gbs, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": gbs / pk["hbm_gbs"],
-                     "traffic": None, "peak_source": f"{pk['source']} (copy bandwidth)", "kernel": "exo_gemv_rowmajor_kernel",
+                     "traffic": None, "peak_source": f"{pk['source']} (copy bandwidth)", "kernel": "exo_gemv_colmajor_kernel" if col else "exo_gemv_rowmajor_kernel",
                      "algorithmic_bytes": abytes, "flop": flop},
         "e2e": {"value": flop / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": int(hA.nbytes + hx.nbytes),
                 "d2h_bytes_per_step": int(4 * M), "ms_per_step": e2e_ms, "steps": k},
@@ -624,13 +627,14 @@ def run_gemv(args, rank, world, local_rank):
     }
     if not args.no_cublas:
         xs = dx
+        mat = (lambda t: t.view(N, M).t()) if col else (lambda t: t.view(M, N))
         for _ in range(3):
-            torch.mv(dAs[0].view(M, N), xs, out=dy)
+            torch.mv(mat(dAs[0]), xs, out=dy)
         torch.cuda.synchronize(dev)
         g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         g0.record(stream)
         for i in range(args.steps):
-            torch.mv(dAs[i % n_sets].view(M, N), xs, out=dy)
+            torch.mv(mat(dAs[i % n_sets]), xs, out=dy)
         g1.record(stream)
         torch.cuda.synchronize(dev)
         cms = g0.elapsed_time(g1) / args.steps
@@ -639,7 +643,7 @@ def run_gemv(args, rank, world, local_rank):
         import oracle
         rows = min(M, max(1, int(2e9 / max(N, 1))))
         t0 = time.perf_counter()
-        oracle.gemv(rows, N, hA, N, hx, np.zeros(rows, np.float32), 1.0, 0.0)
+        oracle.gemv(rows, N, hA, lda, hx, np.zeros(rows, np.float32), 1.0, 0.0, layout=1 if col else 0)
         dt = time.perf_counter() - t0
         line["cpu_baseline"] = {"value": 2.0 * rows * N / dt / 1e12, "unit": UNIT, "cores": oracle.num_threads(),
                                 "kind": "oracle", "sample": f"rows 0..{rows} of {args.workload}, {dt:.2f} s wall"}
@@ -651,7 +655,7 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if args.workload.startswith("gemv_"):
+    if args.workload.startswith(("gemv_", "gemvc_")):
         if args.impl == "reference":
             raise SystemExit("the reference arm times GEMM workloads")
         run_gemv(args, rank, world, local_rank)
@@ -661,7 +665,7 @@ def main():
             raise SystemExit("the reference arm times one workload; pick e.g. --workload sweep_1000x1000x1000")
         run_sweep(args, rank, world, local_rank)
         return
-    if args.workload not in WORKLOADS and not args.workload.startswith(("sweep_", "batched_", "tf32_")):
+    if args.workload not in WORKLOADS and not args.workload.startswith(("sweep_", "batched_", "tf32_", "gemv_", "gemvc_")):
         raise SystemExit(f"unknown workload {args.workload}")
     if args.impl == "reference":
         run_reference(args, rank, world)

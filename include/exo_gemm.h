@@ -274,6 +274,19 @@ exo_gemm_status_t exo_gemm_run_static(const exo_gemm_desc_t* desc, const void* A
 exo_gemm_status_t exo_gemv_run(int64_t M, int64_t N, const float* A, int64_t lda, const float* x, float* y,
                                float alpha, float beta, void* cuda_stream);
 
+/*
+ * The same product for a COLUMN-major A (M contiguous, leading dimension lda >= M), the other
+ * storage order BLAS Sgemv takes.  A lane owns consecutive rows, so every warp load of a
+ * column is contiguous; the columns are split over the warps of a CTA and over the CTAs of
+ * a thread-block cluster, and the partial sums are added through shared and distributed
+ * shared memory in warp and CTA order (the result does not depend on timing).  128-bit
+ * loads when A is 16-byte aligned, lda % 4 == 0 and M >= 128; scalar loads otherwise.  Same argument
+ * rules, ownership and errors as exo_gemv_run (ERR_INVALID_ARG for lda < M; ERR_UNSUPPORTED
+ * if M needs 2^31 or more CTAs).
+ */
+exo_gemm_status_t exo_gemv_run_colmajor(int64_t M, int64_t N, const float* A, int64_t lda, const float* x, float* y,
+                                        float alpha, float beta, void* cuda_stream);
+
 /* Frees the plan and its device status block.  NULL is a no-op returning OK. */
 exo_gemm_status_t exo_gemm_destroy(exo_gemm_handle_t plan);
 

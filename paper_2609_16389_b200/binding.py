@@ -19,7 +19,7 @@ EXPORTED_SYMBOLS = (
     "exo_gemm_validate", "exo_gemm_create", "exo_gemm_run", "exo_gemm_check", "exo_gemm_plan_preview",
     "exo_gemm_get_info", "exo_gemm_destroy", "exo_gemm_status_string", "exo_gemm_last_cuda_error",
     "exo_gemm_schedule_enumerate", "exo_gemm_debug_set", "exo_gemm_run_static", "exo_gemm_schedule_work",
-    "exo_gemm_create_batched", "exo_gemv_run", "exo_gemm_has_shared_operand_clusters",
+    "exo_gemm_create_batched", "exo_gemv_run", "exo_gemm_has_shared_operand_clusters", "exo_gemv_run_colmajor",
 )
 
 
@@ -96,6 +96,8 @@ def lib():
         L.exo_gemm_debug_set.argtypes = [vp, i32, i64]
         L.exo_gemv_run.argtypes = [i64, i64, vp, i64, vp, vp, ctypes.c_float, ctypes.c_float, vp]
         L.exo_gemv_run.restype = ctypes.c_int
+        L.exo_gemv_run_colmajor.argtypes = [i64, i64, vp, i64, vp, vp, ctypes.c_float, ctypes.c_float, vp]
+        L.exo_gemv_run_colmajor.restype = ctypes.c_int
         L.exo_gemm_schedule_work.argtypes = [i64, i32, i32, i32, i32, i32, ctypes.POINTER(i64), ctypes.POINTER(i32),
                                              ctypes.POINTER(i32), ctypes.POINTER(i32), i64]
         L.exo_gemm_schedule_work.restype = i64
@@ -194,6 +196,11 @@ def exo_gemm_run_static(desc: Desc, a_ptr: int, b_ptr: int, c_ptr: int, alpha: f
 def exo_gemv_run(M: int, N: int, a_ptr: int, lda: int, x_ptr: int, y_ptr: int, alpha: float, beta: float,
                  stream: int = 0) -> int:
     return lib().exo_gemv_run(M, N, a_ptr, lda, x_ptr, y_ptr, alpha, beta, stream)
+
+
+def exo_gemv_run_colmajor(M: int, N: int, a_ptr: int, lda: int, x_ptr: int, y_ptr: int, alpha: float, beta: float,
+                          stream: int = 0) -> int:
+    return lib().exo_gemv_run_colmajor(M, N, a_ptr, lda, x_ptr, y_ptr, alpha, beta, stream)
 
 
 def exo_gemm_schedule_enumerate(tiles_m, tiles_n, band, along_m, num_workers, worker):

@@ -366,6 +366,62 @@ def test_gemv_unaligned_operands_take_the_scalar_path_and_bad_arguments_are_refu
     assert B.exo_gemv_run(4, 8, 0, 8, dx.data_ptr(), dy.data_ptr(), 1.0, 0.0) == B.ERR_NULL
 
 
+COL_GEMV_CASES = [
+    # M, N, lda, alpha, beta
+    (1, 1, 4, 1.0, 0.0), (7, 3, 8, 2.0, 0.0), (100, 17, 100, 1.0, 0.5),          # few columns: clusters of 1
+    (128, 64, 128, 1.0, 0.0), (129, 65, 132, -1.0, 1.0),                           # scalar path, clusters of 2
+    (511, 300, 512, 1.0, 0.0), (512, 256, 512, 0.5, 0.0),                          # 128-bit path from M = 512
+    (515, 1000, 516, 1.0, -2.0), (2048, 2049, 2048, 1.0, 0.0),                     # ragged last row group, odd N
+    (1000, 333, 1003, 1.0, 1.0),                                                   # lda % 4 != 0: scalar path
+    (5000, 40, 5000, 1.0, 0.0), (4096, 0, 4096, 1.0, 3.0), (300, 700, 300, 0.0, 0.5),
+]
+
+
+@pytest.mark.parametrize("M,N,lda,alpha,beta", COL_GEMV_CASES)
+def test_gemv_column_major_against_the_oracle(M, N, lda, alpha, beta):
+    import torch
+    rng = np.random.default_rng(M * 11 + N)
+    A = rng.uniform(-1, 1, size=max(N, 1) * lda).astype(np.float32)
+    x = rng.uniform(-1, 1, size=max(N, 1)).astype(np.float32)
+    y = rng.uniform(-1, 1, size=M).astype(np.float32)
+    if beta == 0.0:
+        y[:] = np.nan
+    if alpha == 0.0:
+        A[:] = np.nan                                  # alpha == 0: A and x are not read
+    dev = torch.device("cuda:0")
+    dA, dx, dy = harness._to_device(A, dev), harness._to_device(x, dev), harness._to_device(y, dev)
+    s = torch.cuda.current_stream(dev).cuda_stream
+    assert B.exo_gemv_run_colmajor(M, N, dA.data_ptr(), lda, dx.data_ptr(), dy.data_ptr(), alpha, beta, s) == B.OK
+    torch.cuda.synchronize(dev)
+    first = dy.cpu().numpy().view(np.float32).copy()
+    yref, den = oracle.gemv(M, N, np.nan_to_num(A), lda, x[:N].copy(), np.nan_to_num(y), alpha, beta, layout=1)
+    assert oracle.max_error(first.astype(np.float64), yref, den) <= TOL
+    # the partial sums of a cluster are added in CTA order: a second run gives the same bits
+    dy.copy_(torch.from_numpy(y.view(np.uint8)))
+    assert B.exo_gemv_run_colmajor(M, N, dA.data_ptr(), lda, dx.data_ptr(), dy.data_ptr(), alpha, beta, s) == B.OK
+    torch.cuda.synchronize(dev)
+    assert np.array_equal(dy.cpu().numpy().view(np.float32), first, equal_nan=True)
+
+
+def test_gemv_column_major_unaligned_base_and_bad_arguments():
+    import torch
+    M, N, lda = 640, 200, 640
+    rng = np.random.default_rng(5)
+    A = rng.uniform(-1, 1, size=N * lda + 1).astype(np.float32)
+    x = rng.uniform(-1, 1, size=N).astype(np.float32)
+    y = np.zeros(M, np.float32)
+    dev = torch.device("cuda:0")
+    dA, dx, dy = harness._to_device(A, dev), harness._to_device(x, dev), harness._to_device(y, dev)
+    assert B.exo_gemv_run_colmajor(M, N, dA.data_ptr() + 4, lda, dx.data_ptr(), dy.data_ptr(), 1.0, 0.0) == B.OK
+    torch.cuda.synchronize(dev)
+    got = dy.cpu().numpy().view(np.float32).astype(np.float64)
+    yref, den = oracle.gemv(M, N, A[1:].copy(), lda, x, y, 1.0, 0.0, layout=1)
+    assert oracle.max_error(got, yref, den) <= TOL
+    assert B.exo_gemv_run_colmajor(-1, 4, dA.data_ptr(), 4, dx.data_ptr(), dy.data_ptr(), 1.0, 0.0) == B.ERR_INVALID_ARG
+    assert B.exo_gemv_run_colmajor(8, 4, dA.data_ptr(), 4, dx.data_ptr(), dy.data_ptr(), 1.0, 0.0) == B.ERR_INVALID_ARG
+    assert B.exo_gemv_run_colmajor(4, 8, 0, 8, dx.data_ptr(), dy.data_ptr(), 1.0, 0.0) == B.ERR_NULL
+
+
 # ------------------------------------------------------------------ strided batch
 BATCH_CASES = [
     # M, N, K, ab, cd, la, lb, lc, alpha, beta, batch, pad (extra elements between matrices), shared operand
