@@ -100,8 +100,8 @@ typedef enum { EXO_GEMM_ROW_MAJOR = 0, EXO_GEMM_COL_MAJOR = 1 } exo_gemm_layout_
  * multiplied as tf32 (the tensor core reads sign, exponent and the upper 10 fraction
  * bits of each fp32 operand and ignores the rest; products are accumulated in fp32):
  * this is the precision of the paper's own Section 6 kernels and of
- * CUBLAS_TF32_TENSOR_OP_MATH.  FP32 operands must have K contiguous (A row-major,
- * B column-major); other FP32 layouts return ERR_UNSUPPORTED.  Because operands and
+ * CUBLAS_TF32_TENSOR_OP_MATH (M/N-contiguous FP32 operands are staged with the 128-byte
+ * swizzle in 32-byte atoms that tcgen05 wants for transposed 32-bit operands).  Because operands and
  * results move by TMA, every leading dimension times its element size must be a
  * multiple of 16 bytes (16-bit: ld % 8 == 0, fp32: ld % 4 == 0) and every base
  * pointer passed to exo_gemm_run must be 16-byte aligned.  Legal BLAS calls

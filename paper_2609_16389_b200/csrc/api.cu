@@ -95,7 +95,8 @@ static EncodeTiledFn get_encode_fn() {
 // 2-D tensor map over a matrix whose contiguous dimension has `inner` elements and
 // whose other dimension has `outer` elements `ld` elements apart.
 static CUresult encode_2d(CUtensorMap* map, int dtype, const void* base, uint64_t inner, uint64_t outer,
-                          uint64_t ld, uint32_t box_inner, uint32_t box_outer, bool operand) {
+                          uint64_t ld, uint32_t box_inner, uint32_t box_outer, bool operand,
+                          bool atom32 = false /* M/N-contiguous fp32 operand: 128-byte swizzle in 32-byte atoms */) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return CUDA_ERROR_NOT_FOUND;
   const CUtensorMapDataType dt = dtype == EXO_GEMM_FP32   ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
@@ -106,7 +107,7 @@ static CUresult encode_2d(CUtensorMap* map, int dtype, const void* base, uint64_
   cuuint32_t box[2] = {box_inner, box_outer};
   cuuint32_t estr[2] = {1, 1};
   return fn(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-            CU_TENSOR_MAP_SWIZZLE_128B,
+            atom32 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
             operand ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_NONE,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
 }
@@ -114,7 +115,7 @@ static CUresult encode_2d(CUtensorMap* map, int dtype, const void* base, uint64_
 // The same with a third dimension: `batch` matrices `batch_stride` elements apart, boxes one matrix deep.
 static CUresult encode_3d(CUtensorMap* map, int dtype, const void* base, uint64_t inner, uint64_t outer,
                           uint64_t ld, uint64_t batch, uint64_t batch_stride, uint32_t box_inner,
-                          uint32_t box_outer, bool operand) {
+                          uint32_t box_outer, bool operand, bool atom32 = false) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return CUDA_ERROR_NOT_FOUND;
   const CUtensorMapDataType dt = dtype == EXO_GEMM_FP32   ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
@@ -127,7 +128,7 @@ static CUresult encode_3d(CUtensorMap* map, int dtype, const void* base, uint64_
   cuuint32_t box[3] = {box_inner, box_outer, 1};
   cuuint32_t estr[3] = {1, 1, 1};
   return fn(map, dt, 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-            CU_TENSOR_MAP_SWIZZLE_128B,
+            atom32 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
             operand ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_NONE,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
 }
@@ -469,12 +470,13 @@ exo_gemm_status_t exo_gemm_run(exo_gemm_handle_t plan, const void* A, const void
   const int b_rows = cfg.tile_n / cfg.cta_group;
   const int a_rows = kBlockM * cfg.mrep / cfg.pairs;  // pairs that share A fetch half of a CTA's rows each
   const uint32_t c_box = d.c_dtype == EXO_GEMM_FP32 ? 32 : 64;
+  const bool atom32 = d.ab_dtype == EXO_GEMM_FP32;   // only read for M/N-contiguous operands
   if (cn.batch <= 1) {
     if (read_ab) {
-      r = cn.a_mn_major ? encode_2d(&tm_a, d.ab_dtype, opA, cn.M, cn.K, cn.lda, sub_k, stage_k, true)
+      r = cn.a_mn_major ? encode_2d(&tm_a, d.ab_dtype, opA, cn.M, cn.K, cn.lda, sub_k, stage_k, true, atom32)
                         : encode_2d(&tm_a, d.ab_dtype, opA, cn.K, cn.M, cn.lda, sub_k, a_rows, true);
       if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return EXO_GEMM_ERR_CUDA; }
-      r = cn.b_mn_major ? encode_2d(&tm_b, d.ab_dtype, opB, cn.N, cn.K, cn.ldb, sub_k, stage_k, true)
+      r = cn.b_mn_major ? encode_2d(&tm_b, d.ab_dtype, opB, cn.N, cn.K, cn.ldb, sub_k, stage_k, true, atom32)
                         : encode_2d(&tm_b, d.ab_dtype, opB, cn.K, cn.N, cn.ldb, sub_k, b_rows, true);
       if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return EXO_GEMM_ERR_CUDA; }
     }
@@ -483,11 +485,11 @@ exo_gemm_status_t exo_gemm_run(exo_gemm_handle_t plan, const void* A, const void
   } else {  // strided batch: the matrix index is the third tensor-map coordinate
     if (read_ab) {
       r = cn.a_mn_major
-              ? encode_3d(&tm_a, d.ab_dtype, opA, cn.M, cn.K, cn.lda, cn.batch, cn.stride_a, sub_k, stage_k, true)
+              ? encode_3d(&tm_a, d.ab_dtype, opA, cn.M, cn.K, cn.lda, cn.batch, cn.stride_a, sub_k, stage_k, true, atom32)
               : encode_3d(&tm_a, d.ab_dtype, opA, cn.K, cn.M, cn.lda, cn.batch, cn.stride_a, sub_k, a_rows, true);
       if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return EXO_GEMM_ERR_CUDA; }
       r = cn.b_mn_major
-              ? encode_3d(&tm_b, d.ab_dtype, opB, cn.N, cn.K, cn.ldb, cn.batch, cn.stride_b, sub_k, stage_k, true)
+              ? encode_3d(&tm_b, d.ab_dtype, opB, cn.N, cn.K, cn.ldb, cn.batch, cn.stride_b, sub_k, stage_k, true, atom32)
               : encode_3d(&tm_b, d.ab_dtype, opB, cn.K, cn.N, cn.ldb, cn.batch, cn.stride_b, sub_k, b_rows, true);
       if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return EXO_GEMM_ERR_CUDA; }
     }

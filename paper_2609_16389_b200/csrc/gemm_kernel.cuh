@@ -275,8 +275,12 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                     for (int h = 0; h < KSUB; ++h)
                       load_shared(a_dst + h * kATileBytes + pair_id * (kATileBytes / 2), k0 + h * (int32_t)p.sub_k,
                                   a_mn0 + (int32_t)pair_id * (kBlockM / 2));
-                  } else {  // two boxes of 64 rows: one each
+                  } else if (!p.tf32) {  // two boxes of 64 rows: one each
                     load_shared(a_dst + pair_id * MN_BOX_BYTES, a_mn0 + 64 * (int32_t)pair_id, k0);
+                  } else {               // fp32 storage: four boxes of 32 rows, two each
+#pragma unroll
+                    for (int b = 0; b < 2; ++b)
+                      load_shared(a_dst + (2 * pair_id + b) * (MN_BOX_BYTES / 2), a_mn0 + 32 * (int32_t)(2 * pair_id + b), k0);
                   }
                 }
               } else if (SHARE && !p.a.mn_major) {  // substituted pair: both 64-row halves, same tensor map
@@ -288,17 +292,23 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
               } else if (!p.a.mn_major) {
 #pragma unroll
                 for (int h = 0; h < KSUB; ++h) load(a_dst + h * (kATileBytes * MREP), &tm_a, k0 + h * (int32_t)p.sub_k, a_mn0);
-              } else {
+              } else if (!p.tf32) {
 #pragma unroll
                 for (int b = 0; b < A_BOXES; ++b) load(a_dst + b * MN_BOX_BYTES, &tm_a, a_mn0 + 64 * b, k0);
+              } else {  // fp32 storage: 32 elements per 128 bytes, twice as many boxes of half the size
+#pragma unroll
+                for (int b = 0; b < 2 * A_BOXES; ++b) load(a_dst + b * (MN_BOX_BYTES / 2), &tm_a, a_mn0 + 32 * b, k0);
               }
               if (!do_b) {
               } else if (!p.b.mn_major) {
 #pragma unroll
                 for (int h = 0; h < KSUB; ++h) load(b_dst + h * (B_ROWS * 128), &tm_b, k0 + h * (int32_t)p.sub_k, b_mn0);
-              } else {
+              } else if (!p.tf32) {
 #pragma unroll
                 for (int b = 0; b < B_BOXES; ++b) load(b_dst + b * MN_BOX_BYTES, &tm_b, b_mn0 + 64 * b, k0);
+              } else {
+#pragma unroll
+                for (int b = 0; b < 2 * B_BOXES; ++b) load(b_dst + b * (MN_BOX_BYTES / 2), &tm_b, b_mn0 + 32 * b, k0);
               }
             };
             if (!batched) {

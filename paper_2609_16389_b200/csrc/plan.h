@@ -82,10 +82,6 @@ inline exo_gemm_status_t validate_desc(const exo_gemm_desc_t* d) {
   // beyond here the call is a legal BLAS call; what follows is this library's supported set
   // fp32 operands are multiplied as tf32 (the precision of the paper's own kernels) into an fp32 C
   if (d->c_dtype != EXO_GEMM_FP32 && d->c_dtype != d->ab_dtype) return EXO_GEMM_ERR_UNSUPPORTED;
-  // tf32 operands must have K contiguous (A row-major, B column-major): the M/N-contiguous form
-  // needs a different shared-memory swizzle (32-byte atoms) that this library does not stage
-  if (d->ab_dtype == EXO_GEMM_FP32 && (d->a_layout != EXO_GEMM_ROW_MAJOR || d->b_layout != EXO_GEMM_COL_MAJOR))
-    return EXO_GEMM_ERR_UNSUPPORTED;
   // the persistent scheduler indexes tiles (at least 128 x 64 each) and k-blocks with 32 bits
   if (((d->M + 127) / 128) * ((d->N + 63) / 64) >= (1LL << 31)) return EXO_GEMM_ERR_UNSUPPORTED;
   // a matrix that is never touched (empty problem, K == 0) has no stride rule
@@ -382,6 +378,12 @@ inline OperandStaging make_staging(int mn_major, int rows, int ksub, int ab_byte
   } else {
     const uint32_t sub_k = (uint32_t)sub_block_k(ab_bytes);   // k-rows per sub-block: 64 or 32
     const uint32_t umma_k = sub_k / 4;                        // k-rows per MMA: 16 or 8
+    if (ab_bytes == 4) {
+      // An M/N-contiguous 32-bit operand takes the 128-byte swizzle with 32-byte atomicity (the pattern
+      // repeats every 4 rows of 128 bytes, not every 8): layout type 1 and a 512-byte stride between
+      // groups of 4 k-rows; the TMA maps of such operands use the matching swizzle mode.
+      s.desc_hi = (512u >> 4) | version | (1u << 29);
+    }
     // one TMA box per group of 128 bytes of M/N elements: sub_k*ksub k-rows of 128 bytes; the kernel
     // issues rows / 64 of them per stage (16-bit operands; fp32 operands are K-contiguous only)
     const uint32_t box_bytes = (uint32_t)ksub * sub_k * 128u;

@@ -80,6 +80,8 @@ def test_validate_rejects_bad_arguments():
 
 def test_validate_unsupported_but_legal_blas_calls():
     assert B.exo_gemm_validate(good(ab_dtype=B.FP32, c_dtype=B.FP32)) == B.OK        # tf32 mode
+    for la, lb in ((1, 1), (0, 0), (1, 0)):                                          # ... in every operand layout
+        assert B.exo_gemm_validate(good(ab_dtype=B.FP32, c_dtype=B.FP32, a_layout=la, b_layout=lb)) == B.OK
     assert B.exo_gemm_validate(good(ab_dtype=B.FP32, c_dtype=B.BF16)) == B.ERR_UNSUPPORTED
     assert B.exo_gemm_validate(good(ab_dtype=B.FP32, K=130)) == B.ERR_UNSUPPORTED     # 520 bytes per row
     assert B.exo_gemm_validate(good(ab_dtype=B.FP32, K=132)) == B.OK

@@ -313,9 +313,38 @@ def test_tf32_operands(lc, shape, g, bn, ksub):
     check_full(p, flags_for(g, bn, ksub=ksub) if g else 0, literal=True)
 
 
-def test_tf32_other_layouts_are_refused():
-    for la, lb in ((1, 1), (0, 0), (1, 0)):
-        assert B.exo_gemm_validate(B.make_desc(128, 128, 64, FP32, FP32, la, lb, 0)) == B.ERR_UNSUPPORTED
+@pytest.mark.parametrize("la,lb", [(1, 1), (0, 0), (1, 0)])
+@pytest.mark.parametrize("shape", [(256, 256, 128), (300, 264, 200), (1024, 768, 520)])
+@pytest.mark.parametrize("g,bn", [(0, 0), (1, 64), (1, 128), (2, 128), (2, 256)])
+def test_tf32_operands_with_m_or_n_contiguous(la, lb, shape, g, bn):
+    # transposed 32-bit operands go through the 128-byte swizzle with 32-byte atoms
+    M, N, K = shape
+    for lc in (0, 1):
+        p = synth.Problem("tf32_mn", M, N, K, FP32, FP32, la, lb, lc, 1.5, 0.5, seed=M + K + la + 2 * lb).generate()
+        check_full(p, (flags_for(g, bn) if g else 0) | B.flag_split_k(1))
+
+
+def test_tf32_m_or_n_contiguous_on_the_tall_tile_and_in_a_batch():
+    import torch
+    p = synth.Problem("tf32_tall", 1024, 512, 264, FP32, FP32, 1, 0, 0, 1.0, 0.0, seed=6).generate()
+    cbuf, info = harness.gemm_host(p, B.flag_split_k(1), flags2=B.flag2_cta_rows(256))
+    assert info["tile_m"] == 512
+    got = oracle.logical_view(cbuf, p.M, p.N, 0, p.ldc, FP32)
+    cref, den = oracle.gemm_problem(p)
+    assert oracle.max_error(got, cref, den) <= TOL
+    bp = synth.BatchedProblem("tf32_batch", 3, 264, 328, 136, FP32, FP32, 1, 0, 0, 1.0, 0.0, seed=7).generate()
+    dev = torch.device("cuda:0")
+    dA, dB, dC = (harness._to_device(x, dev) for x in (bp.A, bp.B, bp.C))
+    with B.Plan(harness.desc_of(bp, B.flag_split_k(1)), batch=(3, bp.stride_a, bp.stride_b, bp.stride_c)) as plan:
+        plan.run(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), 1.0, 0.0, torch.cuda.current_stream(dev).cuda_stream)
+        torch.cuda.synchronize(dev)
+        plan.check()
+    out = dC.cpu().numpy().view(np.float32)
+    for i in range(3):
+        q = bp.matrix(i)
+        got = oracle.logical_view(out[i * bp.stride_c:(i + 1) * bp.stride_c], 264, 328, 0, q.ldc, FP32)
+        cref, den = oracle.gemm_problem(q)
+        assert oracle.max_error(got, cref, den) <= TOL
 
 
 def test_tf32_large_sampled():

@@ -53,6 +53,7 @@ CASES = [
     (640, 900, 320, FP16, FP32, 0, 1, 1, -1.0, 1.0, 0),                       # column-major C (operands swap)
     (768, 1536, 1024, FP16, FP16, 0, 1, 0, 1.0, 0.0, B.flag_k_subblocks(2)),  # two sub-blocks per stage
     (512, 1024, 520, FP32, FP32, 0, 1, 0, 1.0, 0.0, 0),                       # tf32 operands
+    (512, 1024, 264, FP32, FP32, 1, 0, 0, 1.0, 0.0, 0),                       # tf32, A with M contiguous: two 32-row boxes each
     (2048, 4096, 512, BF16, FP32, 0, 1, 0, 1.0, 0.0, B.flag_grid_limit(8)),   # persistent: 64 slots' worth of tiles on 2 slots
 ]
 
