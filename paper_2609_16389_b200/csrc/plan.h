@@ -199,7 +199,9 @@ inline int split_factor(int64_t tiles, int64_t workers, int64_t K, int ksub, con
   if (K < 2048 && o.split == 0) return 1;
   const int64_t k_blocks = (K + kBlockK * ksub - 1) / (kBlockK * ksub);
   int64_t f = workers / tail;
-  const int64_t by_k = (K / kBlockK) / 4;   // every slice keeps at least 256 k-elements
+  // every slice keeps at least 256 k-elements; behind whole waves at least 1024 (measured at K = 2048:
+  // three slices of 683 lose 5 % against the uncut tile, at K = 3072 three slices of 1024 win 4-7 %)
+  const int64_t by_k = (K / kBlockK) / (o.split == 0 && tiles >= workers ? 16 : 4);
   if (f > by_k) f = by_k;
   if (f > 8) f = 8;
   if (o.split >= 2 && o.split < f) f = o.split;
@@ -225,10 +227,13 @@ inline double estimate_clocks(int64_t M, int64_t N, int64_t K, int64_t batch, in
   // decode and the last store's latency do not shrink with the tile: at K = 512 the 256-column tile is
   // 20-27 % faster than two 128-column ones)
   const double drain = 1500.0 + 16.0 * bn;
-  double per_tile = mainloop > drain ? mainloop : drain;  // small K: the epilogue bounds a tile
+  // small K: the epilogue bounds a tile.  On top of either, about 2500 clocks per tile that neither hides
+  // (measured: 23.7 against 21.7 us per 64-k-block tile at 4096^3; at K = 1000 one 256-column tile beats two
+  // 128-column ones by 9-14 % where their main loops alone would tie)
+  double per_tile = (mainloop > drain ? mainloop : drain) + 2500.0;
   if (mrep == 2) {  // two accumulators per tile, less operand traffic, but the epilogue is not hidden
     mainloop = 2.0 * mainloop / kTallGain;
-    per_tile = mainloop + kTallDrain;
+    per_tile = mainloop + kTallDrain + 2.0 * 2500.0;   // it replaces two 128-row tiles and their fixed costs
   }
   const int64_t full_waves = tiles / max_workers;
   const int64_t tail = tiles % max_workers;
@@ -236,7 +241,7 @@ inline double estimate_clocks(int64_t M, int64_t N, int64_t K, int64_t batch, in
   if (tail > 0) {
     const int f = split_factor(tiles, max_workers, K, ksub, o);
     // slice + exchange of partial sums (the tall tile's partials are twice as large and nothing hides them)
-    if (f > 1) t += mainloop / f + (30.0 + 8.0 * (f - 1)) * bn * mrep * mrep;
+    if (f > 1) t += mainloop / f + 2500.0 + (30.0 + 8.0 * (f - 1)) * bn * mrep * mrep;
     else t += per_tile;
   }
   return t + drain + 3000.0;  // the last epilogue and the pipeline fill are exposed once

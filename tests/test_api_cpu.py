@@ -329,7 +329,9 @@ def test_tall_tile_flags_and_preview():
     assert info.tile_m == 256
     # the K-slices' scratch covers both accumulators of both CTAs
     st, info = B.exo_gemm_plan_preview(good(M=2560, N=3840, K=2048, flags2=TALL), 148)
-    assert (info.tail_tiles, info.split_k, info.workspace_bytes) == (1, 8, 7 * 512 * 256 * 4)
+    assert (info.tail_tiles, info.split_k, info.workspace_bytes) == (1, 2, 1 * 512 * 256 * 4)   # slices of 1024 k
+    st, info = B.exo_gemm_plan_preview(good(M=2560, N=3840, K=2048, flags2=TALL, flags=B.flag_split_k(8)), 148)
+    assert (info.tail_tiles, info.split_k, info.workspace_bytes) == (1, 8, 7 * 512 * 256 * 4)   # on request: 256 k
 
 
 def test_smoke_cases_are_in_the_supported_set():

@@ -79,7 +79,7 @@ def test_tall_tile_padding_untouched_and_nan_c_ignored_when_beta_is_zero():
         assert np.isnan(flat[i * 512 + 500:(i + 1) * 512]).all(), i
 
 
-@pytest.mark.parametrize("split", [0, 2, 5])
+@pytest.mark.parametrize("split", [0, 3, 8])
 def test_tall_tail_tiles_cut_along_k(split):
     # 5 x 15 = 75 pair tiles: one more than the 74 pairs of a B200, so one tile is cut along K
     import torch
@@ -98,7 +98,7 @@ def test_tall_tail_tiles_cut_along_k(split):
         assert oracle.max_error(got[rows, cols], cref, den) <= TOL, info
         assert oracle.freivalds(p, got) <= TOL, info
         if info["grid"] == 148:
-            assert info["tail_tiles"] == 1 and info["split_k"] == (split if split else 8)
+            assert info["tail_tiles"] == 1 and info["split_k"] == (split if split else 2)   # own choice: slices of 1024 k
             assert info["workspace_bytes"] == (info["split_k"] - 1) * 512 * 256 * 4
         for _ in range(2):   # fixed reduction order: repeated runs of the plan agree bit for bit
             dp.reset_c()
