@@ -182,25 +182,43 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
 
   if (threadIdx.x == 0) EXO_TRACE(2, 4095, 0, 4096);
   // ---------------------------------------------------------------- setup
-  if (threadIdx.x == 0) {
-    for (uint32_t s = 0; s < STAGES; ++s) {
-      ptx::mbar_init(full_bar(s), 1);
-      ptx::mbar_init(empty_bar(s), quad ? 2 : 1);  // every pair whose CTAs fill the stage releases it
+  // An epilogue warp prepares the barriers, a lane each: the producer and MMA warps spend the same time
+  // on their first work item (below), whose parameter loads and divisions would otherwise sit between
+  // the end of the setup and the first copy.
+  if (warp == 2) {
+    if (lane == 0) {
+      ptx::prefetch_tensormap(&tm_a);
+      ptx::prefetch_tensormap(&tm_b);
     }
-    for (uint32_t a = 0; a < 2; ++a) {
-      ptx::mbar_init(tfull_bar(a), 1);
-      ptx::mbar_init(tempty_bar(a), kEpiWarps * CTA_GROUP);
+    // the barrier words are consecutive: full[kMaxStages], empty[kMaxStages], tfull[2], tempty[2], C_in
+    constexpr uint32_t kBarriers = 2 * kMaxStages + 4 + kMaxEpiBufs * kEpiWarps;
+    for (uint32_t i = lane; i < kBarriers; i += 32u) {
+      uint32_t count = 1;
+      if (i >= (uint32_t)kMaxStages && i < 2u * kMaxStages) count = quad ? 2u : 1u;  // every pair whose CTAs fill the stage releases it
+      if (i >= 2u * kMaxStages + 2u && i < 2u * kMaxStages + 4u) count = kEpiWarps * CTA_GROUP;
+      ptx::mbar_init(bar0 + 8u * i, count);
     }
-    for (uint32_t w = 0; w < kEpiWarps; ++w)
-      for (uint32_t b = 0; b < kMaxEpiBufs; ++b) ptx::mbar_init(cin_bar(w, b), 1);
     ptx::fence_mbar_init();
-    ptx::prefetch_tensormap(&tm_a);
-    ptx::prefetch_tensormap(&tm_b);
-    ptx::prefetch_tensormap(&tm_c);
+    if (lane == 0) ptx::prefetch_tensormap(&tm_c);
   }
   if (warp == 1) {
     ptx::tmem_alloc<CTA_GROUP>(tmem_slot, TMEM_COLS);
     ptx::tmem_relinquish<CTA_GROUP>();
+  }
+  // The first work item depends on kernel parameters only, so the warps that need it first compute it
+  // while the barriers are being set up (the epilogue warps need theirs a whole main loop later).
+  const bool batched = p.batch > 1;
+  auto tile_coord = [&](int64_t t, uint32_t* bz) {
+    *bz = batched ? (uint32_t)t / p.tiles_per_batch : 0u;  // which matrix of the batch
+    return raster_decode(p.raster, batched ? (uint32_t)t - *bz * p.tiles_per_batch : t);
+  };
+  WorkItem wi_first{};
+  TileCoord tc_first{};
+  uint32_t bz_first = 0;
+  bool have_first = false;
+  if (warp < 2 || warp == (uint32_t)kProducerBWarp) {
+    have_first = work_item(p.work, worker, num_workers, 0, nkb, &wi_first);
+    if (have_first && warp != 1) tc_first = tile_coord(wi_first.tile, &bz_first);
   }
   ptx::tc_fence_before_sync();
   __syncthreads();
@@ -216,7 +234,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   // dependent launch it overlaps the tail of the previous kernel in the stream.  From here on global
   // memory is read and written: wait for that kernel, then let our own successor start likewise.
   ptx::grid_dependency_wait();
-  ptx::grid_launch_dependents();
+  if (warp == 2) ptx::grid_launch_dependents();  // one warp speaks for the CTA; not one that is in a hurry
 
   bool ok = true;
   if (threadIdx.x == 0) EXO_TRACE(2, 4094, 0, 4096);
@@ -232,12 +250,16 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     // in a pair, both CTAs' loads are counted on the leader's full barrier
     const uint32_t full0 = PAIR ? ptx::map_to_cta(full_bar(0), leader) : full_bar(0);
     for (int64_t it = 0; ok; ++it) {
-      WorkItem wi;
-      if (!work_item(p.work, worker, num_workers, it, nkb, &wi)) break;
+      WorkItem wi = wi_first;
+      TileCoord tc = tc_first;
+      uint32_t bz = bz_first;
+      if (it == 0) {
+        if (!have_first) break;
+      } else {
+        if (!work_item(p.work, worker, num_workers, it, nkb, &wi)) break;
+        tc = tile_coord(wi.tile, &bz);
+      }
       const int64_t t = wi.tile;
-      const bool batched = p.batch > 1;
-      const uint32_t bz = batched ? (uint32_t)t / p.tiles_per_batch : 0u;  // which matrix of the batch
-      const TileCoord tc = raster_decode(p.raster, batched ? (uint32_t)t - bz * p.tiles_per_batch : t);
       const int32_t a_mn0 = tc.m * (CTA_M * CTA_GROUP) + (int32_t)cta_rank * CTA_M;
       const int32_t b_mn0 = (tc.n * NPAIR + (int32_t)pair_id) * BN + (int32_t)cta_rank * B_ROWS;
       for (int32_t kb = wi.kb_begin; kb < wi.kb_end; ++kb) {
@@ -378,8 +400,12 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         }
       };
       for (int64_t it = 0; ok; ++it) {
-        WorkItem wi;
-        if (!work_item(p.work, worker, num_workers, it, nkb, &wi)) break;
+        WorkItem wi = wi_first;
+        if (it == 0) {
+          if (!have_first) break;
+        } else if (!work_item(p.work, worker, num_workers, it, nkb, &wi)) {
+          break;
+        }
         const int64_t t = wi.tile;
         if constexpr (MREP == 1) {
           // the epilogue (of both CTAs) must have drained this accumulator
@@ -452,9 +478,8 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       WorkItem wi;
       if (!work_item(p.work, worker, num_workers, it, nkb, &wi)) break;
       const int64_t t = wi.tile;
-      const bool batched = p.batch > 1;
-      const uint32_t bz = batched ? (uint32_t)t / p.tiles_per_batch : 0u;
-      const TileCoord tc = raster_decode(p.raster, batched ? (uint32_t)t - bz * p.tiles_per_batch : t);
+      uint32_t bz;
+      const TileCoord tc = tile_coord(t, &bz);
       const int32_t col0 = (tc.n * NPAIR + (int32_t)pair_id) * BN;
       // one pass per accumulator of the tile: a single one, or (tall tile) rows 0..127 then 128..255 of the CTA
 #pragma unroll 1
@@ -687,9 +712,11 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   }
 
   // ---------------------------------------------------------------- teardown
-  if (*(volatile uint32_t*)p.status != kStatusOk) {
-    // Some wait was abandoned: give copies and MMAs still in flight time to land
-    // before shared and tensor memory are released.
+  if (!ok) {
+    // This thread abandoned a wait: give copies and MMAs still in flight time to land before shared
+    // and tensor memory are released.  (Every thread that gives up passes here with ok == false, and
+    // the barriers below hold the rest of the CTA and of the cluster back until it has slept; reading
+    // the status word from global memory instead would put a memory round trip on every CTA's exit.)
     for (int i = 0; i < 200; ++i) __nanosleep(1000);
   }
   ptx::tc_fence_before_sync();
