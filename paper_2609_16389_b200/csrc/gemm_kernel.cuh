@@ -205,6 +205,10 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     ptx::tmem_alloc<CTA_GROUP>(tmem_slot, TMEM_COLS);
     ptx::tmem_relinquish<CTA_GROUP>();
   }
+  // Arrive at the cluster barrier as early as possible (a warp's arrival follows its own share of the
+  // setup and publishes it) and wait as late as possible: the barrier's latency then overlaps the
+  // first work item's arithmetic instead of following it.
+  if constexpr (PAIR) ptx::cluster_arrive();
   // The first work item depends on kernel parameters only, so the warps that need it first compute it
   // while the barriers are being set up (the epilogue warps need theirs a whole main loop later).
   const bool batched = p.batch > 1;
@@ -222,19 +226,16 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   }
   ptx::tc_fence_before_sync();
   __syncthreads();
-  if constexpr (PAIR) {  // peer barriers must be initialised before anything remote touches them
-    ptx::cluster_arrive();
-    ptx::cluster_wait();
-  }
+  if constexpr (PAIR) ptx::cluster_wait();  // peer barriers and tensor memory exist before anything remote touches them
   ptx::tc_fence_after_sync();
   uint32_t tmem_base;
   asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot) : "memory");
 
   // Everything above touched only this CTA's shared and tensor memory, so with programmatic
-  // dependent launch it overlaps the tail of the previous kernel in the stream.  From here on global
-  // memory is read and written: wait for that kernel, then let our own successor start likewise.
-  ptx::grid_dependency_wait();
-  if (warp == 2) ptx::grid_launch_dependents();  // one warp speaks for the CTA; not one that is in a hurry
+  // dependent launch it overlaps the tail of the previous kernel in the stream.  Each role waits for
+  // that kernel itself, as late as it can: the copying lanes right before their first copy, the
+  // epilogue warps before they first touch C or the split workspace; the MMA warp never touches
+  // global memory.
 
   bool ok = true;
   if (threadIdx.x == 0) EXO_TRACE(2, 4094, 0, 4096);
@@ -270,6 +271,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         if (ptx::elect_one()) {
           EXO_TRACE(0, issued, 0, 4096);
           if (cta_rank == 0 && do_a) ptx::mbar_arrive_expect_tx(full_bar(s), STAGE_BYTES * CTA_GROUP);
+          if (issued == 0) ptx::grid_dependency_wait();  // the operands may be the previous kernel's output
           if (!skip) {
             const uint32_t a_dst = stage0 + s * STAGE_BYTES;
             const uint32_t b_dst = a_dst + A_BYTES;
@@ -457,6 +459,8 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     // Warp w reads TMEM lanes 32*(w%4)..+31 (a hardware rule) and, of the tile's column
     // chunks (128 bytes of C per row each), those with index == half (mod 2).
     constexpr int UPC = CW / 32;                       // 32-column TMEM loads per chunk
+    if (warp == 2) ptx::grid_launch_dependents();      // one warp speaks for the CTA: our own successor may start likewise
+    ptx::grid_dependency_wait();                       // C and the split workspace may still be in use by the previous kernel
     const uint32_t quad = warp & 3u;
     const uint32_t ew = warp - 2u;
     const int32_t half = (int32_t)(ew >> 2);
