@@ -314,7 +314,10 @@ int64_t exo_gemm_schedule_enumerate(int32_t tiles_m, int32_t tiles_n, int32_t ba
  * tail tiles (the paper's Section 6 measures split-K variants of its GEMM against
  * wave quantisation; here only the tiles of the partial last wave are cut, into
  * `split` slices each, slice 0 owning the output and taking `owner_extra` k-blocks
- * more than an even share).  `tiles` tiles, `num_workers` workers; writes tile index, slice and k-block range [begin, end) of
+ * more than an even share).  The items come in the order the worker executes them:
+ * a contributing slice (slice > 0) before the worker's whole tiles, the owning slice
+ * after them, so that the partial sums are in memory before the owner needs them.
+ * `tiles` tiles, `num_workers` workers; writes tile index, slice and k-block range [begin, end) of
  * `num_k_blocks` per item (capacity `cap`); returns the item count, or -1 on bad
  * arguments (including tail_tiles * split > num_workers).  Needs no GPU.
  */

@@ -162,8 +162,10 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   auto tfull_bar = [&](uint32_t a) { return bar0 + 8u * (2 * kMaxStages + a); };
   auto tempty_bar = [&](uint32_t a) { return bar0 + 8u * (2 * kMaxStages + 2 + a); };
   auto cin_bar = [&](uint32_t w, uint32_t b) { return bar0 + 8u * (2 * kMaxStages + 4 + kMaxEpiBufs * w + b); };
-  const uint32_t tmem_slot = bar0 + 8u * (2 * kMaxStages + 4 + kMaxEpiBufs * kEpiWarps);
-  static_assert(8 * (2 * kMaxStages + 4 + kMaxEpiBufs * kEpiWarps) + 4 <= kBarrierBytes, "barrier area");
+  // "the accumulator of the owning slice holds the other slices' sum": used at most once per launch
+  const uint32_t tfilled_bar = bar0 + 8u * (2 * kMaxStages + 4 + kMaxEpiBufs * kEpiWarps);
+  const uint32_t tmem_slot = tfilled_bar + 8u;
+  static_assert(8 * (2 * kMaxStages + 5 + kMaxEpiBufs * kEpiWarps) + 4 <= kBarrierBytes, "barrier area");
 
   const uint32_t warp = threadIdx.x >> 5;
   const uint32_t lane = threadIdx.x & 31u;
@@ -190,12 +192,12 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       ptx::prefetch_tensormap(&tm_a);
       ptx::prefetch_tensormap(&tm_b);
     }
-    // the barrier words are consecutive: full[kMaxStages], empty[kMaxStages], tfull[2], tempty[2], C_in
-    constexpr uint32_t kBarriers = 2 * kMaxStages + 4 + kMaxEpiBufs * kEpiWarps;
+    // the barrier words are consecutive: full[kMaxStages], empty[kMaxStages], tfull[2], tempty[2], C_in, tfilled
+    constexpr uint32_t kBarriers = 2 * kMaxStages + 5 + kMaxEpiBufs * kEpiWarps;
     for (uint32_t i = lane; i < kBarriers; i += 32u) {
       uint32_t count = 1;
       if (i >= (uint32_t)kMaxStages && i < 2u * kMaxStages) count = quad ? 2u : 1u;  // every pair whose CTAs fill the stage releases it
-      if (i >= 2u * kMaxStages + 2u && i < 2u * kMaxStages + 4u) count = kEpiWarps * CTA_GROUP;
+      if ((i >= 2u * kMaxStages + 2u && i < 2u * kMaxStages + 4u) || i == kBarriers - 1u) count = kEpiWarps * CTA_GROUP;
       ptx::mbar_init(bar0 + 8u * i, count);
     }
     ptx::fence_mbar_init();
@@ -409,11 +411,19 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
           break;
         }
         const int64_t t = wi.tile;
+        // The owning slice of a tail tile that follows at least two whole tiles starts from an accumulator
+        // into which the epilogue warps have already written the other slices' partial sums.
+        const bool preloaded = MREP == 1 && wi.slices > 1 && wi.slice == 0 && it >= 2;
         if constexpr (MREP == 1) {
           // the epilogue (of both CTAs) must have drained this accumulator
           ok = wait_barrier<PAIR>(tempty_bar(acc), acc_ph ^ 1u, p, WaitSite{kRoleMma, 100 + acc, (uint32_t)t, 0});
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
+          if (preloaded) {  // ... and have filled it again (a barrier of its own: this happens once per launch)
+            ok = wait_barrier<PAIR>(tfilled_bar, 0u, p, WaitSite{kRoleMma, 110 + acc, (uint32_t)t, 0});
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+          }
           ptx::tc_fence_after_sync();
         }
         for (int32_t kb = wi.kb_begin; kb < wi.kb_end; ++kb) {
@@ -440,7 +450,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             if (ptx::elect_one()) {  // the same lane every time: commits track this thread's MMAs
               if (r == 0) EXO_TRACE(1, consumed, 0, 4096);
               // the second 128-row block of A lies 16 KB after the first in every staging layout
-              issue_stage(tmem_base + a_acc * BN, a_desc + (uint64_t)(r * (kATileBytes >> 4)), b_desc, first_kb, k_left);
+              issue_stage(tmem_base + a_acc * BN, a_desc + (uint64_t)(r * (kATileBytes >> 4)), b_desc, first_kb && !preloaded, k_left);
               if (r == MREP - 1) ptx::umma_commit<CTA_GROUP>(empty_bar(s), kStageMask);  // stage free once these MMAs completed
               if (last_kb) ptx::umma_commit<CTA_GROUP>(tfull_bar(a_acc), pair_mask);      // accumulator complete
               if (r == MREP - 1) EXO_TRACE(1, consumed, 1, 4096);
@@ -470,13 +480,66 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     const bool has_acc = nkb > 0;
     const bool scale = p.alpha != 1.f;
     const float alpha = p.alpha, beta = p.beta;
-    uint32_t piece[8];  // where this thread's eight 16-byte pieces of a 128-byte row go (swizzled)
-#pragma unroll
-    for (int j = 0; j < 8; ++j) piece[j] = buf0 + lane * 128u + (((uint32_t)j ^ (lane & 7u)) << 4);
+    // where this thread's j-th 16-byte piece of a 128-byte row goes (swizzled); recomputed at every use:
+    // eight precomputed addresses would be eight registers held across the whole role
+    const uint32_t my_row = buf0 + lane * 128u, my_xor = (lane & 7u) << 4;
+    auto piece = [&](int j) { return my_row + (((uint32_t)j << 4) ^ my_xor); };
     // running chunk counter: staging buffer g % EPI_BUFS, its C_in barrier phase (g / EPI_BUFS) & 1
     uint32_t g = 0;
     const bool two_bufs = EPI_BUFS == 2;
     uint32_t acc = 0, acc_ph = 0;
+
+    // Partial accumulators of the K-slices of a tail tile travel through a private fp32 workspace in a
+    // layout where a warp's 16-byte pieces are contiguous (coalesced both ways): [tail tile][slice-1]
+    // [cta][warp][accumulator][chunk][unit][piece][lane]; a unit is 32 lanes x 32 columns x 4 bytes.
+    constexpr uint32_t kUnitBytes = 8u * 512u;
+    auto ws_addr = [&](const WorkItem& w, int32_t slice_m1, int32_t r, int32_t i, int32_t q) {
+      const uint64_t idx = ((((uint64_t)w.tail_index * (uint32_t)(w.slices - 1) + (uint32_t)slice_m1) * CLUSTER +
+                             slot_rank) * kEpiWarps + ew) * (uint32_t)(MREP * ((NCHUNK + 1) / 2) * UPC) +
+                           (uint32_t)((r * ((NCHUNK + 1) / 2) + i) * UPC + q);
+      return reinterpret_cast<char*>(p.split_ws) + idx * kUnitBytes + lane * 16u;
+    };
+    // how many of a tile's column chunks are this warp's, given the tile and the warp's first row
+    auto chunks_of = [&](int32_t row0, int32_t col0) {
+      int32_t nch = 0;  // chunks of the tile that hold any valid column, if this warp's rows exist
+      if (row0 < p.M) {
+        nch = (p.N - col0 + CW - 1) / CW;
+        if (nch > NCHUNK) nch = NCHUNK;
+      }
+      return nch > half ? (nch - half + 1) / 2 : 0;
+    };
+    // Bounded wait until every warp of every contributing slice of a tail tile has delivered its
+    // partials.  One lane polls, with a pause between polls: this can run beside a main loop, whose
+    // copy-issuing warps share the instruction issue slots and the memory pipeline with this warp.
+    auto wait_partials = [&](const WorkItem& w, int32_t r) {
+      const uint32_t* flag = p.split_flags + w.tail_index * NPAIR + (int32_t)pair_id;
+      const long long t_start = clock64();
+      uint32_t spins = 0;
+      for (;;) {
+        bool ready = lane == 0 && (int32_t)(ptx::ld_acquire_gpu(flag) - p.split_target) >= 0;
+        ready = __shfl_sync(0xffffffffu, ready, 0);
+        if (ready) {
+          (void)ptx::ld_acquire_gpu(flag);  // every lane orders its own reads of the partials after the counter
+          return true;
+        }
+        __nanosleep(200);
+        if ((++spins & 63u) == 0u) {
+          bool give_up = *(volatile uint32_t*)p.status != kStatusOk;
+          if (!give_up && (uint64_t)(clock64() - t_start) > p.timeout_cycles) {
+            if (atomicCAS(p.status, (uint32_t)kStatusOk, (uint32_t)kStatusTimeout) == kStatusOk) {
+              p.status[1] = kRoleEpiloguePartials;
+              p.status[2] = (uint32_t)w.tail_index;
+              p.status[3] = (uint32_t)w.tile;
+              p.status[4] = (uint32_t)r;
+              p.status[5] = blockIdx.x;
+              __threadfence();
+            }
+            give_up = true;
+          }
+          if (__any_sync(0xffffffffu, give_up)) return false;
+        }
+      }
+    };
 
     for (int64_t it = 0;; ++it) {
       WorkItem wi;
@@ -485,17 +548,64 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       uint32_t bz;
       const TileCoord tc = tile_coord(t, &bz);
       const int32_t col0 = (tc.n * NPAIR + (int32_t)pair_id) * BN;
+      if constexpr (MREP == 1) {
+        // If this worker's next (and last) item is the owning slice of a tail tile and at least one whole
+        // tile came before this one, the other slices' partial sums were published a whole tile's time
+        // ago (contributing slices are computed first).  Write their sum into that item's accumulator
+        // now, while this item's main loop runs: the MMA warp then accumulates on top of it and the
+        // owner's epilogue is an ordinary one.  (With a single whole tile before the slice the partials
+        // arrive too late for that; the owner then adds them in its epilogue.)
+        WorkItem nx;
+        if (it >= 1 && work_item(p.work, worker, num_workers, it + 1, nkb, &nx) && nx.slices > 1 && nx.slice == 0) {
+          uint32_t bz2;
+          const TileCoord tc2 = tile_coord(nx.tile, &bz2);
+          const int32_t n_mine = chunks_of(tc2.m * (CTA_M * CTA_GROUP) + (int32_t)cta_rank * CTA_M + (int32_t)quad * 32,
+                                           (tc2.n * NPAIR + (int32_t)pair_id) * BN);
+          if (n_mine > 0) {
+            ok = wait_partials(nx, 0);
+            if (!ok) break;
+            const uint32_t tnext = tmem_base + ((quad * 32u) << 16) + (acc ^ 1u) * BN;
+#pragma unroll 1
+            for (int32_t u = 0; u < n_mine * UPC * 2; ++u) {  // 16 columns at a time and rolled: this runs
+              // beside a main loop and must not raise the kernel's register count
+              const int32_t i = u / (UPC * 2), q = (u / 2) % UPC, h = u & 1;
+              uint32_t sum[16];
+              for (int32_t sm1 = 0; sm1 < nx.slices - 1; ++sm1) {  // in slice order
+                const char* src = ws_addr(nx, sm1, 0, i, q) + h * 2048;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  uint32_t a0, a1, a2, a3;
+                  ptx::ld_global_cg_v4(src + j * 512, a0, a1, a2, a3);
+                  if (sm1 == 0) {
+                    sum[4 * j + 0] = a0; sum[4 * j + 1] = a1; sum[4 * j + 2] = a2; sum[4 * j + 3] = a3;
+                  } else {
+                    sum[4 * j + 0] = __float_as_uint(__uint_as_float(sum[4 * j + 0]) + __uint_as_float(a0));
+                    sum[4 * j + 1] = __float_as_uint(__uint_as_float(sum[4 * j + 1]) + __uint_as_float(a1));
+                    sum[4 * j + 2] = __float_as_uint(__uint_as_float(sum[4 * j + 2]) + __uint_as_float(a2));
+                    sum[4 * j + 3] = __float_as_uint(__uint_as_float(sum[4 * j + 3]) + __uint_as_float(a3));
+                  }
+                }
+              }
+              ptx::tmem_st_32x16(tnext + (uint32_t)((half + 2 * i) * CW + q * 32 + h * 16), sum);
+            }
+            ptx::tmem_st_wait();
+          }
+          // every epilogue warp of the CTA group reports "filled" to the MMA-issuing CTA
+          ptx::tc_fence_before_sync();
+          __syncwarp();
+          if (ptx::elect_one()) {
+            if constexpr (PAIR) ptx::mbar_arrive_cluster(ptx::map_to_cta(tfilled_bar, leader));
+            else ptx::mbar_arrive(tfilled_bar);
+          }
+        }
+      }
+      const bool preloaded = MREP == 1 && wi.slices > 1 && wi.slice == 0 && it >= 2;  // see above
       // one pass per accumulator of the tile: a single one, or (tall tile) rows 0..127 then 128..255 of the CTA
 #pragma unroll 1
       for (int32_t r = 0; r < MREP; ++r) {
       const uint32_t cur = MREP == 1 ? acc : (uint32_t)r;
       const int32_t row0 = tc.m * (CTA_M * CTA_GROUP) + (int32_t)cta_rank * CTA_M + r * kBlockM + (int32_t)quad * 32;
-      int32_t nch = 0;  // chunks of this tile that hold any valid column, if this warp's rows exist
-      if (row0 < p.M) {
-        nch = (p.N - col0 + CW - 1) / CW;
-        if (nch > NCHUNK) nch = NCHUNK;
-      }
-      const int32_t mine = nch > half ? (nch - half + 1) / 2 : 0;  // how many of them are this warp's
+      const int32_t mine = chunks_of(row0, col0);  // how many of the tile's chunks are this warp's
       if (has_acc) {
         ok = wait_barrier<PAIR>(tfull_bar(cur), acc_ph, p, WaitSite{kRoleEpilogue, 200 + cur, (uint32_t)t, 0});
         ok = __all_sync(0xffffffffu, ok);
@@ -519,31 +629,21 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       if (mine == 0 && has_acc) release_acc();
 
       // ---- a slice of a tail tile (the tile's K range is cut into wi.slices parts)
-      // Partial accumulators travel through a private fp32 workspace in a layout where a warp's
-      // 16-byte pieces are contiguous (coalesced both ways): [tail tile][slice-1][cta][warp][chunk]
-      // [unit][piece][lane].
-      constexpr uint32_t kUnitBytes = 8u * 512u;  // 32 lanes x 32 columns x 4 bytes
       const bool contributor = wi.slices > 1 && wi.slice != 0;
-      const bool owner = wi.slices > 1 && wi.slice == 0;
-      auto ws_unit = [&](int32_t slice_m1, int32_t i, int32_t q) {
-        const uint64_t idx = ((((uint64_t)wi.tail_index * (uint32_t)(wi.slices - 1) + (uint32_t)slice_m1) * CLUSTER +
-                               slot_rank) * kEpiWarps + ew) * (uint32_t)(MREP * ((NCHUNK + 1) / 2) * UPC) +
-                             (uint32_t)((r * ((NCHUNK + 1) / 2) + i) * UPC + q);
-        return reinterpret_cast<char*>(p.split_ws) + idx * kUnitBytes + lane * 16u;
-      };
+      const bool owner = wi.slices > 1 && wi.slice == 0 && !preloaded;  // has to add the partials itself
       if (contributor) {
         // raw accumulators out, then one arrival per warp on the tile's counter
         for (int32_t i = 0; i < mine; ++i) {
 #pragma unroll
           for (int32_t q = 0; q < UPC; ++q) {
-            uint32_t r[32];
-            tmem_load(r, i, q);
+            uint32_t raw[32];
+            tmem_load(raw, i, q);
             ptx::tmem_ld_wait();
             if (i + 1 == mine && q == UPC - 1) release_acc();
-            char* dst = ws_unit(wi.slice - 1, i, q);
+            char* dst = ws_addr(wi, wi.slice - 1, r, i, q);
 #pragma unroll
             for (int j = 0; j < 8; ++j)
-              ptx::st_global_v4(dst + j * 512, r[4 * j + 0], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+              ptx::st_global_v4(dst + j * 512, raw[4 * j + 0], raw[4 * j + 1], raw[4 * j + 2], raw[4 * j + 3]);
           }
         }
         __threadfence();  // each lane's partials are visible GPU-wide before the arrival below
@@ -552,29 +652,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         continue;
       }
       if (owner && mine > 0) {
-        // wait (bounded) until every warp of every other slice has delivered its partials
-        const uint32_t* flag = p.split_flags + wi.tail_index * NPAIR + (int32_t)pair_id;
-        const long long t_start = clock64();
-        uint32_t spins = 0;
-        for (;;) {
-          const bool ready = (int32_t)(ptx::ld_acquire_gpu(flag) - p.split_target) >= 0;
-          if (__all_sync(0xffffffffu, ready)) break;
-          if ((++spins & 63u) == 0u) {
-            bool give_up = *(volatile uint32_t*)p.status != kStatusOk;
-            if (!give_up && (uint64_t)(clock64() - t_start) > p.timeout_cycles) {
-              if (atomicCAS(p.status, (uint32_t)kStatusOk, (uint32_t)kStatusTimeout) == kStatusOk) {
-                p.status[1] = kRoleEpiloguePartials;
-                p.status[2] = (uint32_t)wi.tail_index;
-                p.status[3] = (uint32_t)t;
-                p.status[4] = 0;
-                p.status[5] = blockIdx.x;
-                __threadfence();
-              }
-              give_up = true;
-            }
-            if (__any_sync(0xffffffffu, give_up)) { ok = false; break; }
-          }
-        }
+        ok = wait_partials(wi, r);
         if (!ok) break;
       }
       auto issue_cin = [&](uint32_t gg, int32_t i) {  // elected lane only: C_in of this warp's i-th chunk
@@ -637,7 +715,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             }
             if (owner) {  // add the other slices' partial sums, in slice order
               for (int32_t sm1 = 0; sm1 < wi.slices - 1; ++sm1) {
-                const char* src = ws_unit(sm1, i, q);
+                const char* src = ws_addr(wi, sm1, r, i, q);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                   uint32_t a0, a1, a2, a3;
@@ -659,18 +737,18 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                 for (int j = 0; j < 8; ++j) {
                   if (has_beta) {
                     uint32_t c0, c1, c2, c3;
-                    ptx::ld_shared_v4(piece[j] + boff, c0, c1, c2, c3);
+                    ptx::ld_shared_v4(piece(j) + boff, c0, c1, c2, c3);
                     cur[4 * j + 0] = __float_as_uint(fmaf(beta, __uint_as_float(c0), __uint_as_float(cur[4 * j + 0])));
                     cur[4 * j + 1] = __float_as_uint(fmaf(beta, __uint_as_float(c1), __uint_as_float(cur[4 * j + 1])));
                     cur[4 * j + 2] = __float_as_uint(fmaf(beta, __uint_as_float(c2), __uint_as_float(cur[4 * j + 2])));
                     cur[4 * j + 3] = __float_as_uint(fmaf(beta, __uint_as_float(c3), __uint_as_float(cur[4 * j + 3])));
                   }
-                  ptx::st_shared_v4(piece[j] + boff, cur[4 * j + 0], cur[4 * j + 1], cur[4 * j + 2], cur[4 * j + 3]);
+                  ptx::st_shared_v4(piece(j) + boff, cur[4 * j + 0], cur[4 * j + 1], cur[4 * j + 2], cur[4 * j + 3]);
                 }
               } else {
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {  // 32 columns = four 16-byte pieces of 8 halves
-                  const uint32_t addr = piece[4 * q + j] + boff;
+                  const uint32_t addr = piece(4 * q + j) + boff;
                   float x[8];
 #pragma unroll
                   for (int k = 0; k < 8; ++k) x[k] = __uint_as_float(cur[8 * j + k]);

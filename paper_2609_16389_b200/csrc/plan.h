@@ -193,15 +193,23 @@ inline int split_factor(int64_t tiles, int64_t workers, int64_t K, int ksub, con
   const int64_t tail = tiles % workers;
   if (tail == 0 || o.split == 1 || o.no_workspace) return 1;
   // A short K loop leaves no main-loop time to save, and the exchange of partial sums (a round trip
-  // through L2 plus the extra output traffic) costs about as much as a dozen k-blocks.  Measured: behind
-  // whole waves at K = 512 the split is 20-27 % slower; for problems smaller than one wave it loses 28 % at
-  // K = 512 and 3 % at K = 1000, and wins 13-35 % from K = 2048 on.
-  if (K < 2048 && o.split == 0) return 1;
+  // through L2 plus the extra output traffic) costs about as much as a dozen k-blocks.
+  // Behind whole waves the contributing slices run first and the exchange is off the critical path
+  // except for the owner's reading.  Measured there (one whole wave + 22 tiles of 256 x 256 on 74 pairs,
+  // against the uncut tiles): two slices -19 % at K = 512, +3 to +5 % at K = 1000 and 1536, +7 to +8 % at
+  // 2048, +8 to +10 % at 4096; three slices 0 %, -1 to -4 %, +4 to +5 %, +7 to +9 %: a further slice pays
+  // only where it still keeps 2048 k-elements.
+  // Problems smaller than one wave run all slices side by side and the owner waits for the others:
+  // the split loses 28 % at K = 512 and 3 % at K = 1000, and wins 13-35 % from K = 2048 on.
+  // (With three or more whole waves in front, the workers that start with a slice run out of step with
+  // the rest for longer than the shorter last wave saves at K = 1024: -0.7 % at 4096 x 4096 x 1024.)
+  const bool behind_waves = tiles >= workers;
+  if (o.split == 0 && K < (behind_waves && tiles / workers <= 2 ? 960 : 2048)) return 1;
   const int64_t k_blocks = (K + kBlockK * ksub - 1) / (kBlockK * ksub);
   int64_t f = workers / tail;
-  // every slice keeps at least 256 k-elements; behind whole waves at least 1024 (measured at K = 2048:
-  // three slices of 683 lose 5 % against the uncut tile, at K = 3072 three slices of 1024 win 4-7 %)
-  const int64_t by_k = (K / kBlockK) / (o.split == 0 && tiles >= workers ? 16 : 4);
+  // every slice keeps at least 256 k-elements
+  int64_t by_k = (K / kBlockK) / 4;
+  if (o.split == 0 && behind_waves) by_k = K / 2048 > 2 ? K / 2048 : 2;
   if (f > by_k) f = by_k;
   if (f > 8) f = 8;
   if (o.split >= 2 && o.split < f) f = o.split;
@@ -240,8 +248,11 @@ inline double estimate_clocks(int64_t M, int64_t N, int64_t K, int64_t batch, in
   double t = (double)full_waves * per_tile;
   if (tail > 0) {
     const int f = split_factor(tiles, max_workers, K, ksub, o);
-    // slice + exchange of partial sums (the tall tile's partials are twice as large and nothing hides them)
-    if (f > 1) t += mainloop / f + 2500.0 + (30.0 + 8.0 * (f - 1)) * bn * mrep * mrep;
+    // slice + exchange of partial sums (the tall tile's partials are twice as large and nothing hides them).
+    // Behind whole waves only the owner's reading of the partials is exposed (about 4000 clocks per
+    // contributing slice of a 256-column tile); side by side, publishing and the round trip are as well.
+    const double exchange = (full_waves > 0 ? 16.0 * (f - 1) : 30.0 + 8.0 * (f - 1)) * bn * mrep * mrep;
+    if (f > 1) t += mainloop / f + 2500.0 + exchange;
     else t += per_tile;
   }
   return t + drain + 3000.0;  // the last epilogue and the pipeline fill are exposed once
@@ -307,11 +318,13 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
     const int64_t k_scaled = c.K * (c.ab_bytes / 2);  // in 16-bit-element units: 64 per sub-block
     const int64_t k_blocks = (k_scaled + kBlockK * cfg.ksub - 1) / (kBlockK * cfg.ksub);
     cfg.split = split_factor(tiles, workers, k_scaled, cfg.ksub, o);
-    // Publishing a 128 x N fp32 partial takes a contributor about as long as 8 k-blocks of 64
-    // (128*N*4 bytes at ~30 B/clk against 2*N clocks of MMA per k-block); let the owner compute that
-    // much longer, so that the partials are there when it finishes.
+    // Behind whole waves the contributing slices are computed first and the owning slice last, so the
+    // partials are in memory long before they are asked for and K is cut evenly.  In a problem of less
+    // than one wave all slices run side by side: publishing a 128 x N fp32 partial takes a contributor
+    // about as long as 8 k-blocks of 64 (128*N*4 bytes at ~30 B/clk against 2*N clocks of MMA per
+    // k-block), so there the owner computes that much longer.
     cfg.owner_extra = 0;
-    if (cfg.split > 1) {
+    if (cfg.split > 1 && cfg.full_tiles == 0) {
       int64_t extra = 8 / cfg.ksub;
       const int64_t room = k_blocks / cfg.split - 1;   // every other slice keeps at least one k-block
       if (extra > room / 2) extra = room / 2;

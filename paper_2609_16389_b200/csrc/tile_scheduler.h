@@ -82,22 +82,32 @@ struct WorkItem {
 };
 
 // The i-th work item of `worker`; returns false when the worker has no i-th item.
+// A worker whose unit of a tail tile is a contributing slice (slice > 0) computes that unit FIRST and
+// its whole tiles afterwards: its partial sums then reach memory a whole tile's time before the owning
+// slice (slice 0, computed LAST by its worker) asks for them, and neither side ever waits.
+// The owners are workers 0 .. tail_tiles-1 and the contributors the workers after them: a worker that
+// starts with a slice stays out of step with the others for the whole launch, and tiles that run in step
+// share their operand panels in L2, so each group is kept contiguous in the tile order.
 EXO_HD bool work_item(const WorkPlan& w, int64_t worker, int64_t num_workers, int64_t i, int32_t num_k_blocks,
                       WorkItem* out) {
-  const int64_t t = worker + i * num_workers;
-  if (t < w.full_tiles) {
-    out->tile = t;
-    out->tail_index = -1;
-    out->slice = 0;
-    out->slices = 1;
-    out->kb_begin = 0;
-    out->kb_end = num_k_blocks;
-    return true;
+  const bool has_unit = worker < (int64_t)w.tail_tiles * w.split;
+  const bool early = has_unit && worker >= w.tail_tiles;  // a contributing slice (split > 1 follows)
+  if (!(early && i == 0)) {
+    const int64_t t = worker + (early ? i - 1 : i) * num_workers;
+    if (t < w.full_tiles) {
+      out->tile = t;
+      out->tail_index = -1;
+      out->slice = 0;
+      out->slices = 1;
+      out->kb_begin = 0;
+      out->kb_end = num_k_blocks;
+      return true;
+    }
+    if (early || !has_unit) return false;
+    if (t - w.full_tiles != worker) return false;           // only the wave right after the full ones
   }
-  if (t - w.full_tiles != worker) return false;             // only the wave right after the full ones
-  if (worker >= (int64_t)w.tail_tiles * w.split) return false;
-  const int32_t ti = (int32_t)((uint32_t)worker / (uint32_t)w.split);
-  const int32_t sl = (int32_t)((uint32_t)worker - (uint32_t)ti * (uint32_t)w.split);
+  const int32_t sl = (int32_t)((uint32_t)worker / (uint32_t)w.tail_tiles);
+  const int32_t ti = (int32_t)((uint32_t)worker - (uint32_t)sl * (uint32_t)w.tail_tiles);
   out->tile = w.full_tiles + ti;
   out->tail_index = w.split > 1 ? ti : -1;
   out->slice = sl;

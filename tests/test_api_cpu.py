@@ -219,6 +219,24 @@ def test_work_schedule_covers_every_tile_and_k_block_exactly_once(tiles, workers
     assert longest == -(-tiles // workers)      # nobody does more items than the wave count
 
 
+def test_contributing_slices_come_first_and_owning_slices_last():
+    # 256 tiles on 74 workers, tail tiles cut in two: workers 0..33 own a tail tile and compute their
+    # slice after their whole tiles; workers 34..67 contribute and compute theirs before; the rest have none
+    tiles, workers, split, nkb = 256, 74, 2, 64
+    full = (tiles // workers) * workers
+    for w in range(workers):
+        items = B.exo_gemm_schedule_work(tiles, workers, split, nkb, w, 0)
+        unit = [k for k, (tile, sl, b, e) in enumerate(items) if tile >= full]
+        if w < 34:
+            assert unit == [len(items) - 1] and items[-1][:2] == (full + w, 0) and items[-1][2:] == (0, 32)
+        elif w < 68:
+            assert unit == [0] and items[0][:2] == (full + w - 34, 1) and items[0][2:] == (32, 64)
+        else:
+            assert unit == []
+        whole = [tile for tile, sl, b, e in items if tile < full]
+        assert whole == [w + k * workers for k in range(3)]
+
+
 def test_work_schedule_rejects_impossible_splits():
     with pytest.raises(ValueError):
         B.exo_gemm_schedule_work(256, 74, 3, 64, 0)      # 34 tail tiles x 3 slices > 74 workers

@@ -188,6 +188,9 @@ SPLIT_CASES = [
     # (M, N, K, ab, cd, alpha, beta, g, bn, grid): tiles vs workers chosen so that a tail exists
     (1280, 1280, 1024, BF16, FP32, 1.0, 0.0, 2, 256, 16),    # 25 tiles on 8 pairs: 1 tail tile, up to 4 slices
     (1280, 1000, 2048, FP16, FP16, -0.5, 1.5, 2, 256, 24),   # 20 tiles on 12 pairs: 8 tail tiles -> no room: 1 slice
+    (512, 1280, 1024, BF16, BF16, 1.0, 0.5, 2, 256, 16),     # 10 tiles on 8 pairs: one whole wave, then 2 tail tiles (the
+                                                             # owner adds the partials in its epilogue; with two or more
+                                                             # whole waves, as above, they are written into its accumulator)
     (1000, 1160, 1544, BF16, BF16, 1.0, 1.0, 1, 128, 36),    # 80 tiles on 36 CTAs: 8 tail tiles, 4 slices, ragged K
     (640, 520, 4096, FP16, FP32, 2.0, 0.0, 2, 128, 0),       # 15 tiles on 74 pairs: split-K of a small problem
     (512, 512, 12288, BF16, FP32, 1.0, 0.0, 1, 64, 0),       # 32 tiles on 148 CTAs, long K
