@@ -221,6 +221,30 @@ def test_tail_tiles_cut_along_k(case, split):
         dp.close()
 
 
+def test_tail_slices_of_a_strided_batch():
+    # 5 matrices x 6 tiles on 13 pairs: two whole waves, then 4 tail tiles cut in two (owners' accumulators
+    # preloaded with the contributors' sums), tiles of different matrices side by side
+    import torch
+    M, N, K, batch = 600, 384, 1024, 5
+    bp = synth.BatchedProblem("split_batch", batch, M, N, K, BF16, BF16, 0, 1, 0, 1.0, 0.5, seed=23).generate()
+    dev = torch.device("cuda:0")
+    dA, dB, dC = (harness._to_device(x, dev) for x in (bp.A, bp.B, bp.C))
+    desc = harness.desc_of(bp, flags_for(2, 256, 26, split=2))
+    with B.Plan(desc, batch=(batch, bp.stride_a, bp.stride_b, bp.stride_c)) as plan:
+        info = plan.info()
+        assert (info["grid"], info["tail_tiles"], info["split_k"]) == (26, 4, 2), info
+        plan.run(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), 1.0, 0.5, torch.cuda.current_stream(dev).cuda_stream)
+        torch.cuda.synchronize(dev)
+        plan.check()
+    out = dC.cpu().numpy().view(np.uint16)
+    for i in range(batch):
+        q = bp.matrix(i)
+        got = oracle.logical_view(out[i * bp.stride_c:(i + 1) * bp.stride_c], M, N, 0, q.ldc, BF16)
+        cref, den = oracle.gemm_problem(q)
+        gate = TOL * den + oracle.output_rounding_slack(cref, BF16)
+        assert (np.abs(got - cref) <= gate).all(), (i, info)
+
+
 def test_split_plan_recovers_after_a_timed_out_run():
     import torch
     p = synth.Problem("split_tmo", 640, 520, 4096, BF16, FP32, 0, 1, 0, 1.0, 0.0, seed=77).generate()

@@ -108,6 +108,19 @@ def test_tail_slots_cut_along_k(flags2, split):
         dp.close()
 
 
+@pytest.mark.parametrize("flags2", [B.FLAG2_SHARE_ALWAYS, B.FLAG2_SHARE_SUBSTITUTED])
+def test_owning_slice_behind_two_whole_waves_starts_from_the_other_slices_sum(flags2):
+    # 3 x 5 = 15 slots of work on 7 slots of CTAs: two whole waves, then one tail slot cut in two; its
+    # owners find the partial sums written into their accumulators before their slice starts
+    p = synth.Problem("share_preload", 768, 2560, 1024, BF16, FP32, 0, 1, 0, 1.0, 0.5, seed=6).generate()
+    flags = B.flag_grid_limit(28) | B.flag_split_k(2)
+    bits, got, info = run(p, flags, flags2)
+    assert (info["grid"], info["tail_tiles"], info["split_k"]) == (28, 1, 2), info
+    assert_parity(p, got, info)
+    again, _, _ = run(p, flags, flags2)
+    assert np.array_equal(again.view(np.uint8), bits.view(np.uint8))
+
+
 def test_strided_batch_on_shared_operand_clusters():
     import torch
     M, N, K, batch = 384, 640, 320, 5
