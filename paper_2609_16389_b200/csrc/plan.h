@@ -121,6 +121,7 @@ struct Canonical {
   int64_t lda, ldb, ldc;
   int swapped;
   int ab_bytes;                          // 2 (bf16/fp16) or 4 (fp32 storage, tf32 math)
+  int c_bytes;                           // 2 or 4: element size of C
   int64_t batch;                         // matrices in a strided batch (1 = plain GEMM)
   int64_t stride_a, stride_b, stride_c;  // elements between consecutive matrices (canonical operands)
 };
@@ -129,6 +130,7 @@ inline Canonical canonicalize(const exo_gemm_desc_t& d, int64_t batch = 1, int64
                               int64_t stride_b = 0, int64_t stride_c = 0) {
   Canonical c;
   c.ab_bytes = elem_bytes(d.ab_dtype);
+  c.c_bytes = elem_bytes(d.c_dtype);
   c.batch = batch;
   c.stride_c = stride_c;
   c.stride_a = d.c_layout == EXO_GEMM_COL_MAJOR ? stride_b : stride_a;
@@ -293,21 +295,26 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
   cfg.pairs = best_p;
   cfg.mrep = best_r;
   cfg.ksub = best_r == 2 ? 1 : (o.ksub ? o.ksub : default_ksub(best_g, best_n));
-  // Two staging buffers per epilogue warp let a warp fill one while the TMA store still
-  // reads the other; they cost 32 KB of ring.  Short K: the epilogue bounds a tile, so staging
-  // depth matters more than ring depth.  Otherwise the ring takes the space: the time between a
-  // stage's release and its reuse has to cover a commit, the producer's wake-up and an L2 or DRAM
-  // round trip (measured: 6 stages instead of 5 give +1.3 to +4.6 % for K >= 2048).
-  const bool want_two = c.K * (c.ab_bytes / 2) <= 1024 && max_stages(best_g, best_n, cfg.ksub, 2, best_r) >= 3;
-  cfg.epi_bufs = o.epi_bufs ? o.epi_bufs : (want_two ? 2 : 1);
-  cfg.stages = max_stages(best_g, best_n, cfg.ksub, cfg.epi_bufs, best_r);
-  if (o.stages && o.stages < cfg.stages) cfg.stages = o.stages < 2 ? 2 : o.stages;
   cfg.tiles_m = (int)((c.M + 128 * best_g * best_r - 1) / (128 * best_g * best_r));
   cfg.tiles_n = (int)((c.N + best_n * best_p - 1) / (best_n * best_p));
   int64_t workers = best_p == 2 ? max_quads : (best_g == 2 ? max_pairs : sm_count);
   if (o.grid_limit && o.grid_limit / (best_g * best_p) < workers) workers = o.grid_limit / (best_g * best_p);
   if (workers < 1) workers = 1;
   const int64_t tiles = (int64_t)cfg.tiles_m * cfg.tiles_n * c.batch;
+  // Two staging buffers per epilogue warp let a warp fill one while the TMA store still
+  // reads the other; they cost 32 KB of ring.  Short K: the epilogue bounds a tile, so staging
+  // depth matters more than ring depth.  Otherwise the ring takes the space: the time between a
+  // stage's release and its reuse has to cover a commit, the producer's wake-up and an L2 or DRAM
+  // round trip (measured: 6 stages instead of 5 give +1.3 to +4.6 % for K >= 2048).
+  // A 16-bit C halves the epilogue's stores: at K <= 512 and three or more tiles per worker one buffer
+  // and a deeper ring are then ahead again (measured +2.5 to +7 %; with one or two tiles per worker
+  // -1 to -2 %, and at K = 1000 neutral to -2.7 %).
+  const int64_t k16 = c.K * (c.ab_bytes / 2);
+  const bool want_two = k16 <= 1024 && !(c.c_bytes == 2 && k16 <= 512 && tiles >= 3 * workers) &&
+                        max_stages(best_g, best_n, cfg.ksub, 2, best_r) >= 3;
+  cfg.epi_bufs = o.epi_bufs ? o.epi_bufs : (want_two ? 2 : 1);
+  cfg.stages = max_stages(best_g, best_n, cfg.ksub, cfg.epi_bufs, best_r);
+  if (o.stages && o.stages < cfg.stages) cfg.stages = o.stages < 2 ? 2 : o.stages;
   // Wave quantisation: the tiles that do not fill a whole wave are cut along K so that the
   // last wave takes 1/split of a tile's time (split-K applied to the tail only; for a problem
   // smaller than one wave that is plain split-K).
