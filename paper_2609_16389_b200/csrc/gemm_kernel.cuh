@@ -670,6 +670,21 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       // The chunk loop stays rolled: eight warps interleave, which hides the TMEM load
       // latency as well as a software pipeline did, at a fraction of the code size.
       uint32_t v[UPC][32];
+      // An owner that adds the partial sums itself keeps the first contributing slice's next unit on its
+      // way from L2 while it converts and stores the current one (one round trip per unit otherwise).
+      // Only where a chunk is one unit (fp32 C): with two units in registers the 32 more do not fit into
+      // the 168 registers a thread of this kernel can have (352 threads are allocated as 384).
+      constexpr bool kPrefetchPartials = UPC == 1;
+      uint32_t pf[kPrefetchPartials ? 32 : 1];
+      auto prefetch_partial = [&](int32_t i, int32_t q) {
+        if constexpr (kPrefetchPartials) {
+          const char* src = ws_addr(wi, 0, r, i, q);
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            ptx::ld_global_cg_v4(src + j * 512, pf[4 * j + 0], pf[4 * j + 1], pf[4 * j + 2], pf[4 * j + 3]);
+        }
+      };
+      if (owner && mine > 0) prefetch_partial(0, 0);
 #pragma unroll 1
       for (int32_t i = 0; i < mine; ++i) {
         if (ok) {
@@ -714,7 +729,12 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
               for (int k = 0; k < 32; ++k) cur[k] = 0u;
             }
             if (owner) {  // add the other slices' partial sums, in slice order
-              for (int32_t sm1 = 0; sm1 < wi.slices - 1; ++sm1) {
+              if constexpr (kPrefetchPartials) {
+#pragma unroll
+                for (int k = 0; k < 32; ++k) cur[k] = __float_as_uint(__uint_as_float(cur[k]) + __uint_as_float(pf[k]));
+                if (i + 1 < mine) prefetch_partial(i + 1, 0);
+              }
+              for (int32_t sm1 = kPrefetchPartials ? 1 : 0; sm1 < wi.slices - 1; ++sm1) {
                 const char* src = ws_addr(wi, sm1, r, i, q);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
