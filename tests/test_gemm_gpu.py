@@ -271,6 +271,35 @@ def test_split_plan_recovers_after_a_timed_out_run():
         dp.close()
 
 
+def test_plan_with_a_preloaded_owning_slice_recovers_after_a_timed_out_run():
+    # 25 tiles on 8 pairs: three whole waves, then one tail tile cut in two; pair 0 owns it (its slice comes
+    # last, on an accumulator preloaded with pair 1's partial sums).  Pair 0 abandons its first tile: the
+    # run reports the timeout, the arrival counters are put back, the next run is bit-identical to a good one
+    import torch
+    p = synth.Problem("preload_tmo", 1280, 1280, 1024, BF16, FP32, 0, 1, 0, 1.0, 0.0, seed=78).generate()
+    dp = harness.DeviceProblem(p, flags_for(2, 256, 16, split=2))
+    try:
+        info = dp.plan.info()
+        assert (info["tail_tiles"], info["split_k"]) == (1, 2), info
+        dp.run()
+        torch.cuda.synchronize()
+        dp.plan.check()
+        good_bits = dp.result_buffer().copy()
+        assert B.exo_gemm_debug_set(dp.plan.handle, 20, 5) == B.OK
+        dp.run()
+        torch.cuda.synchronize()
+        st, detail = B.exo_gemm_check(dp.plan.handle)
+        assert st == B.ERR_DEVICE_TIMEOUT, detail
+        for _ in range(2):
+            dp.reset_c()
+            dp.run()
+            torch.cuda.synchronize()
+            dp.plan.check()
+            assert np.array_equal(dp.result_buffer(), good_bits)
+    finally:
+        dp.close()
+
+
 def test_bounded_wait_reports_timeout_and_the_plan_stays_usable():
     import torch
     p = synth.Problem("tmo", 512, 512, 1024, BF16, FP32, 0, 1, 0, 1.0, 0.0, seed=10).generate()
