@@ -181,6 +181,12 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   const int64_t worker = blockIdx.x / CLUSTER;
   const int64_t num_workers = gridDim.x / CLUSTER;
   const int32_t nkb = p.num_k_blocks;
+  // From which item index on an owning slice of a tail tile finds the other slices' sum preloaded in
+  // its accumulator (see the epilogue role): the partials must have been published and read back while
+  // the item before it ran.  Two whole tiles in front always leave that time; a single one does if the
+  // K loop is long (measured behind one whole wave: -1.4 % at K = 3072, +1.4 to +2.1 % at 4096, +4 % at
+  // 8192).
+  const int64_t preload_from = (int64_t)nkb * STAGE_K >= 4096 ? 1 : 2;
 
   if (threadIdx.x == 0) EXO_TRACE(2, 4095, 0, 4096);
   // ---------------------------------------------------------------- setup
@@ -413,7 +419,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         const int64_t t = wi.tile;
         // The owning slice of a tail tile that follows at least two whole tiles starts from an accumulator
         // into which the epilogue warps have already written the other slices' partial sums.
-        const bool preloaded = MREP == 1 && wi.slices > 1 && wi.slice == 0 && it >= 2;
+        const bool preloaded = MREP == 1 && wi.slices > 1 && wi.slice == 0 && it >= preload_from;
         if constexpr (MREP == 1) {
           // the epilogue (of both CTAs) must have drained this accumulator
           ok = wait_barrier<PAIR>(tempty_bar(acc), acc_ph ^ 1u, p, WaitSite{kRoleMma, 100 + acc, (uint32_t)t, 0});
@@ -556,7 +562,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         // owner's epilogue is an ordinary one.  (With a single whole tile before the slice the partials
         // arrive too late for that; the owner then adds them in its epilogue.)
         WorkItem nx;
-        if (it >= 1 && work_item(p.work, worker, num_workers, it + 1, nkb, &nx) && nx.slices > 1 && nx.slice == 0) {
+        if (it + 1 >= preload_from && work_item(p.work, worker, num_workers, it + 1, nkb, &nx) && nx.slices > 1 && nx.slice == 0) {
           uint32_t bz2;
           const TileCoord tc2 = tile_coord(nx.tile, &bz2);
           const int32_t n_mine = chunks_of(tc2.m * (CTA_M * CTA_GROUP) + (int32_t)cta_rank * CTA_M + (int32_t)quad * 32,
@@ -599,7 +605,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
           }
         }
       }
-      const bool preloaded = MREP == 1 && wi.slices > 1 && wi.slice == 0 && it >= 2;  // see above
+      const bool preloaded = MREP == 1 && wi.slices > 1 && wi.slice == 0 && it >= preload_from;  // see above
       // one pass per accumulator of the tile: a single one, or (tall tile) rows 0..127 then 128..255 of the CTA
 #pragma unroll 1
       for (int32_t r = 0; r < MREP; ++r) {

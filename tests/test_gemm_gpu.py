@@ -191,6 +191,7 @@ SPLIT_CASES = [
     (512, 1280, 1024, BF16, BF16, 1.0, 0.5, 2, 256, 16),     # 10 tiles on 8 pairs: one whole wave, then 2 tail tiles (the
                                                              # owner adds the partials in its epilogue; with two or more
                                                              # whole waves, as above, they are written into its accumulator)
+    (512, 1280, 4096, FP16, FP32, 1.0, 0.0, 2, 256, 16),     # the same with a K loop long enough for that after one whole wave
     (1000, 1160, 1544, BF16, BF16, 1.0, 1.0, 1, 128, 36),    # 80 tiles on 36 CTAs: 8 tail tiles, 4 slices, ragged K
     (640, 520, 4096, FP16, FP32, 2.0, 0.0, 2, 128, 0),       # 15 tiles on 74 pairs: split-K of a small problem
     (512, 512, 12288, BF16, FP32, 1.0, 0.0, 1, 64, 0),       # 32 tiles on 148 CTAs, long K
