@@ -49,6 +49,8 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the sustained run and the short runs of the other configurations")
     ap.add_argument("--no-cublas", action="store_true")
     ap.add_argument("--flags", type=int, default=0, help="EXO_GEMM_FLAG_* overrides (experiments)")
     ap.add_argument("--share", default="auto", choices=["auto", "never", "always"],
@@ -128,10 +130,13 @@ class ClockSampler:
         self._thr = threading.Thread(target=self._run, daemon=True)
         self._thr.start()
 
-    def stop(self):
+    def stop(self, skip_first: int = 0):
+        """``skip_first`` drops that many leading samples (taken while the GPU was still ramping up)."""
         self._stop.set()
         if self._thr:
             self._thr.join(timeout=10)
+        if skip_first and len(self.samples) > skip_first + 2:
+            self.samples = self.samples[skip_first:]
         sm = [float(s[0]) for s in self.samples if s and s[0].replace(".", "").isdigit()]
         mx = [float(s[1]) for s in self.samples if len(s) > 1 and s[1].replace(".", "").isdigit()]
         reasons = set()
@@ -140,8 +145,14 @@ class ClockSampler:
             for i, n in enumerate(names):
                 if len(s) > 3 + i and s[3 + i].lower().startswith("active"):
                     reasons.add(n)
+        pw = []
+        for smp in self.samples:
+            try:
+                pw.append(float(smp[2]))
+            except (IndexError, ValueError):
+                pass
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(sm), "power_w_max": max(pw) if pw else None}
 
 
 def aggregate_over_ranks(local_ms: float, local_flop: float, world: int, device=None):
@@ -215,6 +226,12 @@ def run_ours(args, rank, world, local_rank):
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py: no CUDA device; the GEMM path has no CPU fallback")
+    if world > 1:
+        # several GPUs: the base library only (it holds no cluster-multicast load), whatever files are present
+        if args.share == "always":
+            raise SystemExit("bench.py: --share always is a single-GPU option (the shared-operand clusters "
+                             "are not part of a multi-GPU program)")
+        os.environ["EXO_GEMM_BASE_ONLY"] = "1"
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     if world > 1:
@@ -313,6 +330,26 @@ def run_ours(args, rank, world, local_rank):
     clocks = sampler.stop()
     plan.check()
 
+    # --- sustained: the same back-to-back launches for about a second of device time, with clock samples
+    # taken inside that region only (the K-step region above is over before the sampler's second reading)
+    sustained = None
+    if world == 1 and not args.no_extras:
+        n_long = int(min(200000, max(args.steps, np.ceil(1000.0 / max(total_ms / args.steps, 1e-3)))))
+        long_sampler = ClockSampler(local_rank)
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        s0.record(stream)
+        long_sampler.start()
+        for i in range(n_long):
+            step(i)
+        s1.record(stream)
+        barrier()
+        long_clocks = long_sampler.stop(skip_first=2)
+        plan.check()
+        long_ms = s0.elapsed_time(s1)
+        sustained = {"tflops": flop * n_long / (long_ms * 1e-3) / 1e12, "steps": n_long, "seconds": long_ms * 1e-3,
+                     "clocks": long_clocks}
+
     value, max_ms = aggregate_over_ranks(total_ms, flop * args.steps, world, dev)
     e2e_value, _ = aggregate_over_ranks(e2e_ms, flop, world, dev)
 
@@ -365,6 +402,24 @@ def run_ours(args, rank, world, local_rank):
         }
         if cublas is not None:
             line["cublas"] = cublas
+        if sustained is not None:
+            speak = pk["tflops_sustained"] * (1.1 / 2.25 if p.ab_dtype == synth.FP32 else 1.0)
+            sustained["peak"] = speak
+            sustained["frac"] = sustained["tflops"] / speak
+            sustained["peak_source"] = f"{pk['source']} (sustained cuBLAS bf16)"
+            line["sustained"] = sustained
+        if world == 1 and not args.no_extras and args.workload == DEFAULT_WORKLOAD:
+            # the other benchmark configurations, a short run each (their own bench lines: --workload NAME)
+            line["configs"] = {}
+            for name in ("cfg1_256", "cfg3_8192", "cfg4a_skinny", "cfg4b_skinny"):
+                try:
+                    line["configs"][name] = measure_config(name, dev, max(3, min(args.steps, 20)), pk)
+                except Exception as e:   # a side measurement never fails the headline
+                    line["configs"][name] = {"error": repr(e)}
+            line["configs"][args.workload] = {"M": p.M, "N": p.N, "K": p.K, "tflops": value, "frac": roofline["frac"],
+                                              "parity": sampled_parity(p, sets[(args.steps - 1) % n_sets][2].cpu().numpy()
+                                                                       .view(synth.storage_np_dtype(p.c_dtype)))
+                                              if p.beta == 0.0 else None}
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(p, args.workload)
         print(json.dumps(line), flush=True)
@@ -373,6 +428,60 @@ def run_ours(args, rank, world, local_rank):
     if world > 1:
         import torch.distributed as dist
         dist.destroy_process_group()
+
+
+def sampled_parity(p, cbuf, n=1 << 14):
+    """Oracle error metric of a finished GEMM on n random entries of C (the oracle computes them one by one)."""
+    import oracle
+    rng = np.random.default_rng(p.seed)
+    r, c = rng.integers(0, p.M, n), rng.integers(0, p.N, n)
+    got = oracle.logical_view(cbuf, p.M, p.N, p.c_layout, p.ldc, p.c_dtype)[r, c]
+    cref, den = oracle.gemm_problem_entries(p, r, c)
+    return {"max_error_metric": oracle.max_error(got, cref, den), "tolerance": oracle.TOLERANCE, "entries": int(n)}
+
+
+def measure_config(name, dev, steps, pk):
+    """A short run of one benchmark configuration: TFLOP/s over `steps` launches back to back (operand sets
+    rotated past L2), roofline fraction, the plan, and the oracle's verdict on sampled entries."""
+    import torch
+    from paper_2609_16389_b200 import binding as B
+    from paper_2609_16389_b200 import harness, synth
+    p = make_problem(name)
+    set_bytes = p.A.nbytes + p.B.nbytes + p.C.nbytes
+    n_sets = int(min(8, max(2, np.ceil(2.0 * L2_BYTES / set_bytes))))
+    sets = [(harness._to_device(p.A, dev), harness._to_device(p.B, dev), harness._to_device(p.C, dev)) for _ in range(n_sets)]
+    stream = torch.cuda.current_stream(dev)
+    with B.Plan(harness.desc_of(p, 0, dev.index or 0)) as plan:
+        info = plan.info()
+
+        def step(i):
+            a, b, c = sets[i % n_sets]
+            plan.run(a.data_ptr(), b.data_ptr(), c.data_ptr(), p.alpha, p.beta, stream.cuda_stream)
+
+        # parity first, on a fresh C (beta != 0 updates C in place, so later steps change it again)
+        step(0)
+        torch.cuda.synchronize(dev)
+        plan.check()
+        parity = sampled_parity(p, sets[0][2].cpu().numpy().view(synth.storage_np_dtype(p.c_dtype)))
+        for i in range(3):
+            step(i)
+        torch.cuda.synchronize(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(steps):
+            step(i)
+        e1.record(stream)
+        torch.cuda.synchronize(dev)
+        plan.check()
+        ms = e0.elapsed_time(e1) / steps
+    tf = p.flop / (ms * 1e-3) / 1e12
+    roof = min(pk["tflops_burst"], p.flop / p.algorithmic_bytes * pk["hbm_gbs"] / 1e3)
+    return {"M": p.M, "N": p.N, "K": p.K, "tflops": tf, "ms_per_step": ms, "steps": steps,
+            "roofline_tflops": roof, "frac": tf / roof,
+            "hbm_gbs": p.algorithmic_bytes / (ms * 1e-3) / 1e9,
+            "plan": {k: info[k] for k in ("cta_group", "tile_m", "tile_n", "tile_k", "stages", "epilogue_buffers",
+                                          "split_k", "tail_tiles", "grid")},
+            "l2_sets": n_sets, "parity": parity}
 
 
 def time_cublas(p, dev, steps, n_sets, ours_step=None):

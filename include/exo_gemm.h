@@ -121,7 +121,8 @@ typedef struct {
 /* What a plan decided; filled by exo_gemm_get_info. */
 typedef struct {
   int32_t cta_group;      /* 1 or 2 SMs per tile                                               */
-  int32_t tile_m, tile_n; /* output tile of one CTA group (tile_m = 128 * cta_group)           */
+  int32_t tile_m, tile_n; /* output tile of one CTA group: tile_m = 128 * cta_group rows, or
+                             256 * cta_group (= 512) for the tall tile, EXO_GEMM_FLAG2_CTA_ROWS  */
   int32_t tile_k;         /* k-elements staged per pipeline stage (64 or 128; tf32: 32 or 64)  */
   int32_t stages;         /* depth of the shared-memory operand ring                           */
   int32_t grid;           /* CTAs launched (persistent)                                        */
@@ -144,7 +145,9 @@ typedef struct {
 
 /*
  * Pure argument check; needs no GPU and touches no CUDA state.  Returns OK,
- * ERR_NULL, ERR_INVALID_ARG or ERR_UNSUPPORTED by the rules above.
+ * ERR_NULL, ERR_INVALID_ARG or ERR_UNSUPPORTED by the rules above.  (What is legal
+ * follows BLAS Sgemm, the routine the paper's Section 6 measures its GEMM kernels
+ * against; what is supported is that set cut down to what TMA can address.)
  */
 exo_gemm_status_t exo_gemm_validate(const exo_gemm_desc_t* desc);
 
@@ -179,7 +182,11 @@ exo_gemm_status_t exo_gemm_create_batched(exo_gemm_handle_t* out, const exo_gemm
 
 /*
  * Enqueues C = alpha*A*B + beta*C on cuda_stream (a cudaStream_t; NULL = the
- * legacy default stream) and returns without synchronising.
+ * legacy default stream) and returns without synchronising.  This is the operation
+ * of the paper's GEMM kernels (Section 6; "D += matmul(A, B)" in the Section 2.2
+ * listings) with the alpha/beta form of BLAS Sgemm; one call is one launch of a
+ * persistent, warp-specialised kernel (the kernel class of the paper's Section 4.2
+ * code generation: persistent task loop, one code path per named warp group).
  *
  *   A, B, C   DEVICE pointers, 16-byte aligned, laid out as the descriptor says.
  *             The caller owns them and keeps them alive until the stream has
@@ -206,10 +213,15 @@ exo_gemm_status_t exo_gemm_run(exo_gemm_handle_t plan, const void* A, const void
                                float alpha, float beta, void* cuda_stream);
 
 /*
- * Reads the plan's device status block (a blocking 32-byte copy; call it after
- * synchronising the stream(s) the plan ran on).  Returns OK or
- * ERR_DEVICE_TIMEOUT, and clears the block.  detail, if not NULL, receives 8
- * words: {code, role, barrier, tile, k_block, cta, 0, 0}.
+ * Reads the plan's device status block (a blocking 32-byte device-to-host copy on the
+ * legacy default stream; call it after synchronising the stream(s) the plan ran on).
+ * Returns OK or ERR_DEVICE_TIMEOUT, and clears the block.  detail, if not NULL, receives 8
+ * words: {code, role, barrier, tile, k_block, cta, 0, 0}.  After a timeout it also puts
+ * the arrival counters of a K-slicing plan back to zero; that reset and the launches of
+ * exo_gemm_run on the same plan exclude one another (a lock inside the plan), so the
+ * call is safe beside runs from other host threads.  (The paper's kernels have no such
+ * status: its Section 5 checks synchronisation before the kernel ever runs; a library
+ * that runs on shared GPUs bounds every device-side wait instead and reports here.)
  */
 exo_gemm_status_t exo_gemm_check(exo_gemm_handle_t plan, uint32_t* detail);
 
@@ -331,6 +343,8 @@ int64_t exo_gemm_schedule_work(int64_t tiles, int32_t num_workers, int32_t split
  * first CTA's producer skips issuing the loads of that k-block (counted from the
  * start of the CTA's work), so that one wait runs out and the kernel returns an
  * error status without trapping.  The settings apply to one run, then reset.
+ * plan == NULL: the settings apply to the next exo_gemm_run_static call of this
+ * process instead (that entry point has no plan to attach them to).
  */
 exo_gemm_status_t exo_gemm_debug_set(exo_gemm_handle_t plan, int32_t timeout_ms, int64_t skip_k_block);
 

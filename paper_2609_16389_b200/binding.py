@@ -72,7 +72,10 @@ def lib():
     if _lib is None:
         # EXO_GEMM_LIBRARY overrides (a development build); otherwise the variant library -- the base
         # library plus the shared-operand cluster kernels -- where its sources are present, else the base one
+        # (a rank of a multi-GPU job always gets the base library)
         path = os.environ.get("EXO_GEMM_LIBRARY") or _build.build_preferred()
+        if _build.multi_gpu_job() and os.path.basename(path) == os.path.basename(_build.SHARE_LIB):
+            raise RuntimeError("the shared-operand cluster library is for single-GPU programs only")
         if not os.path.exists(path):
             raise RuntimeError("libexo_gemm.so is missing: the CUDA path cannot run")
         L = ctypes.CDLL(path)

@@ -67,18 +67,29 @@ def build_share(force: bool = False, verbose: bool = False) -> str:
     return _compile(SHARE_LIB, ["EXO_GEMM_SHARE_PAIRS"], verbose)
 
 
+def multi_gpu_job() -> bool:
+    """True in a process that is one rank of several (torchrun sets WORLD_SIZE)."""
+    try:
+        return int(os.environ.get("WORLD_SIZE", "1")) > 1
+    except ValueError:
+        return False
+
+
 def build_preferred() -> str:
-    """The library a single-GPU program should load: the variant where it can be built, else the base."""
-    if os.environ.get("EXO_GEMM_BASE_ONLY") != "1" and have_share_sources():
+    """The library this process should load: the variant where it can be built and the program runs on
+    one GPU, else the base library.  A rank of a multi-GPU job always gets the base library, whatever
+    files are present: code that spans several GPUs carries no cluster-multicast load."""
+    if os.environ.get("EXO_GEMM_BASE_ONLY") != "1" and not multi_gpu_job() and have_share_sources():
         return build_share()
     return build()
 
 
 def build_all(force: bool = False, verbose: bool = False):
-    out = [build(force, verbose)]
-    if have_share_sources():
-        out.append(build_share(force, verbose))
-    return out
+    """Both libraries (the variant only where its sources are present), compiled side by side."""
+    from concurrent.futures import ThreadPoolExecutor
+    jobs = [build] + ([build_share] if have_share_sources() else [])
+    with ThreadPoolExecutor(len(jobs)) as ex:
+        return list(ex.map(lambda fn: fn(force, verbose), jobs))
 
 
 if __name__ == "__main__":

@@ -147,6 +147,7 @@ struct exo_gemm_plan {
   float* d_split_ws;                   // fp32 partials of the tail tiles' K-slices (NULL if none)
   uint32_t* d_split_flags;             // one arrival counter per tail tile
   std::atomic<uint32_t> split_epoch;   // runs that used the counters so far
+  std::mutex split_mutex;              // taking an epoch + launching, and exo_gemm_check's reset, exclude one another
   std::atomic<int32_t> dbg_timeout_ms;
   std::atomic<int64_t> dbg_skip_k_block;
 };
@@ -179,9 +180,17 @@ exo_gemm_status_t cuda_fail(cudaError_t e) {
 
 // How many clusters of `cluster` CTAs of kernel `probe` can be resident at once (GPC shapes may
 // leave SMs that fit no further cluster).
+// One kernel instantiation serves plans with different shared-memory sizes (ring and staging depth are
+// run-time parameters), and the attribute belongs to the function, not to a launch: every kernel gets
+// the same upper value, never a plan's own size, so plans that live side by side cannot lower it for
+// one another.
+cudaError_t allow_full_smem(KernelFn k) {
+  return cudaFuncSetAttribute((const void*)k, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+}
+
 cudaError_t max_active_clusters(KernelFn probe, int sms, int cluster, int* out) {
   const int smem = kSmemLimit - 1024;  // every plan's shared-memory request is close to the limit
-  cudaError_t e = cudaFuncSetAttribute((const void*)probe, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  cudaError_t e = allow_full_smem(probe);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t lc{};
   lc.gridDim = dim3((unsigned)(sms / cluster * cluster), 1, 1);
@@ -376,7 +385,7 @@ exo_gemm_status_t exo_gemm_create_batched(exo_gemm_handle_t* out, const exo_gemm
   p->split_epoch = 0;
   p->kernel = pick_kernel(p->cfg.cta_group, p->cfg.tile_n, p->cfg.ksub, desc->c_dtype, p->cfg.pairs, p->cfg.mrep);
   p->smem_bytes = smem_bytes_for(p->cfg.cta_group, p->cfg.tile_n, p->cfg.ksub, p->cfg.stages, p->cfg.epi_bufs, p->cfg.mrep);
-  e = cudaFuncSetAttribute((const void*)p->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, p->smem_bytes);
+  e = allow_full_smem(p->kernel);
   if (e != cudaSuccess) { delete p; return cuda_fail(e); }
   e = cudaMalloc((void**)&p->d_status, kStatusBytes);
   if (e != cudaSuccess) { delete p; return cuda_fail(e); }
@@ -407,23 +416,44 @@ exo_gemm_status_t exo_gemm_get_info(exo_gemm_handle_t plan, exo_gemm_info_t* inf
 
 int32_t exo_gemm_has_shared_operand_clusters(void) { return kHaveSharePairs ? 1 : 0; }
 
+// one-shot test settings of the plan-less entry point (exo_gemm_debug_set with a NULL plan)
+static std::atomic<int32_t> g_static_dbg_timeout_ms{0};
+static std::atomic<int64_t> g_static_dbg_skip_k_block{-1};
+
 exo_gemm_status_t exo_gemm_debug_set(exo_gemm_handle_t plan, int32_t timeout_ms, int64_t skip_k_block) {
-  if (!plan) return EXO_GEMM_ERR_NULL;
   if (timeout_ms < 0 || timeout_ms > 10000) return EXO_GEMM_ERR_INVALID_ARG;
+  if (!plan) {
+    g_static_dbg_timeout_ms = timeout_ms;
+    g_static_dbg_skip_k_block = skip_k_block;
+    return EXO_GEMM_OK;
+  }
   plan->dbg_timeout_ms = timeout_ms;
   plan->dbg_skip_k_block = skip_k_block;
   return EXO_GEMM_OK;
 }
 
-exo_gemm_status_t exo_gemm_run(exo_gemm_handle_t plan, const void* A, const void* B, void* C, float alpha,
-                               float beta, void* cuda_stream) {
-  if (!plan) return EXO_GEMM_ERR_NULL;
+}  // extern "C"
+
+namespace {
+
+// The argument checks of a run.  *launch is false for an empty problem (nothing to enqueue).
+exo_gemm_status_t check_run_args(const exo_gemm_plan* plan, const void* A, const void* B, const void* C, float alpha,
+                                 bool* launch) {
+  *launch = false;
   const Canonical& cn = plan->canon;
   if (cn.M == 0 || cn.N == 0) return EXO_GEMM_OK;
   const bool read_ab = alpha != 0.f && cn.K > 0;
   if (!C || (read_ab && (!A || !B))) return EXO_GEMM_ERR_NULL;
   if (((uintptr_t)C & 15u) || (read_ab && (((uintptr_t)A | (uintptr_t)B) & 15u))) return EXO_GEMM_ERR_ALIGNMENT;
+  *launch = true;
+  return EXO_GEMM_OK;
+}
 
+// Tensor maps and the launch, for arguments that passed check_run_args.
+exo_gemm_status_t launch_plan(exo_gemm_plan* plan, const void* A, const void* B, void* C, float alpha, float beta,
+                              void* cuda_stream) {
+  const Canonical& cn = plan->canon;
+  const bool read_ab = alpha != 0.f && cn.K > 0;
   const exo_gemm_desc_t& d = plan->desc;
   const TileConfig& cfg = plan->cfg;
   const void* opA = cn.swapped ? B : A;
@@ -525,13 +555,33 @@ exo_gemm_status_t exo_gemm_run(exo_gemm_handle_t plan, const void* A, const void
     at[2].val.preferredClusterDim.z = 1;
     lc.numAttrs = 3;
   }
-  if (split_now) {  // arrival counters only grow: this run is complete at epoch * arrivals-per-run
+  cudaError_t e;
+  if (split_now) {
+    // Arrival counters only grow: this run is complete at epoch * arrivals-per-run.  The epoch is taken and
+    // the launch enqueued under the plan's lock, so that exo_gemm_check (which puts counters and epoch back
+    // to zero after an abandoned run) never falls between the two on another host thread.
+    std::lock_guard<std::mutex> lock(plan->split_mutex);
     const uint32_t epoch = plan->split_epoch.fetch_add(1) + 1;
     prm.split_target = epoch * (uint32_t)((cfg.split - 1) * kEpiWarps * cfg.cta_group * cfg.mrep);
+    e = cudaLaunchKernelEx(&lc, plan->kernel, tm_a, tm_b, tm_c, prm);
+  } else {
+    e = cudaLaunchKernelEx(&lc, plan->kernel, tm_a, tm_b, tm_c, prm);
   }
-  cudaError_t e = cudaLaunchKernelEx(&lc, plan->kernel, tm_a, tm_b, tm_c, prm);
   if (e != cudaSuccess) return cuda_fail(e);
   return EXO_GEMM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+exo_gemm_status_t exo_gemm_run(exo_gemm_handle_t plan, const void* A, const void* B, void* C, float alpha,
+                               float beta, void* cuda_stream) {
+  if (!plan) return EXO_GEMM_ERR_NULL;
+  bool launch = false;
+  const exo_gemm_status_t st = check_run_args(plan, A, B, C, alpha, &launch);
+  if (st != EXO_GEMM_OK || !launch) return st;
+  return launch_plan(plan, A, B, C, alpha, beta, cuda_stream);
 }
 
 exo_gemm_status_t exo_gemm_check(exo_gemm_handle_t plan, uint32_t* detail) {
@@ -546,6 +596,7 @@ exo_gemm_status_t exo_gemm_check(exo_gemm_handle_t plan, uint32_t* detail) {
   e = cudaMemset(plan->d_status, 0, 32);
   if (e != cudaSuccess) return cuda_fail(e);
   if (plan->d_split_flags) {  // an abandoned run may have left the arrival counters short
+    std::lock_guard<std::mutex> lock(plan->split_mutex);
     e = cudaMemset(plan->d_split_flags, 0, sizeof(uint32_t) * (size_t)plan->cfg.tail_tiles * (size_t)plan->cfg.pairs);
     if (e != cudaSuccess) return cuda_fail(e);
     plan->split_epoch = 0;
@@ -609,8 +660,6 @@ exo_gemm_status_t exo_gemm_run_static(const exo_gemm_desc_t* desc, const void* A
   plan.canon = canonicalize(*desc);
   plan.device = device;
   plan.sm_count = sms;
-  plan.dbg_timeout_ms = 0;
-  plan.dbg_skip_k_block = -1;
   FlagOverrides ov = decode_flags(desc->flags, desc->flags2);
   ov.no_workspace = true;  // K-slicing of the tail tiles needs device scratch this entry point may not allocate
   if (ov.share >= 2 && !kHaveSharePairs) return EXO_GEMM_ERR_UNSUPPORTED;
@@ -621,16 +670,26 @@ exo_gemm_status_t exo_gemm_run_static(const exo_gemm_desc_t* desc, const void* A
   plan.cfg = choose_config(plan.canon, ov, sms, max_pairs, max_quads);
   plan.kernel = pick_kernel(plan.cfg.cta_group, plan.cfg.tile_n, plan.cfg.ksub, desc->c_dtype, plan.cfg.pairs, plan.cfg.mrep);
   plan.smem_bytes = smem_bytes_for(plan.cfg.cta_group, plan.cfg.tile_n, plan.cfg.ksub, plan.cfg.stages, plan.cfg.epi_bufs, plan.cfg.mrep);
-  e = cudaFuncSetAttribute((const void*)plan.kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem_bytes);
+  e = allow_full_smem(plan.kernel);
   if (e != cudaSuccess) return cuda_fail(e);
 
+  // every argument check comes before anything is enqueued, as in exo_gemm_run
+  bool launch = false;
+  st = check_run_args(&plan, A, B, C, alpha, &launch);
+  if (st != EXO_GEMM_OK) return st;
+  if (!launch) {  // empty problem: nothing runs, nothing to report
+    if (detail) memset(detail, 0, 32);
+    return EXO_GEMM_OK;
+  }
   e = static_scratch_for_current_device(device, &plan.d_status);
   if (e != cudaSuccess) return cuda_fail(e);
   // the array keeps the last call's contents: the status words must start at zero
   e = cudaMemsetAsync(plan.d_status, 0, kStatusBytes, (cudaStream_t)cuda_stream);
   if (e != cudaSuccess) return cuda_fail(e);
+  plan.dbg_timeout_ms = g_static_dbg_timeout_ms.exchange(0);
+  plan.dbg_skip_k_block = g_static_dbg_skip_k_block.exchange(-1);
 
-  st = exo_gemm_run(&plan, A, B, C, alpha, beta, cuda_stream);
+  st = launch_plan(&plan, A, B, C, alpha, beta, cuda_stream);
   if (st != EXO_GEMM_OK || !detail) return st;
 
   // blocking mode: wait for the kernel and report what it recorded

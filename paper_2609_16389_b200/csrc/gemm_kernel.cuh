@@ -241,9 +241,8 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
 
   // Everything above touched only this CTA's shared and tensor memory, so with programmatic
   // dependent launch it overlaps the tail of the previous kernel in the stream.  Each role waits for
-  // that kernel itself, as late as it can: the copying lanes right before their first copy, the
-  // epilogue warps before they first touch C or the split workspace; the MMA warp never touches
-  // global memory.
+  // that kernel itself at the start of its role, with every lane: before that wait no thread reads
+  // global memory, the status word included.
 
   bool ok = true;
   if (threadIdx.x == 0) EXO_TRACE(2, 4094, 0, 4096);
@@ -258,6 +257,10 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     int64_t issued = 0;
     // in a pair, both CTAs' loads are counted on the leader's full barrier
     const uint32_t full0 = PAIR ? ptx::map_to_cta(full_bar(0), leader) : full_bar(0);
+    // The operands may be the previous kernel's output, and the status word that the bounded waits poll
+    // may still be about to be cleared by the work before this kernel: every lane waits for it here.  (The
+    // first wait of the loop below passes at once, so this is as late as a wait before the first copy.)
+    ptx::grid_dependency_wait();
     for (int64_t it = 0; ok; ++it) {
       WorkItem wi = wi_first;
       TileCoord tc = tc_first;
@@ -279,7 +282,6 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         if (ptx::elect_one()) {
           EXO_TRACE(0, issued, 0, 4096);
           if (cta_rank == 0 && do_a) ptx::mbar_arrive_expect_tx(full_bar(s), STAGE_BYTES * CTA_GROUP);
-          if (issued == 0) ptx::grid_dependency_wait();  // the operands may be the previous kernel's output
           if (!skip) {
             const uint32_t a_dst = stage0 + s * STAGE_BYTES;
             const uint32_t b_dst = a_dst + A_BYTES;
@@ -371,6 +373,10 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   } else if (warp == 1) {
     // ============================================================ MMA issuer
     if (cta_rank == 0 && nkb > 0) {
+      // This warp touches no user memory, but its bounded waits poll the status word, which the work in
+      // front of this kernel may still be about to clear; its first real wait is for data that the
+      // producers fetch after the same dependency, so this costs no time.
+      ptx::grid_dependency_wait();
       uint32_t s = 0, ph = 0, acc = 0, acc_ph = 0;
       const uint16_t kStageMask = quad ? 0xF : (PAIR ? 3 : 1);  // a stage is released in every CTA that fills it
       const uint16_t pair_mask = (uint16_t)((PAIR ? 3u : 1u) << leader);   // the accumulator belongs to this pair

@@ -21,6 +21,8 @@ Entry recipe
 """
 from __future__ import annotations
 
+import os
+
 import numpy as np
 
 BASE_SEED = 260916389
@@ -173,19 +175,30 @@ def load(buf: np.ndarray, rows: int, cols: int, layout: int, ld: int) -> np.ndar
 # matrices and workloads
 # ----------------------------------------------------------------------------
 def matrix(seed: int, tag: int, rows: int, cols: int, dtype: int, dist: str = "uniform",
-           chunk_rows: int = 2048, operand: bool = False) -> np.ndarray:
-    """Logical rows x cols matrix in storage type (uint16 bits, or float32)."""
+           chunk_rows: int = 512, operand: bool = False) -> np.ndarray:
+    """Logical rows x cols matrix in storage type (uint16 bits, or float32).
+
+    An entry depends on (seed, tag, row, column) only, so row blocks are filled by a few threads side
+    by side (numpy releases the interpreter lock inside its array operations)."""
+    if dist not in ("uniform", "normal"):
+        raise ValueError(dist)
     out = np.empty((rows, cols), dtype=storage_np_dtype(dtype))
     cj = np.arange(cols, dtype=np.int64)
-    for r0 in range(0, rows, chunk_rows):
+
+    def fill(r0):
         ri = np.arange(r0, min(rows, r0 + chunk_rows), dtype=np.int64)
-        if dist == "uniform":
-            x = uniform_pm1(seed, tag, ri, cj)
-        elif dist == "normal":
-            x = normal_01(seed, tag, ri, cj)
-        else:
-            raise ValueError(dist)
+        x = uniform_pm1(seed, tag, ri, cj) if dist == "uniform" else normal_01(seed, tag, ri, cj)
         out[r0:r0 + len(ri)] = round_to_storage(x, dtype, operand)
+
+    starts = range(0, rows, chunk_rows)
+    threads = min(len(starts), os.cpu_count() or 1, 32)
+    if threads <= 1 or rows * cols < (1 << 20):
+        for r0 in starts:
+            fill(r0)
+    else:
+        from concurrent.futures import ThreadPoolExecutor
+        with ThreadPoolExecutor(threads) as ex:
+            list(ex.map(fill, starts))
     return out
 
 
@@ -210,12 +223,15 @@ class Problem:
         self.ldb = ldb if ldb is not None else max(1, min_ld(K, N, b_layout))
         self.ldc = ldc if ldc is not None else max(1, min_ld(M, N, c_layout))
         self.A = self.B = self.C = None
+        # fp32 operands (tf32 math): True draws A and B on the tf32 grid (10 fraction bits), False keeps
+        # the full 24-bit significands of the draw
+        self.tf32_grid = True
 
     def generate(self, pad_a=None, pad_b=None, pad_c=None):
         """Fill A, B and C_in.  C_in is drawn uniform[-1,1] in every case (it is
         only read when beta != 0)."""
-        a = matrix(self.seed, TAG_A, self.M, self.K, self.ab_dtype, self.dist, operand=True)
-        b = matrix(self.seed, TAG_B, self.K, self.N, self.ab_dtype, self.dist, operand=True)
+        a = matrix(self.seed, TAG_A, self.M, self.K, self.ab_dtype, self.dist, operand=self.tf32_grid)
+        b = matrix(self.seed, TAG_B, self.K, self.N, self.ab_dtype, self.dist, operand=self.tf32_grid)
         c = matrix(self.seed, TAG_C, self.M, self.N, self.c_dtype, "uniform")
         self.A = store(a, self.a_layout, self.lda, pad_a)
         self.B = store(b, self.b_layout, self.ldb, pad_b)

@@ -183,6 +183,54 @@ def test_persistent_loop_many_tiles_on_few_ctas():
     check_full(p, flags_for(1, 64, 4, ksub=2, epi=2, stages=3))
 
 
+def test_plans_of_one_kernel_with_different_shared_memory_sizes_live_side_by_side():
+    """One kernel instantiation serves plans whose ring and staging depths differ (run-time
+    parameters), hence different dynamic shared-memory sizes; creating the smaller one must not
+    make launches of the larger one fail.  Two pairs of plans, run in alternation."""
+    import torch
+    dev = torch.device("cuda:0")
+    stream = torch.cuda.current_stream(dev).cuda_stream
+    pairs = [
+        (synth.Problem("k4096", 4096, 384, 4096, BF16, FP32, 0, 1, 0, 1.0, 0.0, seed=41), 0,
+         synth.Problem("k512", 4096, 384, 512, BF16, FP32, 0, 1, 0, 1.0, 0.0, seed=42), 0),
+        (synth.Problem("epi1", 520, 392, 328, FP16, FP32, 0, 0, 0, 1.0, 0.0, seed=43, dist="normal"), flags_for(2, 128, epi=1),
+         synth.Problem("epi2", 520, 392, 328, FP16, FP32, 0, 0, 0, 1.0, 0.0, seed=44, dist="normal"), flags_for(2, 128, epi=2)),
+    ]
+    for pa, fa, pb, fb in pairs:
+        pa.generate(); pb.generate()
+        da = harness.DeviceProblem(pa, fa)
+        db = harness.DeviceProblem(pb, fb)           # created second: must not shrink what da may request
+        try:
+            ia, ib = da.plan.info(), db.plan.info()
+            assert (ia["cta_group"], ia["tile_n"], ia["tile_k"]) == (ib["cta_group"], ib["tile_n"], ib["tile_k"])
+            assert ia["smem_bytes"] != ib["smem_bytes"], (ia, ib)
+            refs = {}
+            for q in (pa, pb):
+                refs[q.name] = oracle.gemm_problem(q)
+            for rep in range(3):
+                for dp in (da, db, da):
+                    dp.reset_c()
+                    dp.run(stream)
+                    torch.cuda.synchronize(dev)
+                    dp.plan.check()
+                    q = dp.p
+                    got = oracle.logical_view(dp.result_buffer(), q.M, q.N, q.c_layout, q.ldc, q.c_dtype)
+                    assert oracle.max_error(got, *refs[q.name]) <= TOL, (q.name, rep)
+            # the plan-less entry point in between must not disturb them either
+            st, _ = B.exo_gemm_run_static(harness.desc_of(pb, fb), db.dA.data_ptr(), db.dB.data_ptr(), db.dC.data_ptr(),
+                                          pb.alpha, pb.beta, stream)
+            assert st == B.OK
+            da.reset_c()
+            da.run(stream)
+            torch.cuda.synchronize(dev)
+            da.plan.check()
+            got = oracle.logical_view(da.result_buffer(), pa.M, pa.N, pa.c_layout, pa.ldc, pa.c_dtype)
+            assert oracle.max_error(got, *refs[pa.name]) <= TOL
+        finally:
+            da.close()
+            db.close()
+
+
 # ------------------------------------------------------------------ K-slices of the tail tiles
 SPLIT_CASES = [
     # (M, N, K, ab, cd, alpha, beta, g, bn, grid): tiles vs workers chosen so that a tail exists
@@ -404,6 +452,59 @@ def test_tf32_m_or_n_contiguous_on_the_tall_tile_and_in_a_batch():
         assert oracle.max_error(got, cref, den) <= TOL
 
 
+def tf32_truncated(buf):
+    """What the tensor core reads of an fp32 operand in tf32 mode: sign, exponent and the upper 10
+    fraction bits; the low 13 fraction bits are dropped (not rounded)."""
+    return (buf.view(np.uint32) & np.uint32(0xFFFFE000)).view(np.float32)
+
+
+@pytest.mark.parametrize("la", [0, 1])
+@pytest.mark.parametrize("lb", [0, 1])
+@pytest.mark.parametrize("lc", [0, 1])
+@pytest.mark.parametrize("shape", [(264, 328, 200), (1000, 520, 1028)])
+def test_tf32_on_general_fp32_operands(la, lb, lc, shape):
+    """Operands with full 24-bit significands, as a caller of the tf32 mode passes them.  The reading
+    of "tf32" (the paper's Section 6 precision, cuBLAS's TF32 tensor-op mode): each operand enters
+    the product with its low 13 fraction bits cleared.  The oracle gets copies cleared that way BY THIS
+    TEST and the literal 1e-3 gate applies; against the oracle on the uncleared operands the error is
+    what tf32 costs and is only reported."""
+    M, N, K = shape
+    p = synth.Problem("tf32_general", M, N, K, FP32, FP32, la, lb, lc, 1.25, -0.5, seed=900 + la + 2 * lb + 4 * lc + M)
+    p.tf32_grid = False
+    p.generate()
+    assert (p.A.view(np.uint32) & 0x1FFF).any() and (p.B.view(np.uint32) & 0x1FFF).any()   # really off the grid
+    cbuf, got, info = run_gpu(p)
+    full_a, full_b = p.A, p.B
+    p.A, p.B = tf32_truncated(full_a), tf32_truncated(full_b)
+    cref, den = oracle.gemm_problem(p)
+    err = oracle.max_error(got, cref, den)
+    assert err <= TOL, (err, info)
+    p.A, p.B = full_a, full_b
+    cref_full, den_full = oracle.gemm_problem(p)
+    err_full = oracle.max_error(got, cref_full, den_full)
+    print(f"tf32 general {shape} layouts {la}{lb}{lc}: {err:.2e} vs cleared operands, {err_full:.2e} vs full fp32 operands")
+    assert err_full <= 4 * TOL        # two operands, each short of its value by at most 2^-10 relative
+
+
+@pytest.mark.parametrize("g,bn", [(1, 128), (2, 256)])
+def test_tf32_drops_the_low_fraction_bits_exactly(g, bn):
+    """A times the identity returns, bit for bit, A with the low 13 fraction bits cleared -- values
+    chosen so that rounding to nearest would give something else (fraction bits 12..10 = 111, 110, 011)."""
+    M, N, K = 256, 256, 64
+    p = synth.Problem("tf32_bits", M, N, K, FP32, FP32, 0, 1, 0, 1.0, 0.0, seed=17)
+    p.tf32_grid = False
+    p.generate()
+    a = p.A.view(np.uint32).reshape(M, K)
+    a &= np.uint32(0xFFFFE000)
+    a |= np.array([0x1C00, 0x1800, 0x0C00, 0x1FFF], dtype=np.uint32)[np.arange(K) % 4][None, :]
+    b = np.zeros((K, N), np.float32)
+    b[np.arange(K), np.arange(K)] = 1.0
+    p.B = synth.store(b, p.b_layout, p.ldb)
+    _, got, _ = run_gpu(p, flags_for(g, bn))
+    want = tf32_truncated(p.A).reshape(M, K).astype(np.float64)
+    assert np.array_equal(got[:, :K], want) and np.all(got[:, K:] == 0.0)
+
+
 def test_tf32_large_sampled():
     p = synth.Problem("tf32_big", 4096, 2048, 4096, FP32, FP32, 0, 1, 0, 1.0, 0.0, seed=4242).generate()
     check_sampled(p)
@@ -568,8 +669,9 @@ def test_strided_batched_gemm(case, g, bn):
 
 
 # ------------------------------------------------------------------ the benchmark configurations
-def structured_sample(M, N, rng, n_random=1 << 14):
-    """Rows/columns next to every 128/256 tile boundary crossed with random partners, plus random entries."""
+def structured_sample(M, N, rng, n_random=1 << 16, block=256):
+    """Rows/columns next to every 128/256 tile boundary crossed with random partners, the four corner
+    blocks and the centre block of C in full (256 x 256 each, clipped), plus 2^16 random entries."""
     def edges(n):
         e = set()
         for t in range(0, n + 1, 128):
@@ -580,6 +682,15 @@ def structured_sample(M, N, rng, n_random=1 << 14):
     er, ec = edges(M), edges(N)
     rows = [np.repeat(er, 8), rng.integers(0, M, 8 * ec.size), rng.integers(0, M, n_random)]
     cols = [rng.integers(0, N, 8 * er.size), np.repeat(ec, 8), rng.integers(0, N, n_random)]
+    bm, bn = min(block, M), min(block, N)
+    for r0 in sorted({0, (M - bm) // 2 // 128 * 128, M - bm}):
+        for c0 in sorted({0, (N - bn) // 2 // 128 * 128, N - bn}):
+            corner = (r0 in (0, M - bm)) and (c0 in (0, N - bn))
+            centre = r0 == (M - bm) // 2 // 128 * 128 and c0 == (N - bn) // 2 // 128 * 128
+            if corner or centre:
+                rr, cc = np.meshgrid(np.arange(r0, r0 + bm), np.arange(c0, c0 + bn), indexing="ij")
+                rows.append(rr.reshape(-1))
+                cols.append(cc.reshape(-1))
     return np.concatenate(rows), np.concatenate(cols)
 
 
@@ -613,12 +724,65 @@ def test_config4_skinny_sampled_and_freivalds(variant):
 
 SWEEP_SUBSET = [(512, 512, 512), (1000, 1000, 1000), (512, 12288, 1000), (3072, 1000, 2048),
                 (1000, 512, 12288), (6144, 2048, 512), (2048, 3072, 6144)]
+# shapes with two large dimensions that are checked whatever the plan classes turn out to be
+SWEEP_LARGE = [(12288, 12288, 12288), (12288, 12288, 512), (12288, 1000, 12288), (6144, 12288, 1000)]
 
 
-@pytest.mark.parametrize("M,N,K", SWEEP_SUBSET)
-def test_shape_sweep_subset(M, N, K):
+def plan_signature(info):
+    """What distinguishes the code paths a plan takes: tile shape, pipeline and staging depth, K-slices
+    of the tail, whether a tail exists, whether whole waves precede it, raster direction."""
+    g = info["cta_group"]
+    workers = max(1, info["grid"] // info["cluster_size"])
+    tiles = info["tiles_m"] * info["tiles_n"]
+    return (g, info["tile_m"], info["tile_n"], info["tile_k"], info["stages"], info["epilogue_buffers"],
+            info["split_k"], info["tail_tiles"] > 0, tiles >= workers and info["tail_tiles"] < tiles, info["raster_along_m"])
+
+
+def sweep_plan_classes(sm_count=148):
+    """The 216 sweep shapes grouped by the plan the library previews for them; per class the shape with
+    the least and the one with the most work."""
+    import itertools
+    classes = {}
+    for M, N, K in itertools.product(synth.SWEEP_DIMS, repeat=3):
+        st, info = B.exo_gemm_plan_preview(B.make_desc(M, N, K, BF16, FP32, 0, 1, 0), sm_count)
+        assert st == B.OK
+        classes.setdefault(plan_signature(info.as_dict()), []).append((M, N, K))
+    return classes
+
+
+def sweep_class_representatives():
+    reps = set(SWEEP_SUBSET) | set(SWEEP_LARGE)
+    for shapes in sweep_plan_classes().values():
+        reps.add(min(shapes, key=lambda s: s[0] * s[1] * s[2]))
+    return sorted(reps, key=lambda s: (s[0] * s[1] * s[2], s))
+
+
+SWEEP_SEEN_SIGNATURES = set()
+
+
+@pytest.mark.parametrize("M,N,K", sweep_class_representatives(), ids=lambda v: str(v))
+def test_shape_sweep_every_plan_class_meets_the_oracle(M, N, K):
+    """Configuration 5: at least one shape of every plan class the library picks over the 216 sweep
+    shapes (and the largest shapes by name) against the oracle: the full matrix where that takes
+    seconds, else corner/centre blocks in full + tile edges + 2^16 random entries + Freivalds."""
     p = synth.sweep_problem(M, N, K).generate()
     if M * N * K <= 2 ** 32:
-        check_full(p, literal=True)
+        *_, info = check_full(p, literal=True)
     else:
-        check_sampled(p)
+        _, info = check_sampled(p)
+    SWEEP_SEEN_SIGNATURES.add(plan_signature(info))
+
+
+def test_shape_sweep_classes_on_this_device_were_all_checked():
+    """The classes above come from a preview for 148 SMs; this asks the device itself for the plan of
+    every sweep shape and requires that each signature it reports was met by the test above."""
+    import itertools
+    if not SWEEP_SEEN_SIGNATURES:
+        pytest.skip("runs after test_shape_sweep_every_plan_class_meets_the_oracle")
+    missing = {}
+    for M, N, K in itertools.product(synth.SWEEP_DIMS, repeat=3):
+        with B.Plan(B.make_desc(M, N, K, BF16, FP32, 0, 1, 0)) as plan:
+            sig = plan_signature(plan.info())
+        if sig not in SWEEP_SEEN_SIGNATURES:
+            missing.setdefault(sig, []).append((M, N, K))
+    assert not missing, missing

@@ -279,6 +279,43 @@ def test_metric_flags_a_single_bad_entry_and_passes_a_small_one():
     assert oracle.max_error(nanc, cref, den) == np.inf
 
 
+def test_output_rounding_slack_is_half_an_ulp_of_the_output_type():
+    """The widened gate of the 16-bit-output tests: slack = u_out * |Cref| with u_out = 2^-8 (bf16),
+    2^-11 (fp16), 0 (fp32).  Pinned against the spacing of the output type itself: at a point halfway
+    between two neighbouring representable values the slack covers the half ulp a correctly rounded
+    result is off by, and stays below a whole ulp -- twice or half the constant fails one of the two."""
+    def bf16_value(bits):
+        return float((np.array([bits], np.uint32) << np.uint32(16)).view(np.float32)[0])
+    for e in (-3, 0, 1, 8, 11):                      # binades [2^e, 2^(e+1))
+        for frac in (0, 1, 37, 127):                 # of the 7 stored fraction bits
+            bits = ((127 + e) << 7) | frac
+            lo, hi = bf16_value(bits), bf16_value(bits + 1)
+            ulp, mid = hi - lo, 0.5 * (lo + hi)
+            for sign in (1.0, -1.0):
+                slack = float(oracle.output_rounding_slack(np.array([sign * mid]), BF16)[0])
+                assert 0.5 * ulp <= slack < ulp, (e, frac, slack, ulp)
+    for x16 in (np.float16(1.0), np.float16(0.3333), np.float16(2048.0), np.float16(3.0e-3), np.float16(60000.0)):
+        lo, ulp = float(x16), float(np.spacing(x16))
+        mid = lo + 0.5 * ulp
+        slack = float(oracle.output_rounding_slack(np.array([-mid]), FP16)[0])
+        assert 0.5 * ulp <= slack < ulp, (x16, slack, ulp)
+    assert np.all(oracle.output_rounding_slack(np.array([1.0, -257.0, 1e30]), FP32) == 0.0)
+    # the gate as the GPU tests apply it, on an all-positive sum that is a bf16 tie: K = 257 ones.
+    # Cref = Den = 257 lies halfway between 256 and 258; the correctly rounded result (either
+    # neighbour) is off by 1 = half an ulp, which the literal 1e-3 * Den = 0.257 rejects and the
+    # widened gate accepts; a result one whole ulp further away is rejected.
+    K = 257
+    cref, den = run(np.ones((3, K)), np.ones((K, 2)), np.zeros((3, 2)), BF16, BF16, 1.0, 0.0)
+    assert np.all(cref == K) and np.all(den == K)
+    rounded = oracle.widen(synth.round_to_storage(cref.astype(np.float32), BF16), BF16)   # storage rounding, not the oracle's
+    assert set(np.unique(rounded)) <= {256.0, 258.0}
+    gate = oracle.TOLERANCE * den + oracle.output_rounding_slack(cref, BF16)
+    assert np.all(np.abs(rounded - cref) > oracle.TOLERANCE * den)
+    assert np.all(np.abs(rounded - cref) <= gate)
+    for wrong in (254.0, 260.0):
+        assert np.all(np.abs(wrong - cref) > gate)
+
+
 def test_freivalds_accepts_truth_and_catches_a_corrupted_tile():
     p = synth.Problem("t", 96, 80, 128, FP16, FP32, 0, 0, 0, 0.5, 1.0, seed=4, dist="normal").generate()
     cref, den = oracle.gemm_problem(p)

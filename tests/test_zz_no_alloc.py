@@ -73,3 +73,53 @@ def test_static_entry_point_checks_its_arguments_like_the_others():
     assert B.exo_gemm_run_static(ok, ptr + 2, ptr, ptr + 32768, 1.0, 0.0)[0] == B.ERR_ALIGNMENT
     assert B.exo_gemm_run_static(ok, 0, ptr, ptr + 32768, 1.0, 0.0)[0] == B.ERR_NULL
     torch.cuda.synchronize()
+
+
+def test_static_entry_point_enqueues_nothing_when_it_refuses_its_arguments():
+    """A refused call must leave the stream untouched: an event recorded after it is complete at once
+    even while the stream is blocked behind ... nothing.  Checked the cheap way: the status array keeps a
+    marker that only an enqueued clear (or kernel) of a refused call could have changed."""
+    import torch
+    dev = torch.device("cuda:0")
+    p = synth.Problem("static_marker", 256, 256, 128, synth.BF16, synth.FP32, 0, 1, 0, 1.0, 0.0, seed=31).generate()
+    dA, dB, dC = (harness._to_device(x, dev) for x in (p.A, p.B, p.C))
+    desc = harness.desc_of(p)
+    # leave a timeout record in the shared status array ...
+    assert B.exo_gemm_debug_set(None, 20, 0) == B.OK
+    st, detail = B.exo_gemm_run_static(desc, dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), 1.0, 0.0, 0, blocking=True)
+    assert st == B.ERR_DEVICE_TIMEOUT and detail[0] == 1, (st, detail)
+    # ... refused calls do not touch it (they return before anything is enqueued) ...
+    assert B.exo_gemm_run_static(desc, dA.data_ptr() + 2, dB.data_ptr(), dC.data_ptr(), 1.0, 0.0)[0] == B.ERR_ALIGNMENT
+    assert B.exo_gemm_run_static(desc, 0, dB.data_ptr(), dC.data_ptr(), 1.0, 0.0)[0] == B.ERR_NULL
+    empty = B.make_desc(0, 256, 128, synth.BF16, synth.FP32, 0, 1, 0)
+    assert B.exo_gemm_run_static(empty, 0, 0, 0, 1.0, 0.0, 0, blocking=True) == (B.OK, [0] * 8)
+    torch.cuda.synchronize(dev)
+    # ... and the next good call clears it and computes correctly
+    dC.copy_(torch.from_numpy(p.C.view(np.uint8)))
+    st, detail = B.exo_gemm_run_static(desc, dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), 1.0, 0.0, 0, blocking=True)
+    assert st == B.OK and detail[0] == 0, (st, detail)
+    got = oracle.logical_view(dC.cpu().numpy().view(np.float32), p.M, p.N, 0, p.ldc, synth.FP32)
+    assert oracle.max_error(got, *oracle.gemm_problem(p)) <= TOL
+
+
+def test_static_entry_point_recovers_after_a_timed_out_call():
+    """The status array keeps the words of a call whose device-side wait gave up; the next call clears
+    them on its stream before its kernel, whose roles read them only after the stream's earlier work is
+    complete.  Two good calls after a bad one give the bits of the plan-based entry point."""
+    import torch
+    dev = torch.device("cuda:0")
+    p = synth.Problem("static_after_timeout", 1000, 520, 1032, synth.BF16, synth.FP32, 0, 1, 0, 1.0, 0.0, seed=33).generate()
+    want_buf, _ = harness.gemm_host(p, B.flag_split_k(1))
+    dA, dB, dC = (harness._to_device(x, dev) for x in (p.A, p.B, p.C))
+    desc = harness.desc_of(p)
+    stream = torch.cuda.current_stream(dev).cuda_stream
+    assert B.exo_gemm_debug_set(None, 20, 3) == B.OK    # CTA 0's producer leaves out its k-block 3: a wait runs out after 20 ms
+    st, detail = B.exo_gemm_run_static(desc, dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), 1.0, 0.0, stream, blocking=True)
+    assert st == B.ERR_DEVICE_TIMEOUT and detail[0] == 1 and detail[5] == 0, (st, detail)
+    for blocking in (False, True):                       # back to back, no host sync before the first
+        dC.copy_(torch.from_numpy(p.C.view(np.uint8)))
+        st, detail = B.exo_gemm_run_static(desc, dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), 1.0, 0.0, stream,
+                                           blocking=blocking)
+        assert st == B.OK and (detail is None or detail[0] == 0), (st, detail)
+        torch.cuda.synchronize(dev)
+        assert np.array_equal(dC.cpu().numpy().view(np.float32), want_buf)
