@@ -46,7 +46,8 @@ typedef enum { EXO_GEMM_ROW_MAJOR = 0, EXO_GEMM_COL_MAJOR = 1 } exo_gemm_layout_
  *   bit  10     raster direction: 0 = library choice, set = bands along M instead of N
  *   bits 12..19 grid limit: launch at most this many CTAs (multiple of cta_group), 0 = all SMs
  *   bits 20..21 k sub-blocks (of 64 elements) per pipeline stage: 1 or 2
- *   bits 22..23 staging buffers per epilogue warp: 1 or 2
+ *   bits 22..23 staging buffers per epilogue warp: 1 or 2 (also keeps the staged epilogue -- registers ->
+ *               swizzled shared memory -> TMA store -- in runs that could store C straight from registers)
  *   bits 24..27 upper limit on the pipeline depth (2..8)
  *   bits 28..31 K-slices per tile of the partial last wave: 1 = never split, 2..8 = at most this many
  */
@@ -141,6 +142,9 @@ typedef struct {
   int32_t batch_count;     /* matrices per launch (1 unless created by exo_gemm_create_batched) */
   int32_t cluster_size;    /* CTAs per cluster: cta_group, or 4 when two pairs share the loads of A
                               (tiles_n then counts 2 * tile_n columns per step)                 */
+  int32_t stages_direct;   /* depth of the operand ring in runs that store C straight from registers
+                              (no staging buffers: beta == 0 and C, ldc and N multiples of 32 bytes);
+                              0 if the plan always stages (EXO_GEMM_FLAG_EPI_BUFFERS given)        */
 } exo_gemm_info_t;
 
 /*

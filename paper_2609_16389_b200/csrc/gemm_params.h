@@ -71,10 +71,11 @@ struct GemmParams {
   uint32_t umma_k;          // k-elements per MMA: 16 or 8
   uint32_t tf32;            // 1: operands are fp32 in memory and multiplied as tf32
   int32_t stages;           // depth of the operand ring (2 .. kMaxStages)
-  int32_t epi_bufs;         // staging buffers per epilogue warp (1 or 2)
+  int32_t epi_bufs;         // staging buffers per epilogue warp: 1 or 2, or 0 = C is stored straight from registers
   Raster raster;
   uint32_t batch;           // matrices in the strided batch (1 = a plain GEMM, 2-D tensor maps)
   uint32_t tiles_per_batch; // raster.tiles_m * raster.tiles_n
+  FastDiv by_tiles_per_batch;
   uint32_t a_z_mask, b_z_mask;  // all ones, or 0 for an operand that every matrix of the batch shares
   float alpha, beta;
   uint32_t idesc;           // tcgen05 instruction descriptor
@@ -83,6 +84,8 @@ struct GemmParams {
   float* split_ws;          // device: fp32 partial accumulators of the slices 1.. of every tail tile
   uint32_t* split_flags;    // device: one arrival counter per tail tile, never reset, only grows
   uint32_t split_target;    // counter value that means "all partials of this run have landed"
+  void* c_ptr;              // C of matrix 0 and its strides in bytes (read by the direct stores only)
+  int64_t ldc_bytes, c_batch_bytes;
   uint32_t* status;         // device: 8 words {code, role, barrier, tile, k_block, cta, -, -}
   uint64_t timeout_cycles;  // bound of every device-side wait, in SM clocks
   int64_t debug_skip_k_block;  // -1, or the producer k-block of CTA 0 whose loads are skipped

@@ -158,6 +158,8 @@ struct TileConfig {
   int owner_extra;         // k-blocks the owning slice takes beyond an even share
   int64_t workspace_bytes; // fp32 partials of slices 1.. of the tail tiles
   int cta_group, tile_n, ksub, stages, epi_bufs;
+  int stages_direct;       // ring depth of a run that stores C straight from registers (no staging buffers);
+                           // 0: this plan always stages (a staging depth was requested)
   int pairs;               // CTA pairs per cluster (2: the pairs share the loads of A; else 1)
   int mrep;                // 128-row blocks of C per CTA (2: the tall tile; else 1)
   int tiles_m, tiles_n;    // tiles of (128 * cta_group) x (tile_n * pairs): what one cluster computes at a time
@@ -317,6 +319,8 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
   cfg.epi_bufs = o.epi_bufs ? o.epi_bufs : (want_two ? 2 : 1);
   cfg.stages = max_stages(best_g, best_n, cfg.ksub, cfg.epi_bufs, best_r);
   if (o.stages && o.stages < cfg.stages) cfg.stages = o.stages < 2 ? 2 : o.stages;
+  cfg.stages_direct = o.epi_bufs ? 0 : max_stages(best_g, best_n, cfg.ksub, 0, best_r);
+  if (o.stages && o.stages < cfg.stages_direct) cfg.stages_direct = o.stages < 2 ? 2 : o.stages;
   // Wave quantisation: the tiles that do not fill a whole wave are cut along K so that the
   // last wave takes 1/split of a tile's time (split-K applied to the tail only; for a problem
   // smaller than one wave that is plain split-K).

@@ -330,6 +330,14 @@ __device__ __forceinline__ void st_global_v4(void* addr, uint32_t a, uint32_t b,
   asm volatile("st.global.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
+// 256-bit store: eight consecutive 32-bit registers to a 32-byte aligned address, i.e. one full sector
+// per lane.  (With 128-bit stores of a row per lane every sector would be written in two halves.)
+__device__ __forceinline__ void st_global_v8(void* addr, const uint32_t* r) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(addr), "r"(r[0]), "r"(r[1]), "r"(r[2]),
+               "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+               : "memory");
+}
+
 // Bypasses L1: the data was written by another SM.
 __device__ __forceinline__ void ld_global_cg_v4(const void* addr, uint32_t& a, uint32_t& b, uint32_t& c,
                                                 uint32_t& d) {

@@ -27,27 +27,71 @@ struct TileCoord {
   int32_t m, n;
 };
 
+// Division of a 31-bit numerator by a divisor fixed per launch, as a multiply and a shift (the
+// round-up method: m = ceil(2^(31+l) / d) with l = ceil(log2 d) gives floor(n / d) exactly for every
+// n < 2^31).  A hardware division costs the scheduling warps about a hundred clocks at every tile.
+struct FastDiv {
+  uint32_t mul, shift;   // shift == 32: the divisor is 1
+};
+
+inline FastDiv make_fast_div(uint32_t d) {
+  FastDiv f;
+  if (d <= 1) { f.mul = 0; f.shift = 32; return f; }
+  uint32_t l = 0;
+  while ((1ull << l) < d) ++l;                                   // ceil(log2 d) >= 1
+  f.mul = (uint32_t)((((uint64_t)1 << (31 + l)) + d - 1) / d);   // <= 2^32 - 1 for d >= 2
+  f.shift = l - 1;
+  return f;
+}
+
+EXO_HD uint32_t fast_div(uint32_t n, const FastDiv& f) {
+#if defined(__CUDA_ARCH__)
+  return f.shift == 32u ? n : (__umulhi(n, f.mul) >> f.shift);
+#else
+  return f.shift == 32u ? n : (uint32_t)(((uint64_t)n * f.mul) >> 32) >> f.shift;
+#endif
+}
+
 struct Raster {
   int32_t tiles_m, tiles_n;
   int32_t band;      // >= 1
   int32_t along_m;   // 0: bands are groups of tile columns; 1: groups of tile rows
+  FastDiv by_per_band, by_band, by_last;   // divisions by band * minor, by band and by the last band's width
 };
+
+// The raster of a tiles_m x tiles_n grid with its division constants (host side).
+inline Raster make_raster(int32_t tiles_m, int32_t tiles_n, int32_t band, int32_t along_m) {
+  Raster r;
+  r.tiles_m = tiles_m;
+  r.tiles_n = tiles_n;
+  r.band = band < 1 ? 1 : band;
+  r.along_m = along_m ? 1 : 0;
+  const uint32_t major = (uint32_t)(r.along_m ? tiles_m : tiles_n);
+  const uint32_t minor = (uint32_t)(r.along_m ? tiles_n : tiles_m);
+  const uint32_t last = major % (uint32_t)r.band;
+  r.by_per_band = make_fast_div((uint32_t)r.band * (minor ? minor : 1u));
+  r.by_band = make_fast_div((uint32_t)r.band);
+  r.by_last = make_fast_div(last ? last : (uint32_t)r.band);
+  return r;
+}
 
 EXO_HD int64_t raster_total(const Raster& r) { return (int64_t)r.tiles_m * r.tiles_n; }
 
 // linear index -> tile coordinate.  Tile counts stay below 2^31 (checked by the host plan), so
-// the arithmetic is 32-bit: these divisions sit on the critical path of every tile.
+// the arithmetic is 32-bit, and the divisions are multiplications by constants the host prepared:
+// they sit on the critical path of every tile.
 EXO_HD TileCoord raster_decode(const Raster& r, int64_t t64) {
   const uint32_t t = (uint32_t)t64;
   // "major" = the banded dimension, "minor" = the other one
   const uint32_t major = (uint32_t)(r.along_m ? r.tiles_m : r.tiles_n);
   const uint32_t minor = (uint32_t)(r.along_m ? r.tiles_n : r.tiles_m);
   const uint32_t per_band = (uint32_t)r.band * minor;
-  const uint32_t b = t / per_band;
+  const uint32_t b = fast_div(t, r.by_per_band);
   const uint32_t in_band = t - b * per_band;
   const uint32_t first = b * (uint32_t)r.band;
-  const uint32_t width = (major - first) < (uint32_t)r.band ? (major - first) : (uint32_t)r.band;  // last band may be narrower
-  const uint32_t i_minor = in_band / width;
+  const bool narrow = (major - first) < (uint32_t)r.band;         // the last band may be narrower
+  const uint32_t width = narrow ? (major - first) : (uint32_t)r.band;
+  const uint32_t i_minor = fast_div(in_band, narrow ? r.by_last : r.by_band);
   const uint32_t i_major = first + (in_band - i_minor * width);
   TileCoord c;
   c.m = (int32_t)(r.along_m ? i_major : i_minor);
