@@ -300,33 +300,8 @@ def run_ours(args, rank, world, local_rank):
 
     # --- end to end: pinned host buffers, H2D + GEMM + D2H inside the timed region
     e2e_steps = max(3, min(args.steps, 20))
-    hA = torch.from_numpy(p.A.view(np.uint8)).pin_memory()
-    hB = torch.from_numpy(p.B.view(np.uint8)).pin_memory()
-    hC = torch.from_numpy(p.C.view(np.uint8)).pin_memory()
-    hOut = torch.empty_like(hC).pin_memory()
-    dA, dB, dC = sets[0]
-    need_c_in = p.beta != 0.0
-    h2d = hA.numel() + hB.numel() + (hC.numel() if need_c_in else 0)
-    d2h = hOut.numel()
-
-    def e2e_step():
-        dA.copy_(hA, non_blocking=True)
-        dB.copy_(hB, non_blocking=True)
-        if need_c_in:
-            dC.copy_(hC, non_blocking=True)
-        plan.run(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), p.alpha, p.beta, stream.cuda_stream)
-        hOut.copy_(dC, non_blocking=True)
-
-    for _ in range(2):
-        e2e_step()
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(e2e_steps):
-        e2e_step()
-    e1.record(stream)
-    barrier()
-    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    e2e = end_to_end(p, dev, stream, plan, sets[0], e2e_steps, barrier, args.flags, flags2, local_rank)
+    e2e_ms, h2d, d2h = e2e["ms_per_step"], e2e["h2d_bytes_per_step"], e2e["d2h_bytes_per_step"]
     clocks = sampler.stop()
     plan.check()
 
@@ -396,7 +371,8 @@ def run_ours(args, rank, world, local_rank):
             "iqr_mean_ms": float(iqr.mean()) if iqr.size else None, "min_ms": float(per_step.min()),
             "roofline": roofline,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
-                    "d2h_bytes_per_step": int(d2h), "ms_per_step": e2e_ms, "steps": e2e_steps},
+                    "d2h_bytes_per_step": int(d2h), "ms_per_step": e2e_ms, "steps": e2e_steps,
+                    "how": e2e["how"], "parity": e2e["parity"]},
             "gpu_launches": args.steps,
             "clocks": clocks,
         }
@@ -482,6 +458,122 @@ def measure_config(name, dev, steps, pk):
             "plan": {k: info[k] for k in ("cta_group", "tile_m", "tile_n", "tile_k", "stages", "epilogue_buffers",
                                           "split_k", "tail_tiles", "grid")},
             "l2_sets": n_sets, "parity": parity}
+
+
+def end_to_end(p, dev, stream, plan, dev_set, steps, barrier, flags, flags2, local_rank):
+    """The same GEMM with HOST buffers: every step uploads its A, B (and C_in if beta != 0) from pinned host
+    memory, computes through exo_gemm_run, and reads its C back to pinned host memory, all inside the
+    timed region.
+
+    Where A and C are row-major the step is pipelined over row bands of C: one stream uploads B and then A
+    band by band, the compute stream runs one exo_gemm_run per band (a plan over a band, base pointers
+    offset) as soon as that band and B have landed, a third stream downloads each finished band of C.
+    PCIe carries both directions at once, and with two sets of device buffers the next step's upload
+    overlaps this step's download.  Otherwise: upload, one GEMM, download, on one stream.
+    """
+    import torch
+    from paper_2609_16389_b200 import binding as B
+    from paper_2609_16389_b200 import harness, synth
+    batch = getattr(p, "batch", 1)
+    hA = torch.from_numpy(p.A.view(np.uint8)).pin_memory()
+    hB = torch.from_numpy(p.B.view(np.uint8)).pin_memory()
+    hC = torch.from_numpy(p.C.view(np.uint8)).pin_memory()
+    hOut = torch.empty_like(hC).pin_memory()
+    need_c_in = p.beta != 0.0
+    h2d = hA.numel() + hB.numel() + (hC.numel() if need_c_in else 0)
+    d2h = hOut.numel()
+    bands = 0
+    if batch == 1 and p.a_layout == synth.ROW_MAJOR and p.c_layout == synth.ROW_MAJOR and p.M >= 2048:
+        for nb in (8, 4, 2):
+            if p.M % (nb * 256) == 0:
+                bands = nb
+                break
+
+    if not bands:
+        dA, dB, dC = dev_set
+
+        def step():
+            dA.copy_(hA, non_blocking=True)
+            dB.copy_(hB, non_blocking=True)
+            if need_c_in:
+                dC.copy_(hC, non_blocking=True)
+            plan.run(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), p.alpha, p.beta, stream.cuda_stream)
+            hOut.copy_(dC, non_blocking=True)
+
+        for _ in range(2):
+            step()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            step()
+        e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1) / steps
+        how = "serial: H2D, one exo_gemm_run, D2H on one stream"
+    else:
+        rows = p.M // bands
+        es_ab, es_c = synth.elem_size(p.ab_dtype), synth.elem_size(p.c_dtype)
+        a_band, c_band = rows * p.lda * es_ab, rows * p.ldc * es_c      # bytes per band (row-major, rows apart by ld)
+        band_desc = B.make_desc(rows, p.N, p.K, p.ab_dtype, p.c_dtype, p.a_layout, p.b_layout, p.c_layout,
+                                p.lda, p.ldb, p.ldc, device=local_rank, flags=flags, flags2=flags2)
+        band_plan = B.Plan(band_desc)
+        dsets = [tuple(torch.empty_like(t) for t in dev_set) for _ in range(2)]
+        up, down = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+        busy = [None, None]     # last event of the step that used a device set (its download), before the set is reused
+
+        def step(k):
+            dA, dB, dC = dsets[k % 2]
+            with torch.cuda.stream(up):
+                if busy[k % 2] is not None:
+                    up.wait_event(busy[k % 2])
+                dB.copy_(hB, non_blocking=True)
+                landed = []
+                for i in range(bands):
+                    dA[i * a_band:(i + 1) * a_band].copy_(hA[i * a_band:(i + 1) * a_band], non_blocking=True)
+                    if need_c_in:
+                        dC[i * c_band:(i + 1) * c_band].copy_(hC[i * c_band:(i + 1) * c_band], non_blocking=True)
+                    ev = torch.cuda.Event()
+                    ev.record(up)
+                    landed.append(ev)
+            for i in range(bands):
+                stream.wait_event(landed[i])
+                band_plan.run(dA.data_ptr() + i * a_band, dB.data_ptr(), dC.data_ptr() + i * c_band, p.alpha, p.beta,
+                              stream.cuda_stream)
+                done = torch.cuda.Event()
+                done.record(stream)
+                with torch.cuda.stream(down):
+                    down.wait_event(done)
+                    hOut[i * c_band:(i + 1) * c_band].copy_(dC[i * c_band:(i + 1) * c_band], non_blocking=True)
+            last = torch.cuda.Event()
+            last.record(down)
+            busy[k % 2] = last
+            return last
+
+        for k in range(2):
+            step(k)
+        barrier()
+        torch.cuda.synchronize(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        up.wait_stream(stream)
+        e0.record(up)
+        stream.wait_event(e0)
+        last = None
+        for k in range(steps):
+            last = step(k)
+        stream.wait_event(last)          # the step's result is on the host when the timed region ends
+        e1.record(stream)
+        barrier()
+        torch.cuda.synchronize(dev)
+        ms = e0.elapsed_time(e1) / steps
+        band_plan.check()
+        band_plan.close()
+        how = (f"pipelined over {bands} row bands of C: upload stream (B, then A band by band), one exo_gemm_run per band, "
+               "download stream; two device buffer sets")
+    parity = None
+    if batch == 1:
+        parity = sampled_parity(p, hOut.numpy().view(synth.storage_np_dtype(p.c_dtype)), 1 << 12)
+    return {"ms_per_step": ms, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "how": how, "parity": parity}
 
 
 def time_cublas(p, dev, steps, n_sets, ours_step=None):

@@ -49,7 +49,7 @@ typedef enum { EXO_GEMM_ROW_MAJOR = 0, EXO_GEMM_COL_MAJOR = 1 } exo_gemm_layout_
  *   bits 22..23 staging buffers per epilogue warp: 1 or 2 (also keeps the staged epilogue -- registers ->
  *               swizzled shared memory -> TMA store -- in runs that could store C straight from registers)
  *   bits 24..27 upper limit on the pipeline depth (2..8)
- *   bits 28..31 K-slices per tile of the partial last wave: 1 = never split, 2..8 = at most this many
+ *   bits 28..31 K-slices per tile of the partial last wave: 1 = never cut, 2..8 = at most this many on average
  */
 #define EXO_GEMM_FLAG_CTA_GROUP(g)  ((uint32_t)(g) & 3u)
 #define EXO_GEMM_FLAG_TILE_N(n)     ((((uint32_t)(n) / 64u) & 15u) << 2)
@@ -136,12 +136,13 @@ typedef struct {
   int32_t sm_count;
   int32_t kernel_launches_per_run; /* 1, or 0 for an empty problem                             */
   int32_t epilogue_buffers; /* staging buffers per epilogue warp (1 or 2)                      */
-  int32_t split_k;         /* K-slices per tile of the partial last wave (1 = none)            */
+  int32_t split_k;         /* the most K-slices a tile of the partial last wave is cut into (1 = none) */
   int32_t tail_tiles;      /* tiles in that partial last wave                                  */
   int32_t workspace_bytes; /* device scratch the plan owns for the slices' partial sums        */
   int32_t batch_count;     /* matrices per launch (1 unless created by exo_gemm_create_batched) */
   int32_t cluster_size;    /* CTAs per cluster: cta_group, or 4 when two pairs share the loads of A
                               (tiles_n then counts 2 * tile_n columns per step)                 */
+  int32_t tail_workers;    /* workers that share the k-blocks of the tail tiles in equal ranges (0 = none) */
   int32_t stages_direct;   /* depth of the operand ring in runs that store C straight from registers
                               (no staging buffers: beta == 0 and C, ldc and N multiples of 32 bytes);
                               0 if the plan always stages (EXO_GEMM_FLAG_EPI_BUFFERS given)        */
@@ -163,7 +164,8 @@ exo_gemm_status_t exo_gemm_validate(const exo_gemm_desc_t* desc);
  * clusterDim and warp configuration, and the persistent task loop of
  * Section 4.2).  Allocates host state, one 32-byte device status block and, if the
  * tiles of a partial last wave are to be cut along K (exo_gemm_info_t.split_k > 1),
- * a device workspace of exo_gemm_info_t.workspace_bytes for their partial sums;
+ * a device workspace of exo_gemm_info_t.workspace_bytes for their partial sums, one
+ * arrival counter per such tile and a 64-byte-per-worker table of who computes what;
  * touches no user matrix.  *out is written only on success.
  */
 exo_gemm_status_t exo_gemm_create(exo_gemm_handle_t* out, const exo_gemm_desc_t* desc);
@@ -328,18 +330,28 @@ int64_t exo_gemm_schedule_enumerate(int32_t tiles_m, int32_t tiles_n, int32_t ba
 /*
  * Host-side enumeration of one worker's work list including the K-slicing of the
  * tail tiles (the paper's Section 6 measures split-K variants of its GEMM against
- * wave quantisation; here only the tiles of the partial last wave are cut, into
- * `split` slices each, slice 0 owning the output and taking `owner_extra` k-blocks
- * more than an even share).  The items come in the order the worker executes them:
- * a contributing slice (slice > 0) before the worker's whole tiles, the owning slice
- * after them, so that the partial sums are in memory before the owner needs them.
- * `tiles` tiles, `num_workers` workers; writes tile index, slice and k-block range [begin, end) of
- * `num_k_blocks` per item (capacity `cap`); returns the item count, or -1 on bad
- * arguments (including tail_tiles * split > num_workers).  Needs no GPU.
+ * wave quantisation; here only the tiles of the partial last wave are cut: their
+ * k-blocks, in tile-major order, are shared out among `tail_workers` workers in equal
+ * consecutive ranges, so a range may cover the end of one tile and the beginning of
+ * the next; the part of a tile that starts at k-block 0 is slice 0 and owns the
+ * output, the other parts contribute partial sums in K order).  The items come in the
+ * order the worker executes them: a contributing part (slice > 0) before the worker's
+ * whole tiles, an owning part after them, so that the partial sums are in memory
+ * before the owner needs them.  `tiles` tiles, `num_workers` workers; tail_workers ==
+ * 0 leaves the tail tiles whole.  A range boundary within `snap` k-blocks of a tile
+ * boundary is moved onto it (parts of a few k-blocks are not worth an exchange; at
+ * most num_k_blocks / 8).  Where tail_workers is a multiple f of the tail tile count, every
+ * tail tile is instead cut into f slices at the same k-blocks, slice s of tail tile t goes to
+ * worker s * tail_tiles + t, and slice 0 takes `owner_extra` k-blocks more than an even
+ * share.  Writes tile index, slice, slices (parts the tile is
+ * cut into; 1 = whole) and k-block range [begin, end) of `num_k_blocks` per item
+ * (capacity `cap`); returns the item count, or -1 on bad arguments (including
+ * tail_workers below the tail tile count, above num_workers, or above the tail's
+ * k-block count).  Needs no GPU.
  */
-int64_t exo_gemm_schedule_work(int64_t tiles, int32_t num_workers, int32_t split, int32_t owner_extra,
-                               int32_t num_k_blocks, int32_t worker, int64_t* out_tile, int32_t* out_slice, int32_t* out_kb_begin,
-                               int32_t* out_kb_end, int64_t cap);
+int64_t exo_gemm_schedule_work(int64_t tiles, int32_t num_workers, int32_t tail_workers, int32_t num_k_blocks, int32_t snap,
+                               int32_t owner_extra, int32_t worker, int64_t* out_tile, int32_t* out_slice, int32_t* out_slices,
+                               int32_t* out_kb_begin, int32_t* out_kb_end, int64_t cap);
 
 /*
  * Test hook for the bounded waits: the next exo_gemm_run on this plan uses

@@ -50,7 +50,7 @@ class Info(ctypes.Structure):
         "cta_group", "tile_m", "tile_n", "tile_k", "stages", "grid", "smem_bytes", "tmem_columns",
         "tiles_m", "tiles_n", "raster_along_m", "raster_band", "swapped", "sm_count",
         "kernel_launches_per_run", "epilogue_buffers", "split_k", "tail_tiles", "workspace_bytes",
-        "batch_count", "cluster_size", "stages_direct")]
+        "batch_count", "cluster_size", "tail_workers", "stages_direct")]
 
     def as_dict(self):
         return {n: getattr(self, n) for n, _ in self._fields_}
@@ -101,8 +101,8 @@ def lib():
         L.exo_gemv_run.restype = ctypes.c_int
         L.exo_gemv_run_colmajor.argtypes = [i64, i64, vp, i64, vp, vp, ctypes.c_float, ctypes.c_float, vp]
         L.exo_gemv_run_colmajor.restype = ctypes.c_int
-        L.exo_gemm_schedule_work.argtypes = [i64, i32, i32, i32, i32, i32, ctypes.POINTER(i64), ctypes.POINTER(i32),
-                                             ctypes.POINTER(i32), ctypes.POINTER(i32), i64]
+        L.exo_gemm_schedule_work.argtypes = [i64, i32, i32, i32, i32, i32, i32, ctypes.POINTER(i64), ctypes.POINTER(i32),
+                                             ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32), i64]
         L.exo_gemm_schedule_work.restype = i64
         L.exo_gemm_run_static.argtypes = [ctypes.POINTER(Desc), vp, vp, vp, ctypes.c_float, ctypes.c_float, vp,
                                           ctypes.POINTER(ctypes.c_uint32)]
@@ -216,18 +216,17 @@ def exo_gemm_schedule_enumerate(tiles_m, tiles_n, band, along_m, num_workers, wo
     return [(om[i], on[i]) for i in range(n)]
 
 
-def exo_gemm_schedule_work(tiles, num_workers, split, num_k_blocks, worker, owner_extra=0):
-    """[(tile, slice, kb_begin, kb_end), ...] for one worker, tail tiles cut into `split` K-slices."""
-    n = lib().exo_gemm_schedule_work(tiles, num_workers, split, owner_extra, num_k_blocks, worker,
-                                     None, None, None, None, 0)
+def exo_gemm_schedule_work(tiles, num_workers, tail_workers, num_k_blocks, worker, snap=0, owner_extra=0):
+    """[(tile, slice, slices, kb_begin, kb_end), ...] for one worker; the k-blocks of the tail tiles are
+    shared among `tail_workers` workers in equal consecutive ranges (0: the tail tiles stay whole)."""
+    n = lib().exo_gemm_schedule_work(tiles, num_workers, tail_workers, num_k_blocks, snap, owner_extra, worker,
+                                     None, None, None, None, None, 0)
     if n < 0:
         raise ValueError("bad work-schedule arguments")
     t = (ctypes.c_int64 * max(n, 1))()
-    s = (ctypes.c_int32 * max(n, 1))()
-    b = (ctypes.c_int32 * max(n, 1))()
-    e = (ctypes.c_int32 * max(n, 1))()
-    lib().exo_gemm_schedule_work(tiles, num_workers, split, owner_extra, num_k_blocks, worker, t, s, b, e, n)
-    return [(t[i], s[i], b[i], e[i]) for i in range(n)]
+    s, c, b, e = ((ctypes.c_int32 * max(n, 1))() for _ in range(4))
+    lib().exo_gemm_schedule_work(tiles, num_workers, tail_workers, num_k_blocks, snap, owner_extra, worker, t, s, c, b, e, n)
+    return [(t[i], s[i], c[i], b[i], e[i]) for i in range(n)]
 
 
 # ---- thin convenience wrapper ---------------------------------------------------------

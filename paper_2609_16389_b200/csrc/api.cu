@@ -146,6 +146,7 @@ struct exo_gemm_plan {
   uint32_t* d_status;
   float* d_split_ws;                   // fp32 partials of the tail tiles' K-slices (NULL if none)
   uint32_t* d_split_flags;             // one arrival counter per tail tile
+  exo::TailItem* d_tail_table;         // the workers' ranges of the tail tiles' k-blocks (4 entries per worker)
   std::atomic<uint32_t> split_epoch;   // runs that used the counters so far
   std::mutex split_mutex;              // taking an epoch + launching, and exo_gemm_check's reset, exclude one another
   std::atomic<int32_t> dbg_timeout_ms;
@@ -237,6 +238,7 @@ void fill_info(const exo_gemm_plan* p, exo_gemm_info_t* info) {
   info->grid = p->cfg.workers * p->cfg.cta_group * p->cfg.pairs;
   info->cluster_size = p->cfg.cta_group * p->cfg.pairs;
   info->stages_direct = p->cfg.stages_direct;
+  info->tail_workers = p->cfg.tail_workers;
   info->smem_bytes = p->smem_bytes;
   info->tmem_columns = 2 * p->cfg.tile_n;
   info->tiles_m = p->cfg.tiles_m;
@@ -293,28 +295,40 @@ int64_t exo_gemm_schedule_enumerate(int32_t tiles_m, int32_t tiles_n, int32_t ba
   return n;
 }
 
-int64_t exo_gemm_schedule_work(int64_t tiles, int32_t num_workers, int32_t split, int32_t owner_extra,
-                               int32_t num_k_blocks, int32_t worker, int64_t* out_tile, int32_t* out_slice, int32_t* out_kb_begin,
-                               int32_t* out_kb_end, int64_t cap) {
-  if (tiles < 0 || num_workers < 1 || split < 1 || owner_extra < 0 || num_k_blocks < 0 || worker < 0 || worker >= num_workers || cap < 0 ||
-      (cap > 0 && (!out_tile || !out_slice || !out_kb_begin || !out_kb_end)))
+int64_t exo_gemm_schedule_work(int64_t tiles, int32_t num_workers, int32_t tail_workers, int32_t num_k_blocks, int32_t snap,
+                               int32_t owner_extra, int32_t worker, int64_t* out_tile, int32_t* out_slice, int32_t* out_slices,
+                               int32_t* out_kb_begin, int32_t* out_kb_end, int64_t cap) {
+  if (tiles < 0 || num_workers < 1 || tail_workers < 0 || tail_workers > num_workers || num_k_blocks < 0 || snap < 0 || owner_extra < 0 || worker < 0 ||
+      worker >= num_workers || cap < 0 ||
+      (cap > 0 && (!out_tile || !out_slice || !out_slices || !out_kb_begin || !out_kb_end)))
     return -1;
-  WorkPlan w;
-  w.full_tiles = (tiles / num_workers) * num_workers;
+  WorkPlan w{};
+  w.waves = (int32_t)(tiles / num_workers);
+  w.full_tiles = (int64_t)w.waves * num_workers;
   w.tail_tiles = (int32_t)(tiles - w.full_tiles);
-  w.split = split;
-  w.owner_extra = owner_extra;
-  if ((int64_t)w.tail_tiles * split > num_workers) return -1;
+  w.tail_workers = tail_workers;
+  TailItem* table = nullptr;
+  if (tail_workers > 0) {
+    // the plans the library makes: every range holds a k-block and no range is longer than a tile
+    if (w.tail_tiles == 0 || tail_workers < w.tail_tiles || (int64_t)tail_workers > (int64_t)w.tail_tiles * num_k_blocks)
+      return -1;
+    table = new (std::nothrow) TailItem[4 * (size_t)num_workers];
+    if (!table) return -1;
+    w.slots = build_tail_table(w.tail_tiles, num_k_blocks, tail_workers, num_workers, table, snap, owner_extra);
+    w.table = table;
+  }
   int64_t n = 0;
   WorkItem wi;
   for (int64_t i = 0; work_item(w, worker, num_workers, i, num_k_blocks, &wi); ++i, ++n) {
     if (n < cap) {
       out_tile[n] = wi.tile;
       out_slice[n] = wi.slice;
+      out_slices[n] = wi.slices;
       out_kb_begin[n] = wi.kb_begin;
       out_kb_end[n] = wi.kb_end;
     }
   }
+  delete[] table;
   return n;
 }
 
@@ -392,14 +406,26 @@ exo_gemm_status_t exo_gemm_create_batched(exo_gemm_handle_t* out, const exo_gemm
   if (e != cudaSuccess) { delete p; return cuda_fail(e); }
   e = cudaMemset(p->d_status, 0, kStatusBytes);
   if (e != cudaSuccess) { cudaFree(p->d_status); delete p; return cuda_fail(e); }
-  if (p->cfg.split > 1) {  // scratch for the K-slices of the tail tiles
+  if (p->cfg.tail_workers > 0) {  // scratch for the K-slices of the tail tiles, and who computes which
     e = cudaMalloc((void**)&p->d_split_ws, (size_t)p->cfg.workspace_bytes);
     const size_t flag_bytes = sizeof(uint32_t) * (size_t)p->cfg.tail_tiles * (size_t)p->cfg.pairs;
     if (e == cudaSuccess) e = cudaMalloc((void**)&p->d_split_flags, flag_bytes);
     if (e == cudaSuccess) e = cudaMemset(p->d_split_flags, 0, flag_bytes);
+    const size_t table_entries = 4 * (size_t)p->cfg.workers;
+    TailItem* table = new (std::nothrow) TailItem[table_entries];
+    if (e == cudaSuccess && !table) e = cudaErrorMemoryAllocation;
+    if (e == cudaSuccess) {
+      const int64_t k_scaled = p->canon.K * (p->canon.ab_bytes / 2);
+      const int32_t nkb = (int32_t)((k_scaled + kBlockK * p->cfg.ksub - 1) / (kBlockK * p->cfg.ksub));
+      build_tail_table(p->cfg.tail_tiles, nkb, p->cfg.tail_workers, p->cfg.workers, table, p->cfg.snap, p->cfg.owner_extra);
+      e = cudaMalloc((void**)&p->d_tail_table, table_entries * sizeof(TailItem));
+    }
+    if (e == cudaSuccess) e = cudaMemcpy(p->d_tail_table, table, table_entries * sizeof(TailItem), cudaMemcpyHostToDevice);
+    delete[] table;
     if (e != cudaSuccess) {
       cudaFree(p->d_split_ws);
       cudaFree(p->d_split_flags);
+      cudaFree(p->d_tail_table);
       cudaFree(p->d_status);
       delete p;
       return cuda_fail(e);
@@ -488,8 +514,9 @@ exo_gemm_status_t launch_plan(exo_gemm_plan* plan, const void* A, const void* B,
   prm.ldc_bytes = cn.ldc * cn.c_bytes;
   prm.c_batch_bytes = cn.stride_c * cn.c_bytes;
   // the tail tiles are cut along K only when there is a K loop to cut and scratch to reduce through
-  const bool split_now = cfg.split > 1 && read_ab && plan->d_split_ws != nullptr;
-  prm.work = WorkPlan{cfg.full_tiles, cfg.tail_tiles, split_now ? cfg.split : 1, split_now ? cfg.owner_extra : 0};
+  const bool split_now = cfg.tail_workers > 0 && read_ab && plan->d_split_ws != nullptr;
+  prm.work = WorkPlan{cfg.full_tiles, (int32_t)(cfg.full_tiles / cfg.workers), cfg.tail_tiles, split_now ? cfg.tail_workers : 0,
+                      cfg.slots, plan->d_tail_table};
   prm.split_ws = plan->d_split_ws;
   prm.split_flags = plan->d_split_flags;
   prm.split_target = 0;
@@ -577,7 +604,7 @@ exo_gemm_status_t launch_plan(exo_gemm_plan* plan, const void* A, const void* B,
     // to zero after an abandoned run) never falls between the two on another host thread.
     std::lock_guard<std::mutex> lock(plan->split_mutex);
     const uint32_t epoch = plan->split_epoch.fetch_add(1) + 1;
-    prm.split_target = epoch * (uint32_t)((cfg.split - 1) * kEpiWarps * cfg.cta_group * cfg.mrep);
+    prm.split_target = epoch * (uint32_t)(kEpiWarps * cfg.cta_group * cfg.mrep);   // per contributing slice of a tile
     e = cudaLaunchKernelEx(&lc, plan->kernel, tm_a, tm_b, tm_c, prm);
   } else {
     e = cudaLaunchKernelEx(&lc, plan->kernel, tm_a, tm_b, tm_c, prm);
@@ -737,6 +764,7 @@ exo_gemm_status_t exo_gemm_destroy(exo_gemm_handle_t plan) {
     }
     if (plan->d_split_ws) cudaFree(plan->d_split_ws);
     if (plan->d_split_flags) cudaFree(plan->d_split_flags);
+    if (plan->d_tail_table) cudaFree(plan->d_tail_table);
   }
   delete plan;
   return st;

@@ -438,7 +438,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         const int64_t t = wi.tile;
         // The owning slice of a tail tile that follows at least two whole tiles starts from an accumulator
         // into which the epilogue warps have already written the other slices' partial sums.
-        const bool preloaded = MREP == 1 && wi.slices > 1 && wi.slice == 0 && it >= preload_from;
+        const bool preloaded = MREP == 1 && wi.slices > 1 && wi.slice == 0 && wi.after_whole && it >= preload_from;
         if constexpr (MREP == 1) {
           // the epilogue (of both CTAs) must have drained this accumulator
           ok = wait_barrier<PAIR>(tempty_bar(acc), acc_ph ^ 1u, p, WaitSite{kRoleMma, 100 + acc, (uint32_t)t, 0});
@@ -521,11 +521,11 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     uint32_t acc = 0, acc_ph = 0;
 
     // Partial accumulators of the K-slices of a tail tile travel through a private fp32 workspace in a
-    // layout where a warp's 16-byte pieces are contiguous (coalesced both ways): [tail tile][slice-1]
+    // layout where a warp's 16-byte pieces are contiguous (coalesced both ways): [tail tile][slot = slice-1]
     // [cta][warp][accumulator][chunk][unit][piece][lane]; a unit is 32 lanes x 32 columns x 4 bytes.
     constexpr uint32_t kUnitBytes = 8u * 512u;
     auto ws_addr = [&](const WorkItem& w, int32_t slice_m1, int32_t r, int32_t i, int32_t q) {
-      const uint64_t idx = ((((uint64_t)w.tail_index * (uint32_t)(w.slices - 1) + (uint32_t)slice_m1) * CLUSTER +
+      const uint64_t idx = ((((uint64_t)w.tail_index * (uint32_t)p.work.slots + (uint32_t)slice_m1) * CLUSTER +
                              slot_rank) * kEpiWarps + ew) * (uint32_t)(MREP * ((NCHUNK + 1) / 2) * UPC) +
                            (uint32_t)((r * ((NCHUNK + 1) / 2) + i) * UPC + q);
       return reinterpret_cast<char*>(p.split_ws) + idx * kUnitBytes + lane * 16u;
@@ -550,10 +550,12 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     // copy-issuing warps share the instruction issue slots and the memory pipeline with this warp.
     auto wait_partials = [&](const WorkItem& w, int32_t r) {
       const uint32_t* flag = p.split_flags + w.tail_index * NPAIR + (int32_t)pair_id;
+      // the counter only grows: every contributing part of every run adds one arrival per warp
+      const uint32_t target = p.split_target * (uint32_t)(w.slices - 1);
       const long long t_start = clock64();
       uint32_t spins = 0;
       for (;;) {
-        bool ready = lane == 0 && (int32_t)(ptx::ld_acquire_gpu(flag) - p.split_target) >= 0;
+        bool ready = lane == 0 && (int32_t)(ptx::ld_acquire_gpu(flag) - target) >= 0;
         ready = __shfl_sync(0xffffffffu, ready, 0);
         if (ready) {
           (void)ptx::ld_acquire_gpu(flag);  // every lane orders its own reads of the partials after the counter
@@ -596,7 +598,8 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         // owner's epilogue is an ordinary one.  (With a single whole tile before the slice the partials
         // arrive too late for that; the owner then adds them in its epilogue.)
         WorkItem nx;
-        if (it + 1 >= preload_from && work_item(p.work, worker, num_workers, it + 1, nkb, &nx) && nx.slices > 1 && nx.slice == 0) {
+        if (it + 1 >= preload_from && work_item(p.work, worker, num_workers, it + 1, nkb, &nx) && nx.slices > 1 && nx.slice == 0 &&
+            nx.after_whole) {
           uint32_t bz2;
           const TileCoord tc2 = tile_coord(nx.tile, &bz2);
           const int32_t n_mine = chunks_of(tc2.m * (CTA_M * CTA_GROUP) + (int32_t)cta_rank * CTA_M + (int32_t)quad * 32,
@@ -640,7 +643,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         }
       }
       EXO_TRACE_TILE(it, 3);
-      const bool preloaded = MREP == 1 && wi.slices > 1 && wi.slice == 0 && it >= preload_from;  // see above
+      const bool preloaded = MREP == 1 && wi.slices > 1 && wi.slice == 0 && wi.after_whole && it >= preload_from;  // see above
       // one pass per accumulator of the tile: a single one, or (tall tile) rows 0..127 then 128..255 of the CTA
 #pragma unroll 1
       for (int32_t r = 0; r < MREP; ++r) {

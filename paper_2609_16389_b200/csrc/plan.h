@@ -153,10 +153,14 @@ inline Canonical canonicalize(const exo_gemm_desc_t& d, int64_t batch = 1, int64
 }
 
 struct TileConfig {
-  int64_t full_tiles;      // tiles dealt round-robin as whole-K work items
-  int tail_tiles, split;   // the tiles of the partial last wave, each cut into `split` K-slices
-  int owner_extra;         // k-blocks the owning slice takes beyond an even share
-  int64_t workspace_bytes; // fp32 partials of slices 1.. of the tail tiles
+  int64_t full_tiles;      // tiles dealt round-robin as whole-K work items (whole waves)
+  int tail_tiles;          // the tiles of the partial last wave
+  int tail_workers;        // workers that share those tiles' k-blocks in equal consecutive ranges (0: not cut)
+  int split;               // the most K-slices any tail tile is cut into (1: not cut) = slots + 1
+  int slots;               // partial-sum slots per tail tile in the workspace
+  int snap;                // range boundaries this close to a tile boundary (k-blocks) are moved onto it
+  int owner_extra;         // whole slices side by side: k-blocks the owning slice takes beyond an even share
+  int64_t workspace_bytes; // fp32 partials of the contributing slices of the tail tiles
   int cta_group, tile_n, ksub, stages, epi_bufs;
   int stages_direct;       // ring depth of a run that stores C straight from registers (no staging buffers);
                            // 0: this plan always stages (a staging depth was requested)
@@ -181,8 +185,13 @@ inline double shape_efficiency(int cta_group, int bn) {
   return bn == 256 ? 0.86 : (bn == 128 ? 0.66 : 0.40);
 }
 
-// Main-loop speed of the shared-operand clusters relative to independent pairs.
+// Main-loop speed of the shared-operand clusters relative to independent pairs.  With operand rows that
+// start on 128-byte boundaries the halved fetches of A do not show as time; with rows that do not
+// (K = 1000 16-bit elements: 2000 bytes) every 128-byte piece of a box straddles two lines, the L2 sees
+// twice the requests, and fetching less pays: +0.2 to +10 %, typically +1.5 %, over the 24 sweep shapes
+// with K = 1000 that take 256 x 256 tiles (never slower).
 constexpr double kShareGain = 1.0;
+constexpr double kShareGainUnalignedRows = 1.02;
 // Main-loop speed of the tall tile (256 rows per CTA) relative to the 128-row tile, and the clocks
 // per tile its exposed epilogue costs.
 constexpr double kTallGain = 1.06;
@@ -191,11 +200,18 @@ constexpr double kTallDrain = 4000.0;
 // k-elements in one 128-byte sub-block row: 64 for 16-bit operands, 32 for fp32 storage.
 inline int sub_block_k(int ab_bytes) { return 128 / ab_bytes; }
 
-// How many K-slices each tile of the partial last wave is cut into (1 = not cut).
+// A part of a tail tile shorter than this many k-blocks is not worth the exchange of its partial sums
+// (reading one back costs the owner about 16 * tile_n clocks, a k-block takes 2 * tile_n * ksub).
+inline int32_t tail_snap(int ksub) { return 8 / ksub; }
+
+// How many workers share the k-blocks of the partial last wave's tiles (0 = those tiles stay whole).
+// The tail's tail * num_k_blocks k-blocks are cut into that many equal consecutive ranges; a tile is then
+// computed by tail_workers / tail workers on average and the last wave takes tail / tail_workers of a
+// tile's time, plus the exchange of partial sums.
 // (K is given in units of 128-byte sub-block rows x 64, i.e. already scaled by the element size.)
-inline int split_factor(int64_t tiles, int64_t workers, int64_t K, int ksub, const FlagOverrides& o) {
+inline int tail_workers_for(int64_t tiles, int64_t workers, int64_t K, int ksub, const FlagOverrides& o, int mrep = 1) {
   const int64_t tail = tiles % workers;
-  if (tail == 0 || o.split == 1 || o.no_workspace) return 1;
+  if (tail == 0 || o.split == 1 || o.no_workspace) return 0;
   // A short K loop leaves no main-loop time to save, and the exchange of partial sums (a round trip
   // through L2 plus the extra output traffic) costs about as much as a dozen k-blocks.
   // Behind whole waves the contributing slices run first and the exchange is off the critical path
@@ -208,26 +224,47 @@ inline int split_factor(int64_t tiles, int64_t workers, int64_t K, int ksub, con
   // (With three or more whole waves in front, the workers that start with a slice run out of step with
   // the rest for longer than the shorter last wave saves at K = 1024: -0.7 % at 4096 x 4096 x 1024.)
   const bool behind_waves = tiles >= workers;
-  if (o.split == 0 && K < (behind_waves && tiles / workers <= 2 ? 960 : 2048)) return 1;
+  if (o.split == 0 && K < (behind_waves && tiles / workers <= 2 ? 960 : 2048)) return 0;
   const int64_t k_blocks = (K + kBlockK * ksub - 1) / (kBlockK * ksub);
-  int64_t f = workers / tail;
-  // every slice keeps at least 256 k-elements
-  int64_t by_k = (K / kBlockK) / 4;
+  // slices per tile, on average: every slice keeps about 256 k-elements at least
+  int64_t per_tile = (K / kBlockK) / 4;
   // (from K = 4096 on the owner finds the partials preloaded in its accumulator even behind a single whole
   // wave, and a third slice of 1365 k-elements wins another 2.7-4 % over two)
-  if (o.split == 0 && behind_waves) by_k = K >= 4096 ? K / 1365 : (K / 2048 > 2 ? K / 2048 : 2);
-  if (f > by_k) f = by_k;
-  if (f > 8) f = 8;
-  if (o.split >= 2 && o.split < f) f = o.split;
-  if (f > k_blocks) f = k_blocks;
-  return f >= 2 ? (int)f : 1;
+  if (o.split == 0 && behind_waves) per_tile = K >= 4096 ? K / 1365 : (K / 2048 > 2 ? K / 2048 : 2);
+  if (per_tile > 8) per_tile = 8;
+  if (o.split >= 2 && o.split < per_tile) per_tile = o.split;
+  if (per_tile > k_blocks) per_tile = k_blocks;
+  // Whole slices where at least two per tile fit the workers: every tail tile is cut at the same k-blocks
+  // into f slices, one per worker (tail * f <= workers).
+  const int64_t f = workers / tail < per_tile ? workers / tail : per_tile;
+  if (f >= 2) return (int)(tail * f);
+  if (per_tile < 2) return 0;
+  // (not for the tall tile, whose partial sums are twice as large and whose epilogue nothing hides: 192 tiles
+  // of 512 x 256 on 74 pairs at K = 12288 measured -8 %)
+  if (mrep == 2 && o.split == 0) return 0;
+  // More than half a wave of tail tiles: no two whole slices per tile fit, so the tail's k-blocks are shared
+  // out among ALL workers in equal consecutive ranges that ignore tile boundaries (most tiles end up in
+  // two parts).  Every worker then starts and ends with a part of a tile and exchanges partial sums, so
+  // this pays only where the K loop is long and the last wave shrinks by a fifth of a tile or more
+  // (measured against the uncut tiles: 48 tiles of 256 x 256 on 74 pairs at K = 12288 +4 %; 58 tiles behind
+  // seven whole waves at K = 2048 -7 %).
+  const int64_t tw = workers;
+  if (o.split == 0) {
+    // time saved against the exchange, both in clocks per column of the tile (a k-block of 64 takes 2;
+    // a part's partial sums cost about 16 behind whole waves and about 38 side by side, as in
+    // estimate_clocks): the saving has to be three times the exchange
+    const double saved = (double)k_blocks * ksub * 2.0 * (1.0 - (double)tail / (double)tw);
+    const double exchange = behind_waves ? 16.0 : 38.0;
+    if (saved < 3.0 * exchange || tail * 5 > tw * 4) return 0;
+  }
+  return (int)tw;
 }
 
 // Estimated time of the whole problem in SM clocks for one candidate tile shape: whole waves of
 // tiles, then the partial last wave (cut along K if that pays), plus what is exposed once per launch.
 inline double estimate_clocks(int64_t M, int64_t N, int64_t K, int64_t batch, int cta_group, int bn,
                               int max_workers, const FlagOverrides& o, int pairs = 1, int mrep = 1,
-                              bool mn_major_operand = false) {
+                              bool mn_major_operand = false, bool unaligned_rows = false) {
   const int64_t tm = (M + 128 * cta_group * mrep - 1) / (128 * cta_group * mrep);
   const int64_t tn = (N + bn * pairs - 1) / (bn * pairs);
   const int64_t tiles = tm * tn * batch;
@@ -235,7 +272,7 @@ inline double estimate_clocks(int64_t M, int64_t N, int64_t K, int64_t batch, in
   const int ksub = o.ksub ? o.ksub : (bn == 256 ? 1 : 2);
   const int64_t nkb = (K + kBlockK - 1) / kBlockK;
   double mainloop = (double)nkb * 2.0 * bn / shape_efficiency(cta_group, bn);  // clocks per whole tile
-  if (pairs == 2) mainloop /= kShareGain;
+  if (pairs == 2) mainloop /= unaligned_rows ? kShareGainUnalignedRows : kShareGain;
   (void)mn_major_operand;  // M/N-contiguous operands run at the same rate (measured 1512 against 1516 TFLOP/s at 8192^3)
   // draining one accumulator: 5-7k clocks at N = 256, but only about a third less at N = 128 (waits, tile
   // decode and the last store's latency do not shrink with the tile: at K = 512 the 256-column tile is
@@ -253,13 +290,18 @@ inline double estimate_clocks(int64_t M, int64_t N, int64_t K, int64_t batch, in
   const int64_t tail = tiles % max_workers;
   double t = (double)full_waves * per_tile;
   if (tail > 0) {
-    const int f = split_factor(tiles, max_workers, K, ksub, o);
-    // slice + exchange of partial sums (the tall tile's partials are twice as large and nothing hides them).
-    // Behind whole waves only the owner's reading of the partials is exposed (about 4000 clocks per
-    // contributing slice of a 256-column tile); side by side, publishing and the round trip are as well.
-    const double exchange = (full_waves > 0 ? 16.0 * (f - 1) : 30.0 + 8.0 * (f - 1)) * bn * mrep * mrep;
-    if (f > 1) t += mainloop / f + 2500.0 + exchange;
-    else t += per_tile;
+    const int tw = tail_workers_for(tiles, max_workers, K, ksub, o, mrep);
+    // a range of the tail + the exchange of partial sums (the tall tile's partials are twice as large and
+    // nothing hides them).  Behind whole waves only the owner's reading of the partials is exposed (about
+    // 4000 clocks per contributing slice of a 256-column tile); side by side, publishing and the round
+    // trip are as well.
+    if (tw > 0) {
+      const int64_t parts = (tw + tail - 1) / tail;
+      const double exchange = (full_waves > 0 ? 16.0 * (parts - 1) : 30.0 + 8.0 * (parts - 1)) * bn * mrep * mrep;
+      t += mainloop * (double)tail / (double)tw + 2500.0 + exchange;
+    } else {
+      t += per_tile;
+    }
   }
   return t + drain + 3000.0;  // the last epilogue and the pipeline fill are exposed once
 }
@@ -272,6 +314,8 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
                                  {1, 256, 1, 1}, {1, 128, 1, 1}, {1, 64, 1, 1}};
   int best_g = 0, best_n = 0, best_p = 1, best_r = 1;
   double best = 0;
+  // operand rows (or columns, for M/N-contiguous storage) that do not start on 128-byte boundaries
+  const bool unaligned_rows = c.K > 0 && (((c.lda * c.ab_bytes) % 128) != 0 || ((c.ldb * c.ab_bytes) % 128) != 0);
   for (int i = 0; i < 7; ++i) {
     const int g = cand[i][0], n = cand[i][1], pr = cand[i][2], mr = cand[i][3];
     if (mr == 2 && (o.mrep == 1 || o.share >= 2 || o.ksub == 2)) continue;
@@ -279,20 +323,35 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
     if (o.cta_group && o.cta_group != g) continue;
     if (o.tile_n && o.tile_n != n) continue;
     if (g == 2 && max_pairs < 1) continue;
-    if (pr == 2 && (max_quads < 1 || o.share < 2)) continue;   // only on request
+    if (pr == 2 && (max_quads < 1 || o.share < 2)) continue;   // as a candidate only on request (but see below)
     if (pr == 1 && o.share >= 2 && max_quads >= 1) continue;
     const int workers = pr == 2 ? max_quads : (g == 2 ? max_pairs : sm_count);
     int w_eff = workers;
     if (o.grid_limit && o.grid_limit / (g * pr) < w_eff) w_eff = o.grid_limit / (g * pr);
     if (w_eff < 1) w_eff = 1;
     double t = estimate_clocks(c.M, c.N, c.K * (c.ab_bytes / 2), c.batch, g, n, w_eff, o, pr, mr,
-                               c.a_mn_major || c.b_mn_major);
+                               c.a_mn_major || c.b_mn_major, unaligned_rows);
     if (mr == 2) t *= 1.03;  // the tall tile's exposed epilogue makes it the riskier choice: it must win clearly
     // candidates come largest tile first; a smaller one has to win by 3 %: the estimate flatters small tiles
     // (their fixed costs per tile are only partly modelled)
     if (best_g == 0 || t < best * 0.97) { best = t; best_g = g; best_n = n; best_p = pr; best_r = mr; }
   }
   if (best_g == 0) { best_g = o.cta_group ? o.cta_group : 1; best_n = o.tile_n ? o.tile_n : 128; }
+  // Where the choice fell on plain pairs of 256 x 256 tiles and the operand rows are not 128-byte aligned,
+  // the same tiles in shared-operand clusters are the faster form (see kShareGainUnalignedRows), unless the
+  // slots of two tiles quantise worse than the single tiles did.
+  // (The library's own tile choices only: a caller who names a tile shape gets plain pairs unless the
+  // clusters are asked for as well.)
+  if (best_g == 2 && best_n == 256 && best_p == 1 && best_r == 1 && o.share == 0 && unaligned_rows && max_quads >= 1 &&
+      o.cta_group == 0 && o.tile_n == 0 && o.mrep == 0 && (o.grid_limit & 3) == 0) {
+    int w_eff = max_quads;
+    if (o.grid_limit && o.grid_limit / 4 < w_eff) w_eff = o.grid_limit / 4;
+    if (w_eff >= 1) {
+      const double t = estimate_clocks(c.M, c.N, c.K * (c.ab_bytes / 2), c.batch, 2, 256, w_eff, o, 2, 1,
+                                       c.a_mn_major || c.b_mn_major, true);
+      if (t <= best) best_p = 2;
+    }
+  }
   TileConfig cfg;
   cfg.cta_group = best_g;
   cfg.tile_n = best_n;
@@ -321,37 +380,51 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
   if (o.stages && o.stages < cfg.stages) cfg.stages = o.stages < 2 ? 2 : o.stages;
   cfg.stages_direct = o.epi_bufs ? 0 : max_stages(best_g, best_n, cfg.ksub, 0, best_r);
   if (o.stages && o.stages < cfg.stages_direct) cfg.stages_direct = o.stages < 2 ? 2 : o.stages;
-  // Wave quantisation: the tiles that do not fill a whole wave are cut along K so that the
-  // last wave takes 1/split of a tile's time (split-K applied to the tail only; for a problem
-  // smaller than one wave that is plain split-K).
+  // Wave quantisation: the k-blocks of the tiles that do not fill a whole wave are shared out evenly among
+  // the workers, so that the last wave takes tail / tail_workers of a tile's time (split-K applied to the
+  // tail only; for a problem smaller than one wave that is split-K with slices of equal length).
   {
     const int64_t full_waves = tiles / workers;
     cfg.full_tiles = full_waves * workers;
     cfg.tail_tiles = (int)(tiles - cfg.full_tiles);
     const int64_t k_scaled = c.K * (c.ab_bytes / 2);  // in 16-bit-element units: 64 per sub-block
-    const int64_t k_blocks = (k_scaled + kBlockK * cfg.ksub - 1) / (kBlockK * cfg.ksub);
-    cfg.split = split_factor(tiles, workers, k_scaled, cfg.ksub, o);
-    // Behind whole waves the contributing slices are computed first and the owning slice last, so the
-    // partials are in memory long before they are asked for and K is cut evenly.  In a problem of less
-    // than one wave all slices run side by side: publishing a 128 x N fp32 partial takes a contributor
-    // about as long as 8 k-blocks of 64 (128*N*4 bytes at ~30 B/clk against 2*N clocks of MMA per
-    // k-block), so there the owner computes that much longer.
+    cfg.tail_workers = tail_workers_for(tiles, workers, k_scaled, cfg.ksub, o, best_r);
+    cfg.slots = 0;
+    cfg.snap = 0;
     cfg.owner_extra = 0;
-    if (cfg.split > 1 && cfg.full_tiles == 0) {
-      int64_t extra = 8 / cfg.ksub;
-      const int64_t room = k_blocks / cfg.split - 1;   // every other slice keeps at least one k-block
-      if (extra > room / 2) extra = room / 2;
-      if (extra < 0) extra = 0;
-      cfg.owner_extra = (int)extra;
+    cfg.split = 1;
+    if (cfg.tail_workers > 0) {   // the exact slot count comes from the table of ranges
+      const int32_t nkb = (int32_t)((k_scaled + kBlockK * cfg.ksub - 1) / (kBlockK * cfg.ksub));
+      TailItem* table = new TailItem[4 * (size_t)workers];
+      cfg.snap = o.split >= 2 ? 0 : tail_snap(cfg.ksub);   // a requested slice count is taken literally
+      // In a problem of less than one wave all slices run side by side: publishing a 128 x N fp32 partial
+      // takes a contributor about as long as 8 k-blocks of 64 (128*N*4 bytes at ~30 B/clk against 2*N
+      // clocks of MMA per k-block), so there the owner computes that much longer.
+      if (cfg.full_tiles == 0 && cfg.tail_workers % cfg.tail_tiles == 0) {
+        const int64_t f = cfg.tail_workers / cfg.tail_tiles;
+        int64_t extra = 8 / cfg.ksub;
+        const int64_t room = nkb / f - 1;   // every other slice keeps at least one k-block
+        if (extra > room / 2) extra = room / 2;
+        cfg.owner_extra = (int)(extra < 0 ? 0 : extra);
+      }
+      cfg.slots = build_tail_table(cfg.tail_tiles, nkb, cfg.tail_workers, (int32_t)workers, table, cfg.snap, cfg.owner_extra);
+      delete[] table;
+      cfg.split = cfg.slots + 1;
+      if (cfg.slots == 0) cfg.tail_workers = 0;
     }
     cfg.workspace_bytes = 0;  // filled in by split_workspace_bytes() once the output type is known
   }
   if (tiles < workers) {  // less than one wave: launch only the CTA groups that get a work item
-    workers = tiles * cfg.split;
+    workers = cfg.tail_workers > 0 ? cfg.tail_workers : tiles;
     if (workers < 1) workers = 1;
   }
   cfg.workers = (int)workers;
   cfg.along_m = o.along_m;
+  // Ranges of the tail's k-blocks that ignore tile boundaries put consecutive tiles on consecutive workers,
+  // a fraction of a tile out of step: the operand panel that neighbouring tiles share stays in L2 only if
+  // it is the small one, so the raster walks the shorter side of the tile grid first (6144 x 512 x 12288:
+  // +9 % with bands along M, 512 x 6144 x 12288: -9 %; with whole tiles the direction measured +-0.5 %).
+  if (cfg.tail_workers > 0 && cfg.tail_workers % cfg.tail_tiles != 0 && cfg.tiles_m > cfg.tiles_n) cfg.along_m = 1;
   // Tiles that run together should cover a square patch of C: band width G along
   // the banded dimension minimises (W/G)*extent_other + G*extent_banded.
   const double tile_m = 128.0 * best_g * best_r, tile_n = (double)best_n * best_p;
@@ -368,11 +441,11 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
 // Bytes of fp32 partials: per tail tile and slice beyond the first, every epilogue warp of every
 // CTA of the group stores its chunks as 4 KB units (32 rows x 32 fp32 columns).
 inline int64_t split_workspace_bytes(const TileConfig& cfg, int c_dtype) {
-  if (cfg.split <= 1) return 0;
+  if (cfg.tail_workers <= 0) return 0;
   const int cw = c_dtype == EXO_GEMM_FP32 ? 32 : 64;        // columns per epilogue chunk
   const int nchunk = cfg.tile_n / cw;
   const int units_per_warp = ((nchunk + 1) / 2) * (cw / 32);
-  return (int64_t)cfg.tail_tiles * (cfg.split - 1) * cfg.cta_group * cfg.pairs * cfg.mrep * kEpiWarps * units_per_warp * 4096;
+  return (int64_t)cfg.tail_tiles * cfg.slots * cfg.cta_group * cfg.pairs * cfg.mrep * kEpiWarps * units_per_warp * 4096;
 }
 
 inline int smem_bytes_for(int cta_group, int bn, int ksub, int stages, int epi_bufs, int mrep = 1) {

@@ -101,74 +101,187 @@ EXO_HD TileCoord raster_decode(const Raster& r, int64_t t64) {
 
 // ---------------------------------------------------------------------------
 // Work list of one worker.  Tiles are dealt round-robin for as long as whole
-// waves can be filled (`full_tiles` = the largest multiple of the worker count
-// not above the tile count).  The `tail_tiles` tiles left over would occupy only
-// part of a last wave, so each of them is cut along K into `split` slices and
-// the tail_tiles * split <= num_workers units are dealt one per worker: the
-// last wave then takes about 1/split of a tile's time.  (The paper's Section 6
-// kernels use split-K for the same wave-quantisation problem; here the split is
-// applied only where it pays, and the reduction order is fixed.)  split == 1
-// degenerates to plain round-robin.
+// waves can be filled (`waves` waves of `num_workers` tiles).  The `tail_tiles`
+// tiles left over would occupy only part of a last wave.  Their k-blocks,
+// tail_tiles * num_k_blocks in tile-major order, are instead cut into
+// `tail_workers` equal consecutive ranges, one per worker: a range covers the
+// end of one tile and the beginning of the next, so a tile is computed by two
+// or more workers whatever the ratio of tiles to workers is, and the last wave
+// takes tail_tiles / tail_workers of a tile's time.  (The paper's Section 6
+// kernels use split-K against the same wave-quantisation problem; this is
+// split-K applied to the tail only, with slices that need not end at tile
+// boundaries, and with a fixed reduction order.)  The part of a tile that
+// starts at k-block 0 is the owning slice: its worker adds the other parts'
+// partial sums, in K order, and writes the tile.  tail_workers == 0: the tail
+// tiles are whole-K items like the others.
+//
+// The ranges are laid out by the host into a table of four 16-byte entries per
+// worker -- {items that come first, items in all, -, -} and up to three items
+// -- because finding them takes 64-bit divisions that no role should repeat at
+// every tile.
+struct TailItem {
+  int32_t tail_index;  // which tail tile (the tile is full_tiles + tail_index)
+  int32_t kb_begin, kb_end;
+  int32_t slice_info;  // slice | slices << 16: slice 0 owns the tile, slices - 1 others contribute to it
+};
+
 struct WorkPlan {
-  int64_t full_tiles;   // tiles [0, full_tiles) are whole-K work items
-  int32_t tail_tiles;   // tiles [full_tiles, full_tiles + tail_tiles) are cut into slices
-  int32_t split;        // slices per tail tile, >= 1
-  int32_t owner_extra;  // k-blocks slice 0 takes beyond an even share: the other slices finish
-                        // earlier by about the time it takes them to publish their partial sums
+  int64_t full_tiles;    // tiles [0, full_tiles) are whole-K work items: waves * num_workers
+  int32_t waves;
+  int32_t tail_tiles;    // tiles [full_tiles, full_tiles + tail_tiles)
+  int32_t tail_workers;  // workers that share the tail tiles' k-blocks (0: the tail is not cut)
+  int32_t slots;         // partial-sum slots per tail tile in the workspace: the most contributors any tile has
+  const TailItem* table; // device (or host, for the host-side enumeration): 4 entries per worker
 };
 
 struct WorkItem {
   int64_t tile;         // linear tile index (to be decoded by raster_decode)
   int32_t tail_index;   // index among the tail tiles, or -1 for a whole-K item
-  int32_t slice;        // 0 .. slices - 1; slice 0 owns the output tile
-  int32_t slices;
+  int32_t slice;        // 0 .. slices - 1 in K order; slice 0 owns the output tile
+  int32_t slices;       // parts the tile is cut into (1: a whole-K item)
   int32_t kb_begin, kb_end;  // k-blocks [kb_begin, kb_end) of num_k_blocks
+  int32_t after_whole;  // 1: the item before this one (of the same worker) is a whole tile
 };
 
+// Fills the table (4 * num_workers entries) and returns the number of slots per tail tile.
+// Needs tail_tiles <= tail_workers <= num_workers and tail_workers <= tail_tiles * num_k_blocks.
+// A range boundary that falls within `snap` k-blocks of a tile boundary is moved onto it: a part of a
+// few k-blocks saves less main-loop time than the exchange of its partial sums costs.
+//
+// Where the sharing workers are a multiple f of the tail tiles, every tile is cut into f slices at the
+// same k-blocks instead, slice s of tile t goes to worker s * tail_tiles + t, and the owning slice takes
+// `owner_extra` k-blocks more than an even share (for problems of less than one wave, where all slices
+// run side by side and the others need time to publish their sums).  The owners are then workers
+// 0 .. tail_tiles - 1 and the contributors the workers after them: a worker that starts with a slice stays
+// out of step with the others for the whole launch, and tiles that run in step share their operand panels
+// in L2, so each group is kept contiguous in the tile order (measured: +0.5 % against -1 to -2.8 % with
+// owners and contributors interleaved).
+inline int32_t build_tail_table(int32_t tail_tiles, int32_t num_k_blocks, int32_t tail_workers, int32_t num_workers,
+                                TailItem* table, int32_t snap = 0, int32_t owner_extra = 0) {
+  if (tail_workers % tail_tiles == 0) {
+    const int32_t f = tail_workers / tail_tiles;
+    int32_t own = (num_k_blocks + f - 1) / f + (f > 1 ? owner_extra : 0);
+    if (own > num_k_blocks - (f - 1)) own = num_k_blocks - (f - 1);
+    if (own < 1) own = 1;
+    if (f == 1) own = num_k_blocks;
+    for (int32_t w = 0; w < num_workers; ++w) {
+      TailItem* e = table + 4 * w;
+      for (int k = 0; k < 4; ++k) e[k] = TailItem{0, 0, 0, 0};
+      if (w >= tail_workers) continue;
+      const int32_t sl = w / tail_tiles;
+      TailItem it;
+      it.tail_index = w - sl * tail_tiles;
+      it.slice_info = sl | (f << 16);
+      if (sl == 0) {
+        it.kb_begin = 0;
+        it.kb_end = own;
+      } else {   // slices 1.. share the rest evenly, in K order
+        const int64_t rest = num_k_blocks - own;
+        it.kb_begin = own + (int32_t)(rest * (sl - 1) / (f - 1));
+        it.kb_end = own + (int32_t)(rest * sl / (f - 1));
+      }
+      e[1] = it;
+      e[0].tail_index = sl > 0 ? 1 : 0;   // contributing slices come first
+      e[0].kb_begin = 1;
+    }
+    return f - 1;
+  }
+  const int64_t units = (int64_t)tail_tiles * num_k_blocks;
+  if (snap > num_k_blocks / 8) snap = num_k_blocks / 8;
+  if (snap > units / tail_workers / 4) snap = (int32_t)(units / tail_workers / 4);   // never a whole range
+  int64_t* bound = new int64_t[(size_t)tail_workers + 1];
+  for (int32_t j = 0; j <= tail_workers; ++j) {
+    int64_t b = (int64_t)j * units / tail_workers;
+    const int64_t r = b % num_k_blocks;
+    if (r != 0 && r <= snap) b -= r;
+    else if (r != 0 && num_k_blocks - r <= snap) b += num_k_blocks - r;
+    bound[j] = b;
+  }
+  // the worker whose range holds unit u (ranges may be empty after snapping: the last one that starts at or before u)
+  auto holder = [&](int64_t u) {
+    int32_t j = (int32_t)((u * tail_workers) / units);
+    if (j > tail_workers - 1) j = tail_workers - 1;
+    while (j + 1 < tail_workers && bound[j + 1] <= u) ++j;
+    while (j > 0 && bound[j] > u) --j;
+    return j;
+  };
+  int32_t slots = 0;
+  for (int32_t w = 0; w < num_workers; ++w) {
+    TailItem* e = table + 4 * w;
+    for (int k = 0; k < 4; ++k) e[k] = TailItem{0, 0, 0, 0};
+    if (w >= tail_workers) continue;
+    const int64_t b0 = bound[w], b1 = bound[w + 1];
+    int32_t n = 0, lead = 0;
+    TailItem late[2];
+    int32_t n_late = 0;
+    for (int64_t a = b0 / num_k_blocks; a * num_k_blocks < b1 && n + n_late < 3; ++a) {
+      const int64_t lo = a * num_k_blocks, hi = lo + num_k_blocks;
+      TailItem it;
+      it.tail_index = (int32_t)a;
+      it.kb_begin = (int32_t)((b0 > lo ? b0 : lo) - lo);
+      it.kb_end = (int32_t)((b1 < hi ? b1 : hi) - lo);
+      // the tile's parts are the non-empty ranges from the one that holds its first k-block (the owner)
+      // to the one that holds its last; this part's number among them is its place in K order
+      const int32_t first = holder(lo), last = holder(hi - 1);
+      int32_t slice = 0, parts = 0;
+      for (int32_t j = first; j <= last; ++j) {
+        if (bound[j + 1] <= bound[j]) continue;
+        if (j < w) ++slice;
+        ++parts;
+      }
+      if (parts - 1 > slots) slots = parts - 1;
+      it.slice_info = slice | (parts << 16);
+      if (it.kb_begin > 0) { e[1 + n++] = it; ++lead; }   // a contributing part: computed first
+      else if (n_late < 2) late[n_late++] = it;            // whole tiles and owning parts: computed last
+    }
+    for (int32_t k = 0; k < n_late; ++k) e[1 + n++] = late[k];
+    e[0].tail_index = lead;
+    e[0].kb_begin = n;
+  }
+  delete[] bound;
+  return slots;
+}
+
 // The i-th work item of `worker`; returns false when the worker has no i-th item.
-// A worker whose unit of a tail tile is a contributing slice (slice > 0) computes that unit FIRST and
-// its whole tiles afterwards: its partial sums then reach memory a whole tile's time before the owning
-// slice (slice 0, computed LAST by its worker) asks for them, and neither side ever waits.
-// The owners are workers 0 .. tail_tiles-1 and the contributors the workers after them: a worker that
-// starts with a slice stays out of step with the others for the whole launch, and tiles that run in step
-// share their operand panels in L2, so each group is kept contiguous in the tile order.
+// A worker's contributing part of a tail tile (it does not start at k-block 0) comes FIRST and its whole
+// tiles afterwards: the partial sums then reach memory a whole tile's time before the owning part
+// (computed LAST by its worker) asks for them, and neither side ever waits.
 EXO_HD bool work_item(const WorkPlan& w, int64_t worker, int64_t num_workers, int64_t i, int32_t num_k_blocks,
                       WorkItem* out) {
-  const bool has_unit = worker < (int64_t)w.tail_tiles * w.split;
-  const bool early = has_unit && worker >= w.tail_tiles;  // a contributing slice (split > 1 follows)
-  if (!(early && i == 0)) {
-    const int64_t t = worker + (early ? i - 1 : i) * num_workers;
-    if (t < w.full_tiles) {
+  int32_t lead = 0, n_items = 0;
+  const TailItem* e = nullptr;
+  if (w.tail_workers > 0) {
+    e = w.table + 4 * worker;
+    lead = e[0].tail_index;
+    n_items = e[0].kb_begin;
+  }
+  int64_t k;   // index into this worker's tail items, if the i-th item is one
+  if (i < lead) {
+    k = i;
+  } else {
+    const int64_t j = i - lead;
+    const int64_t t = worker + j * num_workers;
+    if (j < w.waves || (w.tail_workers == 0 && t < w.full_tiles + w.tail_tiles)) {
       out->tile = t;
       out->tail_index = -1;
       out->slice = 0;
       out->slices = 1;
       out->kb_begin = 0;
       out->kb_end = num_k_blocks;
+      out->after_whole = j >= 1;
       return true;
     }
-    if (early || !has_unit) return false;
-    if (t - w.full_tiles != worker) return false;           // only the wave right after the full ones
+    k = lead + (j - w.waves);
+    if (w.tail_workers == 0 || k >= n_items) return false;
   }
-  const int32_t sl = (int32_t)((uint32_t)worker / (uint32_t)w.tail_tiles);
-  const int32_t ti = (int32_t)((uint32_t)worker - (uint32_t)sl * (uint32_t)w.tail_tiles);
-  out->tile = w.full_tiles + ti;
-  out->tail_index = w.split > 1 ? ti : -1;
-  out->slice = sl;
-  out->slices = w.split;
-  // slice 0: an even share plus owner_extra; slices 1.. share the rest evenly, in K order
-  int32_t own = (num_k_blocks + w.split - 1) / w.split + (w.split > 1 ? w.owner_extra : 0);
-  if (own > num_k_blocks - (w.split - 1)) own = num_k_blocks - (w.split - 1);
-  if (own < 1) own = 1;
-  if (w.split == 1) own = num_k_blocks;
-  if (sl == 0) {
-    out->kb_begin = 0;
-    out->kb_end = own;
-  } else {
-    const uint32_t rest = (uint32_t)(num_k_blocks - own);   // rest * slice < 2^31: both are small
-    out->kb_begin = own + (int32_t)((rest * (uint32_t)(sl - 1)) / (uint32_t)(w.split - 1));
-    out->kb_end = own + (int32_t)((rest * (uint32_t)sl) / (uint32_t)(w.split - 1));
-  }
+  const TailItem it = e[1 + k];
+  out->tile = w.full_tiles + it.tail_index;
+  out->slice = it.slice_info & 0xFFFF;
+  out->slices = it.slice_info >> 16;
+  out->tail_index = out->slices > 1 ? it.tail_index : -1;
+  out->kb_begin = it.kb_begin;
+  out->kb_end = it.kb_end;
+  out->after_whole = i > lead;   // (items that come first have no whole tile before them)
   return true;
 }
 

@@ -188,76 +188,131 @@ def test_create_fails_cleanly_without_a_gpu():
     assert B.exo_gemm_run(None, 0, 0, 0, 1.0, 0.0, 0) == B.ERR_NULL
 
 
-@pytest.mark.parametrize("tiles,workers,split", [(256, 74, 2), (256, 74, 1), (32, 148, 4), (5, 148, 8), (300, 148, 3),
-                                                  (148, 148, 1), (149, 148, 8), (1, 1, 1), (0, 4, 1)])
-@pytest.mark.parametrize("nkb", [64, 7, 1000])
-@pytest.mark.parametrize("extra", [0, 3])
-def test_work_schedule_covers_every_tile_and_k_block_exactly_once(tiles, workers, split, nkb, extra):
+@pytest.mark.parametrize("tiles,workers,tail_workers", [(256, 74, 68), (256, 74, 74), (256, 74, 0), (32, 148, 128), (5, 148, 40),
+                                                        (300, 148, 7), (300, 148, 148), (148, 148, 0), (149, 148, 8),
+                                                        (48, 74, 74), (96, 74, 74), (1, 1, 0), (0, 4, 0), (75, 74, 3)])
+@pytest.mark.parametrize("nkb", [64, 7, 1000, 192])
+@pytest.mark.parametrize("snap", [0, 4, 8])
+def test_work_schedule_covers_every_tile_and_k_block_exactly_once(tiles, workers, tail_workers, nkb, snap):
     tail = tiles % workers
-    if tail * split > workers or split > nkb:
+    if tail_workers and (tail_workers < tail or tail_workers > tail * nkb or tail == 0):
         pytest.skip("not a plan the library would make")
     cover = {}
     longest = 0
+    loads = []
     for w in range(workers):
-        items = B.exo_gemm_schedule_work(tiles, workers, split, nkb, w, extra)
+        items = B.exo_gemm_schedule_work(tiles, workers, tail_workers, nkb, w, snap)
         longest = max(longest, len(items))
-        for tile, sl, b, e in items:
-            assert 0 <= tile < tiles and 0 <= b < e <= nkb
-            cover.setdefault(tile, []).append((b, e, sl))
+        loads.append(sum(e - b for _, _, _, b, e in items))
+        for tile, sl, n_sl, b, e in items:
+            assert 0 <= tile < tiles and 0 <= b < e <= nkb and 0 <= sl < n_sl
+            cover.setdefault(tile, []).append((b, e, sl, n_sl))
+        # the order of execution: contributing parts first, whole tiles, owning parts last
+        kinds = ["c" if sl > 0 else ("o" if n_sl > 1 else "w") for _, sl, n_sl, _, _ in items]
+        assert "".join(kinds).lstrip("c").rstrip("o").strip("w") == "", kinds
     assert sorted(cover) == list(range(tiles))
     for tile, parts in cover.items():
         parts.sort()
         assert parts[0][0] == 0 and parts[-1][1] == nkb
         assert all(parts[i][1] == parts[i + 1][0] for i in range(len(parts) - 1))      # a partition of K
         assert [p[2] for p in parts] == list(range(len(parts)))                         # slice order = K order
-        is_tail = tile >= tiles - tail
-        assert len(parts) == (split if is_tail else 1)
-        sizes = [e - b for b, e, _ in parts]
-        if len(sizes) > 1:
-            assert max(sizes[1:]) - min(sizes[1:]) <= 1                                 # contributors balanced
-            assert sizes[0] >= min(sizes[1:])                                           # the owner takes no less
-    assert longest == -(-tiles // workers)      # nobody does more items than the wave count
+        assert all(p[3] == len(parts) for p in parts)                                   # every part knows how many there are
+        if tile < tiles - tail or not tail_workers:
+            assert len(parts) == 1
+    if tail_workers:
+        # the tail's k-blocks are shared evenly: nobody holds more than a k-block beyond an even share
+        tail_loads = [l - (tiles // workers) * nkb for l in loads]
+        share = [l for l in tail_loads[:tail_workers]]
+        eff_snap = min(snap, nkb // 8, tail * nkb // tail_workers // 4)
+        assert max(share) - min(share) <= 1 + 2 * eff_snap and sum(share) == tail * nkb
+        for tile, parts in cover.items():                       # no part shorter than the snap distance
+            if len(parts) > 1 and nkb * tail >= tail_workers * (2 * eff_snap + 1):
+                assert min(e - b for b, e, _, _ in parts) > eff_snap, (tile, parts)
+        assert all(l == 0 for l in tail_loads[tail_workers:])
+    assert longest <= tiles // workers + 2
 
 
-def test_contributing_slices_come_first_and_owning_slices_last():
-    # 256 tiles on 74 workers, tail tiles cut in two: workers 0..33 own a tail tile and compute their
-    # slice after their whole tiles; workers 34..67 contribute and compute theirs before; the rest have none
-    tiles, workers, split, nkb = 256, 74, 2, 64
-    full = (tiles // workers) * workers
+def test_contributing_parts_come_first_and_owning_parts_last():
+    # 96 tiles on 74 workers with 192 k-blocks each: one whole wave, then 22 tiles whose 4224 k-blocks are
+    # shared by all 74 workers, 57 or 58 each.  A range that starts inside a tile contributes to it (first
+    # item of its worker); a range that starts a tile owns it (last item).
+    tiles, workers, nkb = 96, 74, 192
+    owners, contributors = {}, {}
     for w in range(workers):
-        items = B.exo_gemm_schedule_work(tiles, workers, split, nkb, w, 0)
-        unit = [k for k, (tile, sl, b, e) in enumerate(items) if tile >= full]
-        if w < 34:
-            assert unit == [len(items) - 1] and items[-1][:2] == (full + w, 0) and items[-1][2:] == (0, 32)
-        elif w < 68:
-            assert unit == [0] and items[0][:2] == (full + w - 34, 1) and items[0][2:] == (32, 64)
-        else:
-            assert unit == []
-        whole = [tile for tile, sl, b, e in items if tile < full]
-        assert whole == [w + k * workers for k in range(3)]
+        items = B.exo_gemm_schedule_work(tiles, workers, workers, nkb, w)
+        whole = [(k, it) for k, it in enumerate(items) if it[2] == 1]
+        assert [it[0] for _, it in whole] == [w]                       # its tile of the whole wave
+        for k, (tile, sl, n_sl, b, e) in enumerate(items):
+            if n_sl == 1:
+                continue
+            assert tile >= workers
+            if sl == 0:
+                assert b == 0 and k > whole[0][0] and k == len(items) - 1
+                owners[tile] = w
+            else:
+                assert b > 0 and k < whole[0][0]
+                contributors.setdefault(tile, []).append((sl, w))
+    assert sorted(owners) == list(range(74, 96))
+    for tile, own in owners.items():
+        cs = sorted(contributors[tile])
+        assert [sl for sl, _ in cs] == list(range(1, len(cs) + 1))
+        assert [w for _, w in cs] == [own + k for k in range(1, len(cs) + 1)]   # consecutive workers, in K order
+        assert 3 <= len(cs) + 1 <= 5                                           # 74 / 22 = 3.4 workers per tile
 
 
-def test_work_schedule_rejects_impossible_splits():
+def test_whole_slices_keep_owners_and_contributors_in_groups():
+    # 256 tiles on 74 workers, the 34 tail tiles cut in two whole slices: workers 0..33 own a tail tile and
+    # compute their slice after their whole tiles; workers 34..67 contribute and compute theirs before; the
+    # rest have none.  With an owner_extra of 3 the owning slice is 3 k-blocks longer.
+    tiles, workers, nkb = 256, 74, 64
+    full = (tiles // workers) * workers
+    for extra in (0, 3):
+        for w in range(workers):
+            items = B.exo_gemm_schedule_work(tiles, workers, 68, nkb, w, owner_extra=extra)
+            unit = [k for k, it in enumerate(items) if it[0] >= full]
+            if w < 34:
+                assert unit == [len(items) - 1] and items[-1] == (full + w, 0, 2, 0, 32 + extra)
+            elif w < 68:
+                assert unit == [0] and items[0] == (full + w - 34, 1, 2, 32 + extra, 64)
+            else:
+                assert unit == []
+            assert [it[0] for it in items if it[0] < full] == [w + k * workers for k in range(3)]
+
+
+def test_work_schedule_rejects_impossible_plans():
     with pytest.raises(ValueError):
-        B.exo_gemm_schedule_work(256, 74, 3, 64, 0)      # 34 tail tiles x 3 slices > 74 workers
+        B.exo_gemm_schedule_work(256, 74, 20, 64, 0)       # fewer sharing workers than the 34 tail tiles
     with pytest.raises(ValueError):
-        B.exo_gemm_schedule_work(10, 4, 0, 8, 0)
+        B.exo_gemm_schedule_work(256, 74, 75, 64, 0)       # more than there are workers
+    with pytest.raises(ValueError):
+        B.exo_gemm_schedule_work(149, 148, 8, 4, 0)        # one tail tile of 4 k-blocks cannot feed 8 workers
+    with pytest.raises(ValueError):
+        B.exo_gemm_schedule_work(148, 148, 8, 64, 0)       # no tail to share
 
 
-def test_plan_preview_splits_the_partial_last_wave():
-    # 4096^3 with 256x256 pair tiles: 256 tiles on 74 pairs = 3 whole waves + 34 tiles, cut in two
+def test_plan_preview_shares_the_partial_last_wave():
+    # 4096^3 with 256x256 pair tiles: 256 tiles on 74 pairs = 3 whole waves + 34 tiles, each cut in two
+    # whole slices (68 of the 74 pairs take one)
     st, info = B.exo_gemm_plan_preview(good(M=4096, N=4096, K=4096, c_dtype=B.BF16), 148)
     i = info.as_dict()
-    assert (i["cta_group"], i["tile_n"]) == (2, 256) and i["tail_tiles"] == 34 and i["split_k"] == 2
+    assert (i["cta_group"], i["tile_n"]) == (2, 256) and i["tail_tiles"] == 34
+    assert i["tail_workers"] == 68 and i["split_k"] == 2
     assert i["workspace_bytes"] == 34 * 1 * 256 * 256 * 4
-    # never split when told not to, and never more slices than fit the workers or the K loop
+    # never cut when told not to, and never more slices than fit the workers or the K loop
     st, info = B.exo_gemm_plan_preview(good(M=4096, N=4096, K=4096, flags=B.flag_split_k(1)), 148)
-    assert info.split_k == 1 and info.workspace_bytes == 0
+    assert info.split_k == 1 and info.workspace_bytes == 0 and info.tail_workers == 0
+    st, info = B.exo_gemm_plan_preview(good(M=4096, N=4096, K=4096, flags=B.flag_split_k(2)), 148)
+    assert info.tail_workers == 68 and info.split_k == 2
     st, info = B.exo_gemm_plan_preview(good(M=512, N=512, K=256), 148)
     assert info.split_k == 1                           # 256 k-elements: nothing to cut
     st, info = B.exo_gemm_plan_preview(good(M=512, N=512, K=12288), 148)
     i = info.as_dict()
-    assert i["split_k"] >= 2 and i["tail_tiles"] * i["split_k"] <= i["grid"] // i["cta_group"]
+    assert i["split_k"] >= 2 and i["tail_tiles"] <= i["tail_workers"] <= i["grid"] // i["cta_group"]
+    # a wave count that whole slices cannot fix: 48 tiles of 256 x 256 on 74 pairs.  No two slices per tile fit,
+    # so the 48 x 192 k-blocks are shared out among all 74 pairs in equal ranges that ignore tile boundaries
+    st, info = B.exo_gemm_plan_preview(good(M=1000, N=3072, K=12288, flags=B.flag_cta_group(2) | B.flag_tile_n(256)), 148)
+    i = info.as_dict()
+    assert i["tail_tiles"] == 48 and i["tail_workers"] == 74 and i["split_k"] in (2, 3)
     assert B.exo_gemm_validate(good(flags=B.flag_split_k(9))) == B.ERR_INVALID_ARG
 
 
@@ -295,7 +350,7 @@ def test_shared_operand_cluster_flags_and_preview():
     # slots of four CTAs, each covering 256 x 512 of C per step; 148 SMs hold 37 of them
     assert st == B.OK and (i["cluster_size"], i["cta_group"], i["tile_m"], i["tile_n"]) == (4, 2, 256, 256)
     assert (i["tiles_m"], i["tiles_n"], i["grid"]) == (32, 16, 148)
-    assert i["tail_tiles"] == 512 % 37 and i["tail_tiles"] * i["split_k"] <= 37
+    assert i["tail_tiles"] == 512 % 37 and (i["tail_workers"] == 0 or i["tail_tiles"] < i["tail_workers"] <= 37)
     # the K-slices' scratch covers both tiles of a slot
     assert i["workspace_bytes"] == i["tail_tiles"] * (i["split_k"] - 1) * 2 * 256 * 256 * 4
     st, info = B.exo_gemm_plan_preview(good(M=600, N=700, K=64, flags2=SUBST, flags=B.flag_grid_limit(4)), 148)

@@ -255,7 +255,8 @@ def test_tail_tiles_cut_along_k(case, split):
                       dist="normal" if ab == FP16 else "uniform").generate()
     flags = flags_for(g, bn, grid, split=split)
     cbuf, got, cref, den, info = check_full(p, flags)
-    assert info["tail_tiles"] * info["split_k"] <= info["grid"] // info["cta_group"]
+    assert info["tail_workers"] == 0 or info["tail_tiles"] < info["tail_workers"] <= info["grid"] // info["cluster_size"]
+    assert (info["split_k"] > 1) == (info["tail_workers"] > 0)
     if split == 0 and case in SPLIT_CASES[3:5]:
         assert info["split_k"] >= 2 and info["workspace_bytes"] > 0
     # the slices are reduced in a fixed order: bitwise reproducible, also across repeated runs of one plan
@@ -735,7 +736,8 @@ def plan_signature(info):
     workers = max(1, info["grid"] // info["cluster_size"])
     tiles = info["tiles_m"] * info["tiles_n"]
     return (g, info["tile_m"], info["tile_n"], info["tile_k"], info["stages"], info["epilogue_buffers"],
-            info["split_k"], info["tail_tiles"] > 0, tiles >= workers and info["tail_tiles"] < tiles, info["raster_along_m"])
+            info["split_k"], info["tail_tiles"] > 0, tiles >= workers and info["tail_tiles"] < tiles, info["raster_along_m"],
+            info["cluster_size"])
 
 
 def sweep_plan_classes(sm_count=148):
