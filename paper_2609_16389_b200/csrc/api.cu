@@ -68,6 +68,10 @@ static KernelFn pick_kernel(int cta_group, int bn, int ksub, int out, int pairs 
 
 static thread_local int g_last_cuda_error = 0;
 
+// K (in 16-bit-element units) from which a run that may store C straight from registers does so, for a
+// 32-bit and for a 16-bit C.
+constexpr int64_t kDirectMinK32 = 2048, kDirectMinK16 = 1024;
+
 #ifdef EXO_GEMM_TRACE
 constexpr size_t kStatusBytes = 32 + 3 * 4096 * 2 * 8;  // status block + clock stamps of CTA 0
 #else
@@ -501,11 +505,13 @@ exo_gemm_status_t launch_plan(exo_gemm_plan* plan, const void* A, const void* B,
   prm.b_z_mask = cn.stride_b ? 0xFFFFFFFFu : 0u;
   // Where nothing has to be read back from C and every row of C starts and ends on a 32-byte boundary,
   // the epilogue can store from registers (one full sector per lane) and the staging buffers' shared
-  // memory goes to the operand ring.  That pays where the main loop bounds a tile (a seventh stage:
-  // +0.8 % at 4096^3, +1.6 % at 6144 x 6144 x 2048); where the epilogue does, a row per lane is the slower
-  // way to store (32 lines per instruction: -8 to -13 % at K = 512, -2 to -4 % at K = 1000), so short K
-  // loops keep the staged path.  So does a request for a staging depth (EXO_GEMM_FLAG_EPI_BUFFERS).
-  const bool direct = cfg.stages_direct > 0 && cn.K * (cn.ab_bytes / 2) >= 2048 && beta == 0.f && ((uintptr_t)C & 31u) == 0 &&
+  // memory goes to the operand ring.  That pays where the main loop bounds a tile (a seventh stage.  fp32 C:
+  // +0.8 % at 4096^3, +1.6 % at 6144 x 6144 x 2048; bf16 C: +6 % at 4096 x 4096 x 1024, +3 % at 8192 x 8192 x
+  // 1024 and 4096 x 4096 x 1536); where the epilogue does, a row per lane is the slower way to store (32
+  // lines per instruction.  fp32 C: -8 to -13 % at K = 512, -2 to -4 % at K = 1000; bf16 C: -3 to -5 % at
+  // K = 512), so short K loops keep the staged path.  So does a request for a staging depth
+  // (EXO_GEMM_FLAG_EPI_BUFFERS).
+  const bool direct = cfg.stages_direct > 0 && cn.K * (cn.ab_bytes / 2) >= (cn.c_bytes == 2 ? kDirectMinK16 : kDirectMinK32) && beta == 0.f && ((uintptr_t)C & 31u) == 0 &&
                       (cn.ldc * cn.c_bytes) % 32 == 0 && (cn.N * cn.c_bytes) % 32 == 0 &&
                       (cn.batch <= 1 || (cn.stride_c * cn.c_bytes) % 32 == 0);
   prm.stages = direct ? cfg.stages_direct : cfg.stages;

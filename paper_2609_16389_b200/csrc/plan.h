@@ -369,12 +369,11 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
   // depth matters more than ring depth.  Otherwise the ring takes the space: the time between a
   // stage's release and its reuse has to cover a commit, the producer's wake-up and an L2 or DRAM
   // round trip (measured: 6 stages instead of 5 give +1.3 to +4.6 % for K >= 2048).
-  // A 16-bit C halves the epilogue's stores: at K <= 512 and three or more tiles per worker one buffer
-  // and a deeper ring are then ahead again (measured +2.5 to +7 %; with one or two tiles per worker
-  // -1 to -2 %, and at K = 1000 neutral to -2.7 %).
+  // A 16-bit C halves the epilogue's stores, and one buffer with the deeper ring is then at least level at
+  // every K (bf16 C, 6 stages + 1 buffer against 5 + 2: +3 to +5 % at K = 1000 .. 1024, +1 % at 512 and 1536,
+  // -0.2 % at 12288 x 12288 x 512).
   const int64_t k16 = c.K * (c.ab_bytes / 2);
-  const bool want_two = k16 <= 1024 && !(c.c_bytes == 2 && k16 <= 512 && tiles >= 3 * workers) &&
-                        max_stages(best_g, best_n, cfg.ksub, 2, best_r) >= 3;
+  const bool want_two = c.c_bytes == 4 && k16 <= 1024 && max_stages(best_g, best_n, cfg.ksub, 2, best_r) >= 3;
   cfg.epi_bufs = o.epi_bufs ? o.epi_bufs : (want_two ? 2 : 1);
   cfg.stages = max_stages(best_g, best_n, cfg.ksub, cfg.epi_bufs, best_r);
   if (o.stages && o.stages < cfg.stages) cfg.stages = o.stages < 2 ? 2 : o.stages;
