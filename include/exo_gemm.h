@@ -44,6 +44,7 @@ typedef enum { EXO_GEMM_ROW_MAJOR = 0, EXO_GEMM_COL_MAJOR = 1 } exo_gemm_layout_
  *   bits 2..5   tile N / 64 (1, 2 or 4  =>  64, 128 or 256 columns per tile)
  *   bits 6..9   raster band width in tiles (1..15)
  *   bit  10     raster direction: 0 = library choice, set = bands along M instead of N
+ *   bit  11     the parts of a cut tail tile meet in C by TMA reduce-add (see EXO_GEMM_FLAG_SPLIT_REDUCE_ADD)
  *   bits 12..19 grid limit: launch at most this many CTAs (multiple of cta_group), 0 = all SMs
  *   bits 20..21 k sub-blocks (of 64 elements) per pipeline stage: 1 or 2
  *   bits 22..23 staging buffers per epilogue warp: 1 or 2 (also keeps the staged epilogue -- registers ->
@@ -55,6 +56,17 @@ typedef enum { EXO_GEMM_ROW_MAJOR = 0, EXO_GEMM_COL_MAJOR = 1 } exo_gemm_layout_
 #define EXO_GEMM_FLAG_TILE_N(n)     ((((uint32_t)(n) / 64u) & 15u) << 2)
 #define EXO_GEMM_FLAG_BAND(b)       (((uint32_t)(b) & 15u) << 6)
 #define EXO_GEMM_FLAG_BANDS_ALONG_M (1u << 10)
+/*
+ * The unordered form of the K split, as in the paper's Section 6 split-K kernels (TMA reduce-add of fp32
+ * partial sums): every part of a cut tile adds alpha * (its partial sum) onto C with
+ * cp.reduce.async.bulk.tensor instead of handing it to the owning part through a workspace.  No
+ * workspace, no waiting; the order of the additions is the memory system's, so results are not
+ * bitwise reproducible from run to run.  fp32 C only (ERR_UNSUPPORTED from validate otherwise);
+ * exo_gemm_run then accepts beta == 1 (C is accumulated onto) and beta == 0 (the run first clears C
+ * with a memset on the same stream) and returns ERR_UNSUPPORTED for any other beta.  Off by default:
+ * the ordered workspace reduction measured level or faster and is deterministic.
+ */
+#define EXO_GEMM_FLAG_SPLIT_REDUCE_ADD (1u << 11)
 #define EXO_GEMM_FLAG_GRID_LIMIT(c) (((uint32_t)(c) & 255u) << 12)
 #define EXO_GEMM_FLAG_K_SUBBLOCKS(k) (((uint32_t)(k) & 3u) << 20)
 #define EXO_GEMM_FLAG_EPI_BUFFERS(b) (((uint32_t)(b) & 3u) << 22)

@@ -27,6 +27,7 @@ def flag_cta_group(g): return g & 3
 def flag_tile_n(n): return ((n // 64) & 15) << 2
 def flag_band(b): return (b & 15) << 6
 FLAG_BANDS_ALONG_M = 1 << 10
+FLAG_SPLIT_REDUCE_ADD = 1 << 11
 def flag_grid_limit(c): return (c & 255) << 12
 def flag_k_subblocks(k): return (k & 3) << 20
 def flag_epi_buffers(b): return (b & 3) << 22

@@ -348,7 +348,7 @@ exo_gemm_status_t exo_gemm_plan_preview(const exo_gemm_desc_t* desc, int32_t sm_
   const FlagOverrides ov = decode_flags(desc->flags, desc->flags2);
   if (ov.share >= 2 && !kHaveSharePairs) return EXO_GEMM_ERR_UNSUPPORTED;
   p.cfg = choose_config(p.canon, ov, sm_count, sm_count / 2, kHaveSharePairs ? sm_count / 4 : 0);
-  p.cfg.workspace_bytes = split_workspace_bytes(p.cfg, desc->c_dtype);
+  p.cfg.workspace_bytes = ov.reduce_add ? 0 : split_workspace_bytes(p.cfg, desc->c_dtype);
   p.smem_bytes = smem_bytes_for(p.cfg.cta_group, p.cfg.tile_n, p.cfg.ksub, p.cfg.stages, p.cfg.epi_bufs, p.cfg.mrep);
   fill_info(&p, info);
   return EXO_GEMM_OK;
@@ -400,7 +400,7 @@ exo_gemm_status_t exo_gemm_create_batched(exo_gemm_handle_t* out, const exo_gemm
   if (ov.share >= 2 && max_quads < 1) { delete p; return EXO_GEMM_ERR_UNSUPPORTED; }
 
   p->cfg = choose_config(p->canon, ov, sms, max_pairs, max_quads);
-  p->cfg.workspace_bytes = split_workspace_bytes(p->cfg, desc->c_dtype);
+  p->cfg.workspace_bytes = ov.reduce_add ? 0 : split_workspace_bytes(p->cfg, desc->c_dtype);
   p->split_epoch = 0;
   p->kernel = pick_kernel(p->cfg.cta_group, p->cfg.tile_n, p->cfg.ksub, desc->c_dtype, p->cfg.pairs, p->cfg.mrep);
   p->smem_bytes = smem_bytes_for(p->cfg.cta_group, p->cfg.tile_n, p->cfg.ksub, p->cfg.stages, p->cfg.epi_bufs, p->cfg.mrep);
@@ -411,10 +411,14 @@ exo_gemm_status_t exo_gemm_create_batched(exo_gemm_handle_t* out, const exo_gemm
   e = cudaMemset(p->d_status, 0, kStatusBytes);
   if (e != cudaSuccess) { cudaFree(p->d_status); delete p; return cuda_fail(e); }
   if (p->cfg.tail_workers > 0) {  // scratch for the K-slices of the tail tiles, and who computes which
-    e = cudaMalloc((void**)&p->d_split_ws, (size_t)p->cfg.workspace_bytes);
     const size_t flag_bytes = sizeof(uint32_t) * (size_t)p->cfg.tail_tiles * (size_t)p->cfg.pairs;
-    if (e == cudaSuccess) e = cudaMalloc((void**)&p->d_split_flags, flag_bytes);
-    if (e == cudaSuccess) e = cudaMemset(p->d_split_flags, 0, flag_bytes);
+    if (ov.reduce_add) {   // the parts meet in C itself: no workspace, no counters
+      p->cfg.workspace_bytes = 0;
+    } else {
+      e = cudaMalloc((void**)&p->d_split_ws, (size_t)p->cfg.workspace_bytes);
+      if (e == cudaSuccess) e = cudaMalloc((void**)&p->d_split_flags, flag_bytes);
+      if (e == cudaSuccess) e = cudaMemset(p->d_split_flags, 0, flag_bytes);
+    }
     const size_t table_entries = 4 * (size_t)p->cfg.workers;
     TailItem* table = new (std::nothrow) TailItem[table_entries];
     if (e == cudaSuccess && !table) e = cudaErrorMemoryAllocation;
@@ -520,7 +524,12 @@ exo_gemm_status_t launch_plan(exo_gemm_plan* plan, const void* A, const void* B,
   prm.ldc_bytes = cn.ldc * cn.c_bytes;
   prm.c_batch_bytes = cn.stride_c * cn.c_bytes;
   // the tail tiles are cut along K only when there is a K loop to cut and scratch to reduce through
-  const bool split_now = cfg.tail_workers > 0 && read_ab && plan->d_split_ws != nullptr;
+  const bool split_now = cfg.tail_workers > 0 && read_ab && plan->d_tail_table != nullptr;
+  const bool reduce_add = split_now && (d.flags & (1u << 11)) != 0;
+  // the reduce-add form needs C to hold beta * C_in before the launch: it can for beta == 1 (as it is) and
+  // beta == 0 (cleared below)
+  if (reduce_add && beta != 0.f && beta != 1.f) return EXO_GEMM_ERR_UNSUPPORTED;
+  prm.reduce_add = reduce_add ? 1u : 0u;
   prm.work = WorkPlan{cfg.full_tiles, (int32_t)(cfg.full_tiles / cfg.workers), cfg.tail_tiles, split_now ? cfg.tail_workers : 0,
                       cfg.slots, plan->d_tail_table};
   prm.split_ws = plan->d_split_ws;
@@ -604,7 +613,14 @@ exo_gemm_status_t launch_plan(exo_gemm_plan* plan, const void* A, const void* B,
     lc.numAttrs = 3;
   }
   cudaError_t e;
-  if (split_now) {
+  if (reduce_add && beta == 0.f) {   // every part adds onto zeros
+    for (int64_t b = 0; b < cn.batch; ++b) {
+      e = cudaMemset2DAsync(static_cast<char*>(C) + b * cn.stride_c * cn.c_bytes, (size_t)(cn.ldc * cn.c_bytes), 0,
+                            (size_t)(cn.N * cn.c_bytes), (size_t)cn.M, (cudaStream_t)cuda_stream);
+      if (e != cudaSuccess) return cuda_fail(e);
+    }
+  }
+  if (split_now && !reduce_add) {
     // Arrival counters only grow: this run is complete at epoch * arrivals-per-run.  The epoch is taken and
     // the launch enqueued under the plan's lock, so that exo_gemm_check (which puts counters and epoch back
     // to zero after an abandoned run) never falls between the two on another host thread.

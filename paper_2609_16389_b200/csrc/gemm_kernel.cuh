@@ -438,7 +438,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         const int64_t t = wi.tile;
         // The owning slice of a tail tile that follows at least two whole tiles starts from an accumulator
         // into which the epilogue warps have already written the other slices' partial sums.
-        const bool preloaded = MREP == 1 && wi.slices > 1 && wi.slice == 0 && wi.after_whole && it >= preload_from;
+        const bool preloaded = MREP == 1 && wi.slices > 1 && wi.slice == 0 && wi.after_whole && it >= preload_from && !p.reduce_add;
         if constexpr (MREP == 1) {
           // the epilogue (of both CTAs) must have drained this accumulator
           ok = wait_barrier<PAIR>(tempty_bar(acc), acc_ph ^ 1u, p, WaitSite{kRoleMma, 100 + acc, (uint32_t)t, 0});
@@ -502,7 +502,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     const int32_t half = (int32_t)(ew >> 2);
     const uint32_t buf0 = epi0 + ew * EPI_BUFS * kEpiBufBytes;
     const uint32_t tempty0 = PAIR ? ptx::map_to_cta(tempty_bar(0), leader) : tempty_bar(0);
-    const bool has_beta = p.beta != 0.f;
+    const bool has_beta_arg = p.beta != 0.f;
     const bool has_acc = nkb > 0;
     const bool scale = p.alpha != 1.f;
     const float alpha = p.alpha, beta = p.beta;
@@ -510,8 +510,9 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     // eight precomputed addresses would be eight registers held across the whole role
     const uint32_t my_row = buf0 + lane * 128u, my_xor = (lane & 7u) << 4;
     auto piece = [&](int j) { return my_row + (((uint32_t)j << 4) ^ my_xor); };
-    // running chunk counter: staging buffer g % EPI_BUFS, its C_in barrier phase (g / EPI_BUFS) & 1
-    uint32_t g = 0;
+    // running chunk counter: staging buffer g % EPI_BUFS; bit b of cin_phase = the phase of buffer b's C_in
+    // barrier (a tile whose parts are added onto C fetches no C_in, so the phases do not follow g)
+    uint32_t g = 0, cin_phase = 0;
     const bool two_bufs = EPI_BUFS == 2;
     // No staging buffers at all: the plan found that this run can store its result straight from
     // registers (beta == 0; C, its leading dimension and N are multiples of 32 bytes), one full 32-byte
@@ -598,8 +599,8 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         // owner's epilogue is an ordinary one.  (With a single whole tile before the slice the partials
         // arrive too late for that; the owner then adds them in its epilogue.)
         WorkItem nx;
-        if (it + 1 >= preload_from && work_item(p.work, worker, num_workers, it + 1, nkb, &nx) && nx.slices > 1 && nx.slice == 0 &&
-            nx.after_whole) {
+        if (it + 1 >= preload_from && !p.reduce_add && work_item(p.work, worker, num_workers, it + 1, nkb, &nx) && nx.slices > 1 &&
+            nx.slice == 0 && nx.after_whole) {
           uint32_t bz2;
           const TileCoord tc2 = tile_coord(nx.tile, &bz2);
           const int32_t n_mine = chunks_of(tc2.m * (CTA_M * CTA_GROUP) + (int32_t)cta_rank * CTA_M + (int32_t)quad * 32,
@@ -643,7 +644,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         }
       }
       EXO_TRACE_TILE(it, 3);
-      const bool preloaded = MREP == 1 && wi.slices > 1 && wi.slice == 0 && wi.after_whole && it >= preload_from;  // see above
+      const bool preloaded = MREP == 1 && wi.slices > 1 && wi.slice == 0 && wi.after_whole && it >= preload_from && !p.reduce_add;  // see above
       // one pass per accumulator of the tile: a single one, or (tall tile) rows 0..127 then 128..255 of the CTA
 #pragma unroll 1
       for (int32_t r = 0; r < MREP; ++r) {
@@ -674,8 +675,14 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       if (mine == 0 && has_acc) release_acc();
 
       // ---- a slice of a tail tile (the tile's K range is cut into wi.slices parts)
-      const bool contributor = wi.slices > 1 && wi.slice != 0;
-      const bool owner = wi.slices > 1 && wi.slice == 0 && !preloaded;  // has to add the partials itself
+      // The unordered alternative (the form of the paper's Section 6 split-K kernels): every part of a cut
+      // tile adds alpha * (its partial sum) onto C with a TMA reduce-add; C holds beta * C_in (beta == 1) or
+      // zeros (the host cleared it) before the launch, nobody waits for anybody, and the order of the
+      // additions, hence the last bits of the result, is left to the memory system.
+      const bool tile_reduce = p.reduce_add != 0 && wi.slices > 1;
+      const bool has_beta = has_beta_arg && !tile_reduce;
+      const bool contributor = wi.slices > 1 && wi.slice != 0 && !tile_reduce;
+      const bool owner = wi.slices > 1 && wi.slice == 0 && !preloaded && !tile_reduce;  // has to add the partials itself
       if (contributor) {
         // raw accumulators out, then one arrival per warp on the tile's counter
         for (int32_t i = 0; i < mine; ++i) {
@@ -761,9 +768,10 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
           __syncwarp();
           EXO_TRACE_CHUNK(g, 0);
           if (has_beta && !direct) {
-            ok = wait_barrier<false>(cin_bar(ew, b), (two_bufs ? (g >> 1) : g) & 1u, p,
+            ok = wait_barrier<false>(cin_bar(ew, b), (cin_phase >> b) & 1u, p,
                                      WaitSite{kRoleEpilogueCin, 300 + b, (uint32_t)t, (uint32_t)i});
             ok = __all_sync(0xffffffffu, ok);
+            cin_phase ^= 1u << b;
           }
 #pragma unroll
           for (int32_t q = 0; q < UPC; ++q) {
@@ -860,8 +868,14 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             ptx::fence_proxy_async_smem();  // generic-proxy writes -> visible to the TMA store
             __syncwarp();
             if (ptx::elect_one()) {
-              if (batched) ptx::tma_store_3d(&tm_c, col, row0, (int32_t)bz, buf0 + boff);
-              else ptx::tma_store_2d(&tm_c, col, row0, buf0 + boff);
+              if (tile_reduce) {
+                if (batched) ptx::tma_reduce_add_3d(&tm_c, col, row0, (int32_t)bz, buf0 + boff);
+                else ptx::tma_reduce_add_2d(&tm_c, col, row0, buf0 + boff);
+              } else if (batched) {
+                ptx::tma_store_3d(&tm_c, col, row0, (int32_t)bz, buf0 + boff);
+              } else {
+                ptx::tma_store_2d(&tm_c, col, row0, buf0 + boff);
+              }
               ptx::bulk_commit();
             }
             EXO_TRACE_CHUNK(g, 3);

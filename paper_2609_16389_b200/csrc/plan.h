@@ -14,6 +14,7 @@ inline int elem_bytes(int dtype) { return dtype == EXO_GEMM_FP32 ? 4 : 2; }
 struct FlagOverrides {
   int split;       // 0 = auto, 1 = never split, 2..8 = slices per tail tile (if they fit)
   bool no_workspace;  // set by the allocation-free entry point: nothing that needs device scratch
+  bool reduce_add;    // the parts of a cut tile meet in C by TMA reduce-add instead of in a workspace
   int epi_bufs;    // 0 = auto
   int stages;      // 0 = as many as fit, else an upper limit
   int ksub;        // 0 = auto
@@ -39,6 +40,7 @@ inline FlagOverrides decode_flags(uint32_t f, uint32_t f2 = 0) {
   o.stages = (int)((f >> 24) & 15u);
   o.split = (int)((f >> 28) & 15u);
   o.no_workspace = false;
+  o.reduce_add = (f & (1u << 11)) != 0;
   o.share = (int)(f2 & 3u);
   o.mrep = (int)((f2 >> 2) & 3u);
   return o;
@@ -67,7 +69,6 @@ inline exo_gemm_status_t validate_desc(const exo_gemm_desc_t* d) {
   if (((d->flags >> 28) & 15u) > 8u) return EXO_GEMM_ERR_INVALID_ARG;
   if (((d->flags >> 20) & 3u) == 3u || ((d->flags >> 22) & 3u) == 3u) return EXO_GEMM_ERR_INVALID_ARG;
   if (((d->flags >> 24) & 15u) == 1u || ((d->flags >> 24) & 15u) > (uint32_t)kMaxStages) return EXO_GEMM_ERR_INVALID_ARG;
-  if (d->flags & (1u << 11)) return EXO_GEMM_ERR_INVALID_ARG;
   const FlagOverrides o = decode_flags(d->flags, d->flags2);
   if (o.cta_group == 3) return EXO_GEMM_ERR_INVALID_ARG;
   if (o.tile_n != 0 && o.tile_n != 64 && o.tile_n != 128 && o.tile_n != 256) return EXO_GEMM_ERR_INVALID_ARG;
@@ -82,6 +83,8 @@ inline exo_gemm_status_t validate_desc(const exo_gemm_desc_t* d) {
   // beyond here the call is a legal BLAS call; what follows is this library's supported set
   // fp32 operands are multiplied as tf32 (the precision of the paper's own kernels) into an fp32 C
   if (d->c_dtype != EXO_GEMM_FP32 && d->c_dtype != d->ab_dtype) return EXO_GEMM_ERR_UNSUPPORTED;
+  // the reduce-add form of the K split adds fp32 partial sums onto an fp32 C
+  if ((d->flags & (1u << 11)) && d->c_dtype != EXO_GEMM_FP32) return EXO_GEMM_ERR_UNSUPPORTED;
   // the persistent scheduler indexes tiles (at least 128 x 64 each) and k-blocks with 32 bits
   if (((d->M + 127) / 128) * ((d->N + 63) / 64) >= (1LL << 31)) return EXO_GEMM_ERR_UNSUPPORTED;
   // a matrix that is never touched (empty problem, K == 0) has no stride rule
@@ -377,7 +380,7 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
   cfg.epi_bufs = o.epi_bufs ? o.epi_bufs : (want_two ? 2 : 1);
   cfg.stages = max_stages(best_g, best_n, cfg.ksub, cfg.epi_bufs, best_r);
   if (o.stages && o.stages < cfg.stages) cfg.stages = o.stages < 2 ? 2 : o.stages;
-  cfg.stages_direct = o.epi_bufs ? 0 : max_stages(best_g, best_n, cfg.ksub, 0, best_r);
+  cfg.stages_direct = (o.epi_bufs || o.reduce_add) ? 0 : max_stages(best_g, best_n, cfg.ksub, 0, best_r);
   if (o.stages && o.stages < cfg.stages_direct) cfg.stages_direct = o.stages < 2 ? 2 : o.stages;
   // Wave quantisation: the k-blocks of the tiles that do not fill a whole wave are shared out evenly among
   // the workers, so that the last wave takes tail / tail_workers of a tile's time (split-K applied to the

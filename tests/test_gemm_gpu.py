@@ -271,6 +271,70 @@ def test_tail_tiles_cut_along_k(case, split):
         dp.close()
 
 
+REDUCE_ADD_CASES = [
+    # (M, N, K, ab, beta, g, bn, grid)
+    (1280, 1280, 1024, BF16, 0.0, 2, 256, 16),   # three whole waves, one tail tile in two parts
+    (512, 1280, 4096, FP16, 1.0, 2, 256, 16),    # one whole wave, two tail tiles, accumulate onto C
+    (1000, 1160, 1544, BF16, 1.0, 1, 128, 36),   # 8 tail tiles in 4 parts, ragged everywhere
+    (640, 520, 4096, FP16, 0.0, 2, 128, 0),      # less than one wave: every tile is cut
+    (1000, 1536, 3072, BF16, 0.0, 2, 256, 10),   # 24 tiles on 5 pairs: 4 tail tiles shared by all 5 in ranges that ignore tile boundaries
+]
+
+
+@pytest.mark.parametrize("case", REDUCE_ADD_CASES, ids=lambda c: "x".join(str(v) for v in c[:3]))
+def test_tail_parts_meet_in_c_by_tma_reduce_add(case):
+    """The unordered form of the K split (the paper's Section 6 split-K kernels reduce with TMA): every part
+    of a cut tile adds its partial sum onto C.  Same tolerance; the order of the additions is not fixed, so
+    repeated runs need not agree bit for bit."""
+    M, N, K, ab, beta, g, bn, grid = case
+    p = synth.Problem("reduce_add", M, N, K, ab, FP32, 0, 1, 0, 0.75, beta, seed=M + N + K,
+                      dist="normal" if ab == FP16 else "uniform").generate()
+    if beta == 0.0:
+        p.C[:] = np.nan                                # cleared by the run, never read
+    flags = flags_for(g, bn, grid) | B.FLAG_SPLIT_REDUCE_ADD
+    if K < 4096:
+        flags |= B.flag_split_k(2)                     # short K loops are cut on request only
+    q = p
+    if beta == 0.0:                                    # the oracle must not see the NaNs either
+        import copy
+        q = copy.copy(p)
+        q.C = np.zeros_like(p.C)
+    cbuf, info = harness.gemm_host(p, flags)
+    assert info["split_k"] >= 2 and info["workspace_bytes"] == 0, info
+    got = oracle.logical_view(cbuf, M, N, 0, p.ldc, FP32)
+    cref, den = oracle.gemm_problem(q)
+    assert oracle.max_error(got, cref, den) <= TOL, info
+
+
+def test_reduce_add_refuses_what_it_cannot_do():
+    import torch
+    assert B.exo_gemm_validate(B.make_desc(512, 512, 4096, BF16, BF16, 0, 1, 0, flags=B.FLAG_SPLIT_REDUCE_ADD)) == B.ERR_UNSUPPORTED
+    p = synth.Problem("reduce_beta", 640, 520, 4096, BF16, FP32, 0, 1, 0, 1.0, 0.5, seed=3).generate()
+    dp = harness.DeviceProblem(p, flags_for(2, 128) | B.FLAG_SPLIT_REDUCE_ADD)
+    try:
+        assert dp.plan.info()["split_k"] >= 2
+        st = B.exo_gemm_run(dp.plan.handle, dp.dA.data_ptr(), dp.dB.data_ptr(), dp.dC.data_ptr(), 1.0, 0.5, 0)
+        assert st == B.ERR_UNSUPPORTED                  # beta must be 0 or 1
+        torch.cuda.synchronize()
+        dp.plan.check()
+    finally:
+        dp.close()
+
+
+def test_long_k_case_of_the_papers_evaluation():
+    """1024 x 1024 x 65536, the long-K regime of the paper's Section 6 (where it measures its split-K
+    variants): sampled entries and the whole-matrix check, for the ordered split and the reduce-add form."""
+    p = synth.sweep_problem(1024, 1024, 65536).generate()
+    for flags in (0, B.FLAG_SPLIT_REDUCE_ADD):
+        cbuf, got, info = run_gpu(p, flags)
+        assert info["split_k"] >= 2, info
+        rng = np.random.default_rng(5)
+        r, c = structured_sample(p.M, p.N, rng, n_random=1 << 13, block=64)
+        cref, den = oracle.gemm_problem_entries(p, r, c)
+        assert oracle.max_error(got[r, c], cref, den) <= TOL, info
+        assert oracle.freivalds(p, got) <= TOL, info
+
+
 def test_tail_slices_of_a_strided_batch():
     # 5 matrices x 6 tiles on 13 pairs: two whole waves, then 4 tail tiles cut in two (owners' accumulators
     # preloaded with the contributors' sums), tiles of different matrices side by side
