@@ -223,7 +223,9 @@ exo_gemm_status_t exo_gemm_create_batched(exo_gemm_handle_t* out, const exo_gemm
  * handle may be used from several host threads (tensor maps are built on the
  * caller's stack), but runs of ONE plan whose exo_gemm_info_t.split_k > 1 must not
  * overlap on the GPU (enqueue them on one stream, or order the streams): they
- * share the plan's partial-sum workspace and arrival counters.  Device-side waits are bounded: if one gives up, the kernel
+ * share the plan's partial-sum workspace and arrival counters.  Nothing in a launch's parameters depends
+ * on how often the plan has run (the counters of a K-slicing plan keep their own run count on the device),
+ * so exo_gemm_run may be captured into a CUDA graph and the graph replayed.  Device-side waits are bounded: if one gives up, the kernel
  * records where in the plan's status block and exits cleanly; a later
  * exo_gemm_check reports EXO_GEMM_ERR_DEVICE_TIMEOUT.
  */
@@ -235,9 +237,8 @@ exo_gemm_status_t exo_gemm_run(exo_gemm_handle_t plan, const void* A, const void
  * legacy default stream; call it after synchronising the stream(s) the plan ran on).
  * Returns OK or ERR_DEVICE_TIMEOUT, and clears the block.  detail, if not NULL, receives 8
  * words: {code, role, barrier, tile, k_block, cta, 0, 0}.  After a timeout it also puts
- * the arrival counters of a K-slicing plan back to zero; that reset and the launches of
- * exo_gemm_run on the same plan exclude one another (a lock inside the plan), so the
- * call is safe beside runs from other host threads.  (The paper's kernels have no such
+ * the counters of a K-slicing plan back to zero (an abandoned run leaves them out of
+ * step), so call it while no run of the plan is in flight.  (The paper's kernels have no such
  * status: its Section 5 checks synchronisation before the kernel ever runs; a library
  * that runs on shared GPUs bounds every device-side wait instead and reports here.)
  */

@@ -149,10 +149,8 @@ struct exo_gemm_plan {
   int smem_bytes;
   uint32_t* d_status;
   float* d_split_ws;                   // fp32 partials of the tail tiles' K-slices (NULL if none)
-  uint32_t* d_split_flags;             // one arrival counter per tail tile
+  uint32_t* d_split_flags;             // two counters per tail tile: arrivals of contributing warps, owner warps done
   exo::TailItem* d_tail_table;         // the workers' ranges of the tail tiles' k-blocks (4 entries per worker)
-  std::atomic<uint32_t> split_epoch;   // runs that used the counters so far
-  std::mutex split_mutex;              // taking an epoch + launching, and exo_gemm_check's reset, exclude one another
   std::atomic<int32_t> dbg_timeout_ms;
   std::atomic<int64_t> dbg_skip_k_block;
 };
@@ -401,7 +399,6 @@ exo_gemm_status_t exo_gemm_create_batched(exo_gemm_handle_t* out, const exo_gemm
 
   p->cfg = choose_config(p->canon, ov, sms, max_pairs, max_quads);
   p->cfg.workspace_bytes = ov.reduce_add ? 0 : split_workspace_bytes(p->cfg, desc->c_dtype);
-  p->split_epoch = 0;
   p->kernel = pick_kernel(p->cfg.cta_group, p->cfg.tile_n, p->cfg.ksub, desc->c_dtype, p->cfg.pairs, p->cfg.mrep);
   p->smem_bytes = smem_bytes_for(p->cfg.cta_group, p->cfg.tile_n, p->cfg.ksub, p->cfg.stages, p->cfg.epi_bufs, p->cfg.mrep);
   e = allow_full_smem(p->kernel);
@@ -411,7 +408,7 @@ exo_gemm_status_t exo_gemm_create_batched(exo_gemm_handle_t* out, const exo_gemm
   e = cudaMemset(p->d_status, 0, kStatusBytes);
   if (e != cudaSuccess) { cudaFree(p->d_status); delete p; return cuda_fail(e); }
   if (p->cfg.tail_workers > 0) {  // scratch for the K-slices of the tail tiles, and who computes which
-    const size_t flag_bytes = sizeof(uint32_t) * (size_t)p->cfg.tail_tiles * (size_t)p->cfg.pairs;
+    const size_t flag_bytes = 2 * sizeof(uint32_t) * (size_t)p->cfg.tail_tiles * (size_t)p->cfg.pairs;
     if (ov.reduce_add) {   // the parts meet in C itself: no workspace, no counters
       p->cfg.workspace_bytes = 0;
     } else {
@@ -534,7 +531,7 @@ exo_gemm_status_t launch_plan(exo_gemm_plan* plan, const void* A, const void* B,
                       cfg.slots, plan->d_tail_table};
   prm.split_ws = plan->d_split_ws;
   prm.split_flags = plan->d_split_flags;
-  prm.split_target = 0;
+  prm.split_arrivals = (uint32_t)(kEpiWarps * cfg.cta_group * cfg.mrep);
   prm.alpha = read_ab ? alpha : 0.f;
   prm.beta = beta;
   prm.idesc = make_idesc(d.ab_dtype, cn.a_mn_major, cn.b_mn_major, 128 * cfg.cta_group, cfg.tile_n);
@@ -620,17 +617,9 @@ exo_gemm_status_t launch_plan(exo_gemm_plan* plan, const void* A, const void* B,
       if (e != cudaSuccess) return cuda_fail(e);
     }
   }
-  if (split_now && !reduce_add) {
-    // Arrival counters only grow: this run is complete at epoch * arrivals-per-run.  The epoch is taken and
-    // the launch enqueued under the plan's lock, so that exo_gemm_check (which puts counters and epoch back
-    // to zero after an abandoned run) never falls between the two on another host thread.
-    std::lock_guard<std::mutex> lock(plan->split_mutex);
-    const uint32_t epoch = plan->split_epoch.fetch_add(1) + 1;
-    prm.split_target = epoch * (uint32_t)(kEpiWarps * cfg.cta_group * cfg.mrep);   // per contributing slice of a tile
-    e = cudaLaunchKernelEx(&lc, plan->kernel, tm_a, tm_b, tm_c, prm);
-  } else {
-    e = cudaLaunchKernelEx(&lc, plan->kernel, tm_a, tm_b, tm_c, prm);
-  }
+  // (The arrival counters of a K-slicing plan need nothing from the host per run: which run this is follows
+  // from a second counter on the device, so the same parameters can be replayed from a CUDA graph.)
+  e = cudaLaunchKernelEx(&lc, plan->kernel, tm_a, tm_b, tm_c, prm);
   if (e != cudaSuccess) return cuda_fail(e);
   return EXO_GEMM_OK;
 }
@@ -659,11 +648,9 @@ exo_gemm_status_t exo_gemm_check(exo_gemm_handle_t plan, uint32_t* detail) {
   if (h[0] == kStatusOk) return EXO_GEMM_OK;
   e = cudaMemset(plan->d_status, 0, 32);
   if (e != cudaSuccess) return cuda_fail(e);
-  if (plan->d_split_flags) {  // an abandoned run may have left the arrival counters short
-    std::lock_guard<std::mutex> lock(plan->split_mutex);
-    e = cudaMemset(plan->d_split_flags, 0, sizeof(uint32_t) * (size_t)plan->cfg.tail_tiles * (size_t)plan->cfg.pairs);
+  if (plan->d_split_flags) {  // an abandoned run may have left the counters of the tail tiles out of step
+    e = cudaMemset(plan->d_split_flags, 0, 2 * sizeof(uint32_t) * (size_t)plan->cfg.tail_tiles * (size_t)plan->cfg.pairs);
     if (e != cudaSuccess) return cuda_fail(e);
-    plan->split_epoch = 0;
   }
   return EXO_GEMM_ERR_DEVICE_TIMEOUT;
 }

@@ -495,6 +495,12 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     // chunks (128 bytes of C per row each), the left (half == 0) or the right half.
     constexpr int UPC = CW / 32;                       // 32-column TMEM loads per chunk
     constexpr int kHalfChunks = (NCHUNK + 1) / 2;      // chunks per warp of a lane quadrant
+    constexpr uint32_t kOwnerWarps = kEpiWarps * CTA_GROUP;   // epilogue warps of the CTA group that owns a tile
+    // this warp is done with the partial sums of tail tile `ti` (see wait_partials)
+    auto partials_consumed = [&](int32_t ti) {
+      __syncwarp();
+      if (ptx::elect_one()) ptx::red_release_gpu_add(p.split_flags + 2 * (ti * NPAIR + (int32_t)pair_id) + 1, 1u);
+    };
     if (warp == 2) ptx::grid_launch_dependents();      // one warp speaks for the CTA: our own successor may start likewise
     ptx::grid_dependency_wait();                       // C and the split workspace may still be in use by the previous kernel
     const uint32_t quad = warp & 3u;
@@ -550,9 +556,17 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     // partials.  One lane polls, with a pause between polls: this can run beside a main loop, whose
     // copy-issuing warps share the instruction issue slots and the memory pipeline with this warp.
     auto wait_partials = [&](const WorkItem& w, int32_t r) {
-      const uint32_t* flag = p.split_flags + w.tail_index * NPAIR + (int32_t)pair_id;
-      // the counter only grows: every contributing part of every run adds one arrival per warp
-      const uint32_t target = p.split_target * (uint32_t)(w.slices - 1);
+      // Two words per tail tile (and pair): arrivals of contributing warps, and owner warps that are done with
+      // the tile's partial sums.  Both only grow.  Every warp of the owning CTA group adds one to the second
+      // word per run, so its value tells which run of the plan this is without any word from the host: the
+      // counters work the same when the launches are replayed from a CUDA graph.  (A warp reads the word
+      // before it adds its own one, and at most kOwnerWarps - 1 others have added theirs by then.)
+      const uint32_t* flag = p.split_flags + 2 * (w.tail_index * NPAIR + (int32_t)pair_id);
+      uint32_t target = 0;
+      if (lane == 0) {
+        const uint32_t run = ptx::ld_acquire_gpu(flag + 1) / kOwnerWarps;
+        target = (run + 1u) * p.split_arrivals * (uint32_t)(w.slices - 1);
+      }
       const long long t_start = clock64();
       uint32_t spins = 0;
       for (;;) {
@@ -634,6 +648,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             }
             ptx::tmem_st_wait();
           }
+          partials_consumed(nx.tail_index);
           // every epilogue warp of the CTA group reports "filled" to the MMA-issuing CTA
           ptx::tc_fence_before_sync();
           __syncwarp();
@@ -700,7 +715,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         }
         __threadfence();  // each lane's partials are visible GPU-wide before the arrival below
         __syncwarp();
-        if (ptx::elect_one()) ptx::red_release_gpu_add(p.split_flags + wi.tail_index * NPAIR + (int32_t)pair_id, 1u);
+        if (ptx::elect_one()) ptx::red_release_gpu_add(p.split_flags + 2 * (wi.tail_index * NPAIR + (int32_t)pair_id), 1u);
         continue;
       }
       if (owner && mine > 0) {
@@ -888,6 +903,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       if (!ok) break;
       }  // accumulators of the tile
       if (!ok) break;
+      if (wi.slices > 1 && wi.slice == 0 && !preloaded && p.reduce_add == 0) partials_consumed(wi.tail_index);
       if (warp == 2 && lane == 0) EXO_TRACE(2, it, 1, 4096);
       if (MREP == 2 || (acc ^= 1u) == 0u) acc_ph ^= 1u;
     }

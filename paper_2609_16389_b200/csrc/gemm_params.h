@@ -82,9 +82,9 @@ struct GemmParams {
   OperandStaging a, b;
   WorkPlan work;            // whole-K tiles round-robin, then the tail tiles cut along K
   float* split_ws;          // device: fp32 partial accumulators of the slices 1.. of every tail tile
-  uint32_t* split_flags;    // device: one arrival counter per tail tile, never reset, only grows
+  uint32_t* split_flags;    // device: per tail tile {arrivals of contributing warps, owner warps done}; both only grow
   uint32_t reduce_add;      // 1: the parts of a cut tile add onto C (TMA reduce) instead of meeting in the workspace
-  uint32_t split_target;    // counter value that means "all partials of this run have landed"
+  uint32_t split_arrivals;  // arrivals per contributing part of a tile and run: its epilogue warps (x accumulators)
   void* c_ptr;              // C of matrix 0 and its strides in bytes (read by the direct stores only)
   int64_t ldc_bytes, c_batch_bytes;
   uint32_t* status;         // device: 8 words {code, role, barrier, tile, k_block, cta, -, -}

@@ -335,6 +335,43 @@ def test_long_k_case_of_the_papers_evaluation():
         assert oracle.freivalds(p, got) <= TOL, info
 
 
+@pytest.mark.parametrize("case", [(512, 1280, 4096, 2, 256, 16), (640, 520, 4096, 2, 128, 0), (1280, 1280, 2048, 2, 256, 16)],
+                         ids=lambda c: "x".join(str(v) for v in c[:3]))
+def test_k_slicing_plan_replayed_from_a_cuda_graph(case):
+    """Three runs of one K-slicing plan captured into a CUDA graph, the graph replayed five times, eager runs
+    in between: every result has the bits of the first eager run.  (The arrival counters of the tail tiles
+    take their run count from the device, so replaying identical launch parameters is sound.)"""
+    import torch
+    M, N, K, g, bn, grid = case
+    p = synth.Problem("graph", M, N, K, BF16, FP32, 0, 1, 0, 1.0, 0.0, seed=M + K).generate()
+    dp = harness.DeviceProblem(p, flags_for(g, bn, grid))
+    try:
+        assert dp.plan.info()["split_k"] >= 2
+        dp.run()
+        torch.cuda.synchronize()
+        dp.plan.check()
+        want = dp.result_buffer().copy()
+        cref, den = oracle.gemm_problem(p)
+        assert oracle.max_error(oracle.logical_view(want, M, N, 0, p.ldc, FP32), cref, den) <= TOL
+        side = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            for _ in range(3):
+                dp.run()
+        for rep in range(5):
+            dp.dC.fill_(0xFF)                           # NaN patterns: every replay has to write all of C again
+            graph.replay()
+            torch.cuda.synchronize()
+            assert np.array_equal(dp.result_buffer(), want), rep
+            if rep % 2:
+                dp.run()                                # an eager run between replays
+                torch.cuda.synchronize()
+                assert np.array_equal(dp.result_buffer(), want), rep
+        dp.plan.check()
+    finally:
+        dp.close()
+
+
 def test_tail_slices_of_a_strided_batch():
     # 5 matrices x 6 tiles on 13 pairs: two whole waves, then 4 tail tiles cut in two (owners' accumulators
     # preloaded with the contributors' sums), tiles of different matrices side by side
