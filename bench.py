@@ -49,6 +49,9 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--verify", action="store_true",
+                    help="sweep only: host-generated inputs for one operand set of every shape and the oracle's "
+                         "verdict on 4096 sampled entries per shape (adds several minutes)")
     ap.add_argument("--no-extras", action="store_true",
                     help="skip the sustained run and the short runs of the other configurations")
     ap.add_argument("--no-cublas", action="store_true")
@@ -678,10 +681,12 @@ def cpu_baseline(p, workload):
 def run_sweep(args, rank, world, local_rank):
     """The shape sweep: M, N, K each in {512, 1000, 2048, 3072, 6144, 12288}, bf16 in, fp32 out.
 
-    Timing only (parity of sweep shapes is covered by the GPU tests on host-generated inputs):
-    operands are drawn on the device, uniform[-1, 1) rounded to bf16.  Every shape gets its own plan,
-    3 warm-up and `--steps` timed launches; the line reports whole-sweep throughput and, per shape,
-    TFLOP/s and the fraction of roofline(shape) = min(tensor peak, AI x HBM bandwidth).
+    Operands are drawn on the device, uniform[-1, 1) rounded to bf16 (with --verify one operand set per
+    shape is the seeded host-generated problem and its result is checked by the oracle on sampled
+    entries; otherwise parity of the sweep is what the GPU tests cover, one shape per plan class).  Every
+    shape gets its own plan, 3 warm-up launches and `--steps` launches replayed from a CUDA graph; the
+    line reports whole-sweep throughput and, per shape, TFLOP/s and the fraction of
+    roofline(shape) = min(tensor peak, AI x HBM bandwidth).
     """
     import itertools
     import torch
@@ -694,56 +699,84 @@ def run_sweep(args, rank, world, local_rank):
     pk = peaks()
     stream = torch.cuda.current_stream(dev)
     steps = max(3, min(args.steps, 20))
+    side = torch.cuda.Stream(dev)
     rows, tot_flop, tot_ms, launches = [], 0.0, 0.0, 0
     sampler = ClockSampler(local_rank)
     sampler.start()
+    from paper_2609_16389_b200 import harness
+    worst_parity = 0.0
     for (M, N, K) in itertools.product(synth.SWEEP_DIMS, repeat=3):
         set_bytes = 2 * (M * K + K * N) + 4 * M * N
         n_sets = int(min(8, max(1, np.ceil(2.0 * L2_BYTES / set_bytes))))
         sets = [((torch.rand(M, K, device=dev) * 2 - 1).to(torch.bfloat16),
                  (torch.rand(N, K, device=dev) * 2 - 1).to(torch.bfloat16),
                  torch.empty(M, N, device=dev, dtype=torch.float32)) for _ in range(n_sets)]
+        prob = None
+        if args.verify:     # operand set 0 holds the seeded host-generated problem of this shape
+            prob = synth.sweep_problem(M, N, K).generate()
+            sets[0] = (harness._to_device(prob.A, dev), harness._to_device(prob.B, dev), harness._to_device(prob.C, dev))
         plan = B.Plan(B.make_desc(M, N, K, B.BF16, B.FP32, B.ROW_MAJOR, B.COL_MAJOR, B.ROW_MAJOR,
                                   device=local_rank, flags=args.flags))
 
-        def step(i):
+        def step(i, s=None):
             a, b, c = sets[i % n_sets]
-            plan.run(a.data_ptr(), b.data_ptr(), c.data_ptr(), 1.0, 0.0, stream.cuda_stream)
+            plan.run(a.data_ptr(), b.data_ptr(), c.data_ptr(), 1.0, 0.0, (s or stream).cuda_stream)
 
         for i in range(3):
             step(i)
         torch.cuda.synchronize(dev)
+        # `steps` launches captured into one CUDA graph and replayed: what is timed is the kernels back to back,
+        # not the host's launch rate (which would bound every shape under ~10 us)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            for i in range(steps):
+                step(i, side)
+        graph.replay()
+        torch.cuda.synchronize(dev)
+        reps = 3 if 2.0 * M * N * K > 1e11 else 10
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
-        for i in range(steps):
-            step(i)
+        for _ in range(reps):
+            graph.replay()
         e1.record(stream)
         torch.cuda.synchronize(dev)
         plan.check()
-        ms = e0.elapsed_time(e1) / steps
+        ms = e0.elapsed_time(e1) / (steps * reps)
         info = plan.info()
-        plan.close()
         flop = 2.0 * M * N * K
         ai = flop / set_bytes
         roof = min(pk["tflops_burst"], ai * pk["hbm_gbs"] / 1e3)
         tf = flop / (ms * 1e-3) / 1e12
-        rows.append({"M": M, "N": N, "K": K, "us": round(ms * 1e3, 2), "tflops": round(tf, 1),
-                     "roofline_tflops": round(roof, 1), "frac": round(tf / roof, 3),
-                     "plan": [info["cta_group"], info["tile_n"], info["tile_k"], info["split_k"]],
-                     "l2_sets": n_sets})
+        row = {"M": M, "N": N, "K": K, "us": round(ms * 1e3, 2), "tflops": round(tf, 1),
+               "roofline_tflops": round(roof, 1), "frac": round(tf / roof, 3),
+               "plan": [info["cta_group"], info["tile_m"], info["tile_n"], info["tile_k"], info["split_k"], info["cluster_size"]],
+               "l2_sets": n_sets}
+        if prob is not None:
+            step(0)
+            torch.cuda.synchronize(dev)
+            plan.check()
+            par = sampled_parity(prob, sets[0][2].cpu().numpy().view(np.float32), 1 << 12)
+            row["parity"] = float("%.3g" % par["max_error_metric"])
+            worst_parity = max(worst_parity, par["max_error_metric"])
+        plan.close()
+        rows.append(row)
         tot_flop += flop * steps
         tot_ms += ms * steps
-        launches += steps
-        del sets
+        launches += steps * (reps + 1) + 3
+        del sets, graph
     clocks = sampler.stop()
     fr = np.array([r["frac"] for r in rows])
     line = {
         "metric": METRIC, "value": tot_flop / (tot_ms * 1e-3) / 1e12, "unit": UNIT, "n_gpus": 1, "steps": steps,
         "warmup": 3, "ms_per_step": tot_ms / launches, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "bf16 in, fp32 accumulate", "data": "synthetic (device-generated, timing only)",
+        "vs_baseline": None, "dtype": "bf16 in, fp32 accumulate",
+        "data": "synthetic (device-generated for timing" + ("; operand set 0 of every shape seeded on the host and checked by the oracle)" if args.verify else ")"),
         "config": {"workload": "sweep_216", "shapes": len(rows), "dims": list(synth.SWEEP_DIMS),
                    "layouts": "Ar Bc Cr", "c_dtype": "fp32",
-                   "l2": "operand sets rotated to exceed 2x L2 where 8 sets suffice, else L2-warm (l2_sets per shape)"},
+                   "l2": "operand sets rotated to exceed 2x L2 where 8 sets suffice, else L2-warm (l2_sets per shape)",
+                   "timing": f"{steps} launches per shape captured into a CUDA graph, the graph replayed 3 or 10 times between two events",
+                   "parity": ({"entries_per_shape": 4096, "worst_max_error_metric": worst_parity, "tolerance": 1e-3}
+                              if args.verify else "per plan class in tests/test_gemm_gpu.py; per shape with --verify")},
         "roofline": {"bound": "mixed", "achieved": float(np.exp(np.log(fr).mean())), "peak": 1.0, "unit": "fraction",
                      "frac": float(np.exp(np.log(fr).mean())), "traffic": None,
                      "note": "geometric mean over shapes of TFLOP/s / min(measured tensor peak, AI x measured HBM GB/s)",

@@ -512,7 +512,12 @@ exo_gemm_status_t launch_plan(exo_gemm_plan* plan, const void* A, const void* B,
   // lines per instruction.  fp32 C: -8 to -13 % at K = 512, -2 to -4 % at K = 1000; bf16 C: -3 to -5 % at
   // K = 512), so short K loops keep the staged path.  So does a request for a staging depth
   // (EXO_GEMM_FLAG_EPI_BUFFERS).
-  const bool direct = cfg.stages_direct > 0 && cn.K * (cn.ab_bytes / 2) >= (cn.c_bytes == 2 ? kDirectMinK16 : kDirectMinK32) && beta == 0.f && ((uintptr_t)C & 31u) == 0 &&
+  // (An fp32 C is twice the bytes: the last tile's drain, which nothing hides, takes the row-per-lane stores
+  // 9.7 k clocks against 6 k staged, so there the path also wants six or more tiles per worker to pay:
+  // 2048^3 and 4096 x 4096 x 2048 -4 %, 2048 x 2048 x 4096 -2 %, 6144 x 6144 x 2048 +1.8 %.)
+  const bool long_enough = cn.c_bytes == 2 ? cn.K * (cn.ab_bytes / 2) >= kDirectMinK16
+                                           : (cn.K * (cn.ab_bytes / 2) >= kDirectMinK32 && cfg.full_tiles >= 6 * (int64_t)cfg.workers);
+  const bool direct = cfg.stages_direct > 0 && long_enough && beta == 0.f && ((uintptr_t)C & 31u) == 0 &&
                       (cn.ldc * cn.c_bytes) % 32 == 0 && (cn.N * cn.c_bytes) % 32 == 0 &&
                       (cn.batch <= 1 || (cn.stride_c * cn.c_bytes) % 32 == 0);
   prm.stages = direct ? cfg.stages_direct : cfg.stages;
