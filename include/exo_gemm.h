@@ -61,7 +61,8 @@ typedef enum { EXO_GEMM_ROW_MAJOR = 0, EXO_GEMM_COL_MAJOR = 1 } exo_gemm_layout_
  * partial sums): every part of a cut tile adds alpha * (its partial sum) onto C with
  * cp.reduce.async.bulk.tensor instead of handing it to the owning part through a workspace.  No
  * workspace, no waiting; the order of the additions is the memory system's, so results are not
- * bitwise reproducible from run to run.  fp32 C only (ERR_UNSUPPORTED from validate otherwise);
+ * bitwise reproducible from run to run.  fp32 C only (ERR_UNSUPPORTED from validate otherwise), plain
+ * tiles only (ERR_INVALID_ARG together with SHARE_ALWAYS / SHARE_SUBSTITUTED or CTA_ROWS(256));
  * exo_gemm_run then accepts beta == 1 (C is accumulated onto) and beta == 0 (the run first clears C
  * with a memset on the same stream) and returns ERR_UNSUPPORTED for any other beta.  Off by default:
  * the ordered workspace reduction measured level or faster and is deterministic.

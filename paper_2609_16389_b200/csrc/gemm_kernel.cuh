@@ -142,7 +142,10 @@ struct NoShare {
 // tiles, so a tile's epilogue overlaps the next tile's main loop.  2 (the "tall" tile, 256 x BN per
 // CTA): both accumulators belong to one tile -- A_lo and A_hi are multiplied with the same B block, so
 // a quarter less operand data enters shared memory per flop -- and the epilogue is exposed.
-template <int CTA_GROUP, int BN, int OUT, int KSUB, class Share = NoShare, int MREP = 1>
+// REDUCE: the kernel can add the parts of a cut tile onto C (p.reduce_add); compiled only into the few
+// instantiations that plans with that flag use -- the extra paths cost the others 1-2 % where the epilogue
+// bounds a tile.
+template <int CTA_GROUP, int BN, int OUT, int KSUB, class Share = NoShare, int MREP = 1, bool REDUCE = false>
 __global__ void __launch_bounds__(kNumThreads, 1)
 exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                 const __grid_constant__ CUtensorMap tm_c, const GemmParams p) {
@@ -151,6 +154,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   constexpr int STAGE_BYTES = stage_bytes(CTA_GROUP, BN, KSUB, MREP);
   constexpr int A_BYTES = KSUB * kATileBytes * MREP; // the A part of a stage
   constexpr int CTA_M = kBlockM * MREP;              // rows of C per CTA
+  static_assert(!REDUCE || (OUT == kOutFp32 && MREP == 1 && Share::kPairs == 1), "reduce-add: fp32 C, plain tiles");
   static_assert(MREP == 1 || (MREP == 2 && CTA_GROUP == 2 && BN == 256 && KSUB == 1 && Share::kPairs == 1),
                 "the tall tile exists for 2-CTA 256-column tiles only");
   constexpr uint32_t TMEM_COLS = 2 * BN;             // two accumulators; 128, 256 or 512 columns
@@ -438,7 +442,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         const int64_t t = wi.tile;
         // The owning slice of a tail tile that follows at least two whole tiles starts from an accumulator
         // into which the epilogue warps have already written the other slices' partial sums.
-        const bool preloaded = MREP == 1 && wi.slices > 1 && wi.slice == 0 && wi.after_whole && it >= preload_from && !p.reduce_add;
+        const bool preloaded = MREP == 1 && wi.slices > 1 && wi.slice == 0 && wi.after_whole && it >= preload_from && !(REDUCE && p.reduce_add);
         if constexpr (MREP == 1) {
           // the epilogue (of both CTAs) must have drained this accumulator
           ok = wait_barrier<PAIR>(tempty_bar(acc), acc_ph ^ 1u, p, WaitSite{kRoleMma, 100 + acc, (uint32_t)t, 0});
@@ -613,7 +617,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         // owner's epilogue is an ordinary one.  (With a single whole tile before the slice the partials
         // arrive too late for that; the owner then adds them in its epilogue.)
         WorkItem nx;
-        if (it + 1 >= preload_from && !p.reduce_add && work_item(p.work, worker, num_workers, it + 1, nkb, &nx) && nx.slices > 1 &&
+        if (it + 1 >= preload_from && !(REDUCE && p.reduce_add) && work_item(p.work, worker, num_workers, it + 1, nkb, &nx) && nx.slices > 1 &&
             nx.slice == 0 && nx.after_whole) {
           uint32_t bz2;
           const TileCoord tc2 = tile_coord(nx.tile, &bz2);
@@ -659,7 +663,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         }
       }
       EXO_TRACE_TILE(it, 3);
-      const bool preloaded = MREP == 1 && wi.slices > 1 && wi.slice == 0 && wi.after_whole && it >= preload_from && !p.reduce_add;  // see above
+      const bool preloaded = MREP == 1 && wi.slices > 1 && wi.slice == 0 && wi.after_whole && it >= preload_from && !(REDUCE && p.reduce_add);  // see above
       // one pass per accumulator of the tile: a single one, or (tall tile) rows 0..127 then 128..255 of the CTA
 #pragma unroll 1
       for (int32_t r = 0; r < MREP; ++r) {
@@ -694,7 +698,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       // tile adds alpha * (its partial sum) onto C with a TMA reduce-add; C holds beta * C_in (beta == 1) or
       // zeros (the host cleared it) before the launch, nobody waits for anybody, and the order of the
       // additions, hence the last bits of the result, is left to the memory system.
-      const bool tile_reduce = p.reduce_add != 0 && wi.slices > 1;
+      const bool tile_reduce = REDUCE && p.reduce_add != 0 && wi.slices > 1;
       const bool has_beta = has_beta_arg && !tile_reduce;
       const bool contributor = wi.slices > 1 && wi.slice != 0 && !tile_reduce;
       const bool owner = wi.slices > 1 && wi.slice == 0 && !preloaded && !tile_reduce;  // has to add the partials itself
@@ -886,6 +890,9 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
               if (tile_reduce) {
                 if (batched) ptx::tma_reduce_add_3d(&tm_c, col, row0, (int32_t)bz, buf0 + boff);
                 else ptx::tma_reduce_add_2d(&tm_c, col, row0, buf0 + boff);
+              } else if (p.c_evict_first) {
+                if (batched) ptx::tma_store_3d_hint(&tm_c, col, row0, (int32_t)bz, buf0 + boff, ptx::policy_evict_first());
+                else ptx::tma_store_2d_hint(&tm_c, col, row0, buf0 + boff, ptx::policy_evict_first());
               } else if (batched) {
                 ptx::tma_store_3d(&tm_c, col, row0, (int32_t)bz, buf0 + boff);
               } else {
@@ -903,7 +910,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       if (!ok) break;
       }  // accumulators of the tile
       if (!ok) break;
-      if (wi.slices > 1 && wi.slice == 0 && !preloaded && p.reduce_add == 0) partials_consumed(wi.tail_index);
+      if (wi.slices > 1 && wi.slice == 0 && !preloaded && !(REDUCE && p.reduce_add)) partials_consumed(wi.tail_index);
       if (warp == 2 && lane == 0) EXO_TRACE(2, it, 1, 4096);
       if (MREP == 2 || (acc ^= 1u) == 0u) acc_ph ^= 1u;
     }

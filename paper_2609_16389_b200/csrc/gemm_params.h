@@ -83,6 +83,7 @@ struct GemmParams {
   WorkPlan work;            // whole-K tiles round-robin, then the tail tiles cut along K
   float* split_ws;          // device: fp32 partial accumulators of the slices 1.. of every tail tile
   uint32_t* split_flags;    // device: per tail tile {arrivals of contributing warps, owner warps done}; both only grow
+  uint32_t c_evict_first;   // 1: the stores of C carry the L2 evict-first priority
   uint32_t reduce_add;      // 1: the parts of a cut tile add onto C (TMA reduce) instead of meeting in the workspace
   uint32_t split_arrivals;  // arrivals per contributing part of a tile and run: its epilogue warps (x accumulators)
   void* c_ptr;              // C of matrix 0 and its strides in bytes (read by the direct stores only)

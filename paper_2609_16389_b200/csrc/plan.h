@@ -80,6 +80,8 @@ inline exo_gemm_status_t validate_desc(const exo_gemm_desc_t* d) {
   // so does forcing the tall tile, which has no shared-operand form
   if (o.mrep == 2 && (o.cta_group == 1 || (o.tile_n != 0 && o.tile_n != 256) || o.ksub == 2 || o.share >= 2))
     return EXO_GEMM_ERR_INVALID_ARG;
+  // the reduce-add form of the K split exists for plain tiles only
+  if ((d->flags & (1u << 11)) && (o.share >= 2 || o.mrep == 2)) return EXO_GEMM_ERR_INVALID_ARG;
   // beyond here the call is a legal BLAS call; what follows is this library's supported set
   // fp32 operands are multiplied as tf32 (the precision of the paper's own kernels) into an fp32 C
   if (d->c_dtype != EXO_GEMM_FP32 && d->c_dtype != d->ab_dtype) return EXO_GEMM_ERR_UNSUPPORTED;
@@ -321,7 +323,7 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
   const bool unaligned_rows = c.K > 0 && (((c.lda * c.ab_bytes) % 128) != 0 || ((c.ldb * c.ab_bytes) % 128) != 0);
   for (int i = 0; i < 7; ++i) {
     const int g = cand[i][0], n = cand[i][1], pr = cand[i][2], mr = cand[i][3];
-    if (mr == 2 && (o.mrep == 1 || o.share >= 2 || o.ksub == 2)) continue;
+    if (mr == 2 && (o.mrep == 1 || o.share >= 2 || o.ksub == 2 || o.reduce_add)) continue;
     if (mr == 1 && o.mrep == 2 && max_pairs >= 1) continue;
     if (o.cta_group && o.cta_group != g) continue;
     if (o.tile_n && o.tile_n != n) continue;
@@ -346,7 +348,7 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
   // (The library's own tile choices only: a caller who names a tile shape gets plain pairs unless the
   // clusters are asked for as well.)
   if (best_g == 2 && best_n == 256 && best_p == 1 && best_r == 1 && o.share == 0 && unaligned_rows && max_quads >= 1 &&
-      o.cta_group == 0 && o.tile_n == 0 && o.mrep == 0 && (o.grid_limit & 3) == 0) {
+      o.cta_group == 0 && o.tile_n == 0 && o.mrep == 0 && !o.reduce_add && (o.grid_limit & 3) == 0) {
     int w_eff = max_quads;
     if (o.grid_limit && o.grid_limit / 4 < w_eff) w_eff = o.grid_limit / 4;
     if (w_eff >= 1) {
