@@ -328,7 +328,8 @@ int64_t exo_gemm_schedule_work(int64_t tiles, int32_t num_workers, int32_t tail_
     table = new (std::nothrow) TailItem[4 * (size_t)num_workers];
     if (!table) return -1;
     w.slots = build_tail_table(w.tail_tiles, num_k_blocks, tail_workers, num_workers, table, snap, owner_extra);
-    w.table = table;
+    w.owner_extra = owner_extra;
+    w.table = tail_workers % w.tail_tiles == 0 ? nullptr : table;   // whole slices are found by arithmetic, as on the device
   }
   int64_t n = 0;
   WorkItem wi;
@@ -526,8 +527,11 @@ exo_gemm_status_t launch_plan(exo_gemm_plan* plan, const void* A, const void* B,
   // (An fp32 C is twice the bytes: the last tile's drain, which nothing hides, takes the row-per-lane stores
   // 9.7 k clocks against 6 k staged, so there the path also wants six or more tiles per worker to pay:
   // 2048^3 and 4096 x 4096 x 2048 -4 %, 2048 x 2048 x 4096 -2 %, 6144 x 6144 x 2048 +1.8 %.)
+  // (Problems of less than one wave whose tiles are all cut along K are the exception: +1 to +5 % with the
+  // registers-to-global path, whose owner adds the partial sums in registers anyway.)
   const bool long_enough = cn.c_bytes == 2 ? cn.K * (cn.ab_bytes / 2) >= kDirectMinK16
-                                           : (cn.K * (cn.ab_bytes / 2) >= kDirectMinK32 && cfg.full_tiles >= 6 * (int64_t)cfg.workers);
+                                           : (cn.K * (cn.ab_bytes / 2) >= kDirectMinK32 &&
+                                              (cfg.full_tiles >= 6 * (int64_t)cfg.workers || (cfg.full_tiles == 0 && cfg.tail_workers > 0)));
   const bool direct = cfg.stages_direct > 0 && long_enough && beta == 0.f && ((uintptr_t)C & 31u) == 0 &&
                       (cn.ldc * cn.c_bytes) % 32 == 0 && (cn.N * cn.c_bytes) % 32 == 0 &&
                       (cn.batch <= 1 || (cn.stride_c * cn.c_bytes) % 32 == 0);
@@ -542,14 +546,15 @@ exo_gemm_status_t launch_plan(exo_gemm_plan* plan, const void* A, const void* B,
   prm.ldc_bytes = cn.ldc * cn.c_bytes;
   prm.c_batch_bytes = cn.stride_c * cn.c_bytes;
   // the tail tiles are cut along K only when there is a K loop to cut and scratch to reduce through
-  const bool split_now = cfg.tail_workers > 0 && read_ab && plan->d_tail_table != nullptr;
+  const bool split_now = cfg.tail_workers > 0 && read_ab && plan->d_tail_table != nullptr;   // (the table exists for every cutting plan)
   const bool reduce_add = split_now && (d.flags & (1u << 11)) != 0;
   // the reduce-add form needs C to hold beta * C_in before the launch: it can for beta == 1 (as it is) and
   // beta == 0 (cleared below)
   if (reduce_add && beta != 0.f && beta != 1.f) return EXO_GEMM_ERR_UNSUPPORTED;
   prm.reduce_add = reduce_add ? 1u : 0u;
+  const bool whole_slices = cfg.tail_workers > 0 && cfg.tail_workers % cfg.tail_tiles == 0;
   prm.work = WorkPlan{cfg.full_tiles, (int32_t)(cfg.full_tiles / cfg.workers), cfg.tail_tiles, split_now ? cfg.tail_workers : 0,
-                      cfg.slots, plan->d_tail_table};
+                      cfg.slots, cfg.owner_extra, whole_slices ? nullptr : plan->d_tail_table};
   prm.split_ws = plan->d_split_ws;
   prm.split_flags = plan->d_split_flags;
   prm.split_arrivals = (uint32_t)(kEpiWarps * cfg.cta_group * cfg.mrep);

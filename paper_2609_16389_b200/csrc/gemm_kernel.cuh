@@ -559,18 +559,22 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     // Bounded wait until every warp of every contributing slice of a tail tile has delivered its
     // partials.  One lane polls, with a pause between polls: this can run beside a main loop, whose
     // copy-issuing warps share the instruction issue slots and the memory pipeline with this warp.
-    auto wait_partials = [&](const WorkItem& w, int32_t r) {
+    // the run count of a tail tile's counters, read by lane 0 (see wait_partials); asked for early -- at the
+    // top of the owning item, a main loop before the answer is needed -- so that its round trip to L2 is
+    // not added to the wait
+    auto owner_run_of = [&](const WorkItem& w) {
+      uint32_t run = 0;
+      if (lane == 0) run = ptx::ld_acquire_gpu(p.split_flags + 2 * (w.tail_index * NPAIR + (int32_t)pair_id) + 1) / kOwnerWarps;
+      return run;
+    };
+    auto wait_partials = [&](const WorkItem& w, int32_t r, uint32_t run) {
       // Two words per tail tile (and pair): arrivals of contributing warps, and owner warps that are done with
       // the tile's partial sums.  Both only grow.  Every warp of the owning CTA group adds one to the second
       // word per run, so its value tells which run of the plan this is without any word from the host: the
       // counters work the same when the launches are replayed from a CUDA graph.  (A warp reads the word
       // before it adds its own one, and at most kOwnerWarps - 1 others have added theirs by then.)
       const uint32_t* flag = p.split_flags + 2 * (w.tail_index * NPAIR + (int32_t)pair_id);
-      uint32_t target = 0;
-      if (lane == 0) {
-        const uint32_t run = ptx::ld_acquire_gpu(flag + 1) / kOwnerWarps;
-        target = (run + 1u) * p.split_arrivals * (uint32_t)(w.slices - 1);
-      }
+      const uint32_t target = (run + 1u) * p.split_arrivals * (uint32_t)(w.slices - 1);   // lane 0's is the real one
       const long long t_start = clock64();
       uint32_t spins = 0;
       for (;;) {
@@ -624,7 +628,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
           const int32_t n_mine = chunks_of(tc2.m * (CTA_M * CTA_GROUP) + (int32_t)cta_rank * CTA_M + (int32_t)quad * 32,
                                            (tc2.n * NPAIR + (int32_t)pair_id) * BN);
           if (n_mine > 0) {
-            ok = wait_partials(nx, 0);
+            ok = wait_partials(nx, 0, owner_run_of(nx));
             if (!ok) break;
             const uint32_t tnext = tmem_base + ((quad * 32u) << 16) + (acc ^ 1u) * BN;
 #pragma unroll 1
@@ -664,6 +668,8 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       }
       EXO_TRACE_TILE(it, 3);
       const bool preloaded = MREP == 1 && wi.slices > 1 && wi.slice == 0 && wi.after_whole && it >= preload_from && !(REDUCE && p.reduce_add);  // see above
+      uint32_t owner_run = 0;
+      if (wi.slices > 1 && wi.slice == 0 && !preloaded && !(REDUCE && p.reduce_add)) owner_run = owner_run_of(wi);
       // one pass per accumulator of the tile: a single one, or (tall tile) rows 0..127 then 128..255 of the CTA
 #pragma unroll 1
       for (int32_t r = 0; r < MREP; ++r) {
@@ -723,7 +729,7 @@ exo_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         continue;
       }
       if (owner && mine > 0) {
-        ok = wait_partials(wi, r);
+        ok = wait_partials(wi, r, owner_run);
         if (!ok) break;
       }
       auto issue_cin = [&](uint32_t gg, int32_t i) {  // elected lane only: C_in of this warp's i-th chunk

@@ -254,6 +254,9 @@ inline int tail_workers_for(int64_t tiles, int64_t workers, int64_t K, int ksub,
   // (measured against the uncut tiles: 48 tiles of 256 x 256 on 74 pairs at K = 12288 +4 %; 58 tiles behind
   // seven whole waves at K = 2048 -7 %).
   const int64_t tw = workers;
+  // (Behind whole waves and with a very long K loop the tall tile is the better answer to such a tail: 192
+  // tiles of 256 x 256 at K = 12288 measured 3-11 % slower in ranges than as 96 tall tiles.)
+  if (o.split == 0 && behind_waves && K > 8192) return 0;
   if (o.split == 0) {
     // time saved against the exchange, both in clocks per column of the tile (a k-block of 64 takes 2;
     // a part's partial sums cost about 16 behind whole waves and about 38 side by side, as in
@@ -303,7 +306,11 @@ inline double estimate_clocks(int64_t M, int64_t N, int64_t K, int64_t batch, in
     if (tw > 0) {
       const int64_t parts = (tw + tail - 1) / tail;
       const double exchange = (full_waves > 0 ? 16.0 * (parts - 1) : 30.0 + 8.0 * (parts - 1)) * bn * mrep * mrep;
-      t += mainloop * (double)tail / (double)tw + 2500.0 + exchange;
+      // (ranges that ignore tile boundaries run about a sixth slower than their length says: tiles of one row or
+      // column no longer fetch the same k-blocks at the same time, so fewer operand loads meet in L2.
+      // Measured: 48 tiles on 74 pairs at K = 12288 gained 3-7 % where the ranges' length promised 35 %.)
+      const double out_of_step = tw % tail != 0 ? 1.15 : 1.0;
+      t += out_of_step * mainloop * (double)tail / (double)tw + 2500.0 + exchange;
     } else {
       t += per_tile;
     }
@@ -347,14 +354,29 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
   // slots of two tiles quantise worse than the single tiles did.
   // (The library's own tile choices only: a caller who names a tile shape gets plain pairs unless the
   // clusters are asked for as well.)
-  if (best_g == 2 && best_n == 256 && best_p == 1 && best_r == 1 && o.share == 0 && unaligned_rows && max_quads >= 1 &&
+  // The same where the tail of the plain pairs would be shared out in ranges that ignore tile boundaries:
+  // the two pairs of a cluster work on neighbouring tiles at the same k-blocks, which gives back part of the
+  // operand sharing in L2 that such ranges lose (3072 x 1000 x 12288 +7.8 %, 12288 x 1000 x 6144 +5.2 %,
+  // 6144 x 2048 x 6144 +3.2 %, 6144 x 512 x 12288 +2 %).
+  bool ranges = false;
+  if (best_g == 2 && best_n == 256 && best_p == 1 && best_r == 1 && max_pairs >= 1) {
+    int64_t w_pairs = max_pairs;
+    if (o.grid_limit && o.grid_limit / 2 < w_pairs) w_pairs = o.grid_limit / 2;
+    const int64_t tiles_pairs = ((c.M + 255) / 256) * ((c.N + 255) / 256) * c.batch;
+    if (w_pairs >= 1) {
+      const int64_t tail = tiles_pairs % w_pairs;
+      const int tw = tail_workers_for(tiles_pairs, w_pairs, c.K * (c.ab_bytes / 2), default_ksub(2, 256), o, 1);
+      ranges = tw > 0 && tail > 0 && tw % tail != 0;
+    }
+  }
+  if (best_g == 2 && best_n == 256 && best_p == 1 && best_r == 1 && o.share == 0 && (unaligned_rows || ranges) && max_quads >= 1 &&
       o.cta_group == 0 && o.tile_n == 0 && o.mrep == 0 && !o.reduce_add && (o.grid_limit & 3) == 0) {
     int w_eff = max_quads;
     if (o.grid_limit && o.grid_limit / 4 < w_eff) w_eff = o.grid_limit / 4;
     if (w_eff >= 1) {
       const double t = estimate_clocks(c.M, c.N, c.K * (c.ab_bytes / 2), c.batch, 2, 256, w_eff, o, 2, 1,
                                        c.a_mn_major || c.b_mn_major, true);
-      if (t <= best) best_p = 2;
+      if (t <= best * (ranges ? 1.03 : 1.0)) best_p = 2;
     }
   }
   TileConfig cfg;

@@ -131,7 +131,9 @@ struct WorkPlan {
   int32_t tail_tiles;    // tiles [full_tiles, full_tiles + tail_tiles)
   int32_t tail_workers;  // workers that share the tail tiles' k-blocks (0: the tail is not cut)
   int32_t slots;         // partial-sum slots per tail tile in the workspace: the most contributors any tile has
-  const TailItem* table; // device (or host, for the host-side enumeration): 4 entries per worker
+  int32_t owner_extra;   // whole slices: k-blocks the owning slice takes beyond an even share
+  const TailItem* table; // ranges: device (or host, for the host-side enumeration) table, 4 entries per worker;
+                         // NULL: tail_workers is a multiple of tail_tiles and every tile is cut into whole slices
 };
 
 struct WorkItem {
@@ -250,7 +252,13 @@ EXO_HD bool work_item(const WorkPlan& w, int64_t worker, int64_t num_workers, in
                       WorkItem* out) {
   int32_t lead = 0, n_items = 0;
   const TailItem* e = nullptr;
-  if (w.tail_workers > 0) {
+  // whole slices: every sharing worker has exactly one part, found by arithmetic (the table is for ranges
+  // only: its two dependent loads would sit in front of the first copy of every worker of a small problem)
+  const bool whole_slices = w.tail_workers > 0 && w.table == nullptr;
+  if (whole_slices) {
+    n_items = worker < w.tail_workers ? 1 : 0;
+    lead = n_items && worker >= w.tail_tiles ? 1 : 0;   // a contributing slice
+  } else if (w.tail_workers > 0) {
     e = w.table + 4 * worker;
     lead = e[0].tail_index;
     n_items = e[0].kb_begin;
@@ -274,6 +282,29 @@ EXO_HD bool work_item(const WorkPlan& w, int64_t worker, int64_t num_workers, in
     k = lead + (j - w.waves);
     if (w.tail_workers == 0 || k >= n_items) return false;
   }
+  out->after_whole = i > lead;   // (items that come first have no whole tile before them)
+  if (whole_slices) {
+    const int32_t f = w.slots + 1;
+    const int32_t sl = (int32_t)((uint32_t)worker / (uint32_t)w.tail_tiles);
+    const int32_t ti = (int32_t)((uint32_t)worker - (uint32_t)sl * (uint32_t)w.tail_tiles);
+    out->tile = w.full_tiles + ti;
+    out->tail_index = ti;
+    out->slice = sl;
+    out->slices = f;
+    // slice 0: an even share plus owner_extra; slices 1.. share the rest evenly, in K order
+    int32_t own = (num_k_blocks + f - 1) / f + w.owner_extra;
+    if (own > num_k_blocks - (f - 1)) own = num_k_blocks - (f - 1);
+    if (own < 1) own = 1;
+    if (sl == 0) {
+      out->kb_begin = 0;
+      out->kb_end = own;
+    } else {
+      const uint32_t rest = (uint32_t)(num_k_blocks - own);   // rest * slice < 2^31: both are small
+      out->kb_begin = own + (int32_t)((rest * (uint32_t)(sl - 1)) / (uint32_t)(f - 1));
+      out->kb_end = own + (int32_t)((rest * (uint32_t)sl) / (uint32_t)(f - 1));
+    }
+    return true;
+  }
   const TailItem it = e[1 + k];
   out->tile = w.full_tiles + it.tail_index;
   out->slice = it.slice_info & 0xFFFF;
@@ -281,7 +312,6 @@ EXO_HD bool work_item(const WorkPlan& w, int64_t worker, int64_t num_workers, in
   out->tail_index = out->slices > 1 ? it.tail_index : -1;
   out->kb_begin = it.kb_begin;
   out->kb_end = it.kb_end;
-  out->after_whole = i > lead;   // (items that come first have no whole tile before them)
   return true;
 }
 
