@@ -331,6 +331,11 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
   for (int i = 0; i < 7; ++i) {
     const int g = cand[i][0], n = cand[i][1], pr = cand[i][2], mr = cand[i][3];
     if (mr == 2 && (o.mrep == 1 || o.share >= 2 || o.ksub == 2 || o.reduce_add)) continue;
+    // The tall tile is the library's own choice only for problems of up to four waves of it: measured
+    // against the 128-row tile it wins 2-6 % there at long K (6144^3, 6144 x 6144 x 12288, 4608 x 4096 x 16384)
+    // and loses 2-5 % on larger problems (8192^3 with any C, 12288 x 6144 x 6144, 12288^3).
+    if (mr == 2 && o.mrep == 0 && max_pairs >= 1 &&
+        ((c.M + 511) / 512) * ((c.N + 255) / 256) * c.batch > 4 * (int64_t)max_pairs) continue;
     if (mr == 1 && o.mrep == 2 && max_pairs >= 1) continue;
     if (o.cta_group && o.cta_group != g) continue;
     if (o.tile_n && o.tile_n != n) continue;
@@ -349,6 +354,19 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
     if (best_g == 0 || t < best * 0.97) { best = t; best_g = g; best_n = n; best_p = pr; best_r = mr; }
   }
   if (best_g == 0) { best_g = o.cta_group ? o.cta_group : 1; best_n = o.tile_n ? o.tile_n : 128; }
+  // Short K loops on one or two waves of 256 x 256 tiles: where 256 x 128 tiles fill their waves clearly
+  // better they win (K = 512, 96 tiles of 256 x 256 on 74 pairs = 65 % against 192 on 222 = 86 %: +4 to +6 %
+  // with a bf16 C, +0.4 to +2 % with an fp32 C), which the clock estimate above, made for many waves, does not
+  // see; where both fill alike the wider tile stays (144 tiles: -8 to -14 % with 128 columns).
+  if (best_g == 2 && best_n == 256 && best_p == 1 && best_r == 1 && max_pairs >= 1 && o.cta_group == 0 && o.tile_n == 0 &&
+      o.mrep == 0 && o.share < 2 && o.grid_limit == 0 && c.K * (c.ab_bytes / 2) <= 512) {
+    const int64_t t256 = ((c.M + 255) / 256) * ((c.N + 255) / 256) * c.batch;
+    const int64_t t128 = ((c.M + 255) / 256) * ((c.N + 127) / 128) * c.batch;
+    const int64_t w = max_pairs;
+    const double fill256 = (double)t256 / (double)(((t256 + w - 1) / w) * w);
+    const double fill128 = (double)t128 / (double)(((t128 + w - 1) / w) * w);
+    if (t256 <= 2 * w && fill128 >= fill256 + 0.15) best_n = 128;
+  }
   // Where the choice fell on plain pairs of 256 x 256 tiles and the operand rows are not 128-byte aligned,
   // the same tiles in shared-operand clusters are the faster form (see kShareGainUnalignedRows), unless the
   // slots of two tiles quantise worse than the single tiles did.
@@ -400,7 +418,9 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
   // every K (bf16 C, 6 stages + 1 buffer against 5 + 2: +3 to +5 % at K = 1000 .. 1024, +1 % at 512 and 1536,
   // -0.2 % at 12288 x 12288 x 512).
   const int64_t k16 = c.K * (c.ab_bytes / 2);
-  const bool want_two = c.c_bytes == 4 && k16 <= 1024 && max_stages(best_g, best_n, cfg.ksub, 2, best_r) >= 3;
+  // (except at K <= 512 with fewer than three tiles per worker, where the second buffer measured +1 to +3 %)
+  const bool want_two = (c.c_bytes == 4 ? k16 <= 1024 : (k16 <= 512 && tiles < 3 * workers)) &&
+                        max_stages(best_g, best_n, cfg.ksub, 2, best_r) >= 3;
   cfg.epi_bufs = o.epi_bufs ? o.epi_bufs : (want_two ? 2 : 1);
   cfg.stages = max_stages(best_g, best_n, cfg.ksub, cfg.epi_bufs, best_r);
   if (o.stages && o.stages < cfg.stages) cfg.stages = o.stages < 2 ? 2 : o.stages;
