@@ -76,9 +76,9 @@ def test_static_entry_point_checks_its_arguments_like_the_others():
 
 
 def test_static_entry_point_enqueues_nothing_when_it_refuses_its_arguments():
-    """A refused call must leave the stream untouched: an event recorded after it is complete at once
-    even while the stream is blocked behind ... nothing.  Checked the cheap way: the status array keeps a
-    marker that only an enqueued clear (or kernel) of a refused call could have changed."""
+    """A call that is refused (misaligned or NULL operand) or has nothing to do (M == 0) returns before
+    it enqueues anything, also right after a call whose device-side wait ran out; the next good call
+    clears the status words on its stream and computes the oracle's result."""
     import torch
     dev = torch.device("cuda:0")
     p = synth.Problem("static_marker", 256, 256, 128, synth.BF16, synth.FP32, 0, 1, 0, 1.0, 0.0, seed=31).generate()
