@@ -105,6 +105,20 @@ typedef enum { EXO_GEMM_ROW_MAJOR = 0, EXO_GEMM_COL_MAJOR = 1 } exo_gemm_layout_
 #define EXO_GEMM_FLAG2_CTA_ROWS(r) ((((uint32_t)(r) / 128u) & 3u) << 2)
 
 /*
+ * flags2, bits 4-5: the one-tile-per-CTA kernel for problems of less than one wave (the small
+ * matrices of the paper's Section 6, where a run is a chain of latencies rather than a stream of
+ * tiles).  One CTA per 128 x 64 or 128 x 128 tile, all launched at once; the copies of the first
+ * k-blocks are issued before the CTA's set-up barrier, C_in is fetched during the main loop, and
+ * no warp waits for another at the end.  It never cuts K and has no strided-batch form.
+ * 0 = the library decides, 1 = never, 2 = always (ERR_INVALID_ARG together with CTA_GROUP(2),
+ * TILE_N(256), a SHARE_ALWAYS / SHARE_SUBSTITUTED or CTA_ROWS(256) request, SPLIT_K(2..),
+ * SPLIT_REDUCE_ADD or a GRID_LIMIT; a batched plan ignores it).  3 is invalid.
+ */
+#define EXO_GEMM_FLAG2_LEAN_AUTO 0u
+#define EXO_GEMM_FLAG2_LEAN_NEVER (1u << 4)
+#define EXO_GEMM_FLAG2_LEAN_ALWAYS (2u << 4)
+
+/*
  * Problem descriptor.  Logical shapes: A is M x K, B is K x N, C is M x N.
  * Leading dimensions are in elements: for a row-major matrix ld >= #columns, for
  * a column-major matrix ld >= #rows.
@@ -129,7 +143,7 @@ typedef struct {
   int32_t device;                       /* CUDA device ordinal; -1 = the current device        */
   int64_t lda, ldb, ldc;                /* elements                                            */
   uint32_t flags;                       /* 0, or EXO_GEMM_FLAG_* overrides                     */
-  uint32_t flags2;                      /* 0, or EXO_GEMM_FLAG2_*; bits 4.. must be 0          */
+  uint32_t flags2;                      /* 0, or EXO_GEMM_FLAG2_*; bits 6.. must be 0          */
 } exo_gemm_desc_t;
 
 /* What a plan decided; filled by exo_gemm_get_info. */
@@ -159,6 +173,8 @@ typedef struct {
   int32_t stages_direct;   /* depth of the operand ring in runs that store C straight from registers
                               (no staging buffers: beta == 0 and C, ldc and N multiples of 32 bytes);
                               0 if the plan always stages (EXO_GEMM_FLAG_EPI_BUFFERS given)        */
+  int32_t lean_kernel;     /* 1: the one-tile-per-CTA kernel runs this plan (EXO_GEMM_FLAG2_LEAN_*): grid =
+                              tiles_m * tiles_n CTAs at once, one accumulator, `stages` = its ring         */
 } exo_gemm_info_t;
 
 /*

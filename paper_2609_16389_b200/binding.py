@@ -34,6 +34,7 @@ def flag_epi_buffers(b): return (b & 3) << 22
 def flag_max_stages(s): return (s & 15) << 24
 def flag_split_k(f): return (f & 15) << 28
 FLAG2_SHARE_AUTO, FLAG2_SHARE_NEVER, FLAG2_SHARE_ALWAYS, FLAG2_SHARE_SUBSTITUTED = 0, 1, 2, 3
+FLAG2_LEAN_AUTO, FLAG2_LEAN_NEVER, FLAG2_LEAN_ALWAYS = 0, 1 << 4, 2 << 4
 def flag2_cta_rows(r): return ((r // 128) & 3) << 2
 
 
@@ -51,7 +52,7 @@ class Info(ctypes.Structure):
         "cta_group", "tile_m", "tile_n", "tile_k", "stages", "grid", "smem_bytes", "tmem_columns",
         "tiles_m", "tiles_n", "raster_along_m", "raster_band", "swapped", "sm_count",
         "kernel_launches_per_run", "epilogue_buffers", "split_k", "tail_tiles", "workspace_bytes",
-        "batch_count", "cluster_size", "tail_workers", "stages_direct")]
+        "batch_count", "cluster_size", "tail_workers", "stages_direct", "lean_kernel")]
 
     def as_dict(self):
         return {n: getattr(self, n) for n, _ in self._fields_}

@@ -10,6 +10,7 @@
 
 #include "../../include/exo_gemm.h"
 #include "gemm_kernel.cuh"
+#include "lean_kernel.cuh"
 #include "plan.h"
 #ifdef EXO_GEMM_SHARE_PAIRS
 #include "cluster4/share_pairs.cuh"
@@ -75,6 +76,30 @@ static KernelFn pick_kernel(int cta_group, int bn, int ksub, int out, int pairs 
   if (mrep == 2) return pick_tall(out);
   if (pairs == 2) return ksub == 2 ? pick_shared<2>(out) : pick_shared<1>(out);
   return ksub == 2 ? pick_shape<2>(cta_group, bn, out) : pick_shape<1>(cta_group, bn, out);
+}
+
+// the one-tile-per-CTA kernel: 128 x 64 or 128 x 128 tiles
+template <int BN, int KSUB>
+static KernelFn pick_lean_out(int out) {
+  switch (out) {
+    case EXO_GEMM_BF16: return exo_gemm_lean_kernel<BN, kOutBf16, KSUB>;
+    case EXO_GEMM_FP16: return exo_gemm_lean_kernel<BN, kOutFp16, KSUB>;
+    default:            return exo_gemm_lean_kernel<BN, kOutFp32, KSUB>;
+  }
+}
+static KernelFn pick_lean(int bn, int ksub, int out) {
+  if (bn == 128) return ksub == 2 ? pick_lean_out<128, 2>(out) : pick_lean_out<128, 1>(out);
+  return ksub == 2 ? pick_lean_out<64, 2>(out) : pick_lean_out<64, 1>(out);
+}
+
+// kernel and dynamic shared memory of a plan's configuration
+static KernelFn kernel_of(const TileConfig& cfg, int c_dtype, bool reduce) {
+  if (cfg.lean) return pick_lean(cfg.tile_n, cfg.ksub, c_dtype);
+  return pick_kernel(cfg.cta_group, cfg.tile_n, cfg.ksub, c_dtype, cfg.pairs, cfg.mrep, reduce);
+}
+static int smem_of(const TileConfig& cfg, int c_dtype) {
+  if (cfg.lean) return lean_smem_bytes(cfg.tile_n, cfg.ksub, cfg.stages, c_dtype == EXO_GEMM_FP32 ? 4 : 2, cfg.lean);
+  return smem_bytes_for(cfg.cta_group, cfg.tile_n, cfg.ksub, cfg.stages, cfg.epi_bufs, cfg.mrep);
 }
 
 static thread_local int g_last_cuda_error = 0;
@@ -248,12 +273,13 @@ void fill_info(const exo_gemm_plan* p, exo_gemm_info_t* info) {
   info->tile_n = p->cfg.tile_n;
   info->tile_k = sub_block_k(p->canon.ab_bytes) * p->cfg.ksub;
   info->stages = p->cfg.stages;
-  info->grid = p->cfg.workers * p->cfg.cta_group * p->cfg.pairs;
-  info->cluster_size = p->cfg.cta_group * p->cfg.pairs;
+  info->grid = p->cfg.workers * p->cfg.cta_group * p->cfg.pairs * (p->cfg.lean ? p->cfg.lean : 1);
+  info->cluster_size = p->cfg.lean ? p->cfg.lean : p->cfg.cta_group * p->cfg.pairs;
   info->stages_direct = p->cfg.stages_direct;
   info->tail_workers = p->cfg.tail_workers;
   info->smem_bytes = p->smem_bytes;
   info->tmem_columns = 2 * p->cfg.tile_n;
+  info->lean_kernel = p->cfg.lean ? 1 : 0;
   info->tiles_m = p->cfg.tiles_m;
   info->tiles_n = p->cfg.tiles_n;
   info->raster_along_m = p->cfg.along_m;
@@ -262,7 +288,7 @@ void fill_info(const exo_gemm_plan* p, exo_gemm_info_t* info) {
   info->sm_count = p->sm_count;
   info->kernel_launches_per_run = (p->canon.M == 0 || p->canon.N == 0) ? 0 : 1;
   info->epilogue_buffers = p->cfg.epi_bufs;
-  info->split_k = p->cfg.split;
+  info->split_k = p->cfg.lean ? p->cfg.lean : p->cfg.split;
   info->tail_tiles = p->cfg.tail_tiles;
   info->batch_count = (int32_t)p->canon.batch;
   info->workspace_bytes = (int32_t)(p->cfg.workspace_bytes > 2147483647LL ? 2147483647LL : p->cfg.workspace_bytes);
@@ -359,7 +385,7 @@ exo_gemm_status_t exo_gemm_plan_preview(const exo_gemm_desc_t* desc, int32_t sm_
   if (ov.share >= 2 && !kHaveSharePairs) return EXO_GEMM_ERR_UNSUPPORTED;
   p.cfg = choose_config(p.canon, ov, sm_count, sm_count / 2, kHaveSharePairs ? sm_count / 4 : 0);
   p.cfg.workspace_bytes = ov.reduce_add ? 0 : split_workspace_bytes(p.cfg, desc->c_dtype);
-  p.smem_bytes = smem_bytes_for(p.cfg.cta_group, p.cfg.tile_n, p.cfg.ksub, p.cfg.stages, p.cfg.epi_bufs, p.cfg.mrep);
+  p.smem_bytes = smem_of(p.cfg, desc->c_dtype);
   fill_info(&p, info);
   return EXO_GEMM_OK;
 }
@@ -411,8 +437,8 @@ exo_gemm_status_t exo_gemm_create_batched(exo_gemm_handle_t* out, const exo_gemm
 
   p->cfg = choose_config(p->canon, ov, sms, max_pairs, max_quads);
   p->cfg.workspace_bytes = ov.reduce_add ? 0 : split_workspace_bytes(p->cfg, desc->c_dtype);
-  p->kernel = pick_kernel(p->cfg.cta_group, p->cfg.tile_n, p->cfg.ksub, desc->c_dtype, p->cfg.pairs, p->cfg.mrep, ov.reduce_add);
-  p->smem_bytes = smem_bytes_for(p->cfg.cta_group, p->cfg.tile_n, p->cfg.ksub, p->cfg.stages, p->cfg.epi_bufs, p->cfg.mrep);
+  p->kernel = kernel_of(p->cfg, desc->c_dtype, ov.reduce_add);
+  p->smem_bytes = smem_of(p->cfg, desc->c_dtype);
   e = allow_full_smem(p->kernel);
   if (e != cudaSuccess) { delete p; return cuda_fail(e); }
   e = cudaMalloc((void**)&p->d_status, kStatusBytes);
@@ -532,7 +558,7 @@ exo_gemm_status_t launch_plan(exo_gemm_plan* plan, const void* A, const void* B,
   const bool long_enough = cn.c_bytes == 2 ? cn.K * (cn.ab_bytes / 2) >= kDirectMinK16
                                            : (cn.K * (cn.ab_bytes / 2) >= kDirectMinK32 &&
                                               (cfg.full_tiles >= 6 * (int64_t)cfg.workers || (cfg.full_tiles == 0 && cfg.tail_workers > 0)));
-  const bool direct = cfg.stages_direct > 0 && long_enough && beta == 0.f && ((uintptr_t)C & 31u) == 0 &&
+  const bool direct = !cfg.lean && cfg.stages_direct > 0 && long_enough && beta == 0.f && ((uintptr_t)C & 31u) == 0 &&
                       (cn.ldc * cn.c_bytes) % 32 == 0 && (cn.N * cn.c_bytes) % 32 == 0 &&
                       (cn.batch <= 1 || (cn.stride_c * cn.c_bytes) % 32 == 0);
   prm.stages = direct ? cfg.stages_direct : cfg.stages;
@@ -610,14 +636,14 @@ exo_gemm_status_t launch_plan(exo_gemm_plan* plan, const void* A, const void* B,
   DeviceGuard guard(plan->device);
   if (guard.err != cudaSuccess) return cuda_fail(guard.err);
   cudaLaunchConfig_t lc{};
-  lc.gridDim = dim3((unsigned)(cfg.workers * cfg.cta_group * cfg.pairs), 1, 1);
-  lc.blockDim = dim3(kNumThreads, 1, 1);
+  lc.gridDim = dim3((unsigned)(cfg.workers * cfg.cta_group * cfg.pairs * (cfg.lean ? cfg.lean : 1)), 1, 1);
+  lc.blockDim = dim3(cfg.lean ? (unsigned)lean_threads(cfg.tile_n, (int)cn.c_bytes) : (unsigned)kNumThreads, 1, 1);
   lc.dynamicSmemBytes = direct ? smem_bytes_for(cfg.cta_group, cfg.tile_n, cfg.ksub, cfg.stages_direct, 0, cfg.mrep)
                                : plan->smem_bytes;
   lc.stream = (cudaStream_t)cuda_stream;
   cudaLaunchAttribute at[3];
   at[0].id = cudaLaunchAttributeClusterDimension;
-  at[0].val.clusterDim.x = (unsigned)cfg.cta_group;
+  at[0].val.clusterDim.x = (unsigned)(cfg.lean ? cfg.lean : cfg.cta_group);
   at[0].val.clusterDim.y = 1;
   at[0].val.clusterDim.z = 1;
   // Programmatic dependent launch: this kernel's CTAs may start (barrier set-up, TMEM allocation)
@@ -745,8 +771,8 @@ exo_gemm_status_t exo_gemm_run_static(const exo_gemm_desc_t* desc, const void* A
   if (e != cudaSuccess) return cuda_fail(e);
   if (ov.share >= 2 && max_quads < 1) return EXO_GEMM_ERR_UNSUPPORTED;
   plan.cfg = choose_config(plan.canon, ov, sms, max_pairs, max_quads);
-  plan.kernel = pick_kernel(plan.cfg.cta_group, plan.cfg.tile_n, plan.cfg.ksub, desc->c_dtype, plan.cfg.pairs, plan.cfg.mrep);
-  plan.smem_bytes = smem_bytes_for(plan.cfg.cta_group, plan.cfg.tile_n, plan.cfg.ksub, plan.cfg.stages, plan.cfg.epi_bufs, plan.cfg.mrep);
+  plan.kernel = kernel_of(plan.cfg, desc->c_dtype, false);
+  plan.smem_bytes = smem_of(plan.cfg, desc->c_dtype);
   e = allow_full_smem(plan.kernel);
   if (e != cudaSuccess) return cuda_fail(e);
 

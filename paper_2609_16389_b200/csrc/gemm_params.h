@@ -40,6 +40,23 @@ EXO_CX int max_stages(int cta_group, int bn, int ksub, int epi_bufs, int mrep = 
   return n > kMaxStages ? kMaxStages : n;
 }
 
+// The one-tile-per-CTA kernel (lean_kernel.cuh): 1-CTA tiles of 128 x bn, bn = 64 or 128.
+// epilogue warps of a lean tile: one per TMEM lane quadrant and per half of the column chunks
+EXO_CX int lean_epi_warps(int bn, int c_bytes) { return (bn * c_bytes / 128) >= 2 ? 8 : 4; }
+EXO_CX int lean_threads(int bn, int c_bytes) { return 64 + 32 * lean_epi_warps(bn, c_bytes); }
+// the peers' partial sums of the rows a CTA finishes when `split` CTAs (a cluster of 1, 2 or 4) share a tile's K loop
+EXO_CX int lean_recv_bytes(int bn, int split) { return split > 1 ? (split - 1) * (4 / split) * (bn / 32) * kEpiBufBytes : 0; }
+// shared memory of a lean CTA: the operand ring, one staging buffer per column chunk and quadrant,
+// the receive buffer, barriers, alignment slack
+EXO_CX int lean_smem_bytes(int bn, int ksub, int stages, int c_bytes, int split) {
+  return stages * stage_bytes(1, bn, ksub) + 4 * (bn * c_bytes / 128) * kEpiBufBytes + lean_recv_bytes(bn, split) + kBarrierBytes + 1024;
+}
+EXO_CX int lean_max_stages(int bn, int ksub, int c_bytes, int split) {
+  const int n = (kSmemLimit - 1024 - kBarrierBytes - 4 * (bn * c_bytes / 128) * kEpiBufBytes - lean_recv_bytes(bn, split)) /
+                stage_bytes(1, bn, ksub);
+  return n > kMaxStages ? kMaxStages : n;
+}
+
 // How one operand is staged.  K-major: per 64-k sub-block one TMA box {64 k, rows},
 // sub-blocks rows*128 bytes apart.  MN-major: rows/64 boxes {64 mn, 64*ksub k}.
 struct OperandStaging {

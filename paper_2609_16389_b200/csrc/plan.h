@@ -26,6 +26,7 @@ struct FlagOverrides {
   int share;       // clusters of two CTA pairs sharing the loads of A: 0 = auto, 1 = never, 2 = always,
                    // 3 = always, but every slot launched as two plain pairs (exercises the substitute path)
   int mrep;        // 128-row blocks of C per CTA: 0 = auto, 1, or 2 (the tall 2-CTA tile, 512 x 256 per pair)
+  int lean;        // the one-tile-per-CTA kernel for problems of less than one wave: 0 = auto, 1 = never, 2 = always
 };
 
 inline FlagOverrides decode_flags(uint32_t f, uint32_t f2 = 0) {
@@ -43,12 +44,13 @@ inline FlagOverrides decode_flags(uint32_t f, uint32_t f2 = 0) {
   o.reduce_add = (f & (1u << 11)) != 0;
   o.share = (int)(f2 & 3u);
   o.mrep = (int)((f2 >> 2) & 3u);
+  o.lean = (int)((f2 >> 4) & 3u);
   return o;
 }
 
 inline exo_gemm_status_t validate_desc(const exo_gemm_desc_t* d) {
   if (!d) return EXO_GEMM_ERR_NULL;
-  if ((d->flags2 & ~15u) != 0 || ((d->flags2 >> 2) & 3u) == 3u) return EXO_GEMM_ERR_INVALID_ARG;
+  if ((d->flags2 & ~63u) != 0 || ((d->flags2 >> 2) & 3u) == 3u || ((d->flags2 >> 4) & 3u) == 3u) return EXO_GEMM_ERR_INVALID_ARG;
   const int64_t kMaxDim = 2147483647LL;
   if (d->M < 0 || d->N < 0 || d->K < 0 || d->M > kMaxDim || d->N > kMaxDim || d->K > kMaxDim)
     return EXO_GEMM_ERR_INVALID_ARG;
@@ -82,6 +84,11 @@ inline exo_gemm_status_t validate_desc(const exo_gemm_desc_t* d) {
     return EXO_GEMM_ERR_INVALID_ARG;
   // the reduce-add form of the K split exists for plain tiles only
   if ((d->flags & (1u << 11)) && (o.share >= 2 || o.mrep == 2)) return EXO_GEMM_ERR_INVALID_ARG;
+  // the one-tile-per-CTA kernel has 1-CTA tiles of 128 x 64 or 128 x 128, cuts K over a cluster of 2 or 4 only and
+  // takes every tile at once
+  if (o.lean == 2 && (o.cta_group == 2 || o.tile_n == 256 || o.share >= 2 || o.mrep == 2 || (o.split >= 2 && o.split != 2 && o.split != 4) ||
+                      (d->flags & (1u << 11)) || o.grid_limit != 0))
+    return EXO_GEMM_ERR_INVALID_ARG;
   // beyond here the call is a legal BLAS call; what follows is this library's supported set
   // fp32 operands are multiplied as tf32 (the precision of the paper's own kernels) into an fp32 C
   if (d->c_dtype != EXO_GEMM_FP32 && d->c_dtype != d->ab_dtype) return EXO_GEMM_ERR_UNSUPPORTED;
@@ -174,6 +181,8 @@ struct TileConfig {
   int tiles_m, tiles_n;    // tiles of (128 * cta_group) x (tile_n * pairs): what one cluster computes at a time
   int band, along_m;
   int workers;  // CTA groups launched
+  int lean;     // > 0: the one-tile-per-CTA kernel runs this plan (workers = tiles, `stages` is its ring) with clusters of
+                // this many CTAs (1, 2 or 4) sharing each tile's K loop
 };
 
 // Sub-blocks of 64 k-elements per pipeline stage.  Two per stage halves the number of
@@ -318,6 +327,30 @@ inline double estimate_clocks(int64_t M, int64_t N, int64_t K, int64_t batch, in
   return t + drain + 3000.0;  // the last epilogue and the pipeline fill are exposed once
 }
 
+// Whether the one-tile-per-CTA kernel is the library's own choice, and with which tile width and how many
+// CTAs per tile.  Measured against the persistent kernel's plan on every sweep shape of up to 300 tiles
+// (launches replayed from CUDA graphs, bf16 and fp32 C): while 128 x 64 tiles fit the SMs at one CTA each it wins
+// 12-30 % up to K = 2048; with room for two or four CTAs per tile a K loop from about 1000 on is cut over a
+// cluster (512 x 512: +15 to +55 % up to K = 12288; 512 x 1000: +13 to +27 % up to K = 3072, level at 6144);
+// 128 x 128 tiles win at K = 512 only (+18 to +26 %; +2 to +6 % at K = 1000); beyond one wave of those the
+// persistent kernel's larger tiles are faster at every K.
+inline bool lean_is_faster(const Canonical& c, const FlagOverrides& o, int sm_count, int* bn, int* split) {
+  const int64_t k16 = c.K * (c.ab_bytes / 2);
+  const int64_t t64 = ((c.M + 127) / 128) * ((c.N + 63) / 64), t128 = ((c.M + 127) / 128) * ((c.N + 127) / 128);
+  *split = 1;
+  if (k16 <= 0 || t128 <= 0) return false;
+  if (t64 <= sm_count) {
+    *bn = 64;
+    if (k16 >= 960 && o.split == 0 && !o.no_workspace) *split = t64 * 4 <= sm_count ? 4 : (t64 * 2 <= sm_count ? 2 : 1);
+    return k16 <= (*split == 4 ? 16384 : (*split == 2 ? 4096 : 2048));
+  }
+  if (t128 <= sm_count) {
+    *bn = 128;
+    return k16 <= 768;
+  }
+  return false;
+}
+
 inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int sm_count,
                                 int max_pairs /* co-resident 2-CTA clusters */,
                                 int max_quads = 0 /* co-resident 4-CTA clusters; 0: variant not available */) {
@@ -397,7 +430,33 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
       if (t <= best * (ranges ? 1.03 : 1.0)) best_p = 2;
     }
   }
+  // Problems of less than one wave: the one-tile-per-CTA kernel (lean_kernel.cuh), 128 x 64 tiles while they
+  // fit the SMs at one per SM, else 128 x 128.
+  bool lean = false;
+  int lean_split = 1;   // CTAs (a cluster) that share a lean tile's K loop: 1, 2 or 4
+  if (o.lean != 1 && c.batch <= 1 && !o.reduce_add && o.share < 2 && o.mrep != 2 && o.cta_group != 2 && o.tile_n != 256 &&
+      o.grid_limit == 0 && (o.split < 2 || o.split == 2 || o.split == 4)) {
+    const int ksub = o.ksub ? o.ksub : 2;
+    const int64_t nkb_all = (c.K * (c.ab_bytes / 2) + kBlockK * ksub - 1) / (kBlockK * ksub);
+    int bn = 64, split = 1;
+    if (o.lean == 2) {   // on request: 128 x 64 tiles while a CTA per tile fits the SMs, else 128 x 128; K cut as asked
+      const int64_t t64 = ((c.M + 127) / 128) * ((c.N + 63) / 64);
+      bn = o.tile_n ? o.tile_n : (t64 <= sm_count ? 64 : 128);
+      split = o.split >= 2 ? o.split : 1;
+      lean = true;
+    } else if (o.tile_n == 0 && o.cta_group == 0 && o.ksub == 0 && o.stages == 0 && o.epi_bufs == 0 && o.band == 0 &&
+               o.along_m == 0 && o.split < 2) {
+      // (the library's own choice only where the caller names no parameter of the persistent kernel)
+      lean = lean_is_faster(c, o, sm_count, &bn, &split);
+    }
+    if (lean) {
+      best_g = 1; best_n = bn; best_p = 1; best_r = 1;
+      lean_split = split;
+      while (lean_split > 1 && lean_split > nkb_all) lean_split /= 2;   // every CTA of a cluster gets a k-block
+    }
+  }
   TileConfig cfg;
+  cfg.lean = lean ? lean_split : 0;
   cfg.cta_group = best_g;
   cfg.tile_n = best_n;
   cfg.pairs = best_p;
@@ -409,6 +468,7 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
   if (o.grid_limit && o.grid_limit / (best_g * best_p) < workers) workers = o.grid_limit / (best_g * best_p);
   if (workers < 1) workers = 1;
   const int64_t tiles = (int64_t)cfg.tiles_m * cfg.tiles_n * c.batch;
+  if (lean) workers = tiles < 1 ? 1 : tiles;   // a cluster per tile, all at once
   // Two staging buffers per epilogue warp let a warp fill one while the TMA store still
   // reads the other; they cost 32 KB of ring.  Short K: the epilogue bounds a tile, so staging
   // depth matters more than ring depth.  Otherwise the ring takes the space: the time between a
@@ -426,6 +486,17 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
   if (o.stages && o.stages < cfg.stages) cfg.stages = o.stages < 2 ? 2 : o.stages;
   cfg.stages_direct = (o.epi_bufs || o.reduce_add) ? 0 : max_stages(best_g, best_n, cfg.ksub, 0, best_r);
   if (o.stages && o.stages < cfg.stages_direct) cfg.stages_direct = o.stages < 2 ? 2 : o.stages;
+  if (lean) {  // a ring no deeper than a CTA's K loop: with every k-block resident no stage is ever waited for
+    const int64_t nkb_all = (k16 + kBlockK * cfg.ksub - 1) / (kBlockK * cfg.ksub);
+    const int64_t nkb = (nkb_all + lean_split - 1) / lean_split;
+    cfg.stages = lean_max_stages(best_n, cfg.ksub, c.c_bytes, lean_split);
+    if (nkb < cfg.stages) cfg.stages = nkb < 1 ? 1 : (int)nkb;
+    if (o.stages && o.stages < cfg.stages) cfg.stages = o.stages;
+    // (a cluster's CTAs stage their partial sums, 4 quadrants x 128 bytes x tile_n, in the ring once their MMAs are done)
+    while (lean_split > 1 && cfg.stages * stage_bytes(1, best_n, cfg.ksub) < 16 * best_n * 32) ++cfg.stages;
+    cfg.stages_direct = 0;
+    cfg.epi_bufs = 1;
+  }
   // Wave quantisation: the k-blocks of the tiles that do not fill a whole wave are shared out evenly among
   // the workers, so that the last wave takes tail / tail_workers of a tile's time (split-K applied to the
   // tail only; for a problem smaller than one wave that is split-K with slices of equal length).

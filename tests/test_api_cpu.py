@@ -339,7 +339,7 @@ def test_shared_operand_cluster_flags_and_preview():
         assert B.exo_gemm_validate(good(flags2=f2, flags=B.flag_tile_n(128))) == B.ERR_INVALID_ARG
         assert B.exo_gemm_validate(good(flags2=f2, flags=B.flag_grid_limit(6))) == B.ERR_INVALID_ARG
         assert B.exo_gemm_validate(good(flags2=f2, flags=B.flag_grid_limit(8) | B.flag_tile_n(256))) == B.OK
-    assert B.exo_gemm_validate(good(flags2=16)) == B.ERR_INVALID_ARG
+    assert B.exo_gemm_validate(good(flags2=64)) == B.ERR_INVALID_ARG
     have = B.exo_gemm_has_shared_operand_clusters()
     assert have in (0, 1)
     st, info = B.exo_gemm_plan_preview(good(M=8192, N=8192, K=8192, flags2=ALWAYS), 148)
@@ -405,6 +405,56 @@ def test_tall_tile_flags_and_preview():
     assert (info.tail_tiles, info.split_k, info.workspace_bytes) == (1, 2, 1 * 512 * 256 * 4)   # slices of 1024 k
     st, info = B.exo_gemm_plan_preview(good(M=2560, N=3840, K=2048, flags2=TALL, flags=B.flag_split_k(8)), 148)
     assert (info.tail_tiles, info.split_k, info.workspace_bytes) == (1, 8, 7 * 512 * 256 * 4)   # on request: 256 k
+
+
+def test_lean_kernel_flags_and_preview():
+    LEAN, NEVER = B.FLAG2_LEAN_ALWAYS, B.FLAG2_LEAN_NEVER
+    assert (LEAN, NEVER) == (32, 16)
+    assert B.exo_gemm_validate(good(flags2=LEAN)) == B.OK and B.exo_gemm_validate(good(flags2=NEVER)) == B.OK
+    assert B.exo_gemm_validate(good(flags2=48)) == B.ERR_INVALID_ARG                       # lean field 3
+    assert B.exo_gemm_validate(good(flags2=64)) == B.ERR_INVALID_ARG                       # bits 6.. are reserved
+    for f, f2 in [(B.flag_cta_group(2), LEAN), (B.flag_tile_n(256), LEAN), (B.flag_split_k(3), LEAN), (B.flag_split_k(8), LEAN),
+                  (B.flag_grid_limit(8), LEAN), (1 << 11, LEAN), (0, LEAN | B.flag2_cta_rows(256)),
+                  (0, LEAN | B.FLAG2_SHARE_ALWAYS)]:
+        assert B.exo_gemm_validate(good(flags=f, flags2=f2)) == B.ERR_INVALID_ARG, (f, f2)
+    assert B.exo_gemm_validate(good(flags=B.flag_split_k(1) | B.flag_tile_n(128), flags2=LEAN | B.FLAG2_SHARE_NEVER)) == B.OK
+    # 128 x 64 tiles while a CTA per tile fits the SMs, else 128 x 128; a ring no deeper than the K loop
+    st, info = B.exo_gemm_plan_preview(good(M=256, N=256, K=256, flags2=LEAN), 148)
+    i = info.as_dict()
+    assert st == B.OK and (i["lean_kernel"], i["cta_group"], i["tile_m"], i["tile_n"], i["tile_k"]) == (1, 1, 128, 64, 128)
+    assert (i["tiles_m"], i["tiles_n"], i["grid"], i["stages"], i["tmem_columns"], i["split_k"]) == (2, 4, 8, 2, 128, 1)
+    # fp32 C: two 4 KB staging buffers per TMEM lane quadrant; a stage holds 128 rows of A and 64 of B, 128 k each
+    assert i["smem_bytes"] == 2 * 49152 + 8 * 4096 + 512 + 1024
+    st, info = B.exo_gemm_plan_preview(good(M=1024, N=1024, K=4096, c_dtype=B.BF16, flags2=LEAN), 148)
+    i = info.as_dict()
+    assert (i["lean_kernel"], i["tile_n"], i["grid"], i["stages"]) == (1, 64, 128, 4) and i["smem_bytes"] <= 232448
+    st, info = B.exo_gemm_plan_preview(good(M=1024, N=2048, K=512, flags2=LEAN), 148)
+    assert (info.lean_kernel, info.tile_n, info.grid, info.stages) == (1, 128, 128, 2)      # 64 KB of staging for an fp32 C
+    st, info = B.exo_gemm_plan_preview(good(M=1024, N=2048, K=512, flags2=LEAN, flags=B.flag_tile_n(64)), 148)
+    assert (info.lean_kernel, info.tile_n, info.grid) == (1, 64, 256)                      # more CTAs than SMs: they queue
+    st, info = B.exo_gemm_plan_preview(good(M=1024, N=2048, K=512, flags2=NEVER), 148)
+    assert info.lean_kernel == 0
+    # the library's own choice: one wave of 128 x 64 tiles up to K = 2048, a cluster per tile from K ~ 1000 on where
+    # the SMs have room for it, 128 x 128 tiles at K = 512 only; never when the caller names a persistent-kernel parameter
+    for (M, N, K), want in {(256, 256, 256): (1, 64, 1, 8), (512, 512, 512): (1, 64, 1, 32), (512, 512, 2048): (1, 64, 4, 128),
+                            (512, 1000, 3072): (1, 64, 2, 128), (1000, 1000, 1000): (1, 64, 1, 128), (512, 1000, 6144): (0,),
+                            (1000, 1000, 3072): (0,), (512, 3072, 512): (1, 128, 1, 96), (512, 3072, 1000): (0,),
+                            (2048, 2048, 512): (0,), (4096, 4096, 4096): (0,)}.items():
+        st, info = B.exo_gemm_plan_preview(good(M=M, N=N, K=K), 148)
+        got = (info.lean_kernel, info.tile_n, info.split_k, info.grid) if info.lean_kernel else (0,)
+        assert st == B.OK and got == want, (M, N, K, got)
+    st, info = B.exo_gemm_plan_preview(good(M=512, N=512, K=2048, flags=B.flag_split_k(1)), 148)
+    assert (info.lean_kernel, info.split_k, info.grid) == (1, 1, 32)                    # "never cut K" is kept
+    for f in (B.flag_tile_n(64), B.flag_cta_group(1), B.flag_max_stages(3), B.flag_epi_buffers(1), B.flag_band(2), B.flag_split_k(4)):
+        st, info = B.exo_gemm_plan_preview(good(M=512, N=512, K=512, flags=f), 148)
+        assert info.lean_kernel == 0, f
+    # K cut over a cluster of 2 or 4 CTAs per tile; the partial sums travel through shared memory, not a workspace
+    st, info = B.exo_gemm_plan_preview(good(M=512, N=512, K=1000, flags2=LEAN, flags=B.flag_split_k(4)), 148)
+    i = info.as_dict()
+    assert (i["lean_kernel"], i["split_k"], i["cluster_size"], i["grid"], i["stages"], i["workspace_bytes"]) == (1, 4, 4, 128, 2, 0)
+    assert i["smem_bytes"] == 2 * 49152 + 8 * 4096 + 3 * 2 * 4096 + 512 + 1024         # + three peers' 32 x 64 fp32 parts
+    st, info = B.exo_gemm_plan_preview(good(M=512, N=512, K=128, flags2=LEAN, flags=B.flag_split_k(4)), 148)
+    assert (info.split_k, info.cluster_size, info.grid) == (1, 1, 32)                   # one k-block: nothing to cut
 
 
 def test_smoke_cases_are_in_the_supported_set():

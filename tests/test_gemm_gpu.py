@@ -186,23 +186,27 @@ def test_persistent_loop_many_tiles_on_few_ctas():
 def test_plans_of_one_kernel_with_different_shared_memory_sizes_live_side_by_side():
     """One kernel instantiation serves plans whose ring and staging depths differ (run-time
     parameters), hence different dynamic shared-memory sizes; creating the smaller one must not
-    make launches of the larger one fail.  Two pairs of plans, run in alternation."""
+    make launches of the larger one fail.  Three pairs of plans (two of the persistent kernel, one of the
+    one-tile-per-CTA kernel), each run in alternation."""
     import torch
     dev = torch.device("cuda:0")
     stream = torch.cuda.current_stream(dev).cuda_stream
+    PERS, LEAN = B.FLAG2_LEAN_NEVER, B.FLAG2_LEAN_ALWAYS
     pairs = [
         (synth.Problem("k4096", 4096, 384, 4096, BF16, FP32, 0, 1, 0, 1.0, 0.0, seed=41), 0,
-         synth.Problem("k512", 4096, 384, 512, BF16, FP32, 0, 1, 0, 1.0, 0.0, seed=42), 0),
+         synth.Problem("k512", 4096, 384, 512, BF16, FP32, 0, 1, 0, 1.0, 0.0, seed=42), 0, PERS),
         (synth.Problem("epi1", 520, 392, 328, FP16, FP32, 0, 0, 0, 1.0, 0.0, seed=43, dist="normal"), flags_for(2, 128, epi=1),
-         synth.Problem("epi2", 520, 392, 328, FP16, FP32, 0, 0, 0, 1.0, 0.0, seed=44, dist="normal"), flags_for(2, 128, epi=2)),
+         synth.Problem("epi2", 520, 392, 328, FP16, FP32, 0, 0, 0, 1.0, 0.0, seed=44, dist="normal"), flags_for(2, 128, epi=2), PERS),
+        (synth.Problem("lean512", 520, 392, 512, BF16, FP32, 0, 1, 0, 1.0, 0.0, seed=45), 0,
+         synth.Problem("lean128", 520, 392, 128, BF16, FP32, 0, 1, 0, 1.0, 0.0, seed=46), 0, LEAN),
     ]
-    for pa, fa, pb, fb in pairs:
+    for pa, fa, pb, fb, f2 in pairs:
         pa.generate(); pb.generate()
-        da = harness.DeviceProblem(pa, fa)
-        db = harness.DeviceProblem(pb, fb)           # created second: must not shrink what da may request
+        da = harness.DeviceProblem(pa, fa, flags2=f2)
+        db = harness.DeviceProblem(pb, fb, flags2=f2)           # created second: must not shrink what da may request
         try:
             ia, ib = da.plan.info(), db.plan.info()
-            assert (ia["cta_group"], ia["tile_n"], ia["tile_k"]) == (ib["cta_group"], ib["tile_n"], ib["tile_k"])
+            assert (ia["cta_group"], ia["tile_n"], ia["tile_k"], ia["lean_kernel"]) == (ib["cta_group"], ib["tile_n"], ib["tile_k"], ib["lean_kernel"])
             assert ia["smem_bytes"] != ib["smem_bytes"], (ia, ib)
             refs = {}
             for q in (pa, pb):
@@ -217,7 +221,7 @@ def test_plans_of_one_kernel_with_different_shared_memory_sizes_live_side_by_sid
                     got = oracle.logical_view(dp.result_buffer(), q.M, q.N, q.c_layout, q.ldc, q.c_dtype)
                     assert oracle.max_error(got, *refs[q.name]) <= TOL, (q.name, rep)
             # the plan-less entry point in between must not disturb them either
-            st, _ = B.exo_gemm_run_static(harness.desc_of(pb, fb), db.dA.data_ptr(), db.dB.data_ptr(), db.dC.data_ptr(),
+            st, _ = B.exo_gemm_run_static(harness.desc_of(pb, fb, flags2=f2), db.dA.data_ptr(), db.dB.data_ptr(), db.dC.data_ptr(),
                                           pb.alpha, pb.beta, stream)
             assert st == B.OK
             da.reset_c()
@@ -832,13 +836,13 @@ SWEEP_LARGE = [(12288, 12288, 12288), (12288, 12288, 512), (12288, 1000, 12288),
 
 def plan_signature(info):
     """What distinguishes the code paths a plan takes: tile shape, pipeline and staging depth, K-slices
-    of the tail, whether a tail exists, whether whole waves precede it, raster direction."""
+    of the tail, whether a tail exists, whether whole waves precede it, raster direction, which of the two kernels."""
     g = info["cta_group"]
     workers = max(1, info["grid"] // info["cluster_size"])
     tiles = info["tiles_m"] * info["tiles_n"]
     return (g, info["tile_m"], info["tile_n"], info["tile_k"], info["stages"], info["epilogue_buffers"],
             info["split_k"], info["tail_tiles"] > 0, tiles >= workers and info["tail_tiles"] < tiles, info["raster_along_m"],
-            info["cluster_size"])
+            info["cluster_size"], info["lean_kernel"])
 
 
 def sweep_plan_classes(sm_count=148):

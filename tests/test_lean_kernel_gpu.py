@@ -1,0 +1,202 @@
+"""Parity of the one-tile-per-CTA kernel (128 x 64 or 128 x 128 tiles, every tile's CTA launched at once;
+the kernel for the small matrices the paper's Section 6 discusses) against the CPU oracle, through the C ABI.
+The operation is the same GEMM, so the same tolerance applies:
+
+    max |C - Cref| / (sum_k |a b| + |beta c|) <= 1e-3,
+
+widened by half an ulp of a 16-bit output type as in the main parity file.  The order of summation is fixed
+(two accumulators taken in turn by consecutive MMAs, added at the end; with K cut over a cluster the parts are
+added in rank order), so repeated runs must agree bit for bit.
+"""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2609_16389_b200 import binding as B
+from paper_2609_16389_b200 import harness, synth
+from paper_2609_16389_b200.synth import BF16, FP16, FP32
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-3
+NO_SPLIT = B.flag_split_k(1)
+LEAN = B.FLAG2_LEAN_ALWAYS
+PERSISTENT = B.FLAG2_LEAN_NEVER | B.FLAG2_SHARE_NEVER
+
+
+def run(p, flags, flags2):
+    cbuf, info = harness.gemm_host(p, flags, flags2=flags2)
+    return cbuf, oracle.logical_view(cbuf, p.M, p.N, p.c_layout, p.ldc, p.c_dtype), info
+
+
+def assert_parity(p, got, info):
+    cref, den = oracle.gemm_problem(p)
+    gate = TOL * den + oracle.output_rounding_slack(cref, p.c_dtype)
+    bad = np.abs(got - cref) > gate
+    assert not bad.any(), (p.name, int(bad.sum()), np.argwhere(bad)[:5], info)
+
+
+# M, N, K, ab, cd, la, lb, lc, alpha, beta, tile_n (0 = the library's choice), extra flags
+CASES = [
+    (128, 64, 64, BF16, FP32, 0, 1, 0, 1.0, 0.0, 0, 0),                        # exactly one tile, one k-block
+    (256, 256, 256, BF16, FP32, 0, 1, 0, 1.0, 0.0, 0, 0),                      # config 1: 8 tiles of 128 x 64
+    (512, 512, 512, BF16, FP32, 0, 1, 0, 1.0, 0.0, 0, 0),
+    (512, 512, 512, BF16, BF16, 0, 1, 0, 1.0, 0.0, 128, 0),                    # 128 x 128 tiles, 16-bit C (two chunks)
+    (512, 512, 1000, BF16, FP32, 0, 1, 0, 1.0, 0.0, 128, 0),                   # fp32 C, two chunks per warp; ragged K
+    (700, 300, 200, BF16, FP32, 0, 1, 0, 1.0, 0.0, 0, 0),                      # ragged M, N and K
+    (1, 8, 8, BF16, FP32, 0, 1, 0, 2.0, 0.0, 0, 0),
+    (130, 72, 4096, FP16, FP16, 0, 1, 0, 1.0, 0.0, 0, 0),                      # long K: the ring is reused 7 times
+    (384, 520, 2048, BF16, BF16, 0, 1, 0, 1.5, -0.75, 128, B.flag_max_stages(2)),  # 16-bit output, beta, a ring of 2
+    (1000, 520, 264, BF16, FP32, 1, 0, 0, 1.0, 0.5, 0, 0),                     # A with M contiguous, B with N contiguous
+    (1000, 520, 264, BF16, FP32, 1, 0, 0, 1.0, 0.5, 128, B.flag_k_subblocks(1)),
+    (640, 900, 320, FP16, FP32, 0, 1, 1, -1.0, 1.0, 0, 0),                     # column-major C (operands swap)
+    (640, 384, 520, FP32, FP32, 0, 1, 0, 1.0, 0.0, 0, 0),                      # tf32 operands
+    (520, 392, 264, FP32, FP32, 1, 0, 0, 1.25, -0.5, 128, 0),                  # tf32, M/N-contiguous operands
+    (2048, 2048, 512, BF16, FP32, 0, 1, 0, 1.0, 0.0, 128, 0),                  # 256 CTAs: more than the SMs hold at once
+    (1024, 1024, 0, BF16, FP32, 0, 1, 0, 1.0, 0.5, 0, 0),                      # K = 0: C = beta * C
+    (256, 512, 512, BF16, BF16, 0, 1, 0, 0.0, 2.0, 0, 0),                      # alpha = 0: operands never read
+]
+
+# the same through clusters of 2 or 4 CTAs that share a tile's K loop: M, N, K, ab, cd, la, lb, lc, alpha, beta, tile_n, split, extra
+SPLIT_CASES = [
+    (512, 512, 512, BF16, FP32, 0, 1, 0, 1.0, 0.0, 0, 4, 0),                   # one 128-k block per CTA
+    (512, 512, 1000, BF16, FP32, 0, 1, 0, 1.0, 0.0, 0, 4, 0),                  # two each, the last one ragged
+    (512, 512, 1000, BF16, BF16, 0, 1, 0, 1.0, 0.0, 128, 2, 0),
+    (256, 256, 256, BF16, FP32, 0, 1, 0, 1.0, 0.0, 0, 2, 0),
+    (256, 256, 256, BF16, FP32, 0, 1, 0, 1.0, 0.0, 0, 4, B.flag_k_subblocks(1)),   # four 64-k blocks, one per CTA
+    (700, 300, 200, BF16, FP32, 0, 1, 0, 1.0, 0.5, 0, 4, 0),                   # ragged everywhere; two k-blocks for four CTAs -> 2
+    (130, 72, 4096, FP16, FP16, 0, 1, 0, 1.0, 0.0, 0, 4, B.flag_max_stages(2)), # 8 k-blocks per CTA through a ring of 2
+    (1, 8, 8, BF16, FP32, 0, 1, 0, 2.0, 0.0, 0, 4, 0),                         # one k-block: no cluster
+    (384, 520, 2048, BF16, BF16, 0, 1, 0, 1.5, -0.75, 128, 4, 0),
+    (1000, 520, 264, BF16, FP32, 1, 0, 0, 1.0, 0.5, 128, 2, 0),                # M/N-contiguous operands
+    (640, 900, 320, FP16, FP32, 0, 1, 1, -1.0, 1.0, 0, 2, 0),                  # column-major C
+    (640, 384, 520, FP32, FP32, 0, 1, 0, 1.0, 0.0, 0, 4, 0),                   # tf32
+    (520, 392, 264, FP32, FP32, 1, 0, 0, 1.25, -0.5, 128, 4, 0),
+    (1024, 1024, 1024, BF16, FP32, 0, 1, 0, 1.0, 0.0, 128, 4, 0),              # 64 clusters of 4: more than fit at once
+]
+
+
+@pytest.mark.parametrize("case", CASES, ids=lambda c: "x".join(str(v) for v in c[:3]) + f"_{c[3]}{c[4]}{c[5]}{c[6]}{c[7]}_n{c[10]}")
+def test_lean_kernel_matches_the_oracle(case):
+    M, N, K, ab, cd, la, lb, lc, alpha, beta, bn, extra = case
+    p = synth.Problem("lean", M, N, K, ab, cd, la, lb, lc, alpha, beta, seed=M + 3 * N + K,
+                      dist="normal" if ab == FP16 else "uniform").generate()
+    tile = B.flag_tile_n(bn) if bn else 0
+    bits, got, info = run(p, NO_SPLIT | extra | tile, LEAN)
+    assert info["lean_kernel"] == 1 and info["cta_group"] == 1 and info["tile_m"] == 128 and info["cluster_size"] == 1
+    assert info["tile_n"] in (64, 128) and (not bn or info["tile_n"] == bn)
+    assert info["grid"] == info["tiles_m"] * info["tiles_n"] and info["split_k"] == 1
+    assert info["tmem_columns"] == 2 * info["tile_n"] and info["smem_bytes"] <= 232448
+    assert_parity(p, got, info)
+    again, _, _ = run(p, NO_SPLIT | extra | tile, LEAN)
+    assert np.array_equal(again.view(np.uint8), bits.view(np.uint8))
+    # the persistent kernel on the same tile shape meets the same oracle (its summation order differs: one
+    # accumulator there, two taken in turn here)
+    _, got_r, info_r = run(p, NO_SPLIT | extra | B.flag_cta_group(1) | B.flag_tile_n(info["tile_n"]), PERSISTENT)
+    assert info_r["lean_kernel"] == 0 and info_r["tile_n"] == info["tile_n"] and info_r["tile_k"] == info["tile_k"]
+    assert_parity(p, got_r, info_r)
+
+
+@pytest.mark.parametrize("case", SPLIT_CASES, ids=lambda c: "x".join(str(v) for v in c[:3]) + f"_{c[3]}{c[4]}{c[5]}{c[6]}{c[7]}_n{c[10]}_s{c[11]}")
+def test_lean_kernel_with_k_cut_over_a_cluster(case):
+    """The CTAs of a cluster compute consecutive K ranges of one tile and exchange partial sums through
+    distributed shared memory; each finishes a quarter (or half) of the tile's rows, adding the others'
+    parts in rank order: the oracle's result within the tolerance, and the same bits in every run."""
+    M, N, K, ab, cd, la, lb, lc, alpha, beta, bn, split, extra = case
+    p = synth.Problem("lean_split", M, N, K, ab, cd, la, lb, lc, alpha, beta, seed=M + 3 * N + K + split,
+                      dist="normal" if ab == FP16 else "uniform").generate()
+    tile = B.flag_tile_n(bn) if bn else 0
+    bits, got, info = run(p, B.flag_split_k(split) | extra | tile, LEAN)
+    k_blocks = -(-K * (2 if ab == FP32 else 1) // (2 * info["tile_k"] if ab == FP32 else info["tile_k"]))
+    want_split = split
+    while want_split > max(k_blocks, 1):
+        want_split //= 2
+    assert info["lean_kernel"] == 1 and info["split_k"] == want_split == info["cluster_size"], info
+    assert info["grid"] == info["tiles_m"] * info["tiles_n"] * want_split and info["smem_bytes"] <= 232448
+    assert info["workspace_bytes"] == 0
+    assert_parity(p, got, info)
+    for _ in range(2):
+        again, _, _ = run(p, B.flag_split_k(split) | extra | tile, LEAN)
+        assert np.array_equal(again.view(np.uint8), bits.view(np.uint8))
+
+
+def test_lean_kernel_padding_untouched_and_nan_c_ignored_when_beta_is_zero():
+    p = synth.Problem("lean_pad", 600, 500, 136, BF16, FP32, 0, 1, 0, 1.0, 0.0, seed=4, ldc=512).generate()
+    p.C[:] = np.nan
+    bits, got, info = run(p, NO_SPLIT, LEAN)
+    assert info["lean_kernel"] == 1
+    assert_parity(p, got, info)
+    flat = bits.reshape(-1)
+    for i in (0, 1, 127, 128, 255, 256, 511, 512, 598):      # the gap after each row is as it was
+        assert np.isnan(flat[i * 512 + 500:(i + 1) * 512]).all(), i
+
+
+def test_lean_kernel_bounded_wait_reports_timeout_and_the_plan_stays_usable():
+    """The producer of CTA 0 leaves out the loads of one k-block (a stage that never fills): the MMA
+    issuer's wait runs out after 20 ms, every role leaves, tensor memory is freed, the kernel returns,
+    and the same plan computes correctly afterwards."""
+    import torch
+    p = synth.Problem("lean_tmo", 512, 512, 1024, BF16, FP32, 0, 1, 0, 1.0, 0.0, seed=10).generate()
+    # a k-block of the first two (issued before the set-up barrier), one behind them; then with the K loop cut
+    # over a cluster of 4 (CTA 0 has k-blocks 0 and 1: its peers' partial sums arrive, its own never does)
+    for skip, split in ((1, 1), (6, 1), (1, 4)):
+        dp = harness.DeviceProblem(p, B.flag_split_k(split) | B.flag_max_stages(4), flags2=LEAN)
+        try:
+            assert dp.plan.info()["lean_kernel"] == 1 and dp.plan.info()["stages"] == (4 if split == 1 else 2)
+            assert B.exo_gemm_debug_set(dp.plan.handle, 20, skip) == B.OK
+            dp.run()
+            torch.cuda.synchronize()
+            st, detail = B.exo_gemm_check(dp.plan.handle)
+            assert st == B.ERR_DEVICE_TIMEOUT
+            # the wait that runs out first is CTA 0's own, or (cut K) a peer's wait for CTA 0's partial sums,
+            # which starts within a microsecond of it
+            assert detail[0] == 1 and detail[1] in ((1, 2, 3) if split == 1 else (1, 2, 3, 6)) and detail[5] < split, detail
+            dp.reset_c()
+            dp.run()
+            torch.cuda.synchronize()
+            dp.plan.check()
+            got = oracle.logical_view(dp.result_buffer(), p.M, p.N, 0, p.ldc, FP32)
+            cref, den = oracle.gemm_problem(p)
+            assert oracle.max_error(got, cref, den) <= TOL
+        finally:
+            dp.close()
+
+
+def test_lean_kernels_back_to_back_keep_stream_order():
+    """D = (A B) E as two small GEMMs on one stream with no host sync in between, and the pair replayed from
+    a CUDA graph: the second kernel starts early (its set-up overlaps the first kernel) but reads C only
+    after the first has written it."""
+    import torch
+    M, K, N, N2 = 500, 264, 392, 200
+    p1 = synth.Problem("lchain1", M, N, K, BF16, BF16, 0, 1, 0, 1.0, 0.0, seed=41).generate()
+    p2 = synth.Problem("lchain2", M, N2, N, BF16, FP32, 0, 1, 0, 1.0, 0.0, seed=42).generate()
+    dev = torch.device("cuda:0")
+    dA, dB = harness._to_device(p1.A, dev), harness._to_device(p1.B, dev)
+    dE = harness._to_device(p2.B, dev)
+    with B.Plan(harness.desc_of(p1, NO_SPLIT, 0, LEAN)) as g1, B.Plan(harness.desc_of(p2, NO_SPLIT, 0, LEAN)) as g2:
+        assert g1.info()["lean_kernel"] == 1 and g2.info()["lean_kernel"] == 1
+        dC = torch.full((M * N * 2,), 0xFF, dtype=torch.uint8, device=dev)
+        dD = torch.zeros(M * N2 * 4, dtype=torch.uint8, device=dev)
+        side = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            g1.run(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), 1.0, 0.0, side.cuda_stream)
+            g2.run(dC.data_ptr(), dE.data_ptr(), dD.data_ptr(), 1.0, 0.0, side.cuda_stream)
+        ref = None
+        stream = torch.cuda.current_stream(dev).cuda_stream
+        for rep in range(6):
+            dC.fill_(0xFF)                                  # NaN patterns until GEMM 1 writes
+            dD.zero_()
+            if rep % 2:
+                graph.replay()
+            else:
+                g1.run(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), 1.0, 0.0, stream)
+                g2.run(dC.data_ptr(), dE.data_ptr(), dD.data_ptr(), 1.0, 0.0, stream)
+            torch.cuda.synchronize(dev)
+            g1.check(); g2.check()
+            c_host = dC.cpu().numpy().view(np.uint16)
+            d_host = dD.cpu().numpy().view(np.float32)
+            p2.A = c_host.copy()                            # the oracle for GEMM 2 takes GEMM 1's actual output
+            cref, den = oracle.gemm_problem(p2)
+            assert oracle.max_error(d_host.reshape(M, N2).astype(np.float64), cref, den) <= TOL, rep
+            ref = d_host.copy() if ref is None else ref
+            assert np.array_equal(d_host, ref), rep
