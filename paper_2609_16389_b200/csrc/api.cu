@@ -278,7 +278,7 @@ void fill_info(const exo_gemm_plan* p, exo_gemm_info_t* info) {
   info->stages_direct = p->cfg.stages_direct;
   info->tail_workers = p->cfg.tail_workers;
   info->smem_bytes = p->smem_bytes;
-  info->tmem_columns = 2 * p->cfg.tile_n;
+  info->tmem_columns = p->cfg.lean ? p->cfg.tile_n : 2 * p->cfg.tile_n;
   info->lean_kernel = p->cfg.lean ? 1 : 0;
   info->tiles_m = p->cfg.tiles_m;
   info->tiles_n = p->cfg.tiles_n;

@@ -57,9 +57,9 @@ exo_gemm_lean_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
   constexpr int UPC = CW / 32;                       // 32-column TMEM loads per chunk
   constexpr int STAGE_BYTES = stage_bytes(1, BN, KSUB);
   constexpr int A_BYTES = KSUB * kATileBytes;
-  // Two accumulators, taken in turn by consecutive MMAs and added in the epilogue: MMAs into one accumulator
-  // depend on each other, and at N <= 128 one is shorter than the tensor core's accumulate latency.
-  constexpr uint32_t TMEM_COLS = 2 * BN;
+  // (One accumulator.  Two, taken in turn by consecutive MMAs and added in the epilogue, were measured: the
+  // k-block period stayed at 930 clocks, so the MMAs into one accumulator do not wait for one another.)
+  constexpr uint32_t TMEM_COLS = BN;
   constexpr int UNITS = BN / 32;                     // 4 KB units (32 rows x 32 fp32 columns) of a quadrant's partial sums
   const int32_t STAGE_K = (int32_t)p.sub_k * KSUB;
   const int32_t STAGES = p.stages;
@@ -216,12 +216,12 @@ exo_gemm_lean_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         if (k_left >= STAGE_K && !tf32) {
 #pragma unroll
           for (int32_t k = 0; k < kMmaPerStage; ++k)
-            ptx::umma_f16<1>(tmem_base + (uint32_t)(k & 1) * BN, a_desc + k_off(k, a_step, a_sub), b_desc + k_off(k, b_step, b_sub), idesc,
-                             (j != 0 || k >= 2) ? 1u : 0u);
+            ptx::umma_f16<1>(tmem_base, a_desc + k_off(k, a_step, a_sub), b_desc + k_off(k, b_step, b_sub), idesc,
+                             (j != 0 || k != 0) ? 1u : 0u);
         } else {  // tf32, or a ragged last k-block, which skips the MMAs that would only read zero fill
           const int32_t n_mma = k_left >= STAGE_K ? kMmaPerStage : (k_left + umma_k - 1) / umma_k;
           for (int32_t k = 0; k < n_mma; ++k) {
-            const uint32_t accumulate = (j != 0 || k >= 2) ? 1u : 0u, d = tmem_base + (uint32_t)(k & 1) * BN;
+            const uint32_t accumulate = (j != 0 || k != 0) ? 1u : 0u, d = tmem_base;
             if (tf32) ptx::umma_tf32<1>(d, a_desc + k_off(k, a_step, a_sub), b_desc + k_off(k, b_step, b_sub), idesc, accumulate);
             else ptx::umma_f16<1>(d, a_desc + k_off(k, a_step, a_sub), b_desc + k_off(k, b_step, b_sub), idesc, accumulate);
           }
@@ -283,22 +283,6 @@ exo_gemm_lean_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         for (int q = 0; q < UPC; ++q)
           if (i < mine || S > 1) ptx::tmem_ld_32x32(tacc + (uint32_t)((first_chunk + i) * CW + q * 32), v[i][q]);
       ptx::tmem_ld_wait();
-      // ... plus the second accumulator, if this CTA's K range had a second MMA to write it
-      int32_t k_mine = p.K - kb_begin * STAGE_K;
-      if (k_mine > nkb * STAGE_K) k_mine = nkb * STAGE_K;
-      if (k_mine > (int32_t)p.umma_k) {
-#pragma unroll
-        for (int i = 0; i < CPW; ++i)
-#pragma unroll
-          for (int q = 0; q < UPC; ++q)
-            if (i < mine || S > 1) {
-              uint32_t w[32];
-              ptx::tmem_ld_32x32(tacc + (uint32_t)(BN + (first_chunk + i) * CW + q * 32), w);
-              ptx::tmem_ld_wait();
-#pragma unroll
-              for (int k = 0; k < 32; ++k) v[i][q][k] = __float_as_uint(__uint_as_float(v[i][q][k]) + __uint_as_float(w[k]));
-            }
-      }
     } else {
 #pragma unroll
       for (int i = 0; i < CPW; ++i)

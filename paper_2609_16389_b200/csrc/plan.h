@@ -531,6 +531,17 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
     }
     cfg.workspace_bytes = 0;  // filled in by split_workspace_bytes() once the output type is known
   }
+  // One whole tile per worker and nothing after it: the drain is exposed, and with a single staging buffer a
+  // warp waits about 1000 clocks per chunk for the previous store to have read it.  fp32 C, 5 stages + 2 buffers
+  // against 6 + 1: 2048^3 -3.1 %, 2048 x 2048 x 3072 -2.7 %, 1000 x 3072 x 3072 -3.3 %, 2048 x 2048 x 6144 -0.8 % (time);
+  // with a 16-bit C -1 %, not taken.
+  // (256-column tiles, where it was measured: a ring of 32 KB stages goes from 6 to 5; narrower tiles would go from 4 to 3)
+  if (!lean && !o.epi_bufs && c.c_bytes == 4 && best_r == 1 && best_n == 256 && cfg.full_tiles == 0 && cfg.tail_workers == 0 && cfg.epi_bufs == 1 &&
+      max_stages(best_g, best_n, cfg.ksub, 2, best_r) >= 3) {
+    cfg.epi_bufs = 2;
+    cfg.stages = max_stages(best_g, best_n, cfg.ksub, 2, best_r);
+    if (o.stages && o.stages < cfg.stages) cfg.stages = o.stages < 2 ? 2 : o.stages;
+  }
   if (tiles < workers) {  // less than one wave: launch only the CTA groups that get a work item
     workers = cfg.tail_workers > 0 ? cfg.tail_workers : tiles;
     if (workers < 1) workers = 1;

@@ -422,7 +422,7 @@ def test_lean_kernel_flags_and_preview():
     st, info = B.exo_gemm_plan_preview(good(M=256, N=256, K=256, flags2=LEAN), 148)
     i = info.as_dict()
     assert st == B.OK and (i["lean_kernel"], i["cta_group"], i["tile_m"], i["tile_n"], i["tile_k"]) == (1, 1, 128, 64, 128)
-    assert (i["tiles_m"], i["tiles_n"], i["grid"], i["stages"], i["tmem_columns"], i["split_k"]) == (2, 4, 8, 2, 128, 1)
+    assert (i["tiles_m"], i["tiles_n"], i["grid"], i["stages"], i["tmem_columns"], i["split_k"]) == (2, 4, 8, 2, 64, 1)
     # fp32 C: two 4 KB staging buffers per TMEM lane quadrant; a stage holds 128 rows of A and 64 of B, 128 k each
     assert i["smem_bytes"] == 2 * 49152 + 8 * 4096 + 512 + 1024
     st, info = B.exo_gemm_plan_preview(good(M=1024, N=1024, K=4096, c_dtype=B.BF16, flags2=LEAN), 148)
