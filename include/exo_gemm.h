@@ -129,11 +129,17 @@ typedef enum { EXO_GEMM_ROW_MAJOR = 0, EXO_GEMM_COL_MAJOR = 1 } exo_gemm_layout_
  * bits of each fp32 operand and ignores the rest; products are accumulated in fp32):
  * this is the precision of the paper's own Section 6 kernels and of
  * CUBLAS_TF32_TENSOR_OP_MATH (M/N-contiguous FP32 operands are staged with the 128-byte
- * swizzle in 32-byte atoms that tcgen05 wants for transposed 32-bit operands).  Because operands and
- * results move by TMA, every leading dimension times its element size must be a
- * multiple of 16 bytes (16-bit: ld % 8 == 0, fp32: ld % 4 == 0) and every base
- * pointer passed to exo_gemm_run must be 16-byte aligned.  Legal BLAS calls
- * outside this set return EXO_GEMM_ERR_UNSUPPORTED.
+ * swizzle in 32-byte atoms that tcgen05 wants for transposed 32-bit operands).  Operands and
+ * results move by TMA, which addresses rows by a byte stride that is a multiple of 16: a
+ * matrix whose leading dimension times its element size is such a multiple (16-bit:
+ * ld % 8 == 0, fp32: ld % 4 == 0) is used in place and its base pointer passed to
+ * exo_gemm_run must be 16-byte aligned.  Any other leading dimension is legal too: the plan
+ * then owns an aligned copy of that matrix and every run makes one extra pass over it
+ * (operands copied in before the GEMM, C copied out after it and, if beta != 0, in before
+ * it; the base pointer only needs the alignment of its element type; see
+ * exo_gemm_info_t.repacked).  That path has no strided-batch form and is not available to
+ * the allocation-free entry point (ERR_UNSUPPORTED from both).  Legal BLAS calls outside
+ * this set return EXO_GEMM_ERR_UNSUPPORTED.
  */
 typedef struct {
   int64_t M, N, K;
@@ -175,6 +181,9 @@ typedef struct {
                               0 if the plan always stages (EXO_GEMM_FLAG_EPI_BUFFERS given)        */
   int32_t lean_kernel;     /* 1: the one-tile-per-CTA kernel runs this plan (EXO_GEMM_FLAG2_LEAN_*): grid =
                               tiles_m * tiles_n CTAs at once, one accumulator, `stages` = its ring         */
+  int32_t repacked;        /* bit 0 = A, 1 = B, 2 = C: the matrix's leading dimension times its element size is not a
+                              multiple of 16 bytes, so every run copies it through an aligned buffer the plan owns
+                              (counted in workspace_bytes)                                                    */
 } exo_gemm_info_t;
 
 /*
@@ -223,7 +232,8 @@ exo_gemm_status_t exo_gemm_create_batched(exo_gemm_handle_t* out, const exo_gemm
  * persistent, warp-specialised kernel (the kernel class of the paper's Section 4.2
  * code generation: persistent task loop, one code path per named warp group).
  *
- *   A, B, C   DEVICE pointers, 16-byte aligned, laid out as the descriptor says.
+ *   A, B, C   DEVICE pointers, 16-byte aligned (element-aligned for a matrix the plan
+ *             repacks, see the descriptor), laid out as the descriptor says.
  *             The caller owns them and keeps them alive until the stream has
  *             passed the kernel.  C is updated in place; A and B must not
  *             overlap C.  The library never allocates, frees or copies them.
@@ -238,9 +248,10 @@ exo_gemm_status_t exo_gemm_create_batched(exo_gemm_handle_t* out, const exo_gemm
  *
  * All checks happen before the launch; on any error nothing is enqueued.  A
  * handle may be used from several host threads (tensor maps are built on the
- * caller's stack), but runs of ONE plan whose exo_gemm_info_t.split_k > 1 must not
- * overlap on the GPU (enqueue them on one stream, or order the streams): they
- * share the plan's partial-sum workspace and arrival counters.  Nothing in a launch's parameters depends
+ * caller's stack), but runs of ONE plan whose exo_gemm_info_t.split_k > 1 or
+ * .repacked != 0 must not overlap on the GPU (enqueue them on one stream, or order the
+ * streams): they share the plan's partial-sum workspace and arrival counters, or its
+ * aligned copies.  Nothing in a launch's parameters depends
  * on how often the plan has run (the counters of a K-slicing plan keep their own run count on the device),
  * so exo_gemm_run may be captured into a CUDA graph and the graph replayed.  Device-side waits are bounded: if one gives up, the kernel
  * records where in the plan's status block and exits cleanly; a later

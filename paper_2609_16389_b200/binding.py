@@ -52,7 +52,7 @@ class Info(ctypes.Structure):
         "cta_group", "tile_m", "tile_n", "tile_k", "stages", "grid", "smem_bytes", "tmem_columns",
         "tiles_m", "tiles_n", "raster_along_m", "raster_band", "swapped", "sm_count",
         "kernel_launches_per_run", "epilogue_buffers", "split_k", "tail_tiles", "workspace_bytes",
-        "batch_count", "cluster_size", "tail_workers", "stages_direct", "lean_kernel")]
+        "batch_count", "cluster_size", "tail_workers", "stages_direct", "lean_kernel", "repacked")]
 
     def as_dict(self):
         return {n: getattr(self, n) for n, _ in self._fields_}

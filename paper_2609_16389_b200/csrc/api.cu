@@ -11,6 +11,7 @@
 #include "../../include/exo_gemm.h"
 #include "gemm_kernel.cuh"
 #include "lean_kernel.cuh"
+#include "repack.cuh"
 #include "plan.h"
 #ifdef EXO_GEMM_SHARE_PAIRS
 #include "cluster4/share_pairs.cuh"
@@ -176,7 +177,10 @@ static CUresult encode_3d(CUtensorMap* map, int dtype, const void* base, uint64_
 }  // namespace exo
 
 struct exo_gemm_plan {
-  exo_gemm_desc_t desc;
+  exo_gemm_desc_t desc;                // as planned and launched: leading dimensions of repacked matrices rounded up
+  exo_gemm_desc_t user_desc;           // as the caller gave it
+  int repack;                          // 1 = A, 2 = B, 4 = C go through an aligned copy (rows not on 16-byte boundaries)
+  void* d_pack[3];                     // the copies (NULL where not needed)
   exo::Canonical canon;
   exo::TileConfig cfg;
   exo::KernelFn kernel;
@@ -266,6 +270,30 @@ cudaError_t cluster_capacity(int sms, int c_dtype, const FlagOverrides& ov, int*
   return e;
 }
 
+// The descriptor with the leading dimension of every matrix in `mask` (1 = A, 2 = B, 4 = C) replaced by its
+// contiguous extent rounded up to 64 elements: what the plan's aligned copy of that matrix looks like.
+exo_gemm_desc_t aligned_desc(const exo_gemm_desc_t& d, int mask) {
+  exo_gemm_desc_t e = d;
+  int64_t outer, inner;
+  if (mask & 1) { storage_shape(d.a_layout, d.M, d.K, &outer, &inner); e.lda = (inner + 63) / 64 * 64; }
+  if (mask & 2) { storage_shape(d.b_layout, d.K, d.N, &outer, &inner); e.ldb = (inner + 63) / 64 * 64; }
+  if (mask & 4) { storage_shape(d.c_layout, d.M, d.N, &outer, &inner); e.ldc = (inner + 63) / 64 * 64; }
+  return e;
+}
+
+// rows, contiguous elements per row, leading dimension and element size of matrix m (0 = A, 1 = B, 2 = C)
+void matrix_storage(const exo_gemm_desc_t& d, int m, int64_t* outer, int64_t* inner, int64_t* ld, int* bytes) {
+  if (m == 0) { storage_shape(d.a_layout, d.M, d.K, outer, inner); *ld = d.lda; *bytes = elem_bytes(d.ab_dtype); }
+  else if (m == 1) { storage_shape(d.b_layout, d.K, d.N, outer, inner); *ld = d.ldb; *bytes = elem_bytes(d.ab_dtype); }
+  else { storage_shape(d.c_layout, d.M, d.N, outer, inner); *ld = d.ldc; *bytes = elem_bytes(d.c_dtype); }
+}
+
+int64_t pack_bytes(const exo_gemm_desc_t& aligned, int m) {
+  int64_t outer, inner, ld; int bytes;
+  matrix_storage(aligned, m, &outer, &inner, &ld, &bytes);
+  return outer * ld * bytes;
+}
+
 void fill_info(const exo_gemm_plan* p, exo_gemm_info_t* info) {
   memset(info, 0, sizeof(*info));
   info->cta_group = p->cfg.cta_group;
@@ -291,7 +319,11 @@ void fill_info(const exo_gemm_plan* p, exo_gemm_info_t* info) {
   info->split_k = p->cfg.lean ? p->cfg.lean : p->cfg.split;
   info->tail_tiles = p->cfg.tail_tiles;
   info->batch_count = (int32_t)p->canon.batch;
-  info->workspace_bytes = (int32_t)(p->cfg.workspace_bytes > 2147483647LL ? 2147483647LL : p->cfg.workspace_bytes);
+  int64_t scratch = p->cfg.workspace_bytes;
+  for (int m = 0; m < 3; ++m)
+    if (p->repack & (1 << m)) scratch += pack_bytes(p->desc, m);
+  info->workspace_bytes = (int32_t)(scratch > 2147483647LL ? 2147483647LL : scratch);
+  info->repacked = p->repack;
 }
 
 }  // namespace
@@ -378,8 +410,10 @@ exo_gemm_status_t exo_gemm_plan_preview(const exo_gemm_desc_t* desc, int32_t sm_
   if (st != EXO_GEMM_OK) return st;
   if (sm_count < 1) return EXO_GEMM_ERR_INVALID_ARG;
   exo_gemm_plan p{};
-  p.desc = *desc;
-  p.canon = canonicalize(*desc);
+  p.user_desc = *desc;
+  p.repack = repack_mask(*desc);
+  p.desc = aligned_desc(*desc, p.repack);
+  p.canon = canonicalize(p.desc);
   p.sm_count = sm_count;
   const FlagOverrides ov = decode_flags(desc->flags, desc->flags2);
   if (ov.share >= 2 && !kHaveSharePairs) return EXO_GEMM_ERR_UNSUPPORTED;
@@ -421,8 +455,10 @@ exo_gemm_status_t exo_gemm_create_batched(exo_gemm_handle_t* out, const exo_gemm
 
   exo_gemm_plan* p = new (std::nothrow) exo_gemm_plan{};
   if (!p) return EXO_GEMM_ERR_CUDA;
-  p->desc = *desc;
-  p->canon = canonicalize(*desc, batch_count, stride_a, stride_b, stride_c);
+  p->user_desc = *desc;
+  p->repack = repack_mask(*desc);
+  p->desc = aligned_desc(*desc, p->repack);
+  p->canon = canonicalize(p->desc, batch_count, stride_a, stride_b, stride_c);
   p->device = device;
   p->sm_count = sms;
   p->dbg_timeout_ms = 0;
@@ -444,7 +480,14 @@ exo_gemm_status_t exo_gemm_create_batched(exo_gemm_handle_t* out, const exo_gemm
   e = cudaMalloc((void**)&p->d_status, kStatusBytes);
   if (e != cudaSuccess) { delete p; return cuda_fail(e); }
   e = cudaMemset(p->d_status, 0, kStatusBytes);
-  if (e != cudaSuccess) { cudaFree(p->d_status); delete p; return cuda_fail(e); }
+  for (int m = 0; m < 3 && e == cudaSuccess; ++m)   // aligned copies of the matrices whose rows TMA cannot address
+    if (p->repack & (1 << m)) e = cudaMalloc(&p->d_pack[m], (size_t)pack_bytes(p->desc, m));
+  if (e != cudaSuccess) {
+    for (int m = 0; m < 3; ++m) cudaFree(p->d_pack[m]);
+    cudaFree(p->d_status);
+    delete p;
+    return cuda_fail(e);
+  }
   if (p->cfg.tail_workers > 0) {  // scratch for the K-slices of the tail tiles, and who computes which
     const size_t flag_bytes = 2 * sizeof(uint32_t) * (size_t)p->cfg.tail_tiles * (size_t)p->cfg.pairs;
     if (ov.reduce_add) {   // the parts meet in C itself: no workspace, no counters
@@ -470,6 +513,7 @@ exo_gemm_status_t exo_gemm_create_batched(exo_gemm_handle_t* out, const exo_gemm
       cudaFree(p->d_split_flags);
       cudaFree(p->d_tail_table);
       cudaFree(p->d_status);
+      for (int m = 0; m < 3; ++m) cudaFree(p->d_pack[m]);
       delete p;
       return cuda_fail(e);
     }
@@ -514,7 +558,11 @@ exo_gemm_status_t check_run_args(const exo_gemm_plan* plan, const void* A, const
   if (cn.M == 0 || cn.N == 0) return EXO_GEMM_OK;
   const bool read_ab = alpha != 0.f && cn.K > 0;
   if (!C || (read_ab && (!A || !B))) return EXO_GEMM_ERR_NULL;
-  if (((uintptr_t)C & 15u) || (read_ab && (((uintptr_t)A | (uintptr_t)B) & 15u))) return EXO_GEMM_ERR_ALIGNMENT;
+  // 16 bytes for a matrix that TMA addresses in place; its element size for one that is copied first
+  const uintptr_t ab_mask = (uintptr_t)cn.ab_bytes - 1, c_mask = (uintptr_t)cn.c_bytes - 1;
+  if ((uintptr_t)C & ((plan->repack & 4) ? c_mask : 15u)) return EXO_GEMM_ERR_ALIGNMENT;
+  if (read_ab && (((uintptr_t)A & ((plan->repack & 1) ? ab_mask : 15u)) || ((uintptr_t)B & ((plan->repack & 2) ? ab_mask : 15u))))
+    return EXO_GEMM_ERR_ALIGNMENT;
   *launch = true;
   return EXO_GEMM_OK;
 }
@@ -676,6 +724,23 @@ exo_gemm_status_t launch_plan(exo_gemm_plan* plan, const void* A, const void* B,
   return EXO_GEMM_OK;
 }
 
+// One pass of repack.cuh's kernel over matrix m (0 = A, 1 = B, 2 = C) between the caller's layout and the plan's
+// aligned copy, in the direction given.
+exo_gemm_status_t copy_matrix(const exo_gemm_plan* plan, int m, void* dst, const void* src, bool into_aligned, void* cuda_stream) {
+  int64_t outer, inner, ld_user, ld_aligned; int bytes;
+  matrix_storage(plan->user_desc, m, &outer, &inner, &ld_user, &bytes);
+  matrix_storage(plan->desc, m, &outer, &inner, &ld_aligned, &bytes);
+  uint32_t seg = 0, blocks = 0;
+  if (!repack_grid(inner, outer, &seg, &blocks)) return EXO_GEMM_ERR_UNSUPPORTED;
+  const int64_t dst_ld = into_aligned ? ld_aligned : ld_user, src_ld = into_aligned ? ld_user : ld_aligned;
+  if (bytes == 2)
+    exo_repack_kernel<uint16_t><<<blocks, kRepackThreads, 0, (cudaStream_t)cuda_stream>>>((uint16_t*)dst, dst_ld, (const uint16_t*)src, src_ld, inner, seg);
+  else
+    exo_repack_kernel<uint32_t><<<blocks, kRepackThreads, 0, (cudaStream_t)cuda_stream>>>((uint32_t*)dst, dst_ld, (const uint32_t*)src, src_ld, inner, seg);
+  const cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? EXO_GEMM_OK : cuda_fail(e);
+}
+
 }  // namespace
 
 extern "C" {
@@ -684,9 +749,26 @@ exo_gemm_status_t exo_gemm_run(exo_gemm_handle_t plan, const void* A, const void
                                float beta, void* cuda_stream) {
   if (!plan) return EXO_GEMM_ERR_NULL;
   bool launch = false;
-  const exo_gemm_status_t st = check_run_args(plan, A, B, C, alpha, &launch);
+  exo_gemm_status_t st = check_run_args(plan, A, B, C, alpha, &launch);
   if (st != EXO_GEMM_OK || !launch) return st;
-  return launch_plan(plan, A, B, C, alpha, beta, cuda_stream);
+  if (!plan->repack) return launch_plan(plan, A, B, C, alpha, beta, cuda_stream);
+  // Matrices whose rows TMA cannot address travel through the plan's aligned copies: operands in before the
+  // GEMM, C in as well if it is read, C out after it (only its M x N elements: the caller's padding is untouched).
+  DeviceGuard guard(plan->device);
+  if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+  const bool read_ab = alpha != 0.f && plan->canon.K > 0;
+  const void* user[3] = {A, B, C};
+  const void* eff[3] = {A, B, C};
+  for (int m = 0; m < 3; ++m) {
+    if (!(plan->repack & (1 << m))) continue;
+    eff[m] = plan->d_pack[m];
+    if (m < 2 ? !read_ab : beta == 0.f) continue;   // never read: nothing to copy in
+    st = copy_matrix(plan, m, plan->d_pack[m], user[m], /*into_aligned=*/true, cuda_stream);
+    if (st != EXO_GEMM_OK) return st;
+  }
+  st = launch_plan(plan, eff[0], eff[1], const_cast<void*>(eff[2]), alpha, beta, cuda_stream);
+  if (st != EXO_GEMM_OK || !(plan->repack & 4)) return st;
+  return copy_matrix(plan, 2, C, plan->d_pack[2], /*into_aligned=*/false, cuda_stream);
 }
 
 exo_gemm_status_t exo_gemm_check(exo_gemm_handle_t plan, uint32_t* detail) {
@@ -759,7 +841,9 @@ exo_gemm_status_t exo_gemm_run_static(const exo_gemm_desc_t* desc, const void* A
 
   // a plan on the stack: same choices as exo_gemm_create, nothing allocated
   exo_gemm_plan plan{};
+  if (repack_mask(*desc)) return EXO_GEMM_ERR_UNSUPPORTED;   // an aligned copy would be scratch, which this entry point does not own
   plan.desc = *desc;
+  plan.user_desc = *desc;
   plan.canon = canonicalize(*desc);
   plan.device = device;
   plan.sm_count = sms;
@@ -826,6 +910,8 @@ exo_gemm_status_t exo_gemm_destroy(exo_gemm_handle_t plan) {
     if (plan->d_split_ws) cudaFree(plan->d_split_ws);
     if (plan->d_split_flags) cudaFree(plan->d_split_flags);
     if (plan->d_tail_table) cudaFree(plan->d_tail_table);
+    for (int m = 0; m < 3; ++m)
+      if (plan->d_pack[m]) cudaFree(plan->d_pack[m]);
   }
   delete plan;
   return st;

@@ -96,13 +96,27 @@ inline exo_gemm_status_t validate_desc(const exo_gemm_desc_t* d) {
   if ((d->flags & (1u << 11)) && d->c_dtype != EXO_GEMM_FP32) return EXO_GEMM_ERR_UNSUPPORTED;
   // the persistent scheduler indexes tiles (at least 128 x 64 each) and k-blocks with 32 bits
   if (((d->M + 127) / 128) * ((d->N + 63) / 64) >= (1LL << 31)) return EXO_GEMM_ERR_UNSUPPORTED;
-  // a matrix that is never touched (empty problem, K == 0) has no stride rule
-  const bool c_used = d->M > 0 && d->N > 0;
-  const bool ab_used = c_used && d->K > 0;
-  if (ab_used && ((d->lda * elem_bytes(d->ab_dtype)) % 16 || (d->ldb * elem_bytes(d->ab_dtype)) % 16))
-    return EXO_GEMM_ERR_UNSUPPORTED;
-  if (c_used && (d->ldc * elem_bytes(d->c_dtype)) % 16) return EXO_GEMM_ERR_UNSUPPORTED;
+  // (a leading dimension whose byte size is not a multiple of 16 cannot be described by a tensor map: a plan
+  // repacks such a matrix through scratch of its own, see repack_mask; the entry points that own no scratch refuse it)
   return EXO_GEMM_OK;
+}
+
+// Which matrices (1 = A, 2 = B, 4 = C) have rows that do not start on 16-byte boundaries and have to go through
+// an aligned copy.  A matrix that is never touched (empty problem, K == 0) has no stride rule.
+inline int repack_mask(const exo_gemm_desc_t& d) {
+  const bool c_used = d.M > 0 && d.N > 0;
+  const bool ab_used = c_used && d.K > 0;
+  int m = 0;
+  if (ab_used && (d.lda * elem_bytes(d.ab_dtype)) % 16) m |= 1;
+  if (ab_used && (d.ldb * elem_bytes(d.ab_dtype)) % 16) m |= 2;
+  if (c_used && (d.ldc * elem_bytes(d.c_dtype)) % 16) m |= 4;
+  return m;
+}
+
+// Rows (outer) and contiguous elements per row (inner) of a matrix as it lies in memory.
+inline void storage_shape(int32_t layout, int64_t rows, int64_t cols, int64_t* outer, int64_t* inner) {
+  *outer = layout == EXO_GEMM_ROW_MAJOR ? rows : cols;
+  *inner = layout == EXO_GEMM_ROW_MAJOR ? cols : rows;
 }
 
 // Strided batch: `batch` matrices, consecutive ones stride_x elements apart.  A and B may repeat
@@ -114,6 +128,7 @@ inline exo_gemm_status_t validate_batch(const exo_gemm_desc_t* d, int64_t batch,
   const int64_t kMaxStride = 1LL << 38;
   if (sa > kMaxStride || sb > kMaxStride || sc > kMaxStride) return EXO_GEMM_ERR_INVALID_ARG;
   if (batch > 1) {
+    if (repack_mask(*d)) return EXO_GEMM_ERR_UNSUPPORTED;   // the repacking path has no strided-batch form
     const int64_t c_extent = d->c_layout == EXO_GEMM_ROW_MAJOR ? (d->M - 1) * d->ldc + d->N : (d->N - 1) * d->ldc + d->M;
     if (d->M > 0 && d->N > 0 && sc < c_extent) return EXO_GEMM_ERR_INVALID_ARG;  // overlapping outputs
     if ((sa * elem_bytes(d->ab_dtype)) % 16 || (sb * elem_bytes(d->ab_dtype)) % 16 ||

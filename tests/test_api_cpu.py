@@ -1,6 +1,7 @@
 """Host-side tests of the C-ABI library that need no GPU: the library loads and
 exports what the header declares, argument validation, plan preview, and the
 persistent tile schedule."""
+import ctypes
 import os
 import re
 
@@ -83,13 +84,28 @@ def test_validate_unsupported_but_legal_blas_calls():
     for la, lb in ((1, 1), (0, 0), (1, 0)):                                          # ... in every operand layout
         assert B.exo_gemm_validate(good(ab_dtype=B.FP32, c_dtype=B.FP32, a_layout=la, b_layout=lb)) == B.OK
     assert B.exo_gemm_validate(good(ab_dtype=B.FP32, c_dtype=B.BF16)) == B.ERR_UNSUPPORTED
-    assert B.exo_gemm_validate(good(ab_dtype=B.FP32, K=130)) == B.ERR_UNSUPPORTED     # 520 bytes per row
-    assert B.exo_gemm_validate(good(ab_dtype=B.FP32, K=132)) == B.OK
     assert B.exo_gemm_validate(good(ab_dtype=B.BF16, c_dtype=B.FP16)) == B.ERR_UNSUPPORTED
-    assert B.exo_gemm_validate(good(K=100)) == B.ERR_UNSUPPORTED            # lda = 100: 200 bytes, not 16 | it
-    assert B.exo_gemm_validate(good(K=100, lda=104, ldb=104)) == B.OK
-    assert B.exo_gemm_validate(good(N=190)) == B.ERR_UNSUPPORTED            # fp32 C, ldc = 190
-    assert B.exo_gemm_validate(good(N=190, ldc=192)) == B.OK
+
+
+def test_leading_dimensions_tma_cannot_address_are_repacked():
+    """Rows that do not start on 16-byte boundaries are legal: the plan owns an aligned copy of such a matrix
+    (its contiguous extent rounded up to 64 elements) and says so; plans without scratch of their own refuse."""
+    for kw, want in ((dict(ab_dtype=B.FP32, K=130), 3),          # 520 bytes per row of A and of B
+                     (dict(ab_dtype=B.FP32, K=132), 0),
+                     (dict(K=100), 3),                           # 200 bytes
+                     (dict(K=100, lda=104), 2), (dict(K=100, ldb=104), 1), (dict(K=100, lda=104, ldb=104), 0),
+                     (dict(N=190), 4), (dict(N=190, ldc=192), 0),             # fp32 C, ldc = 190
+                     (dict(M=250, N=190, K=100, a_layout=1, c_layout=1), 7),   # col-major A (lda = 250), B (100), col-major C (250)
+                     (dict(M=0, N=190, K=100), 0), (dict(K=0, lda=3, ldb=5), 0)):    # matrices that are never touched
+        d = good(**kw)
+        assert B.exo_gemm_validate(d) == B.OK, kw
+        st, info = B.exo_gemm_plan_preview(d, 148)
+        assert st == B.OK and info.repacked == want, (kw, info.repacked)
+    st, info = B.exo_gemm_plan_preview(good(M=256, N=190, K=100), 148)
+    # A: 256 rows x 128 bf16, B (K x N col-major): 190 rows x 128 bf16, C: 256 rows x 192 fp32
+    assert info.repacked == 7 and info.workspace_bytes == 256 * 128 * 2 + 190 * 128 * 2 + 256 * 192 * 4
+    h = ctypes.c_void_p()
+    assert B.lib().exo_gemm_create_batched(ctypes.byref(h), ctypes.byref(good(K=100)), 4, 1 << 16, 1 << 16, 1 << 16) == B.ERR_UNSUPPORTED
 
 
 def test_benchmark_configs_are_in_the_supported_set():

@@ -893,3 +893,65 @@ def test_shape_sweep_classes_on_this_device_were_all_checked():
         if sig not in SWEEP_SEEN_SIGNATURES:
             missing.setdefault(sig, []).append((M, N, K))
     assert not missing, missing
+
+# ------------------------------------------------------------------ leading dimensions TMA cannot address
+# M, N, K, ab, cd, la, lb, lc, alpha, beta, lda, ldb, ldc (None = the contiguous extent), what is repacked
+REPACK_CASES = [
+    (300, 190, 100, BF16, FP32, 0, 1, 0, 1.0, 0.0, None, None, None, 7),      # every matrix: 200-byte operand rows, 760-byte C rows
+    (300, 190, 100, BF16, FP32, 0, 1, 0, 1.5, -0.5, None, None, None, 7),     # ... and C read back (beta != 0)
+    (257, 129, 77, FP16, FP16, 0, 1, 0, 1.0, 1.0, 79, 83, 131, 7),            # odd leading dimensions beyond the extents
+    (512, 256, 136, BF16, BF16, 0, 1, 0, 1.0, 0.0, None, None, 250 + 7, 4),   # only C (ldc = 257 halves)
+    (512, 256, 100, BF16, FP32, 0, 1, 0, 1.0, 0.0, None, 104, None, 1),       # only A
+    (250, 190, 100, BF16, FP32, 1, 0, 1, -1.0, 0.75, None, None, None, 7),    # M-contiguous A, N-contiguous B, column-major C
+    (260, 132, 130, FP32, FP32, 0, 1, 0, 1.0, 0.0, None, None, 133, 7),       # tf32: 520-byte rows
+    (2048, 1288, 1001, BF16, BF16, 0, 1, 0, 1.0, 0.0, None, None, None, 3),   # the persistent kernel behind the copies
+]
+
+
+@pytest.mark.parametrize("case", REPACK_CASES, ids=lambda c: "x".join(str(v) for v in c[:3]) + f"_{c[3]}{c[4]}{c[5]}{c[6]}{c[7]}_r{c[13]}")
+def test_matrices_whose_rows_tma_cannot_address_go_through_aligned_copies(case):
+    """A legal BLAS call whose leading dimension times the element size is not a multiple of 16 bytes: the plan
+    copies that matrix into an aligned buffer of its own before the GEMM (and C back after it).  Same oracle,
+    same tolerance; the caller's padding between rows is untouched; base pointers need element alignment only."""
+    import torch
+    M, N, K, ab, cd, la, lb, lc, alpha, beta, lda, ldb, ldc, want = case
+    p = synth.Problem("repack", M, N, K, ab, cd, la, lb, lc, alpha, beta, seed=M + 5 * N + 11 * K, lda=lda, ldb=ldb, ldc=ldc,
+                      dist="normal" if ab == FP16 else "uniform").generate()
+    dev = torch.device("cuda:0")
+    # operands and C at addresses that are only element-aligned where the matrix is repacked
+    def shifted(host, repacked, elem):
+        raw = torch.from_numpy(host.view(np.uint8).reshape(-1))
+        off = elem if repacked else 0
+        buf = torch.full((raw.numel() + 64,), 0x7F, dtype=torch.uint8, device=dev)
+        buf[off:off + raw.numel()] = raw.to(dev)
+        return buf, off
+    eb = 4 if ab == FP32 else 2
+    cb = 4 if cd == FP32 else 2
+    dA, oa = shifted(p.A, want & 1, eb)
+    dB, ob = shifted(p.B, want & 2, eb)
+    dC, oc = shifted(p.C, want & 4, cb)
+    with B.Plan(harness.desc_of(p)) as plan:
+        info = plan.info()
+        assert info["repacked"] == want, info
+        stream = torch.cuda.current_stream(dev).cuda_stream
+        for rep in range(2):      # the second run starts from the first one's C when beta != 0: reset it
+            dC[oc:oc + p.C.nbytes] = torch.from_numpy(p.C.view(np.uint8).reshape(-1)).to(dev)
+            plan.run(dA.data_ptr() + oa, dB.data_ptr() + ob, dC.data_ptr() + oc, p.alpha, p.beta, stream)
+            torch.cuda.synchronize(dev)
+            plan.check()
+        out = dC.cpu().numpy()
+    assert (out[:oc] == 0x7F).all() and (out[oc + p.C.nbytes:] == 0x7F).all()        # nothing outside the buffer
+    cbuf = out[oc:oc + p.C.nbytes].view(synth.storage_np_dtype(cd)).reshape(p.C.shape)
+    got = oracle.logical_view(cbuf, M, N, lc, p.ldc, cd)
+    cref, den = oracle.gemm_problem(p)
+    gate = TOL * den + oracle.output_rounding_slack(cref, cd)
+    assert (np.abs(got - cref) <= gate).all(), info
+    # the padding elements of C (between the logical row end and ldc) keep the caller's bits
+    rows, cols = (M, N) if lc == 0 else (N, M)
+    if p.ldc > cols:
+        before = p.C.view(np.uint8).reshape(-1)[: (rows - 1) * p.ldc * cb + cols * cb]
+        after = out[oc:oc + before.size]
+        pad = np.ones(before.size, dtype=bool)
+        for r in range(rows):
+            pad[r * p.ldc * cb: r * p.ldc * cb + cols * cb] = False
+        assert np.array_equal(before[pad], after[pad])
