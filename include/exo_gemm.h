@@ -110,9 +110,15 @@ typedef enum { EXO_GEMM_ROW_MAJOR = 0, EXO_GEMM_COL_MAJOR = 1 } exo_gemm_layout_
  * tiles).  One CTA per 128 x 64 or 128 x 128 tile, all launched at once; the copies of the first
  * k-blocks are issued before the CTA's set-up barrier, C_in is fetched during the main loop, and
  * no warp waits for another at the end.  It never cuts K and has no strided-batch form.
- * 0 = the library decides, 1 = never, 2 = always (ERR_INVALID_ARG together with CTA_GROUP(2),
- * TILE_N(256), a SHARE_ALWAYS / SHARE_SUBSTITUTED or CTA_ROWS(256) request, SPLIT_K(2..),
- * SPLIT_REDUCE_ADD or a GRID_LIMIT; a batched plan ignores it).  3 is invalid.
+ * With SPLIT_K(2) or SPLIT_K(4) the K loop of every tile is cut over a cluster of that many CTAs,
+ * which exchange their partial sums through distributed shared memory (no workspace).  Together
+ * with CTA_GROUP(2) the request means the same kernel structure for a PAIR of CTAs per 256 x 128
+ * or 256 x 256 tile (tcgen05 cta_group::2; K is never cut there); the library never picks that
+ * form on its own (it measured level with the persistent kernel).
+ * 0 = the library decides, 1 = never, 2 = always (ERR_INVALID_ARG together with TILE_N(256)
+ * unless CTA_GROUP(2) is given, a SHARE_ALWAYS / SHARE_SUBSTITUTED or CTA_ROWS(256) request,
+ * SPLIT_K other than 1, 2, 4 (other than 1 with CTA_GROUP(2)), SPLIT_REDUCE_ADD or a
+ * GRID_LIMIT; a batched plan ignores it).  3 is invalid.
  */
 #define EXO_GEMM_FLAG2_LEAN_AUTO 0u
 #define EXO_GEMM_FLAG2_LEAN_NEVER (1u << 4)

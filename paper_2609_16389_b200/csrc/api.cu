@@ -11,6 +11,7 @@
 #include "../../include/exo_gemm.h"
 #include "gemm_kernel.cuh"
 #include "lean_kernel.cuh"
+#include "lean_pair_kernel.cuh"
 #include "repack.cuh"
 #include "plan.h"
 #ifdef EXO_GEMM_SHARE_PAIRS
@@ -93,12 +94,28 @@ static KernelFn pick_lean(int bn, int ksub, int out) {
   return ksub == 2 ? pick_lean_out<64, 2>(out) : pick_lean_out<64, 1>(out);
 }
 
+// ... and its form for a CTA pair per tile: 256 x 128 or 256 x 256
+template <int BN, int KSUB>
+static KernelFn pick_lean_pair_out(int out) {
+  switch (out) {
+    case EXO_GEMM_BF16: return exo_gemm_lean_pair_kernel<BN, kOutBf16, KSUB>;
+    case EXO_GEMM_FP16: return exo_gemm_lean_pair_kernel<BN, kOutFp16, KSUB>;
+    default:            return exo_gemm_lean_pair_kernel<BN, kOutFp32, KSUB>;
+  }
+}
+static KernelFn pick_lean_pair(int bn, int ksub, int out) {
+  if (bn == 256) return ksub == 2 ? pick_lean_pair_out<256, 2>(out) : pick_lean_pair_out<256, 1>(out);
+  return ksub == 2 ? pick_lean_pair_out<128, 2>(out) : pick_lean_pair_out<128, 1>(out);
+}
+
 // kernel and dynamic shared memory of a plan's configuration
 static KernelFn kernel_of(const TileConfig& cfg, int c_dtype, bool reduce) {
+  if (cfg.lean && cfg.cta_group == 2) return pick_lean_pair(cfg.tile_n, cfg.ksub, c_dtype);
   if (cfg.lean) return pick_lean(cfg.tile_n, cfg.ksub, c_dtype);
   return pick_kernel(cfg.cta_group, cfg.tile_n, cfg.ksub, c_dtype, cfg.pairs, cfg.mrep, reduce);
 }
 static int smem_of(const TileConfig& cfg, int c_dtype) {
+  if (cfg.lean && cfg.cta_group == 2) return lean_pair_smem_bytes(cfg.tile_n, cfg.ksub, cfg.stages, c_dtype == EXO_GEMM_FP32 ? 4 : 2);
   if (cfg.lean) return lean_smem_bytes(cfg.tile_n, cfg.ksub, cfg.stages, c_dtype == EXO_GEMM_FP32 ? 4 : 2, cfg.lean);
   return smem_bytes_for(cfg.cta_group, cfg.tile_n, cfg.ksub, cfg.stages, cfg.epi_bufs, cfg.mrep);
 }
@@ -302,7 +319,7 @@ void fill_info(const exo_gemm_plan* p, exo_gemm_info_t* info) {
   info->tile_k = sub_block_k(p->canon.ab_bytes) * p->cfg.ksub;
   info->stages = p->cfg.stages;
   info->grid = p->cfg.workers * p->cfg.cta_group * p->cfg.pairs * (p->cfg.lean ? p->cfg.lean : 1);
-  info->cluster_size = p->cfg.lean ? p->cfg.lean : p->cfg.cta_group * p->cfg.pairs;
+  info->cluster_size = p->cfg.lean ? p->cfg.lean * p->cfg.cta_group : p->cfg.cta_group * p->cfg.pairs;
   info->stages_direct = p->cfg.stages_direct;
   info->tail_workers = p->cfg.tail_workers;
   info->smem_bytes = p->smem_bytes;
@@ -685,13 +702,14 @@ exo_gemm_status_t launch_plan(exo_gemm_plan* plan, const void* A, const void* B,
   if (guard.err != cudaSuccess) return cuda_fail(guard.err);
   cudaLaunchConfig_t lc{};
   lc.gridDim = dim3((unsigned)(cfg.workers * cfg.cta_group * cfg.pairs * (cfg.lean ? cfg.lean : 1)), 1, 1);
-  lc.blockDim = dim3(cfg.lean ? (unsigned)lean_threads(cfg.tile_n, (int)cn.c_bytes) : (unsigned)kNumThreads, 1, 1);
+  lc.blockDim = dim3(!cfg.lean ? (unsigned)kNumThreads
+                               : (cfg.cta_group == 2 ? (unsigned)kLeanPairThreads : (unsigned)lean_threads(cfg.tile_n, (int)cn.c_bytes)), 1, 1);
   lc.dynamicSmemBytes = direct ? smem_bytes_for(cfg.cta_group, cfg.tile_n, cfg.ksub, cfg.stages_direct, 0, cfg.mrep)
                                : plan->smem_bytes;
   lc.stream = (cudaStream_t)cuda_stream;
   cudaLaunchAttribute at[3];
   at[0].id = cudaLaunchAttributeClusterDimension;
-  at[0].val.clusterDim.x = (unsigned)(cfg.lean ? cfg.lean : cfg.cta_group);
+  at[0].val.clusterDim.x = (unsigned)(cfg.lean ? cfg.lean * cfg.cta_group : cfg.cta_group);
   at[0].val.clusterDim.y = 1;
   at[0].val.clusterDim.z = 1;
   // Programmatic dependent launch: this kernel's CTAs may start (barrier set-up, TMEM allocation)

@@ -57,6 +57,20 @@ EXO_CX int lean_max_stages(int bn, int ksub, int c_bytes, int split) {
   return n > kMaxStages ? kMaxStages : n;
 }
 
+// The same for a pair of CTAs per 256 x bn tile (lean_pair_kernel.cuh), bn = 128 or 256: the ring doubles as the
+// epilogue's staging area (128 rows x bn of C per CTA) once the accumulator is complete.
+EXO_CX int lean_pair_ring_bytes(int bn, int ksub, int stages, int c_bytes) {
+  return stages * stage_bytes(2, bn, ksub) > kBlockM * bn * c_bytes ? stages * stage_bytes(2, bn, ksub) : kBlockM * bn * c_bytes;
+}
+EXO_CX int lean_pair_smem_bytes(int bn, int ksub, int stages, int c_bytes) {
+  return lean_pair_ring_bytes(bn, ksub, stages, c_bytes) + kBarrierBytes + 1024;
+}
+EXO_CX int lean_pair_max_stages(int bn, int ksub) {
+  const int n = (kSmemLimit - 1024 - kBarrierBytes) / stage_bytes(2, bn, ksub);
+  return n > kMaxStages ? kMaxStages : n;
+}
+constexpr int kLeanPairThreads = 320;   // producer, MMA issuer, eight epilogue warps
+
 // How one operand is staged.  K-major: per 64-k sub-block one TMA box {64 k, rows},
 // sub-blocks rows*128 bytes apart.  MN-major: rows/64 boxes {64 mn, 64*ksub k}.
 struct OperandStaging {

@@ -6,15 +6,15 @@
 // regime where kernels differ most.  This kernel computes one 128 x BN tile per CTA and shortens
 // every link of that chain:
 //
-//   warp 0             initialises the barriers and issues the copies of the first ring of k-blocks
-//                      BEFORE the CTA-wide set-up barrier (nothing but this warp's own barriers is
-//                      needed for that), then the remaining k-blocks as stages come free
+//   warp 0             initialises the barriers and issues the copies of the first two k-blocks BEFORE
+//                      the CTA-wide set-up barrier (nothing but this warp's own barriers is needed for
+//                      that), then the remaining k-blocks, waiting only for stages that are reused
 //   warp 1             allocates tensor memory, issues the MMAs (one elected lane), frees tensor
 //                      memory as soon as every epilogue warp has read its part of the accumulator
 //   warps 2..          epilogue, four or eight warps: C_in (beta != 0) is fetched while the main loop
 //                      runs, every warp has a staging buffer per column chunk of its own (no buffer
 //                      is ever waited for), and a warp leaves as soon as its own store has read its
-//                      buffer: there is no barrier at the end
+//                      buffer: without a cluster there is no barrier at the end
 //
 // K split across a cluster (the cluster's size, 1, 2 or 4, is the split factor): the CTAs of a cluster
 // compute the same tile over consecutive ranges of k-blocks, each into its own TMEM accumulator, and
@@ -23,9 +23,10 @@
 // fp32 partials in their own operand ring (free by then) and send them with one bulk copy each
 // (cp.async.bulk shared::cta -> shared::cluster, counted in bytes on the receiver's barrier), and the
 // finishing CTA adds them in rank order -- deterministic, no global-memory round trip.  (Ordinary
-// remote stores were measured first: 20 bytes per clock and SM, 4.5 k clocks for the exchange.)  A 128 x 64 MMA costs the tensor
-// core about 80 clocks whatever its share of the peak, so a short problem on few SMs is bound by the
-// number of MMAs per CTA; cutting K over four SMs cuts that by four for an exchange of 24 KB per CTA.
+// remote stores were measured first: 20 bytes per clock and SM, 4.5 k clocks for the exchange.)
+// A k-block of eight 128 x 64 x 16 MMAs costs the issuing thread about 600 clocks whatever the tensor
+// core could do, so a short problem on few SMs is bound by the number of MMAs per CTA; cutting K over
+// four SMs cuts that by four for an exchange of 24 KB per CTA.
 //
 // The code is short on purpose (a CTA runs every basic block exactly once, from a cold instruction
 // cache).  Operand staging, descriptors, tensor maps and the parameter block are those of the

@@ -86,8 +86,9 @@ inline exo_gemm_status_t validate_desc(const exo_gemm_desc_t* d) {
   if ((d->flags & (1u << 11)) && (o.share >= 2 || o.mrep == 2)) return EXO_GEMM_ERR_INVALID_ARG;
   // the one-tile-per-CTA kernel has 1-CTA tiles of 128 x 64 or 128 x 128, cuts K over a cluster of 2 or 4 only and
   // takes every tile at once
-  if (o.lean == 2 && (o.cta_group == 2 || o.tile_n == 256 || o.share >= 2 || o.mrep == 2 || (o.split >= 2 && o.split != 2 && o.split != 4) ||
-                      (d->flags & (1u << 11)) || o.grid_limit != 0))
+  // (with CTA_GROUP(2): one 256 x 128 or 256 x 256 tile per CTA pair, K never cut)
+  if (o.lean == 2 && (o.share >= 2 || o.mrep == 2 || (d->flags & (1u << 11)) || o.grid_limit != 0 ||
+                      (o.cta_group == 2 ? o.split >= 2 : (o.tile_n == 256 || (o.split >= 2 && o.split != 2 && o.split != 4)))))
     return EXO_GEMM_ERR_INVALID_ARG;
   // beyond here the call is a legal BLAS call; what follows is this library's supported set
   // fp32 operands are multiplied as tf32 (the precision of the paper's own kernels) into an fp32 C
@@ -449,7 +450,10 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
   // fit the SMs at one per SM, else 128 x 128.
   bool lean = false;
   int lean_split = 1;   // CTAs (a cluster) that share a lean tile's K loop: 1, 2 or 4
-  if (o.lean != 1 && c.batch <= 1 && !o.reduce_add && o.share < 2 && o.mrep != 2 && o.cta_group != 2 && o.tile_n != 256 &&
+  if (o.lean == 2 && o.cta_group == 2 && c.batch <= 1 && max_pairs >= 1) {   // on request: a CTA pair per 256 x N tile
+    lean = true;
+    best_g = 2; best_n = o.tile_n ? o.tile_n : 256; best_p = 1; best_r = 1;
+  } else if (o.lean != 1 && c.batch <= 1 && !o.reduce_add && o.share < 2 && o.mrep != 2 && o.cta_group != 2 && o.tile_n != 256 &&
       o.grid_limit == 0 && (o.split < 2 || o.split == 2 || o.split == 4)) {
     const int ksub = o.ksub ? o.ksub : 2;
     const int64_t nkb_all = (c.K * (c.ab_bytes / 2) + kBlockK * ksub - 1) / (kBlockK * ksub);
@@ -504,7 +508,7 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
   if (lean) {  // a ring no deeper than a CTA's K loop: with every k-block resident no stage is ever waited for
     const int64_t nkb_all = (k16 + kBlockK * cfg.ksub - 1) / (kBlockK * cfg.ksub);
     const int64_t nkb = (nkb_all + lean_split - 1) / lean_split;
-    cfg.stages = lean_max_stages(best_n, cfg.ksub, c.c_bytes, lean_split);
+    cfg.stages = best_g == 2 ? lean_pair_max_stages(best_n, cfg.ksub) : lean_max_stages(best_n, cfg.ksub, c.c_bytes, lean_split);
     if (nkb < cfg.stages) cfg.stages = nkb < 1 ? 1 : (int)nkb;
     if (o.stages && o.stages < cfg.stages) cfg.stages = o.stages;
     // (a cluster's CTAs stage their partial sums, 4 quadrants x 128 bytes x tile_n, in the ring once their MMAs are done)

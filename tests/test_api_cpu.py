@@ -429,7 +429,7 @@ def test_lean_kernel_flags_and_preview():
     assert B.exo_gemm_validate(good(flags2=LEAN)) == B.OK and B.exo_gemm_validate(good(flags2=NEVER)) == B.OK
     assert B.exo_gemm_validate(good(flags2=48)) == B.ERR_INVALID_ARG                       # lean field 3
     assert B.exo_gemm_validate(good(flags2=64)) == B.ERR_INVALID_ARG                       # bits 6.. are reserved
-    for f, f2 in [(B.flag_cta_group(2), LEAN), (B.flag_tile_n(256), LEAN), (B.flag_split_k(3), LEAN), (B.flag_split_k(8), LEAN),
+    for f, f2 in [(B.flag_cta_group(2) | B.flag_split_k(2), LEAN), (B.flag_tile_n(256), LEAN), (B.flag_split_k(3), LEAN), (B.flag_split_k(8), LEAN),
                   (B.flag_grid_limit(8), LEAN), (1 << 11, LEAN), (0, LEAN | B.flag2_cta_rows(256)),
                   (0, LEAN | B.FLAG2_SHARE_ALWAYS)]:
         assert B.exo_gemm_validate(good(flags=f, flags2=f2)) == B.ERR_INVALID_ARG, (f, f2)
@@ -464,6 +464,13 @@ def test_lean_kernel_flags_and_preview():
     for f in (B.flag_tile_n(64), B.flag_cta_group(1), B.flag_max_stages(3), B.flag_epi_buffers(1), B.flag_band(2), B.flag_split_k(4)):
         st, info = B.exo_gemm_plan_preview(good(M=512, N=512, K=512, flags=f), 148)
         assert info.lean_kernel == 0, f
+    # a CTA pair per 256 x 256 (or 256 x 128) tile on request
+    st, info = B.exo_gemm_plan_preview(good(M=2048, N=2048, K=512, flags2=LEAN, flags=B.flag_cta_group(2)), 148)
+    i = info.as_dict()
+    assert (i["lean_kernel"], i["cta_group"], i["tile_m"], i["tile_n"], i["cluster_size"], i["grid"], i["stages"], i["tmem_columns"]) == (1, 2, 256, 256, 2, 128, 7, 256)
+    assert i["smem_bytes"] == 7 * 32768 + 512 + 1024
+    st, info = B.exo_gemm_plan_preview(good(M=512, N=512, K=128, flags2=LEAN, flags=B.flag_cta_group(2) | B.flag_tile_n(128)), 148)
+    assert (info.tile_n, info.stages, info.grid, info.smem_bytes) == (128, 1, 16, 128 * 128 * 4 + 512 + 1024)   # the ring holds the staged C
     # K cut over a cluster of 2 or 4 CTAs per tile; the partial sums travel through shared memory, not a workspace
     st, info = B.exo_gemm_plan_preview(good(M=512, N=512, K=1000, flags2=LEAN, flags=B.flag_split_k(4)), 148)
     i = info.as_dict()

@@ -117,6 +117,45 @@ def test_lean_kernel_with_k_cut_over_a_cluster(case):
         assert np.array_equal(again.view(np.uint8), bits.view(np.uint8))
 
 
+# one CTA pair per 256 x 128 or 256 x 256 tile: M, N, K, ab, cd, la, lb, lc, alpha, beta, tile_n (0 = 256), extra flags
+PAIR_CASES = [
+    (256, 256, 64, BF16, FP32, 0, 1, 0, 1.0, 0.0, 0, 0),                       # exactly one tile, one k-block
+    (2048, 2048, 512, BF16, FP32, 0, 1, 0, 1.0, 0.0, 0, 0),                    # 64 tiles: one wave of pairs
+    (2048, 2048, 2048, BF16, BF16, 0, 1, 0, 1.0, 0.0, 0, 0),                   # the ring is reused; 16-bit C
+    (512, 3072, 1000, BF16, FP32, 0, 1, 0, 1.0, 0.0, 128, 0),                  # 256 x 128 tiles, ragged K
+    (700, 300, 200, BF16, FP32, 0, 1, 0, 1.0, 0.0, 0, 0),                      # ragged M, N and K; second CTA partly outside
+    (130, 72, 4096, FP16, FP16, 0, 1, 0, 1.0, 0.0, 128, 0),                    # two valid rows in the second CTA
+    (1, 8, 8, BF16, FP32, 0, 1, 0, 2.0, 0.0, 0, 0),
+    (384, 520, 2048, BF16, BF16, 0, 1, 0, 1.5, -0.75, 128, B.flag_max_stages(2)),  # beta, a ring of 2
+    (1000, 520, 264, BF16, FP32, 1, 0, 0, 1.0, 0.5, 0, 0),                     # M/N-contiguous operands, beta
+    (1000, 520, 264, BF16, FP32, 1, 0, 0, 1.0, 0.5, 128, B.flag_k_subblocks(1)),
+    (640, 900, 320, FP16, FP32, 0, 1, 1, -1.0, 1.0, 0, 0),                     # column-major C (operands swap)
+    (640, 384, 520, FP32, FP32, 0, 1, 0, 1.0, 0.0, 0, 0),                      # tf32 operands
+    (520, 392, 264, FP32, FP32, 1, 0, 0, 1.25, -0.5, 128, 0),                  # tf32, M/N-contiguous operands
+    (4096, 4096, 256, BF16, FP32, 0, 1, 0, 1.0, 0.0, 0, 0),                    # 256 pairs: more than fit at once
+    (1024, 1024, 0, BF16, FP32, 0, 1, 0, 1.0, 0.5, 0, 0),                      # K = 0: C = beta * C
+    (256, 512, 512, BF16, BF16, 0, 1, 0, 0.0, 2.0, 0, 0),                      # alpha = 0: operands never read
+]
+
+
+@pytest.mark.parametrize("case", PAIR_CASES, ids=lambda c: "x".join(str(v) for v in c[:3]) + f"_{c[3]}{c[4]}{c[5]}{c[6]}{c[7]}_n{c[10]}")
+def test_lean_pair_kernel_matches_the_oracle_and_the_persistent_kernel(case):
+    """The form for a pair of CTAs per tile (tcgen05 cta_group::2, 256 x 128 or 256 x 256): the oracle's result,
+    and the bits of the persistent kernel on the same tile with its K split switched off."""
+    M, N, K, ab, cd, la, lb, lc, alpha, beta, bn, extra = case
+    p = synth.Problem("lean_pair", M, N, K, ab, cd, la, lb, lc, alpha, beta, seed=M + 3 * N + K + 1,
+                      dist="normal" if ab == FP16 else "uniform").generate()
+    tile = B.flag_tile_n(bn) if bn else 0
+    bits, got, info = run(p, NO_SPLIT | B.flag_cta_group(2) | extra | tile, LEAN)
+    assert info["lean_kernel"] == 1 and info["cta_group"] == 2 and info["tile_m"] == 256 and info["cluster_size"] == 2
+    assert info["tile_n"] == (bn or 256) and info["grid"] == 2 * info["tiles_m"] * info["tiles_n"] and info["split_k"] == 1
+    assert info["tmem_columns"] == info["tile_n"] and info["smem_bytes"] <= 232448
+    assert_parity(p, got, info)
+    ref_bits, _, info_r = run(p, NO_SPLIT | B.flag_cta_group(2) | extra | B.flag_tile_n(info["tile_n"]), PERSISTENT | B.flag2_cta_rows(128))
+    assert info_r["lean_kernel"] == 0 and info_r["tile_n"] == info["tile_n"] and info_r["tile_k"] == info["tile_k"]
+    assert np.array_equal(ref_bits.view(np.uint8), bits.view(np.uint8))
+
+
 def test_lean_kernel_padding_untouched_and_nan_c_ignored_when_beta_is_zero():
     p = synth.Problem("lean_pad", 600, 500, 136, BF16, FP32, 0, 1, 0, 1.0, 0.0, seed=4, ldc=512).generate()
     p.C[:] = np.nan
@@ -136,10 +175,12 @@ def test_lean_kernel_bounded_wait_reports_timeout_and_the_plan_stays_usable():
     p = synth.Problem("lean_tmo", 512, 512, 1024, BF16, FP32, 0, 1, 0, 1.0, 0.0, seed=10).generate()
     # a k-block of the first two (issued before the set-up barrier), one behind them; then with the K loop cut
     # over a cluster of 4 (CTA 0 has k-blocks 0 and 1: its peers' partial sums arrive, its own never does)
-    for skip, split in ((1, 1), (6, 1), (1, 4)):
-        dp = harness.DeviceProblem(p, B.flag_split_k(split) | B.flag_max_stages(4), flags2=LEAN)
+    # ... and the pair form (CTA 0 is the leader of the first pair: its copies of one k-block never come)
+    for skip, split, group in ((1, 1, 1), (6, 1, 1), (1, 4, 1), (1, 1, 2), (6, 1, 2)):
+        dp = harness.DeviceProblem(p, B.flag_split_k(split) | B.flag_max_stages(4) | (B.flag_cta_group(2) if group == 2 else 0), flags2=LEAN)
         try:
             assert dp.plan.info()["lean_kernel"] == 1 and dp.plan.info()["stages"] == (4 if split == 1 else 2)
+            assert dp.plan.info()["cta_group"] == group
             assert B.exo_gemm_debug_set(dp.plan.handle, 20, skip) == B.OK
             dp.run()
             torch.cuda.synchronize()
@@ -147,7 +188,7 @@ def test_lean_kernel_bounded_wait_reports_timeout_and_the_plan_stays_usable():
             assert st == B.ERR_DEVICE_TIMEOUT
             # the wait that runs out first is CTA 0's own, or (cut K) a peer's wait for CTA 0's partial sums,
             # which starts within a microsecond of it
-            assert detail[0] == 1 and detail[1] in ((1, 2, 3) if split == 1 else (1, 2, 3, 6)) and detail[5] < split, detail
+            assert detail[0] == 1 and detail[1] in ((1, 2, 3) if split == 1 else (1, 2, 3, 6)) and detail[5] < split * group, detail
             dp.reset_c()
             dp.run()
             torch.cuda.synchronize()
