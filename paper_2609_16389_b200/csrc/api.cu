@@ -701,7 +701,7 @@ exo_gemm_status_t launch_plan(exo_gemm_plan* plan, const void* A, const void* B,
   DeviceGuard guard(plan->device);
   if (guard.err != cudaSuccess) return cuda_fail(guard.err);
   cudaLaunchConfig_t lc{};
-  lc.gridDim = dim3((unsigned)(cfg.workers * cfg.cta_group * cfg.pairs * (cfg.lean ? cfg.lean : 1)), 1, 1);
+  lc.gridDim = dim3((unsigned)((int64_t)cfg.workers * cfg.cta_group * cfg.pairs * (cfg.lean ? cfg.lean : 1)), 1, 1);
   lc.blockDim = dim3(!cfg.lean ? (unsigned)kNumThreads
                                : (cfg.cta_group == 2 ? (unsigned)kLeanPairThreads : (unsigned)lean_threads(cfg.tile_n, (int)cn.c_bytes)), 1, 1);
   lc.dynamicSmemBytes = direct ? smem_bytes_for(cfg.cta_group, cfg.tile_n, cfg.ksub, cfg.stages_direct, 0, cfg.mrep)

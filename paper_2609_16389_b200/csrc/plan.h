@@ -472,6 +472,8 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
       best_g = 1; best_n = bn; best_p = 1; best_r = 1;
       lean_split = split;
       while (lean_split > 1 && lean_split > nkb_all) lean_split /= 2;   // every CTA of a cluster gets a k-block
+      const int64_t lean_tiles = ((c.M + 127) / 128) * ((c.N + bn - 1) / bn);
+      while (lean_split > 1 && lean_tiles * lean_split >= (1LL << 31)) lean_split /= 2;   // the grid is indexed with 32 bits
     }
   }
   TileConfig cfg;
