@@ -294,9 +294,6 @@ exo_gemm_lean_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     }
     EXO_TRACE_CHUNK(0, 1);
     EXO_TRACE_W(2);
-    ptx::tc_fence_before_sync();
-    __syncwarp();
-    if (ptx::elect_one()) ptx::mbar_arrive(tdone_bar);   // also on the way out of an abandoned wait
     const uint32_t my_xor = (lane & 7u) << 4;
     if (S > 1) {
       // partial sums travel as 4 KB units (32 rows x 32 fp32 columns): lane l's 128 bytes at l * 128, 16-byte pieces swizzled
@@ -414,6 +411,13 @@ exo_gemm_lean_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
           EXO_TRACE_CHUNK(i, 3);
         }
       }
+    }
+    // This warp has read its part of the accumulator (long ago: the arrival is kept off the path to the
+    // stores; tensor memory is only wanted back at the CTA's exit).  Also on the way out of an abandoned wait.
+    ptx::tc_fence_before_sync();
+    __syncwarp();
+    if (ptx::elect_one()) ptx::mbar_arrive(tdone_bar);
+    if (ok) {
       // the stores must have read this warp's buffers before the warp (possibly the CTA's last) leaves
       if (warp == 2 && lane == 0) EXO_TRACE(2, 0, 1, 4096);
       if (ptx::elect_one()) ptx::bulk_wait_read<0>();
