@@ -209,7 +209,15 @@ def output_rounding_slack(cref: np.ndarray, c_dtype: int) -> np.ndarray:
     widened gate |dC| <= 1e-3 * Den + u_out * |Cref|.
     """
     u = {FP32: 0.0, BF16: 2.0 ** -8, FP16: 2.0 ** -11}[c_dtype]
-    return u * np.abs(cref)
+    slack = u * np.abs(cref)
+    if c_dtype != FP32:
+        # Below the smallest normal number the spacing of the output type no longer shrinks with the value
+        # (gradual underflow: 2^-24 for fp16 below 2^-14, 2^-133 for bf16 below 2^-126), so half an ulp is a
+        # constant there.  Zero is representable: no slack at Cref == 0.
+        min_normal, half_spacing = {BF16: (2.0 ** -126, 2.0 ** -134), FP16: (2.0 ** -14, 2.0 ** -25)}[c_dtype]
+        a = np.abs(cref)
+        slack = np.where((a > 0) & (a < min_normal), half_spacing, slack)
+    return slack
 
 
 # ----------------------------------------------------------------------------

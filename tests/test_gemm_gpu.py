@@ -955,3 +955,45 @@ def test_matrices_whose_rows_tma_cannot_address_go_through_aligned_copies(case):
         for r in range(rows):
             pad[r * p.ldc * cb: r * p.ldc * cb + cols * cb] = False
         assert np.array_equal(before[pad], after[pad])
+
+
+# ------------------------------------------------------------------ seeded random problems, the library's own plans
+def _random_problems(n=48, seed=20260916):
+    """Shapes, types, layouts, leading dimensions and scalars drawn from a fixed generator: small enough for the
+    full oracle, spread over every kind of plan the library picks by itself for problems of up to a few waves (the
+    one-tile-per-CTA kernel with and without a cluster, the persistent kernel with and without K-slices, aligned
+    copies of matrices whose rows TMA cannot address)."""
+    rng = np.random.default_rng(seed)
+    out = []
+    for i in range(n):
+        M = int(rng.choice([1, 8, 64, 136, 200, 256, 504, 512, 777, 1000, 1304, 2048, 3072, 4096]))
+        N = int(rng.choice([8, 24, 64, 72, 130, 256, 392, 512, 1000, 1536, 2048, 3072]))
+        K = int(rng.choice([0, 8, 40, 64, 136, 256, 520, 1000, 1024, 2048, 3000]))
+        ab = int(rng.choice([BF16, BF16, FP16, FP32]))
+        cd = FP32 if ab == FP32 else int(rng.choice([FP32, ab]))
+        la, lb, lc = (int(x) for x in rng.integers(0, 2, 3))
+        alpha = float(rng.choice([1.0, 1.0, -0.5, 2.0, 0.0]))
+        beta = float(rng.choice([0.0, 0.0, 1.0, -0.75]))
+        pad = [int(x) for x in rng.choice([0, 0, 0, 8, 8, 16, 3, 5], 3)]     # 3 and 5: rows off the 16-byte grid
+        ext = lambda layout, rows, cols: cols if layout == 0 else rows
+        lda = max(1, ext(la, M, K)) + pad[0]
+        ldb = max(1, ext(lb, K, N)) + pad[1]
+        ldc = max(1, ext(lc, M, N)) + pad[2]
+        out.append((i, M, N, K, ab, cd, la, lb, lc, alpha, beta, lda, ldb, ldc))
+    return out
+
+
+@pytest.mark.parametrize("case", _random_problems(), ids=lambda c: f"{c[0]}_{c[1]}x{c[2]}x{c[3]}_{c[4]}{c[5]}{c[6]}{c[7]}{c[8]}")
+def test_seeded_random_problems_on_the_librarys_own_plans(case):
+    i, M, N, K, ab, cd, la, lb, lc, alpha, beta, lda, ldb, ldc = case
+    p = synth.Problem(f"rand{i}", M, N, K, ab, cd, la, lb, lc, alpha, beta, seed=1000 + i, lda=lda, ldb=ldb, ldc=ldc,
+                      dist="normal" if ab == FP16 else "uniform").generate()
+    before = p.C.copy()
+    cbuf, got, cref, den, info = check_full(p)
+    # what lies between the logical row ends and the leading dimension keeps the caller's bits
+    rows, cols = (M, N) if lc == 0 else (N, M)
+    flat_before, flat_after = before.reshape(-1), cbuf.reshape(-1)
+    for r in (0, rows // 2, rows - 1):
+        if p.ldc > cols and r < rows - 1:
+            a, b = flat_before[r * p.ldc + cols:(r + 1) * p.ldc], flat_after[r * p.ldc + cols:(r + 1) * p.ldc]
+            assert np.array_equal(a.view(np.uint8), b.view(np.uint8)), (r, info)

@@ -299,6 +299,13 @@ def test_output_rounding_slack_is_half_an_ulp_of_the_output_type():
         mid = lo + 0.5 * ulp
         slack = float(oracle.output_rounding_slack(np.array([-mid]), FP16)[0])
         assert 0.5 * ulp <= slack < ulp, (x16, slack, ulp)
+    # fp16 results below the smallest normal number (2^-14): the spacing is 2^-24 whatever the value
+    for x16 in (np.float16(9.0e-6), np.float16(6.0e-5), np.float16(6.0e-8), np.float16(3.0e-7)):
+        lo, ulp = float(x16), float(np.spacing(x16))
+        assert ulp == 2.0 ** -24 and lo < 2.0 ** -14
+        slack = float(oracle.output_rounding_slack(np.array([-(lo + 0.5 * ulp)]), FP16)[0])
+        assert 0.5 * ulp <= slack < ulp, (x16, slack, ulp)
+    assert float(oracle.output_rounding_slack(np.array([0.0]), FP16)[0]) == 0.0
     assert np.all(oracle.output_rounding_slack(np.array([1.0, -257.0, 1e30]), FP32) == 0.0)
     # the gate as the GPU tests apply it, on an all-positive sum that is a bf16 tie: K = 257 ones.
     # Cref = Den = 257 lies halfway between 256 and 258; the correctly rounded result (either
