@@ -416,6 +416,15 @@ inline TileConfig choose_config(const Canonical& c, const FlagOverrides& o, int 
     const double fill128 = (double)t128 / (double)(((t128 + w - 1) / w) * w);
     if (t256 <= 2 * w && fill128 >= fill256 + 0.15) best_n = 128;
   }
+  // Operand rows off the 128-byte grid at K around 1000 with a 16-bit C: the tall tile, which moves a quarter fewer
+  // operand bytes (and L2 requests, of which such rows need twice as many) per flop, measured +4.5 to +6.7 % at
+  // 12288 x 6144, 6144 x 12288, 12288 x 12288, 3072 x 3072 and 6144 x 3072 (x 1000), +0.5 to +1.7 % at 6144 x 6144,
+  // 3072 x 12288 and 12288 x 3072, but -2.6 % with four tile rows (2048 x 12288); with an fp32 C or rows on the grid
+  // (K = 1024) its exposed epilogue loses.
+  if (best_g == 2 && best_n == 256 && best_p == 1 && best_r == 1 && unaligned_rows && c.c_bytes == 2 && c.batch <= 1 &&
+      c.K * (c.ab_bytes / 2) >= 768 && c.K * (c.ab_bytes / 2) <= 1536 && c.M >= 3072 && c.N >= 3072 && max_pairs >= 1 &&
+      o.mrep == 0 && o.cta_group == 0 && o.tile_n == 0 && o.share == 0 && o.ksub != 2 && !o.reduce_add && o.grid_limit == 0)
+    best_r = 2;
   // Where the choice fell on plain pairs of 256 x 256 tiles and the operand rows are not 128-byte aligned,
   // the same tiles in shared-operand clusters are the faster form (see kShareGainUnalignedRows), unless the
   // slots of two tiles quantise worse than the single tiles did.
